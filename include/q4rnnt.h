@@ -1,0 +1,274 @@
+/*
+ * q4rnnt — INT4 x INT4 RNN-T inference with density-ratio LM fusion on one GPU.
+ *
+ * C ABI of the CUDA library.  All tensor pointers are DEVICE pointers owned by
+ * the caller unless a parameter says "host"; they must be 16-byte aligned.  No
+ * entry point allocates, frees, or keeps a copy of anything; work is enqueued
+ * on the stream passed last and the call returns without synchronising (except
+ * q4_poll_status).  Every function returns 0 on success or a negative Q4_ERR_*;
+ * argument errors are detected on the host before anything is launched.
+ *
+ * Number formats
+ *   codes, 4 bit : two per byte, element 2i in bits 0-3, element 2i+1 in bits
+ *                  4-7; two's complement when signed, plain when unsigned.
+ *   codes, 8 bit : one per byte, two's complement (signed only).
+ *   rows         : row-major, k_pad elements per row, k_pad a multiple of 32,
+ *                  elements k..k_pad-1 hold the code of the real value 0 (0 for
+ *                  signed codes, the zero point for unsigned ones).
+ *   weights      : symmetric signed codes with one fp32 scale per output row
+ *                  (W[j,k] ~ scale[j] * q[j,k]); biases and LSTM cell states
+ *                  are fp32 and never quantized (paper Section 3.2).
+ *   LSTM gates   : the 4H rows of w_ih / w_hh / bias are ordered i, f, g, o.
+ * A matrix product needs its weight and its input activation at the same bit
+ * width (both 4 or both 8).
+ */
+#ifndef Q4RNNT_H_
+#define Q4RNNT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define Q4_OK 0
+#define Q4_ERR_NULL (-1)        /* a required pointer is NULL */
+#define Q4_ERR_DIM (-2)         /* a size is non-positive or inconsistent */
+#define Q4_ERR_ALIGN (-3)       /* a pointer or k_pad breaks the alignment rule */
+#define Q4_ERR_BITS (-4)        /* bit width not 4/8, or operands disagree */
+#define Q4_ERR_WORKSPACE (-5)   /* workspace smaller than q4_workspace_bytes says */
+#define Q4_ERR_UNSUPPORTED (-6) /* valid request this build does not implement */
+#define Q4_ERR_CUDA (-7)        /* a CUDA runtime call failed (launch error) */
+#define Q4_ERR_TIMEOUT (-8)     /* a bounded device-side wait expired */
+
+typedef void* q4_stream; /* a cudaStream_t, passed as an opaque handle (NULL = default stream) */
+
+/* Integer weight matrix [rows, k_pad] with per-row scales (device pointers). */
+typedef struct {
+  const void* q;
+  const float* scale;
+  int32_t rows, k, k_pad, bits;
+} q4_mat;
+
+/* Constants of one activation quantizer (paper Eq. 2, Eq. 3):
+ *   code = clamp(rne(x * inv_scale) + zero_point, lo, hi),  x_q = scale * (code - zero_point)
+ * rne = round half to even; [lo,hi] = [-2^(b-1), 2^(b-1)-1] when is_signed (symmetric
+ * quantizer, zero_point 0) or [0, 2^b-1] otherwise (asymmetric). */
+typedef struct {
+  float scale, inv_scale;
+  int32_t zero_point, bits, is_signed;
+} q4_act;
+
+/* Fill *out (host) for a symmetric quantizer with boundary alpha (Section 3.1):
+ * scale = alpha / (2^(b-1) - 1), inv_scale = 1 / scale, both rounded to fp32. */
+int q4_act_symmetric(float alpha, int32_t bits, q4_act* out);
+/* Fill *out (host) for the asymmetric quantizer of Eq. 2 with boundaries lo < hi:
+ * scale = (hi - lo) / (2^b - 1), zero_point = clamp(rne(-lo / scale), 0, 2^b - 1). */
+int q4_act_asymmetric(float lo, float hi, int32_t bits, q4_act* out);
+
+/*
+ * quantize_pack_int4 — Eq. 2 on a [rows, k] matrix of fp16 or fp32 values, written as
+ * packed codes [rows, k_pad] (4 or 8 bit per act->bits).  (Section 3.1.)
+ *   mode 0 (FIX / learned constants): `act` (host) gives the quantizer.
+ *   mode 1 (MAX boundary): symmetric, boundary = largest magnitude over each group; row r
+ *          belongs to group r % n_groups (time-major [T,B,*] data with n_groups = B gives one
+ *          boundary per utterance).  The per-group scale is written to group_scale_out
+ *          [n_groups] (device); an all-zero group gets boundary 1.  act->bits selects the width.
+ *   mode 2 (weights): symmetric, row r uses scale per_row_scale[r] (device), act->bits wide.
+ * x_is_fp16: 1 = half precision input, 0 = fp32.  x rows are dense (k values per row).
+ */
+int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k, int32_t k_pad,
+                       const q4_act* act, int32_t mode, int32_t n_groups,
+                       const float* per_row_scale, void* q_out, float* group_scale_out,
+                       q4_stream stream);
+
+/*
+ * qlstm_layer_forward — one uni- or bidirectional quantized LSTM layer over a batch of
+ * sequences (Sections 3.2 and 3.4).  Time-major.
+ *   xq    [T, B, kx_pad] codes of the layer input, quantizer x_act (zero_point honoured);
+ *         x_scale_b (nullable, [B]) overrides x_act.scale per sequence.
+ *   w_ih  [dirs] host array of matrices [4H, kx_pad]; w_hh [dirs] of [4H, H]; bias [dirs]
+ *         host array of device pointers [4H] (entries or the array may be NULL = no bias).
+ *   Direction 1 consumes the sequence backwards with its own weights.
+ *   Per step and direction: int32 MACs of the input and of the previous cell-output codes,
+ *   de-quantization, sigmoid/tanh gates, c_t = f*c + i*g (fp32), h_t = o*tanh(c_t), and h_t
+ *   is quantized ONCE at the cell output with hid_act; that code is the next step's
+ *   recurrent input.  yq [T, B, dirs*H] receives the code of h_t under out_act (the next
+ *   layer's input quantizer: same boundary, possibly another bit width; made from the same
+ *   fp32 h_t), directions concatenated [forward | backward].
+ *   hq_n [dirs, B, H] codes (hid_act) and c_n [dirs, B, H] fp32 receive the final states
+ *   (nullable).  dbg_acc_ih / dbg_acc_hh [T, B, dirs, 4H] int32 (nullable) receive the raw
+ *   accumulators for parity checks.  h0 = c0 = 0.
+ *   workspace: q4_workspace_bytes(Q4_WS_LSTM_LAYER, {T,B,dirs,H}) bytes, scratch.
+ */
+int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scale_b, int32_t T,
+                        int32_t B, int32_t dirs, const q4_mat* w_ih, const q4_mat* w_hh,
+                        const float* const* bias, const q4_act* hid_act, const q4_act* out_act,
+                        void* yq, void* hq_n, float* c_n, int32_t* dbg_acc_ih,
+                        int32_t* dbg_acc_hh, void* workspace, size_t workspace_bytes,
+                        q4_stream stream);
+
+/*
+ * qlstm_step — one LSTM time step for N independent rows (prediction network and LM
+ * building block; Sections 2 and 3.2).
+ *   xq [*, kx_pad] codes; row n reads xq row x_row_idx[n] when x_row_idx is given (an
+ *   embedding lookup into a pre-quantized table), else row n.
+ *   hq_in [N, H] codes (hid_act), c_in [N, H] fp32; c_out may alias c_in, hq_out must not
+ *   alias hq_in (every output cell reads the whole previous row).
+ *   h_f32_out [N, H] (nullable) receives the fp32 cell output before quantization;
+ *   dbg_acc_ih / dbg_acc_hh [N, 4H] int32 (nullable).
+ */
+int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, const void* hq_in,
+               const float* c_in, int32_t N, const q4_mat* w_ih, const q4_mat* w_hh,
+               const float* bias, const q4_act* hid_act, void* hq_out, float* c_out,
+               float* h_f32_out, int32_t* dbg_acc_ih, int32_t* dbg_acc_hh, q4_stream stream);
+
+/*
+ * q4_linear_forward — quantized linear layer (Section 3.2): out[m, j] = acc[m, j] *
+ * (x_act.scale * w.scale[j]) + bias[j], fp32, out [M, w.rows].  Used for the encoder ->
+ * joint projection.  dbg_acc [M, w.rows] int32 nullable.
+ */
+int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_mat* w,
+                      const float* bias, float* out, int32_t* dbg_acc, q4_stream stream);
+
+/*
+ * qjoint_logprobs — joint network (Section 2): the prediction-network cell output codes pq
+ * [N, Hp] (p_act) are projected to D dims (w_pred, b_pred), combined multiplicatively with
+ * the projected encoder frame e[frame_idx[n]] ([*, D] fp32), z = tanh(e * p), z is quantized
+ * with z_act, passed through the output layer (w_out [V, D], b_out) and a log-softmax.
+ * logp [N, V] fp32.  workspace: q4_workspace_bytes(Q4_WS_JOINT, {N, D}).
+ */
+int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, const q4_act* p_act,
+                    int32_t N, const q4_mat* w_pred, const float* b_pred, const q4_act* z_act,
+                    const q4_mat* w_out, const float* b_out, float* logp, void* workspace,
+                    size_t workspace_bytes, q4_stream stream);
+
+/* One LSTM layer / linear layer inside a model description. */
+typedef struct {
+  q4_mat w_ih, w_hh;
+  const float* bias;
+  q4_act hid_act;
+} q4_lstm;
+typedef struct {
+  q4_mat w;
+  const float* bias;
+} q4_linear;
+/* LSTM language model: embedding (pre-quantized table [V, E_pad] codes under emb_act) ->
+ * n_layers LSTM -> bottleneck (H -> D, fp32) -> quantize (bott_act) -> output (D -> V). */
+typedef struct {
+  const void* emb_q;
+  q4_act emb_act;
+  int32_t n_layers;
+  q4_lstm lstm[2];
+  q4_linear bott;
+  q4_act bott_act;
+  q4_linear out;
+} q4_lm;
+/* Everything the beam step needs (host struct of device pointers). */
+typedef struct {
+  int32_t V, E, D;
+  const void* pred_emb_q; /* [V, E_pad] codes under pred_emb_act */
+  q4_act pred_emb_act;
+  q4_lstm pred_lstm;
+  q4_linear pred_proj; /* Hp -> D */
+  q4_act z_act;
+  q4_linear joint_out; /* D -> V */
+  q4_lm src, tgt;
+} q4_model;
+
+/*
+ * Caller-owned search state for B utterances x W beam slots.  R = B * 2W "state rows" hold
+ * network states (a label extension writes a fresh row; a blank extension keeps its
+ * parent's row, so nothing is copied).  Sizes in elements; codes packed as above.
+ */
+typedef struct {
+  /* per state row */
+  void* pred_hq;    /* [R, Hp] codes */
+  float* pred_c;    /* [R, Hp] */
+  float* pred_p;    /* [R, D]  projected prediction output */
+  void* src_hq;     /* [R, Hs] codes */
+  float* src_c;     /* [R, Hs] */
+  float* src_lp;    /* [R, V]  log P_src(. | labels) */
+  void* tgt_hq[2];  /* [R, Ht] codes per layer */
+  float* tgt_c[2];  /* [R, Ht] */
+  float* tgt_lp;    /* [R, V]  log P_tgt(. | labels) */
+  /* per slot [B*W] */
+  float* score;
+  int32_t* t;         /* frames consumed */
+  int32_t* u;         /* labels emitted */
+  uint64_t* hash;     /* hash of the label string */
+  uint64_t* prev_hash;/* hash of the string without its last label */
+  int32_t* last_tok;
+  int32_t* row;       /* state row of the slot, -1 = slot empty */
+  int32_t* adv_src;   /* pending network advance: state row to read (-1 = zero state) */
+  int32_t* adv_dst;   /* row to write (-1 = nothing pending) */
+  int32_t* adv_tok;   /* symbol to feed */
+  /* history [n_iters, B, W] */
+  int32_t* bp_parent; /* slot in the previous beam, -1 = empty */
+  int32_t* bp_token;  /* 0 = blank */
+  float* bp_score;
+  /* finished hypotheses, best first [B, W] */
+  float* fin_score;
+  int32_t* fin_iter;  /* iteration at which it consumed the last frame */
+  int32_t* fin_slot;  /* its slot in the beam entering that iteration */
+  int32_t* fin_n;     /* [B] */
+  int32_t* status;    /* [1] device status word, 0 = ok */
+} q4_beam_state;
+
+/* Reset `state` for a new batch: slot 0 of every utterance holds the empty hypothesis with
+ * the start symbol (0) pending, everything else empty. */
+int q4_beam_init(q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters, q4_stream stream);
+
+/*
+ * dr_fusion_beam_step — one iteration of alignment-length synchronous beam search with the
+ * density-ratio score of Eq. 1 (Section 2) for B utterances x W slots:
+ *   1. pending network advances: every newly created label extension feeds its label to the
+ *      prediction network, the source LM and the target LM (LSTM steps, projections, LM
+ *      log-softmax);
+ *   2. joint network + log-softmax for every live hypothesis at its frame e[t, b];
+ *   3. proposals: blank (t+1, score + log P(blank)) and, while u < u_max, every label k
+ *      (score + log P(k) + lambda_t log P_tgt(k) - lambda_s log P_src(k) + rho);
+ *      proposals describing the same label string are merged by log-addition; blank
+ *      proposals that consumed the last frame go to the finished list (best W kept); the
+ *      W best others (score descending, then parent slot, then token) become the next beam.
+ * e [T, B, D] fp32 projected encoder frames.  `iter` counts from 0; hypotheses in the beam
+ * entering iteration `iter` satisfy t + u = iter.  mode: 0 (the only one implemented).
+ * workspace: q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D}).
+ */
+int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float* e, int32_t B,
+                        int32_t T, int32_t W, int32_t iter, int32_t u_max, float lambda_t,
+                        float lambda_s, float rho, int32_t mode, void* workspace,
+                        size_t workspace_bytes, q4_stream stream);
+
+/* Label strings of the best finished hypothesis per utterance (the best live one if none
+ * finished): tokens [B, u_max], lens [B], scores [B] (device). */
+int q4_traceback(const q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters,
+                 int32_t u_max, int32_t* tokens, int32_t* lens, float* scores, q4_stream stream);
+
+/*
+ * q4_feature_prologue — log-mel [B, T100, M] fp32 at 100 frames/s -> first and second time
+ * differences (d_t = (x_{t+1} - x_{t-1}) / 2, edges replicated; dd likewise on d) -> frames
+ * (2s, 2s+1) concatenated -> out [T100/2, B, 6M] fp16, time-major.  (Section 2 gives only
+ * the feature dimension; this is the reading documented with the workloads.)
+ */
+int q4_feature_prologue(const float* mel, int32_t B, int32_t T100, int32_t M, void* out_fp16,
+                        q4_stream stream);
+
+#define Q4_WS_LSTM_LAYER 1 /* dims = {T, B, dirs, H} */
+#define Q4_WS_JOINT 2      /* dims = {N, D} */
+#define Q4_WS_BEAM 3       /* dims = {B, W, V, D} */
+size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims);
+
+/* Synchronise `stream`, read the device status word and return 0 or the error it holds. */
+int q4_poll_status(const int32_t* device_status, q4_stream stream);
+
+/* Library version and the number of kernels launched so far by this process (a counter the
+ * benchmark reads to report its launch count). */
+int q4_version(void);
+int64_t q4_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* Q4RNNT_H_ */

@@ -149,6 +149,14 @@ def unpack4(b: np.ndarray, k: int, is_signed: bool) -> np.ndarray:
     return q
 
 
+def activations(x: np.ndarray):
+    """The oracle's fp32 exp, sigmoid and tanh on an array."""
+    x = _c(x, np.float32)
+    ex, sg, th = np.empty_like(x), np.empty_like(x), np.empty_like(x)
+    lib().orc_activations(_p(x), C.c_int64(x.size), _p(ex), _p(sg), _p(th))
+    return ex, sg, th
+
+
 def int_matmul(w: np.ndarray, xq: np.ndarray, zero_point: int = 0) -> np.ndarray:
     w = _c(w, np.int8)
     xq = _c(xq, np.int16)

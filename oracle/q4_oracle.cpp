@@ -7,11 +7,17 @@
 // Conventions
 //   * integer codes are held one per int16 (activations) or int8 (weights);
 //     integer accumulation is exact in int32;
-//   * floating-point stages are evaluated in double and rounded to float only
-//     where the method stores a value (cell state, cell output, linear output,
-//     log-probability, hypothesis score);
+//   * every floating-point value that is later quantized or carried as state
+//     (de-quantized pre-activations, gates, cell state, cell output, linear
+//     outputs, tanh(e*p)) is computed in fp32 by a fixed sequence of IEEE
+//     operations (multiply, add, fused multiply-add, divide), including the
+//     exponential behind sigmoid and tanh: a float decides an integer code
+//     there, so the decision is taken in the precision the kernels use and
+//     is reproducible bit for bit on any IEEE machine;
 //   * the quantizer itself is fp32 by definition (one multiply by a stored
-//     reciprocal, round-half-even, clamp) so that codes are reproducible.
+//     reciprocal, round-half-even, clamp);
+//   * reductions whose order is free (log-softmax) and the hypothesis scores
+//     of Eq. 1 are evaluated in double and rounded to float where stored.
 //
 // Parity status: every function below is pinned by tests/test_oracle_*.py
 // (hand tables, closed forms, brute force).  What no test can pin, because it
@@ -149,18 +155,68 @@ struct OrcLinear {
 };
 
 // Quantized linear layer (Section 3.2: weight and input quantized, bias not):
-// out[m,j] = acc[m,j] * (s_x * s_w[j]) + bias[j].
+// out[m,j] = fma(acc[m,j], s_x * s_w[j], bias[j]) in fp32.
 void orc_linear(const OrcLinear* L, const int16_t* xq, const OrcAct* x_act, int32_t M, float* out,
                 int32_t* acc_out) {
   std::vector<int32_t> acc((size_t)M * L->J);
   orc_int_matmul(L->w, L->J, L->K, xq, x_act->zero_point, M, acc.data());
   for (int32_t m = 0; m < M; ++m)
     for (int32_t j = 0; j < L->J; ++j) {
-      double v = (double)acc[(size_t)m * L->J + j] * ((double)x_act->scale * (double)L->s_w[j]);
-      if (L->bias) v += (double)L->bias[j];
-      out[(size_t)m * L->J + j] = (float)v;
+      const float sc = x_act->scale * L->s_w[j];
+      out[(size_t)m * L->J + j] =
+          std::fmaf((float)acc[(size_t)m * L->J + j], sc, L->bias ? L->bias[j] : 0.0f);
     }
   if (acc_out) std::memcpy(acc_out, acc.data(), acc.size() * sizeof(int32_t));
+}
+
+
+// ------------------------------------------------- fp32 activation functions
+// exp(x) for x in [-86, 88]: n = rne(x*log2(e)); r = x - n*ln2 (two-constant
+// reduction, fused multiply-adds); degree-7 Taylor polynomial in r by Horner's
+// rule with fused multiply-adds; scaling by 2^n through the exponent field.
+static inline float f32_from_bits(uint32_t b) {
+  float f;
+  std::memcpy(&f, &b, 4);
+  return f;
+}
+static inline uint32_t bits_from_f32(float f) {
+  uint32_t b;
+  std::memcpy(&b, &f, 4);
+  return b;
+}
+float orc_exp(float x) {
+  x = std::fmin(std::fmax(x, -86.0f), 88.0f);
+  const float n = std::nearbyintf(x * 0x1.715476p+0f);
+  float r = std::fmaf(n, -0x1.62e400p-1f, x);
+  r = std::fmaf(n, -0x1.7f7d1cp-20f, r);
+  float p = 0x1.a01a02p-13f;               // 1/5040
+  p = std::fmaf(p, r, 0x1.6c16c2p-10f);    // 1/720
+  p = std::fmaf(p, r, 0x1.111112p-7f);     // 1/120
+  p = std::fmaf(p, r, 0x1.555556p-5f);     // 1/24
+  p = std::fmaf(p, r, 0x1.555556p-3f);     // 1/6
+  p = std::fmaf(p, r, 0.5f);
+  p = std::fmaf(p, r, 1.0f);
+  p = std::fmaf(p, r, 1.0f);
+  return f32_from_bits(bits_from_f32(p) + ((uint32_t)(int32_t)n << 23));
+}
+// sigmoid(x) = 1 / (1 + exp(-x)), argument clamped to [-86, 86].
+float orc_sigmoid(float x) {
+  x = std::fmin(std::fmax(x, -86.0f), 86.0f);
+  return 1.0f / (1.0f + orc_exp(-x));
+}
+// tanh(x) = sign(x) * (1 - e) / (1 + e), e = exp(-2 min(|x|, 43)).
+float orc_tanh(float x) {
+  const float a = std::fmin(std::fabs(x), 43.0f);
+  const float e = orc_exp(-2.0f * a);
+  const float t = (1.0f - e) / (1.0f + e);
+  return std::copysign(t, x);
+}
+void orc_activations(const float* x, int64_t n, float* ex, float* sg, float* th) {
+  for (int64_t i = 0; i < n; ++i) {
+    if (ex) ex[i] = orc_exp(x[i]);
+    if (sg) sg[i] = orc_sigmoid(x[i]);
+    if (th) th[i] = orc_tanh(x[i]);
+  }
 }
 
 // ---------------------------------------------------------------- LSTM cell
@@ -173,7 +229,7 @@ struct OrcLstm {
   int32_t K, H;
 };
 
-static inline double sigmoid(double v) { return 1.0 / (1.0 + std::exp(-v)); }
+static inline double sigmoid(double v) { return 1.0 / (1.0 + std::exp(-v)); }  // fp reference only
 
 // One time step for N independent rows.  Cell state is kept in floating point
 // and never quantized; the cell output o * tanh(c) lies in [-1,1] and is
@@ -187,22 +243,22 @@ void orc_lstm_step(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act,
                    int32_t* acc_ih_out, int32_t* acc_hh_out, float* gates_out) {
   const int32_t H = L->H, K = L->K, G = 4 * H;
   std::vector<int32_t> a_ih(G), a_hh(G);
-  std::vector<double> act(G);
+  std::vector<float> act(G);
   for (int32_t n = 0; n < N; ++n) {
     orc_int_matmul(L->w_ih, G, K, xq + (int64_t)n * K, x_act->zero_point, 1, a_ih.data());
     orc_int_matmul(L->w_hh, G, H, hq_in + (int64_t)n * H, hid_act->zero_point, 1, a_hh.data());
-    const double s_x = x_scale_row ? (double)x_scale_row[n] : (double)x_act->scale;
-    const double s_h = (double)hid_act->scale;
+    const float s_x = x_scale_row ? x_scale_row[n] : x_act->scale;
+    const float s_h = hid_act->scale;
     for (int32_t j = 0; j < G; ++j) {
-      double pre = (double)a_ih[j] * (s_x * (double)L->s_wih[j]) +
-                   (double)a_hh[j] * (s_h * (double)L->s_whh[j]);
-      if (L->bias) pre += (double)L->bias[j];
-      act[j] = (j >= 2 * H && j < 3 * H) ? std::tanh(pre) : sigmoid(pre);
+      // de-quantize: each accumulator times (activation scale * row scale), plus bias
+      float pre = std::fmaf((float)a_ih[j], s_x * L->s_wih[j], L->bias ? L->bias[j] : 0.0f);
+      pre = std::fmaf((float)a_hh[j], s_h * L->s_whh[j], pre);
+      act[j] = (j >= 2 * H && j < 3 * H) ? orc_tanh(pre) : orc_sigmoid(pre);
     }
     for (int32_t u = 0; u < H; ++u) {
-      const double i = act[u], f = act[H + u], g = act[2 * H + u], o = act[3 * H + u];
-      const float c = (float)(f * (double)c_in[(int64_t)n * H + u] + i * g);
-      const float h = (float)(o * std::tanh((double)c));
+      const float i = act[u], f = act[H + u], g = act[2 * H + u], o = act[3 * H + u];
+      const float c = std::fmaf(f, c_in[(int64_t)n * H + u], i * g);
+      const float h = o * orc_tanh(c);
       c_out[(int64_t)n * H + u] = c;
       if (h_out) h_out[(int64_t)n * H + u] = h;
       hq_out[(int64_t)n * H + u] = (int16_t)quantize_one(h, *hid_act);
@@ -210,7 +266,7 @@ void orc_lstm_step(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act,
     if (acc_ih_out) std::memcpy(acc_ih_out + (int64_t)n * G, a_ih.data(), G * sizeof(int32_t));
     if (acc_hh_out) std::memcpy(acc_hh_out + (int64_t)n * G, a_hh.data(), G * sizeof(int32_t));
     if (gates_out)
-      for (int32_t j = 0; j < G; ++j) gates_out[(int64_t)n * G + j] = (float)act[j];
+      for (int32_t j = 0; j < G; ++j) gates_out[(int64_t)n * G + j] = act[j];
   }
 }
 
@@ -328,7 +384,7 @@ void orc_joint(const OrcJoint* Jn, const float* e, const float* p, int32_t N, fl
   const int32_t D = Jn->out.K, V = Jn->out.J;
   std::vector<float> z((size_t)N * D), logits((size_t)N * V);
   std::vector<int16_t> zq((size_t)N * D);
-  for (int64_t i = 0; i < (int64_t)N * D; ++i) z[i] = (float)std::tanh((double)e[i] * (double)p[i]);
+  for (int64_t i = 0; i < (int64_t)N * D; ++i) z[i] = orc_tanh(e[i] * p[i]);
   orc_quantize(z.data(), (int64_t)N * D, &Jn->z_act, zq.data());
   orc_linear(&Jn->out, zq.data(), &Jn->z_act, N, logits.data(), acc_out);
   orc_log_softmax(logits.data(), N, V, logp);

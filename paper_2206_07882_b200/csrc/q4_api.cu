@@ -1,0 +1,546 @@
+// C ABI of the library (see include/q4rnnt.h): argument checking on the host, argument
+// blocks for the kernels, launch sequencing.  Nothing here allocates or synchronises.
+#include <math.h>
+#include <string.h>
+
+#include "q4_internal.h"
+
+using namespace q4;
+
+#define Q4_TRY(expr)                               \
+  do {                                             \
+    cudaError_t e__ = (expr);                      \
+    if (e__ != cudaSuccess) return Q4_ERR_CUDA;    \
+  } while (0)
+#define Q4_CHECK(expr)        \
+  do {                        \
+    int r__ = (expr);         \
+    if (r__ != Q4_OK) return r__; \
+  } while (0)
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline cudaStream_t S(q4_stream s) { return reinterpret_cast<cudaStream_t>(s); }
+
+int check_act(const q4_act* a) {
+  if (!a) return Q4_ERR_NULL;
+  if (a->bits != 4 && a->bits != 8) return Q4_ERR_BITS;
+  if (!a->is_signed && a->bits != 4) return Q4_ERR_BITS;  // unsigned codes exist at 4 bit only
+  if (!a->is_signed && (a->zero_point < 0 || a->zero_point > 15)) return Q4_ERR_DIM;
+  if (a->is_signed && a->zero_point != 0) return Q4_ERR_DIM;
+  if (!(a->scale > 0.0f) || !(a->inv_scale > 0.0f)) return Q4_ERR_DIM;
+  return Q4_OK;
+}
+
+int check_mat(const q4_mat* m, int rows, int k_pad_expected) {
+  if (!m || !m->q || !m->scale) return Q4_ERR_NULL;
+  if (m->bits != 4 && m->bits != 8) return Q4_ERR_BITS;
+  if (m->rows <= 0 || m->k <= 0 || m->k_pad < m->k) return Q4_ERR_DIM;
+  if (m->k_pad % 32 != 0) return Q4_ERR_ALIGN;
+  if (rows > 0 && m->rows != rows) return Q4_ERR_DIM;
+  if (k_pad_expected > 0 && m->k_pad != k_pad_expected) return Q4_ERR_DIM;
+  if (!aligned16(m->q) || (reinterpret_cast<uintptr_t>(m->scale) & 3u)) return Q4_ERR_ALIGN;
+  return Q4_OK;
+}
+
+inline long long row_bytes(int k_pad, int bits) { return (long long)k_pad * bits / 8; }
+
+GemmArgs gemm_args(const void* x, long long x_stride, const int32_t* x_idx, const q4_act& xa, int M,
+                   const q4_mat& w, const float* bias, void* out, long long out_stride,
+                   const int32_t* out_idx) {
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.x.base = static_cast<const uint8_t*>(x);
+  g.x.stride = x_stride;
+  g.x.idx = x_idx;
+  g.x_signed = xa.is_signed;
+  g.x_zp = xa.zero_point;
+  g.M = M;
+  g.w = static_cast<const uint8_t*>(w.q);
+  g.w_scale = w.scale;
+  g.bias = bias;
+  g.J = w.rows;
+  g.k_pad = w.k_pad;
+  g.x_scale = xa.scale;
+  g.out = out;
+  g.out_stride = out_stride;
+  g.out_idx = out_idx;
+  return g;
+}
+
+}  // namespace
+
+extern "C" {
+
+int q4_version(void) { return 1; }
+int64_t q4_launch_count(void) { return g_launches; }
+
+int q4_act_symmetric(float alpha, int32_t bits, q4_act* out) {
+  if (!out) return Q4_ERR_NULL;
+  if (bits != 4 && bits != 8) return Q4_ERR_BITS;
+  if (!(alpha > 0.0f)) return Q4_ERR_DIM;
+  const volatile float qmax = (float)((1 << (bits - 1)) - 1);
+  const volatile float s = alpha / qmax;
+  const volatile float inv = 1.0f / s;
+  out->scale = s;
+  out->inv_scale = inv;
+  out->zero_point = 0;
+  out->bits = bits;
+  out->is_signed = 1;
+  return Q4_OK;
+}
+
+int q4_act_asymmetric(float lo, float hi, int32_t bits, q4_act* out) {
+  if (!out) return Q4_ERR_NULL;
+  if (bits != 4) return Q4_ERR_BITS;
+  if (!(hi > lo)) return Q4_ERR_DIM;
+  const volatile float qmax = (float)((1 << bits) - 1);
+  const volatile float s = (hi - lo) / qmax;
+  const volatile float inv = 1.0f / s;
+  const volatile float zr = -lo / s;
+  float z = nearbyintf(zr);
+  z = fminf(fmaxf(z, 0.0f), qmax);
+  out->scale = s;
+  out->inv_scale = inv;
+  out->zero_point = (int32_t)z;
+  out->bits = bits;
+  out->is_signed = 0;
+  return Q4_OK;
+}
+
+size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims) {
+  if (!dims) return 0;
+  if (call_id == Q4_WS_LSTM_LAYER && ndims >= 4) {
+    const size_t T = dims[0], B = dims[1], D = dims[2], H = dims[3];
+    size_t n = 0;
+    n += align_up(D * T * B * 4 * H * sizeof(int32_t));  // input accumulators
+    n += align_up(D * 2 * B * H);                        // recurrent codes, double buffered
+    n += align_up(D * B * H * sizeof(float));            // cell state
+    return n;
+  }
+  if (call_id == Q4_WS_JOINT && ndims >= 2) {
+    const size_t N = dims[0], D = dims[1];
+    return align_up(N * D * sizeof(float)) + align_up(N * D);
+  }
+  if (call_id == Q4_WS_BEAM && ndims >= 4) {
+    const size_t N = (size_t)dims[0] * dims[1], V = dims[2], D = dims[3];
+    return align_up(N * D) * 3 + align_up(N * V * sizeof(float)) + align_up(N * sizeof(int32_t));
+  }
+  return 0;
+}
+
+int q4_poll_status(const int32_t* device_status, q4_stream stream) {
+  if (!device_status) return Q4_ERR_NULL;
+  int32_t h = 0;
+  if (cudaMemcpyAsync(&h, device_status, sizeof(h), cudaMemcpyDeviceToHost, S(stream)) != cudaSuccess)
+    return Q4_ERR_CUDA;
+  if (cudaStreamSynchronize(S(stream)) != cudaSuccess) return Q4_ERR_CUDA;
+  return h == 0 ? Q4_OK : (int)h;
+}
+
+int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k, int32_t k_pad,
+                       const q4_act* act, int32_t mode, int32_t n_groups,
+                       const float* per_row_scale, void* q_out, float* group_scale_out,
+                       q4_stream stream) {
+  if (!x || !q_out || !act) return Q4_ERR_NULL;
+  if (rows < 0 || k <= 0 || k_pad < k) return Q4_ERR_DIM;
+  if (k_pad % 32 != 0 || !aligned16(q_out)) return Q4_ERR_ALIGN;
+  if (act->bits != 4 && act->bits != 8) return Q4_ERR_BITS;
+  if (mode < 0 || mode > 2) return Q4_ERR_UNSUPPORTED;
+  q4_act a = *act;
+  if (mode == 0) {
+    Q4_CHECK(check_act(act));
+  } else {
+    a.is_signed = 1;
+    a.zero_point = 0;
+    a.scale = a.inv_scale = 1.0f;
+    if (mode == 1 && (!group_scale_out || n_groups <= 0)) return group_scale_out ? Q4_ERR_DIM : Q4_ERR_NULL;
+    if (mode == 2 && !per_row_scale) return Q4_ERR_NULL;
+  }
+  if (rows == 0) return Q4_OK;
+  Q4_TRY(launch_quantize(x, x_is_fp16 != 0, rows, k, k_pad, a, mode, n_groups, per_row_scale,
+                         static_cast<uint8_t*>(q_out), group_scale_out, S(stream)));
+  return Q4_OK;
+}
+
+int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_mat* w,
+                      const float* bias, float* out, int32_t* dbg_acc, q4_stream stream) {
+  if (!xq || !out) return Q4_ERR_NULL;
+  Q4_CHECK(check_act(x_act));
+  Q4_CHECK(check_mat(w, 0, 0));
+  if (M < 0) return Q4_ERR_DIM;
+  if (w->bits != x_act->bits) return Q4_ERR_BITS;
+  if (!aligned16(xq) || !aligned16(out)) return Q4_ERR_ALIGN;
+  GemmArgs g = gemm_args(xq, row_bytes(w->k_pad, w->bits), nullptr, *x_act, M, *w, bias, out,
+                         w->rows, nullptr);
+  g.dbg_acc = dbg_acc;
+  Q4_TRY(launch_gemm(g, w->bits, EPI_F32, S(stream)));
+  return Q4_OK;
+}
+
+static int check_lstm(const q4_mat* w_ih, const q4_mat* w_hh, const q4_act* x_act,
+                      const q4_act* hid_act, int* H_out) {
+  Q4_CHECK(check_act(x_act));
+  Q4_CHECK(check_act(hid_act));
+  if (!hid_act->is_signed) return Q4_ERR_UNSUPPORTED;
+  Q4_CHECK(check_mat(w_ih, 0, 0));
+  Q4_CHECK(check_mat(w_hh, 0, 0));
+  if (w_ih->rows != w_hh->rows || w_ih->rows % 4 != 0) return Q4_ERR_DIM;
+  const int H = w_ih->rows / 4;
+  if (w_hh->k != H || w_hh->k_pad != H) return Q4_ERR_DIM;
+  if (H % 32 != 0) return Q4_ERR_ALIGN;
+  if (w_ih->bits != x_act->bits || w_hh->bits != hid_act->bits) return Q4_ERR_BITS;
+  *H_out = H;
+  return Q4_OK;
+}
+
+static void fill_lstm_weights(LstmArgs& a, const q4_mat& w_ih, const q4_mat& w_hh, const float* bias,
+                              const q4_act& x_act, const q4_act& hid_act) {
+  a.x_signed = x_act.is_signed;
+  a.x_zp = x_act.zero_point;
+  a.kx_pad = w_ih.k_pad;
+  a.x_scale = x_act.scale;
+  a.w_ih = static_cast<const uint8_t*>(w_ih.q);
+  a.s_wih = w_ih.scale;
+  a.w_hh = static_cast<const uint8_t*>(w_hh.q);
+  a.s_whh = w_hh.scale;
+  a.bias = bias;
+  a.H = w_ih.rows / 4;
+  a.kh_pad = w_hh.k_pad;
+  a.hid_act = hid_act;
+  a.out_act = hid_act;
+}
+
+int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, const void* hq_in,
+               const float* c_in, int32_t N, const q4_mat* w_ih, const q4_mat* w_hh,
+               const float* bias, const q4_act* hid_act, void* hq_out, float* c_out,
+               float* h_f32_out, int32_t* dbg_acc_ih, int32_t* dbg_acc_hh, q4_stream stream) {
+  if (!xq || !hq_in || !c_in || !hq_out || !c_out) return Q4_ERR_NULL;
+  int H = 0;
+  Q4_CHECK(check_lstm(w_ih, w_hh, x_act, hid_act, &H));
+  if (N < 0) return Q4_ERR_DIM;
+  if (hq_in == hq_out) return Q4_ERR_UNSUPPORTED;
+  if (!aligned16(xq) || !aligned16(hq_in) || !aligned16(hq_out)) return Q4_ERR_ALIGN;
+  if (N == 0) return Q4_OK;
+  LstmArgs2 args;
+  memset(&args, 0, sizeof(args));
+  LstmArgs& a = args.d[0];
+  fill_lstm_weights(a, *w_ih, *w_hh, bias, *x_act, *hid_act);
+  a.x.base = static_cast<const uint8_t*>(xq);
+  a.x.stride = row_bytes(w_ih->k_pad, w_ih->bits);
+  a.x.idx = x_row_idx;
+  a.hin.base = static_cast<const uint8_t*>(hq_in);
+  a.hin.stride = row_bytes(H, hid_act->bits);
+  a.c_in = c_in;
+  a.N = N;
+  a.hq_out = static_cast<uint8_t*>(hq_out);
+  a.hq_stride = a.hin.stride;
+  a.c_out = c_out;
+  a.h_f32 = h_f32_out;
+  a.dbg_ih = dbg_acc_ih;
+  a.dbg_hh = dbg_acc_hh;
+  a.dbg_stride = 4LL * H;
+  Q4_TRY(launch_lstm(args, 1, w_ih->bits, w_hh->bits, S(stream)));
+  return Q4_OK;
+}
+
+int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scale_b, int32_t T,
+                        int32_t B, int32_t dirs, const q4_mat* w_ih, const q4_mat* w_hh,
+                        const float* const* bias, const q4_act* hid_act, const q4_act* out_act,
+                        void* yq, void* hq_n, float* c_n, int32_t* dbg_acc_ih,
+                        int32_t* dbg_acc_hh, void* workspace, size_t workspace_bytes,
+                        q4_stream stream) {
+  if (!xq || !yq || !w_ih || !w_hh || !workspace) return Q4_ERR_NULL;
+  if (T <= 0 || B <= 0 || dirs < 1 || dirs > 2) return Q4_ERR_DIM;
+  int H = 0;
+  for (int d = 0; d < dirs; ++d) {
+    int Hd = 0;
+    Q4_CHECK(check_lstm(&w_ih[d], &w_hh[d], x_act, hid_act, &Hd));
+    if (d == 0) H = Hd;
+    if (Hd != H || w_ih[d].k_pad != w_ih[0].k_pad || w_ih[d].bits != w_ih[0].bits) return Q4_ERR_DIM;
+  }
+  if (!out_act) out_act = hid_act;
+  Q4_CHECK(check_act(out_act));
+  if (!out_act->is_signed) return Q4_ERR_UNSUPPORTED;
+  if (!aligned16(xq) || !aligned16(yq) || !aligned16(workspace)) return Q4_ERR_ALIGN;
+  const int32_t dims[4] = {T, B, dirs, H};
+  if (workspace_bytes < q4_workspace_bytes(Q4_WS_LSTM_LAYER, dims, 4)) return Q4_ERR_WORKSPACE;
+
+  cudaStream_t s = S(stream);
+  const long long TB = (long long)T * B;
+  const int G = 4 * H;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int32_t* acc_ih = reinterpret_cast<int32_t*>(ws);
+  ws += align_up((size_t)dirs * TB * G * sizeof(int32_t));
+  uint8_t* hbuf = ws;  // [dirs][2][B*H bytes]
+  ws += align_up((size_t)dirs * 2 * B * H);
+  float* cbuf = reinterpret_cast<float*>(ws);  // [dirs][B][H]
+  const long long hb = row_bytes(H, hid_act->bits);
+  const long long yb = row_bytes(dirs * H, out_act->bits);
+  const long long xb = row_bytes(w_ih[0].k_pad, w_ih[0].bits);
+
+  // time-parallel input projections for all frames
+  for (int d = 0; d < dirs; ++d) {
+    GemmArgs g = gemm_args(xq, xb, nullptr, *x_act, (int)TB, w_ih[d], nullptr,
+                           acc_ih + (size_t)d * TB * G, G, nullptr);
+    Q4_TRY(launch_gemm(g, w_ih[d].bits, EPI_I32, s));
+  }
+  Q4_TRY(cudaMemsetAsync(hbuf, 0, (size_t)dirs * 2 * B * H, s));
+  Q4_TRY(cudaMemsetAsync(cbuf, 0, (size_t)dirs * B * H * sizeof(float), s));
+
+  for (int st = 0; st < T; ++st) {
+    LstmArgs2 args;
+    memset(&args, 0, sizeof(args));
+    for (int d = 0; d < dirs; ++d) {
+      const int t = d == 0 ? st : T - 1 - st;
+      LstmArgs& a = args.d[d];
+      fill_lstm_weights(a, w_ih[d], w_hh[d], bias ? bias[d] : nullptr, *x_act, *hid_act);
+      a.out_act = *out_act;
+      a.x_scale_vec = x_scale_b;
+      a.x_scale_mod = B;
+      a.acc_pre = acc_ih + ((size_t)d * TB + (size_t)t * B) * G;
+      a.acc_pre_stride = G;
+      a.hin.base = hbuf + ((size_t)d * 2 + (st & 1)) * B * H;
+      a.hin.stride = hb;
+      a.c_in = cbuf + (size_t)d * B * H;
+      a.N = B;
+      a.hq_out = hbuf + ((size_t)d * 2 + ((st + 1) & 1)) * B * H;
+      a.hq_stride = hb;
+      a.c_out = cbuf + (size_t)d * B * H;
+      a.yq_out = static_cast<uint8_t*>(yq) + (size_t)t * B * yb + row_bytes(d * H, out_act->bits);
+      a.yq_stride = yb;
+      if (dbg_acc_ih) a.dbg_ih = dbg_acc_ih + ((size_t)t * B * dirs + d) * G;
+      if (dbg_acc_hh) a.dbg_hh = dbg_acc_hh + ((size_t)t * B * dirs + d) * G;
+      a.dbg_stride = (long long)dirs * G;
+    }
+    Q4_TRY(launch_lstm(args, dirs, w_ih[0].bits, w_hh[0].bits, s));
+  }
+  for (int d = 0; d < dirs; ++d) {
+    if (hq_n)
+      Q4_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(hq_n) + (size_t)d * B * hb,
+                             hbuf + ((size_t)d * 2 + (T & 1)) * B * H, (size_t)B * hb,
+                             cudaMemcpyDeviceToDevice, s));
+    if (c_n)
+      Q4_TRY(cudaMemcpyAsync(c_n + (size_t)d * B * H, cbuf + (size_t)d * B * H,
+                             (size_t)B * H * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  }
+  return Q4_OK;
+}
+
+int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, const q4_act* p_act,
+                    int32_t N, const q4_mat* w_pred, const float* b_pred, const q4_act* z_act,
+                    const q4_mat* w_out, const float* b_out, float* logp, void* workspace,
+                    size_t workspace_bytes, q4_stream stream) {
+  if (!e || !frame_idx || !pq || !logp || !workspace) return Q4_ERR_NULL;
+  Q4_CHECK(check_act(p_act));
+  Q4_CHECK(check_act(z_act));
+  Q4_CHECK(check_mat(w_pred, 0, 0));
+  Q4_CHECK(check_mat(w_out, 0, 0));
+  if (N < 0) return Q4_ERR_DIM;
+  const int D = w_pred->rows, V = w_out->rows;
+  if (w_out->k != D || w_out->k_pad != D || D % 32 != 0) return Q4_ERR_DIM;
+  if (w_pred->bits != p_act->bits || w_out->bits != z_act->bits) return Q4_ERR_BITS;
+  if (!aligned16(pq) || !aligned16(workspace) || !aligned16(e)) return Q4_ERR_ALIGN;
+  const int32_t dims[2] = {N, D};
+  if (workspace_bytes < q4_workspace_bytes(Q4_WS_JOINT, dims, 2)) return Q4_ERR_WORKSPACE;
+  if (N == 0) return Q4_OK;
+  cudaStream_t s = S(stream);
+  float* p = static_cast<float*>(workspace);
+  uint8_t* zq = static_cast<uint8_t*>(workspace) + align_up((size_t)N * D * sizeof(float));
+  GemmArgs g1 = gemm_args(pq, row_bytes(w_pred->k_pad, w_pred->bits), nullptr, *p_act, N, *w_pred,
+                          b_pred, p, D, nullptr);
+  Q4_TRY(launch_gemm(g1, w_pred->bits, EPI_F32, s));
+  Q4_TRY(launch_joint_z(e, frame_idx, nullptr, 1, 1, p, nullptr, N, D, *z_act, zq, nullptr, s));
+  GemmArgs g2 = gemm_args(zq, row_bytes(D, z_act->bits), nullptr, *z_act, N, *w_out, b_out, logp, V,
+                          nullptr);
+  Q4_TRY(launch_gemm(g2, w_out->bits, EPI_F32, s));
+  Q4_TRY(launch_logsoftmax(logp, logp, N, V, V, nullptr, s));
+  return Q4_OK;
+}
+
+int q4_feature_prologue(const float* mel, int32_t B, int32_t T100, int32_t M, void* out_fp16,
+                        q4_stream stream) {
+  if (!mel || !out_fp16) return Q4_ERR_NULL;
+  if (B <= 0 || T100 < 2 || M <= 0) return Q4_ERR_DIM;
+  Q4_TRY(launch_features(mel, B, T100, M, out_fp16, S(stream)));
+  return Q4_OK;
+}
+
+// ------------------------------------------------------------------------ beam search
+static int check_state(const q4_beam_state* st, int n_lm_layers) {
+  if (!st) return Q4_ERR_NULL;
+  const void* req[] = {st->pred_hq, st->pred_c, st->pred_p, st->src_hq, st->src_c, st->src_lp,
+                       st->tgt_hq[0], st->tgt_c[0], st->tgt_lp, st->score, st->t, st->u, st->hash,
+                       st->prev_hash, st->last_tok, st->row, st->adv_src, st->adv_dst, st->adv_tok,
+                       st->bp_parent, st->bp_token, st->bp_score, st->fin_score, st->fin_iter,
+                       st->fin_slot, st->fin_n, st->status};
+  for (const void* p : req)
+    if (!p) return Q4_ERR_NULL;
+  if (n_lm_layers > 1 && (!st->tgt_hq[1] || !st->tgt_c[1])) return Q4_ERR_NULL;
+  return Q4_OK;
+}
+
+int q4_beam_init(q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters, q4_stream stream) {
+  Q4_CHECK(check_state(state, 1));
+  if (B <= 0 || W <= 0 || W > 16 || n_iters < 0) return Q4_ERR_DIM;
+  Q4_TRY(launch_beam_init(*state, B, W, n_iters, S(stream)));
+  return Q4_OK;
+}
+
+// One network's pending advance for all slots: LSTM layers reading the parent's state row and
+// writing the fresh row, then the projection(s).
+static int advance_lstm(const q4_lstm& L, const void* x, long long x_stride, const int32_t* x_idx,
+                        const q4_act& x_act, void* hq, float* c, const q4_beam_state& st, int N,
+                        cudaStream_t s) {
+  LstmArgs2 args;
+  memset(&args, 0, sizeof(args));
+  LstmArgs& a = args.d[0];
+  fill_lstm_weights(a, L.w_ih, L.w_hh, L.bias, x_act, L.hid_act);
+  const int H = a.H;
+  a.x.base = static_cast<const uint8_t*>(x);
+  a.x.stride = x_stride;
+  a.x.idx = x_idx;
+  a.hin.base = static_cast<const uint8_t*>(hq);
+  a.hin.stride = row_bytes(H, L.hid_act.bits);
+  a.hin.idx = st.adv_src;
+  a.c_in = c;
+  a.N = N;
+  a.hq_out = static_cast<uint8_t*>(hq);
+  a.hq_stride = a.hin.stride;
+  a.out_idx = st.adv_dst;
+  a.c_out = c;
+  a.dbg_stride = 4LL * H;
+  Q4_TRY(launch_lstm(args, 1, L.w_ih.bits, L.w_hh.bits, s));
+  return Q4_OK;
+}
+
+static int check_model_lstm(const q4_lstm& L, const q4_act& x_act) {
+  int H = 0;
+  return check_lstm(&L.w_ih, &L.w_hh, &x_act, &L.hid_act, &H);
+}
+
+int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float* e, int32_t B,
+                        int32_t T, int32_t W, int32_t iter, int32_t u_max, float lambda_t,
+                        float lambda_s, float rho, int32_t mode, void* workspace,
+                        size_t workspace_bytes, q4_stream stream) {
+  if (!model || !e || !workspace) return Q4_ERR_NULL;
+  if (mode != 0) return Q4_ERR_UNSUPPORTED;
+  if (B <= 0 || T <= 0 || W <= 0 || W > 16 || iter < 0 || u_max < 0) return Q4_ERR_DIM;
+  const q4_model& m = *model;
+  Q4_CHECK(check_state(state, m.tgt.n_layers));
+  const int V = m.V, D = m.D;
+  if (V <= 1 || D <= 0 || D % 32 != 0 || m.E <= 0) return Q4_ERR_DIM;
+  if (m.src.n_layers < 1 || m.src.n_layers > 2 || m.tgt.n_layers < 1 || m.tgt.n_layers > 2)
+    return Q4_ERR_DIM;
+  if (!m.pred_emb_q || !m.src.emb_q || !m.tgt.emb_q) return Q4_ERR_NULL;
+  Q4_CHECK(check_model_lstm(m.pred_lstm, m.pred_emb_act));
+  Q4_CHECK(check_mat(&m.pred_proj.w, D, m.pred_lstm.w_hh.k_pad));
+  Q4_CHECK(check_act(&m.z_act));
+  Q4_CHECK(check_mat(&m.joint_out.w, V, D));
+  if (m.joint_out.w.bits != m.z_act.bits || m.pred_proj.w.bits != m.pred_lstm.hid_act.bits)
+    return Q4_ERR_BITS;
+  const q4_lm* lms[2] = {&m.src, &m.tgt};
+  for (const q4_lm* lm : lms) {
+    Q4_CHECK(check_model_lstm(lm->lstm[0], lm->emb_act));
+    if (lm->n_layers == 2) Q4_CHECK(check_model_lstm(lm->lstm[1], lm->lstm[0].hid_act));
+    const q4_lstm& last = lm->lstm[lm->n_layers - 1];
+    Q4_CHECK(check_mat(&lm->bott.w, D, last.w_hh.k_pad));
+    Q4_CHECK(check_act(&lm->bott_act));
+    Q4_CHECK(check_mat(&lm->out.w, V, D));
+    if (lm->bott.w.bits != last.hid_act.bits || lm->out.w.bits != lm->bott_act.bits) return Q4_ERR_BITS;
+  }
+  if ((size_t)W * V * sizeof(float) > 200 * 1024) return Q4_ERR_UNSUPPORTED;
+  const int32_t dims[4] = {B, W, V, D};
+  if (workspace_bytes < q4_workspace_bytes(Q4_WS_BEAM, dims, 4)) return Q4_ERR_WORKSPACE;
+  if (!aligned16(workspace) || !aligned16(e)) return Q4_ERR_ALIGN;
+
+  cudaStream_t s = S(stream);
+  const q4_beam_state& st = *state;
+  const int N = B * W;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint8_t* zq = ws;
+  ws += align_up((size_t)N * D);
+  uint8_t* bq_src = ws;
+  ws += align_up((size_t)N * D);
+  uint8_t* bq_tgt = ws;
+  ws += align_up((size_t)N * D);
+  float* logits = reinterpret_cast<float*>(ws);
+  ws += align_up((size_t)N * V * sizeof(float));
+  int32_t* live = reinterpret_cast<int32_t*>(ws);
+
+  // 1. pending advances -------------------------------------------------------------
+  {  // prediction network: embedding row -> LSTM -> projection to D
+    const q4_lstm& L = m.pred_lstm;
+    Q4_CHECK(advance_lstm(L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), st.adv_tok,
+                          m.pred_emb_act, st.pred_hq, st.pred_c, st, N, s));
+    GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), st.adv_dst,
+                           L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, st.adv_dst);
+    Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
+  }
+  for (int which = 0; which < 2; ++which) {
+    const q4_lm& lm = *lms[which];
+    void* hq0 = which == 0 ? st.src_hq : st.tgt_hq[0];
+    float* c0 = which == 0 ? st.src_c : st.tgt_c[0];
+    float* lp = which == 0 ? st.src_lp : st.tgt_lp;
+    uint8_t* bq = which == 0 ? bq_src : bq_tgt;
+    const q4_lstm& L0 = lm.lstm[0];
+    Q4_CHECK(advance_lstm(L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), st.adv_tok,
+                          lm.emb_act, hq0, c0, st, N, s));
+    const void* top = hq0;
+    const q4_lstm* last = &L0;
+    if (lm.n_layers == 2) {
+      if (which == 0) return Q4_ERR_UNSUPPORTED;  // the state block holds one source-LM layer
+      const q4_lstm& L1 = lm.lstm[1];
+      Q4_CHECK(advance_lstm(L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), st.adv_dst,
+                            L0.hid_act, st.tgt_hq[1], st.tgt_c[1], st, N, s));
+      top = st.tgt_hq[1];
+      last = &L1;
+    }
+    GemmArgs gb = gemm_args(top, row_bytes(last->w_hh.k_pad, last->hid_act.bits), st.adv_dst,
+                            last->hid_act, N, lm.bott.w, lm.bott.bias, bq,
+                            row_bytes(D, lm.bott_act.bits), nullptr);
+    gb.out_act = lm.bott_act;
+    Q4_TRY(launch_gemm(gb, lm.bott.w.bits, EPI_QUANT, s));
+    GemmArgs go = gemm_args(bq, row_bytes(D, lm.bott_act.bits), nullptr, lm.bott_act, N, lm.out.w,
+                            lm.out.bias, lp, V, st.adv_dst);
+    Q4_TRY(launch_gemm(go, lm.out.w.bits, EPI_F32, s));
+    Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, st.adv_dst, s));
+  }
+
+  // 2. joint network for every live slot at its frame -----------------------------------
+  Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, zq, live, s));
+  GemmArgs gj = gemm_args(zq, row_bytes(D, m.z_act.bits), live, m.z_act, N, m.joint_out.w,
+                          m.joint_out.bias, logits, V, nullptr);
+  Q4_TRY(launch_gemm(gj, m.joint_out.w.bits, EPI_F32, s));
+
+  // 3. Eq. 1 proposals, merge, finished list, next beam --------------------------------
+  BeamSelArgs sel;
+  memset(&sel, 0, sizeof(sel));
+  sel.logits = logits;
+  sel.src_lp = st.src_lp;
+  sel.tgt_lp = st.tgt_lp;
+  sel.st = st;
+  sel.B = B;
+  sel.T = T;
+  sel.W = W;
+  sel.V = V;
+  sel.iter = iter;
+  sel.u_max = u_max;
+  sel.lambda_t = lambda_t;
+  sel.lambda_s = lambda_s;
+  sel.rho = rho;
+  Q4_TRY(launch_beam_select(sel, s));
+  return Q4_OK;
+}
+
+int q4_traceback(const q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters,
+                 int32_t u_max, int32_t* tokens, int32_t* lens, float* scores, q4_stream stream) {
+  Q4_CHECK(check_state(state, 1));
+  if (!tokens || !lens || !scores) return Q4_ERR_NULL;
+  if (B <= 0 || W <= 0 || W > 16 || n_iters < 0 || u_max <= 0) return Q4_ERR_DIM;
+  Q4_TRY(launch_traceback(*state, B, W, n_iters, u_max, tokens, lens, scores, S(stream)));
+  return Q4_OK;
+}
+
+}  // extern "C"

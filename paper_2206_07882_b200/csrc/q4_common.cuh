@@ -1,0 +1,136 @@
+// Shared device helpers of the CUDA library: operand tile staging (packed codes
+// in global memory -> int8 in shared memory), the quantizer, launch accounting.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/q4rnnt.h"
+
+namespace q4 {
+
+constexpr int TILE = 64;        // rows of each operand per CTA tile
+constexpr int KC = 128;         // K elements staged per chunk
+constexpr int PITCH = KC + 16;  // shared-memory row pitch in bytes (16 B aligned, conflict-free)
+constexpr int NT = 256;         // threads per CTA of the tile kernels
+
+extern int64_t g_launches;      // kernels launched by this process
+
+// Where the rows of an operand live: row n is at base + (idx ? idx[n] : n) * stride bytes;
+// a negative index means "no row" (reads as zeros / is not written).
+struct RowSrc {
+  const uint8_t* base;
+  long long stride;
+  const int32_t* idx;
+};
+
+__device__ __forceinline__ int dp4a(int a, int b, int c) { return __dp4a(a, b, c); }
+
+// 8 packed nibbles -> two words of 4 int8 each (even elements, odd elements).  Both
+// operands of a dot product are unpacked the same way, so the element order inside a
+// word does not matter.  sub = value subtracted from every element (8 via the xor trick
+// for two's complement; the zero point for unsigned codes).
+__device__ __forceinline__ void unpack8(uint32_t w, bool is_signed, uint32_t zp4, uint32_t& even,
+                                        uint32_t& odd) {
+  uint32_t lo = w & 0x0F0F0F0Fu, hi = (w >> 4) & 0x0F0F0F0Fu;
+  if (is_signed) {
+    even = __vsub4(lo ^ 0x08080808u, 0x08080808u);
+    odd = __vsub4(hi ^ 0x08080808u, 0x08080808u);
+  } else {
+    even = __vsub4(lo, zp4);
+    odd = __vsub4(hi, zp4);
+  }
+}
+
+// Stage one K chunk [k0, k0+KC) of a 64-row operand tile into shared memory as int8.
+// rowp[s] = first byte of the global row that belongs in shared row s (nullptr = zeros).
+// Thread t handles 32 elements of row t/4.  BITS = storage width of the codes.
+template <int BITS>
+__device__ __forceinline__ void stage_chunk(int8_t* smem, const uint8_t* const* rowp, int k0,
+                                            int k_pad, bool is_signed, uint32_t zp4, int tid) {
+  const int s = tid >> 2, seg = tid & 3;
+  const int k = k0 + 32 * seg;
+  uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
+  const uint8_t* p = rowp[s];
+  if (p != nullptr && k < k_pad) {
+    if (BITS == 4) {
+      const uint4 v = *reinterpret_cast<const uint4*>(p + (k >> 1));
+      unpack8(v.x, is_signed, zp4, o0.x, o0.y);
+      unpack8(v.y, is_signed, zp4, o0.z, o0.w);
+      unpack8(v.z, is_signed, zp4, o1.x, o1.y);
+      unpack8(v.w, is_signed, zp4, o1.z, o1.w);
+    } else {
+      o0 = *reinterpret_cast<const uint4*>(p + k);
+      o1 = *reinterpret_cast<const uint4*>(p + k + 16);
+    }
+  }
+  uint4* d = reinterpret_cast<uint4*>(smem + s * PITCH + 32 * seg);
+  d[0] = o0;
+  d[1] = o1;
+}
+
+// Eq. 2 in fp32: one multiply by the stored reciprocal, round half to even, add the zero
+// point, clamp.  cvt.rni saturates and maps NaN to 0.
+__device__ __forceinline__ int quantize1(float x, float inv_scale, int zp, int lo, int hi) {
+  int q = __float2int_rn(__fmul_rn(x, inv_scale));
+  q = max(min(q, 1000000000), -1000000000) + zp;
+  return max(min(q, hi), lo);
+}
+__device__ __forceinline__ int act_lo(const q4_act& a) { return a.is_signed ? -(1 << (a.bits - 1)) : 0; }
+__device__ __forceinline__ int act_hi(const q4_act& a) {
+  return a.is_signed ? (1 << (a.bits - 1)) - 1 : (1 << a.bits) - 1;
+}
+
+__device__ __forceinline__ float sigmoidf_acc(float v) { return 1.0f / (1.0f + expf(-v)); }
+
+// ---- argument blocks of the tile kernels -------------------------------------------
+enum { EPI_I32 = 0, EPI_F32 = 1, EPI_QUANT = 2 };
+
+struct GemmArgs {
+  RowSrc x;                 // activation codes
+  int32_t x_signed, x_zp, M;
+  const uint8_t* w;         // weight codes [J, k_pad]
+  const float* w_scale;
+  const float* bias;
+  int32_t J, k_pad;
+  float x_scale;
+  void* out;                // EPI_I32: int32 [*, out_stride]; EPI_F32: float; EPI_QUANT: bytes
+  long long out_stride;     // elements (I32/F32) or bytes (QUANT) between output rows
+  const int32_t* out_idx;   // output row of x row m (nullptr = m; negative = skip)
+  int32_t* dbg_acc;         // optional raw accumulators [M, J]
+  q4_act out_act;           // EPI_QUANT
+};
+
+struct LstmArgs {
+  RowSrc x;                 // input codes (ignored when acc_pre is set)
+  int32_t x_signed, x_zp, kx_pad;
+  float x_scale;
+  const float* x_scale_vec; // optional per-row input scale, indexed n % x_scale_mod
+  int32_t x_scale_mod;
+  const int32_t* acc_pre;   // optional precomputed input accumulators, row n at n*acc_pre_stride
+  long long acc_pre_stride;
+  RowSrc hin;               // previous cell-output codes
+  const float* c_in;        // [*, H], indexed like hin
+  const uint8_t* w_ih;
+  const float* s_wih;
+  const uint8_t* w_hh;
+  const float* s_whh;
+  const float* bias;
+  int32_t H, N, kh_pad;
+  q4_act hid_act, out_act;
+  uint8_t* hq_out;          // recurrent codes, row stride hq_stride bytes, rows via out_idx
+  long long hq_stride;
+  const int32_t* out_idx;
+  float* c_out;             // [*, H] rows via out_idx
+  uint8_t* yq_out;          // optional second code (out_act), row n at n*yq_stride bytes
+  long long yq_stride;
+  float* h_f32;             // optional [N, H]
+  int32_t* dbg_ih;          // optional, row n at n*dbg_stride
+  int32_t* dbg_hh;
+  long long dbg_stride;
+};
+struct LstmArgs2 {
+  LstmArgs d[2];
+};
+
+}  // namespace q4

@@ -1,0 +1,209 @@
+"""GPU parity: qlstm_step (teacher-forced, every step fed the oracle's state) and
+qlstm_layer_forward / the encoder (free-running) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2206_07882_b200 import synth
+from _parity import assert_close, assert_codes_match, gpu_codes, near_tie, pack_codes, to_act
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def Bd():
+    from paper_2206_07882_b200 import binding
+    binding.lib()
+    return binding
+
+
+def step_case(Bd, lw, x_act, hid, xq, hq, c):
+    L = O.Lstm([lw])
+    want = O.lstm_step(L, xq, x_act, hq, c, hid)
+    dl = Bd.DeviceLstm(lw)
+    assert dl.hid_act.scale == hid.scale
+    got = Bd.qlstm_step(pack_codes(xq, x_act), to_act(x_act), pack_codes(hq, hid),
+                        torch.from_numpy(c).cuda(), dl, want_dbg=True)
+    H = c.shape[1]
+    np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), want["acc_ih"])     # bit-exact
+    np.testing.assert_array_equal(got["acc_hh"].cpu().numpy(), want["acc_hh"])
+    assert_close(got["c"].cpu().numpy(), want["c"], "cell state")
+    assert_close(got["h"].cpu().numpy(), want["h"], "cell output")
+    return assert_codes_match(gpu_codes(got["hq"], H, hid), want["hq"], want["h"], hid, "hq")
+
+
+def test_config0_teacher_forced_every_step(Bd):
+    # Single unidirectional INT4 layer: K=64, H=128, B=4, T=50, clip 3.0, seed 0.
+    w = synth.single_layer(seed=0)
+    lw = w["layers"][0]
+    x_act, hid = O.act_symmetric(w["x_clip"], 4), O.act_symmetric(1.0, 4)
+    xq = O.quantize(w["x"], x_act)
+    ref = O.lstm_layer(O.Lstm([lw]), xq, x_act, hid, want=("h", "hq_hid", "c_n"))
+    hq = np.zeros((4, 128), np.int16)
+    c = np.zeros((4, 128), np.float32)
+    ties = 0
+    L = O.Lstm([lw])
+    for t in range(50):
+        ties += step_case(Bd, lw, x_act, hid, xq[t], hq, c)
+        s = O.lstm_step(L, xq[t], x_act, hq, c, hid)          # oracle state feeds the next step
+        hq, c = s["hq"], s["c"]
+    np.testing.assert_array_equal(hq, ref["yq"][49])
+    assert ties <= 2
+
+
+@pytest.mark.parametrize("N,K,H,xb,hb,signed", [(70, 200, 96, 4, 4, True), (5, 32, 32, 4, 4, False),
+                                                 (130, 240, 64, 8, 8, True), (33, 256, 160, 4, 4, False),
+                                                 (64, 64, 32, 8, 4, True), (1, 1280, 640, 4, 4, True)])
+def test_step_shapes_and_formats(Bd, N, K, H, xb, hb, signed):
+    st = synth.Stream(100 + N)
+    lw = synth._lstm(st, "l", K, H, 4, bias_std=0.2, hid_bits=hb)
+    if xb == 8:
+        lw.w_ih = synth._qmat(st, "w8", 4 * H, K, 8)
+    if hb == 8:
+        lw.w_hh = synth._qmat(st, "h8", 4 * H, H, 8)
+    x_act = O.act_symmetric(3.0, xb) if signed else O.act_asymmetric(-1.7, 1.4, 4)
+    hid = O.act_symmetric(0.95, hb)
+    lo, hi = x_act.lo(), x_act.hi()
+    xq = st.integers("xq", (N, K), lo, hi).astype(np.int16)
+    hq = st.integers("hq", (N, H), -(1 << (hb - 1)) + 1, (1 << (hb - 1)) - 1).astype(np.int16)
+    c = st.normal("c", (N, H)).astype(np.float32)
+    step_case(Bd, lw, x_act, hid, xq, hq, c)
+
+
+def test_step_embedding_lookup(Bd):
+    st = synth.Stream(7)
+    V, E, H, N = 50, 32, 64, 20
+    lw = synth._lstm(st, "l", E, H, 4, bias_std=0.1)
+    emb = st.normal("emb", (V, E), 0, 0.5).astype(np.float32)
+    a = O.act_asymmetric(-1.2, 1.6, 4)
+    table = Bd.quantize_pack_int4(torch.from_numpy(emb).cuda(), to_act(a))
+    tok = st.integers("tok", (N,), 0, V - 1).astype(np.int32)
+    hid = O.act_symmetric(1.0, 4)
+    hq = st.integers("hq", (N, H), -7, 7).astype(np.int16)
+    c = st.normal("c", (N, H)).astype(np.float32)
+    got = Bd.qlstm_step(table, to_act(a), pack_codes(hq, hid), torch.from_numpy(c).cuda(),
+                        Bd.DeviceLstm(lw), x_row_idx=torch.from_numpy(tok).cuda(), want_dbg=True)
+    want = O.lstm_step(O.Lstm([lw]), O.quantize(emb[tok], a), a, hq, c, hid)
+    np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), want["acc_ih"])
+    assert_codes_match(gpu_codes(got["hq"], H, hid), want["hq"], want["h"], hid)
+
+
+def layer_case(Bd, T, B, K, H, dirs, xb=4, hb=4, ob=None, seed=0, x_clip=3.0, max_off=1e-4):
+    w = synth.single_layer(seed=seed, T=T, B=B, K=K, H=H, bits=4, dirs=dirs)
+    st = synth.Stream(seed + 77)
+    for d, lw in enumerate(w["layers"]):
+        lw.bias[:] = st.normal(f"b{d}", (4 * H,), 0, 0.1)
+        if xb == 8:
+            lw.w_ih = synth._qmat(st, f"w8{d}", 4 * H, K, 8)
+        if hb == 8:
+            lw.w_hh = synth._qmat(st, f"h8{d}", 4 * H, H, 8)
+        lw.hid_bits = hb
+    ob = ob or hb
+    x_act, hid, out = O.act_symmetric(x_clip, xb), O.act_symmetric(1.0, hb), O.act_symmetric(1.0, ob)
+    xq = O.quantize(w["x"], x_act)
+    ref = O.lstm_layer(O.Lstm(w["layers"]), xq, x_act, hid, out, want=("h", "hq_hid", "c_n", "acc_ih", "acc_hh"))
+    layers = [Bd.DeviceLstm(lw) for lw in w["layers"]]
+    got = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), x_act), to_act(x_act), T, B, layers,
+                                 to_act(out), want_state=True, want_dbg=True)
+    # input accumulators depend on the input only: bit-exact over the whole sequence
+    np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), ref["acc_ih"])
+    yq = gpu_codes(got["yq"], dirs * H, out).reshape(T, B, dirs * H)
+    diff = np.abs(yq.astype(np.int32) - ref["yq"])
+    # free-running: almost all codes identical, none off by more than one step
+    assert (diff > 1).mean() <= max_off, (diff > 1).mean()
+    assert (diff > 0).mean() <= 5e-3, (diff > 0).mean()
+    # recurrent accumulators are exact wherever the previous step's codes agreed
+    hh = got["acc_hh"].cpu().numpy()
+    for d in range(dirs):
+        order = list(range(T)) if d == 0 else list(range(T - 1, -1, -1))
+        ok = np.ones(B, bool)
+        for i, t in enumerate(order):
+            np.testing.assert_array_equal(hh[t, ok, d], ref["acc_hh"][t, ok, d])
+            if hb == ob:
+                ok &= (diff[t, :, d * H:(d + 1) * H] == 0).all(axis=1)
+            else:
+                break
+    c_n = got["c_n"].cpu().numpy()
+    clean = (diff == 0).all(axis=(0, 2))
+    if clean.any():
+        assert_close(c_n[:, clean], ref["c_n"][:, clean], "final cell state")
+        hqn = gpu_codes(got["hq_n"].reshape(dirs * B, -1), H, hid).reshape(dirs, B, H)
+        last = np.stack([ref["hq_hid"][T - 1, :, :H]] + ([ref["hq_hid"][0, :, H:]] if dirs == 2 else []))
+        assert (np.abs(hqn[:, clean] - last[:, clean]) <= 1).all()
+    return diff
+
+
+def test_config0_layer_forward(Bd):
+    diff = layer_case(Bd, T=50, B=4, K=64, H=128, dirs=1, seed=0)
+    assert (diff > 0).sum() <= 8
+
+
+@pytest.mark.parametrize("T,B,K,H,dirs,xb,hb,ob", [(9, 3, 48, 32, 2, 4, 4, 4), (20, 70, 240, 64, 2, 8, 8, 4),
+                                                   (12, 33, 128, 96, 1, 4, 4, 8), (7, 1, 1280, 160, 2, 4, 4, 4)])
+def test_layer_shapes_directions_precisions(Bd, T, B, K, H, dirs, xb, hb, ob):
+    layer_case(Bd, T, B, K, H, dirs, xb, hb, ob, seed=11)
+
+
+def test_layer_per_sequence_input_scale(Bd):
+    T, B, K, H = 8, 5, 64, 32
+    w = synth.single_layer(seed=5, T=T, B=B, K=K, H=H, bits=8, dirs=2)
+    base = O.act_symmetric(1.0, 8)
+    xq = np.empty((T, B, K), np.int16)
+    sc = np.empty(B, np.float32)
+    for b in range(B):
+        a = O.act_symmetric(O.absmax(w["x"][:, b]), 8)
+        xq[:, b] = O.quantize(w["x"][:, b], a)
+        sc[b] = a.scale
+    hid = O.act_symmetric(1.0, 8)
+    ref = O.lstm_layer(O.Lstm(w["layers"]), xq, base, hid, x_scale_b=sc)
+    for lw in w["layers"]:
+        lw.hid_bits = 8
+    got = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), base), to_act(base), T, B,
+                                 [Bd.DeviceLstm(lw) for lw in w["layers"]],
+                                 x_scale_b=torch.from_numpy(sc).cuda())
+    yq = gpu_codes(got["yq"], 2 * H, hid).reshape(T, B, 2 * H)
+    assert (np.abs(yq - ref["yq"]) > 1).mean() <= 1e-4
+    assert (yq != ref["yq"]).mean() <= 1e-2
+
+
+def encoder_case(Bd, enc_w, feats, utts=None):
+    E = enc_w["enc"]
+    T, B, F = feats.shape
+    dev = Bd.Encoder(E)
+    got = dev.forward(torch.from_numpy(feats).cuda(), want_layers=True)
+    sel = list(range(B)) if utts is None else utts
+    ref = O.encoder_forward(E, feats[:, sel, :], want_layers=True)
+    H2 = 2 * enc_w["H"]
+    worst = 0.0
+    for l, yq in enumerate(got["layers"]):
+        a = dev.out_acts[l]
+        g = gpu_codes(yq, H2, a).reshape(T, B, H2)[:, sel]
+        d = np.abs(g.astype(np.int32) - ref["layers"][l]["yq"])
+        worst = max(worst, float((d > 1).mean()))
+        assert (d > 1).mean() <= 1e-4, (l, (d > 1).mean())
+    e = got["e"].cpu().numpy()[:, sel]
+    # projected frames: compare where the last layer's codes agree exactly (else the
+    # difference is one quantization step times a weight, not an arithmetic error)
+    g = gpu_codes(got["yq"], H2, dev.out_acts[-1]).reshape(T, B, H2)[:, sel]
+    same = (g == ref["yq"]).all(axis=2)
+    assert same.mean() > 0.5
+    assert_close(e[same], ref["e"][same], "encoder projection")
+    return worst
+
+
+def test_encoder_reduced(Bd):
+    enc = synth.encoder(seed=1, T=40, B=6, F=48, H=64, L=3, D=32)
+    encoder_case(Bd, enc, enc["features"])
+
+
+def test_encoder_reduced_int8_first_layer_max_input(Bd):
+    enc = synth.encoder(seed=2, T=30, B=5, F=80, H=32, L=3, D=32, first_layer_bits=8, in_max=True)
+    encoder_case(Bd, enc, enc["features"])
+
+
+def test_config1_full_size_sampled_utterances(Bd):
+    # 6-layer bidirectional encoder, 640 cells/direction, 240-dim input, T=500, B=32; the
+    # oracle recomputes two of the 32 utterances (they are independent).
+    enc = synth.encoder(seed=1)
+    encoder_case(Bd, enc, enc["features"], utts=[3, 28])

@@ -1,0 +1,85 @@
+"""GPU parity: quantize_pack_int4 and the feature prologue against the oracle (bit-exact:
+the quantizer is defined in fp32 on both sides)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2206_07882_b200 import synth
+from _parity import gpu_codes, to_act
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def Bd():
+    from paper_2206_07882_b200 import binding
+    binding.lib()
+    return binding
+
+
+CASES = [("sym4", lambda: O.act_symmetric(3.0, 4)), ("sym8", lambda: O.act_symmetric(2.7, 8)),
+         ("asym4", lambda: O.act_asymmetric(-2.5, 3.5, 4)), ("pred", lambda: O.act_symmetric(1.25, 4))]
+
+
+@pytest.mark.parametrize("name,mk", CASES)
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("rows,k", [(1, 32), (7, 45), (200, 240), (1000, 1280), (0, 64)])
+def test_fixed_boundary(Bd, name, mk, dtype, rows, k):
+    a = mk()
+    x = synth.Stream(3).normal(f"x{rows}.{k}", (rows, k), 0.0, 1.5).astype(dtype)
+    if rows:
+        x[0, :min(k, 6)] = np.array([0.0, a.scale * 0.5, -a.scale * 1.5, 100.0, -100.0, a.scale * 2.5], dtype)[:min(k, 6)]
+    got = Bd.quantize_pack_int4(torch.from_numpy(x).cuda(), to_act(a))
+    k_pad = Bd.pad32(k)
+    assert got.shape == (rows, k_pad * a.bits // 8)
+    if rows == 0:
+        return
+    want = O.quantize(x.astype(np.float32), a)
+    np.testing.assert_array_equal(gpu_codes(got, k, a), want)
+    # padding holds the code of the real value 0
+    if k_pad > k:
+        full = gpu_codes(got, k_pad, a)
+        assert (full[:, k:] == (0 if a.is_signed else a.zero_point)).all()
+    # byte-identical to the oracle's storage format
+    if a.bits == 4:
+        np.testing.assert_array_equal(got.cpu().numpy(), O.pack4(want, k_pad, 0 if a.is_signed else a.zero_point))
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("T,B,F", [(6, 3, 40), (50, 8, 240)])
+def test_max_boundary_per_utterance(Bd, bits, T, B, F):
+    x = synth.Stream(4).normal("feat", (T, B, F)).astype(np.float16)
+    x[:, 1, :] = 0                                     # an all-zero utterance: boundary 1
+    base = Bd.q4_act_symmetric(1.0, bits)
+    got, scales = Bd.quantize_pack_int4(torch.from_numpy(x).cuda().reshape(T * B, F), base, mode=1, n_groups=B)
+    codes = gpu_codes(got, F, base).reshape(T, B, F)
+    for b in range(B):
+        a = O.act_symmetric(O.absmax(x[:, b, :].astype(np.float32)), bits)
+        assert scales[b].item() == a.scale
+        np.testing.assert_array_equal(codes[:, b, :], O.quantize(x[:, b, :].astype(np.float32), a))
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_weight_mode_per_row_scale(Bd, bits):
+    st = synth.Stream(5)
+    rows, k = 130, 200
+    w = st.normal("w", (rows, k), 0.0, 0.1).astype(np.float32)
+    s = st.uniform("s", (rows,), 0.01, 0.05).astype(np.float32)
+    m = Bd.DeviceMat.from_float(w, s, bits)
+    a = O.act_symmetric(1.0, bits)
+    np.testing.assert_array_equal(gpu_codes(m.q, k, a), O.quantize_weights(w, s, bits))
+    # integer codes handed over as floats come back exactly
+    q = st.integers("q", (rows, k), -(1 << (bits - 1)), (1 << (bits - 1)) - 1).astype(np.int8)
+    m2 = Bd.DeviceMat.from_codes(q, s, bits)
+    np.testing.assert_array_equal(gpu_codes(m2.q, k, a), q)
+
+
+@pytest.mark.parametrize("B,T100,M", [(1, 4, 1), (3, 20, 40), (2, 1000, 40), (2, 7, 5)])
+def test_feature_prologue(Bd, B, T100, M):
+    mel = synth.logmel(9, B, T100, M)
+    got = Bd.q4_feature_prologue(torch.from_numpy(mel).cuda()).cpu().numpy()
+    assert got.shape == (T100 // 2, B, 6 * M) and got.dtype == np.float16
+    for b in range(B):
+        want = O.features(mel[b]).astype(np.float16)
+        np.testing.assert_array_equal(got[:, b, :], want)

@@ -227,3 +227,27 @@ def test_features_prologue_by_hand():
     dd = np.array([(d[1] - d[0]) / 2, (d[2] - d[0]) / 2, (d[3] - d[1]) / 2, (d[3] - d[2]) / 2])
     want = np.array([[1, d[0], dd[0], 4, d[1], dd[1]], [9, d[2], dd[2], 16, d[3], dd[3]]])
     np.testing.assert_allclose(out, want, atol=1e-6)
+
+
+def test_fp32_activation_functions_against_libm():
+    # The gate non-linearities are fixed fp32 operation sequences (so that codes are
+    # reproducible); here they are pinned to the real functions evaluated in double.
+    x = np.concatenate([np.linspace(-30, 30, 400001), np.linspace(-1e-3, 1e-3, 2001),
+                        np.array([-1e4, -90.0, 90.0, 1e4, 0.0])]).astype(np.float32)
+    ex, sg, th = O.activations(x)
+    xd = x.astype(np.float64)
+    inr = np.abs(xd) <= 30
+    assert np.max(np.abs(ex[inr] / np.exp(xd[inr]) - 1)) < 2e-7
+    assert np.max(np.abs(sg - 1 / (1 + np.exp(-np.clip(xd, -700, 700))))) < 2e-7
+    assert np.max(np.abs(th - np.tanh(xd))) < 2e-7
+    assert (sg >= 0).all() and (sg <= 1).all() and (np.abs(th) <= 1).all()
+    assert th[-1] == 0.0 and sg[-1] == 0.5 and ex[-1] == 1.0
+    # monotone where it matters for quantization: no inversions on a fine grid
+    g = np.linspace(-12, 12, 200001).astype(np.float32)
+    _, sg, th = O.activations(g)
+    assert (np.diff(sg) >= -1.2e-7).all() and (np.diff(th) >= -1.2e-7).all()
+    # odd symmetry of tanh, and sigmoid(x) + sigmoid(-x) = 1 within rounding
+    _, s1, t1 = O.activations(g)
+    _, s2, t2 = O.activations(-g)
+    np.testing.assert_array_equal(t1, -t2)
+    assert np.max(np.abs(s1 + s2 - 1)) < 2e-7
