@@ -81,7 +81,38 @@ __device__ __forceinline__ int act_hi(const q4_act& a) {
   return a.is_signed ? (1 << (a.bits - 1)) - 1 : (1 << a.bits) - 1;
 }
 
-__device__ __forceinline__ float sigmoidf_acc(float v) { return 1.0f / (1.0f + expf(-v)); }
+// Gate non-linearities as a fixed sequence of IEEE fp32 operations (round-to-nearest
+// multiply / fused multiply-add / divide), so that the code a cell output quantizes to does
+// not depend on a math library:
+//   exp(x), x clamped to [-86, 88]: n = rne(x * log2 e); r = x - n ln2 with ln2 split in two
+//   constants; 7th-degree Taylor polynomial in r (Horner); times 2^n via the exponent field.
+__device__ __forceinline__ float exp_fixed(float x) {
+  x = fminf(fmaxf(x, -86.0f), 88.0f);
+  const float n = rintf(__fmul_rn(x, 1.44269502162933349609375f));
+  float r = __fmaf_rn(n, -0.693145751953125f, x);
+  r = __fmaf_rn(n, -1.428606765330187045037746429443359375e-6f, r);
+  float p = 1.98412701138295233249664306640625e-4f;
+  p = __fmaf_rn(p, r, 1.388888922519981861114501953125e-3f);
+  p = __fmaf_rn(p, r, 8.3333335816860198974609375e-3f);
+  p = __fmaf_rn(p, r, 4.1666667908430099487304687500e-2f);
+  p = __fmaf_rn(p, r, 0.16666667163372039794921875f);
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  return __uint_as_float(__float_as_uint(p) + ((uint32_t)(int)n << 23));
+}
+//   sigmoid(x) = 1 / (1 + exp(-x)), x clamped to [-86, 86]
+__device__ __forceinline__ float sigmoid_fixed(float x) {
+  x = fminf(fmaxf(x, -86.0f), 86.0f);
+  return __fdiv_rn(1.0f, __fadd_rn(1.0f, exp_fixed(-x)));
+}
+//   tanh(x) = sign(x) (1 - e) / (1 + e), e = exp(-2 min(|x|, 43))
+__device__ __forceinline__ float tanh_fixed(float x) {
+  const float a = fminf(fabsf(x), 43.0f);
+  const float e = exp_fixed(__fmul_rn(-2.0f, a));
+  const float t = __fdiv_rn(__fsub_rn(1.0f, e), __fadd_rn(1.0f, e));
+  return copysignf(t, x);
+}
 
 // ---- argument blocks of the tile kernels -------------------------------------------
 enum { EPI_I32 = 0, EPI_F32 = 1, EPI_QUANT = 2 };

@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(NT) k_gemm(const __grid_constant__ GemmArgs a)
       for (int j = 0; j < 4; ++j) {
         const int jj = min(jb + j, a.J - 1);
         const float b = a.bias ? a.bias[jj] : 0.0f;
-        v[j] = fmaf((float)acc[i][j], a.x_scale * a.w_scale[jj], b);
+        v[j] = __fmaf_rn((float)acc[i][j], __fmul_rn(a.x_scale, a.w_scale[jj]), b);
       }
       if (EPI == EPI_F32) {
         float* out = reinterpret_cast<float*>(a.out) + (long long)o * a.out_stride;
@@ -274,7 +274,7 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
       for (int g = 0; g < 4; ++g) {
         const int j = g * H + min(cell0 + cc, H - 1);
         const float b = a.bias ? a.bias[j] : 0.0f;
-        pre[r][cc][g] = fmaf((float)acc[r][cc][g], sx * a.s_wih[j], b);
+        pre[r][cc][g] = __fmaf_rn((float)acc[r][cc][g], __fmul_rn(sx, a.s_wih[j]), b);
         if (ok && a.dbg_ih && cell0 + cc < H) a.dbg_ih[(long long)n * a.dbg_stride + j] = acc[r][cc][g];
         acc[r][cc][g] = 0;
       }
@@ -317,13 +317,13 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
       for (int g = 0; g < 4; ++g) {
         const int j = g * H + cell;
         if (a.dbg_hh) a.dbg_hh[(long long)n * a.dbg_stride + j] = acc[r][cc][g];
-        g4[g] = fmaf((float)acc[r][cc][g], sh * a.s_whh[j], pre[r][cc][g]);
+        g4[g] = __fmaf_rn((float)acc[r][cc][g], __fmul_rn(sh, a.s_whh[j]), pre[r][cc][g]);
       }
-      const float ig = sigmoidf_acc(g4[0]), fg = sigmoidf_acc(g4[1]);
-      const float gg = tanhf(g4[2]), og = sigmoidf_acc(g4[3]);
+      const float ig = sigmoid_fixed(g4[0]), fg = sigmoid_fixed(g4[1]);
+      const float gg = tanh_fixed(g4[2]), og = sigmoid_fixed(g4[3]);
       const float cprev = hi >= 0 ? a.c_in[(long long)hi * H + cell] : 0.0f;
-      const float c = fmaf(fg, cprev, ig * gg);
-      const float h = og * tanhf(c);
+      const float c = __fmaf_rn(fg, cprev, __fmul_rn(ig, gg));
+      const float h = __fmul_rn(og, tanh_fixed(c));
       a.c_out[(long long)oi * H + cell] = c;
       if (a.h_f32) a.h_f32[(long long)n * H + cell] = h;
       q[cc] = quantize1(h, a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
@@ -435,8 +435,8 @@ __global__ void __launch_bounds__(256) k_joint_z(const float* e, const int32_t* 
     const float2 ev = *reinterpret_cast<const float2*>(e + (long long)er * D + d);
     const float2 pv = *reinterpret_cast<const float2*>(p + (long long)pr * D + d);
     const int lo = act_lo(za), hi = act_hi(za);
-    q0 = quantize1(tanhf(ev.x * pv.x), za.inv_scale, za.zero_point, lo, hi);
-    q1 = quantize1(tanhf(ev.y * pv.y), za.inv_scale, za.zero_point, lo, hi);
+    q0 = quantize1(tanh_fixed(__fmul_rn(ev.x, pv.x)), za.inv_scale, za.zero_point, lo, hi);
+    q1 = quantize1(tanh_fixed(__fmul_rn(ev.y, pv.y)), za.inv_scale, za.zero_point, lo, hi);
   }
   if (za.bits == 4) {
     zq[(long long)n * half + (d >> 1)] = (uint8_t)((q0 & 0xF) | ((q1 & 0xF) << 4));

@@ -1,0 +1,235 @@
+"""GPU parity: qjoint_logprobs, the prediction/joint path of config 2 and the fused beam
+search (dr_fusion_beam_step) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2206_07882_b200 import synth
+from _parity import gpu_codes, pack_codes, to_act
+
+pytestmark = pytest.mark.gpu
+
+LP_ATOL = 1e-5     # log-softmax: fp32 reduction on the GPU vs double in the oracle, |lp| <= ~20
+
+
+@pytest.fixture(scope="module")
+def Bd():
+    from paper_2206_07882_b200 import binding
+    binding.lib()
+    return binding
+
+
+@pytest.mark.parametrize("N,V,D,Hp,zb", [(5, 64, 32, 64, 4), (70, 1024, 256, 1024, 4), (33, 200, 64, 96, 8)])
+def test_joint_logprobs(Bd, N, V, D, Hp, zb):
+    dw = synth.decoder(seed=5, V=V, E=32, Hp=Hp, D=D, Hs=32, Ht=32, out_bits=zb)
+    dec = O.Decoder(dw)
+    st = synth.Stream(9)
+    R = 40
+    e = st.normal("e", (R, D)).astype(np.float32)
+    fi = st.integers("fi", (N,), 0, R - 1).astype(np.int32)
+    hid = O.act_symmetric(1.0, 4)
+    pq = st.integers("pq", (N, Hp), -7, 7).astype(np.int16)
+    p = O.linear(O.Linear(dw.pred.proj), pq, hid)
+    want = O.joint(dec, e[fi], p)
+    dd = Bd.Decoder(dw)
+    got = Bd.qjoint_logprobs(torch.from_numpy(e).cuda(), torch.from_numpy(fi).cuda(), pack_codes(pq, hid),
+                             to_act(hid), dd.pred_proj, dd.z_act, dd.joint_out).cpu().numpy()
+    assert np.abs(got - want).max() <= LP_ATOL
+    np.testing.assert_allclose(np.exp(got.astype(np.float64)).sum(1), 1.0, atol=1e-5)
+
+
+def pred_joint_gpu(Bd, dd, e_dev, frame_idx, tokens):
+    """Teacher-forced prediction network + joint on the GPU: logp [N,S,V], hq codes [N,S,Hp]."""
+    N, S = tokens.shape
+    Hp, V = dd.pred_lstm.H, dd.V
+    hq = torch.zeros((N, Hp // 2), dtype=torch.uint8, device="cuda")
+    c = torch.zeros((N, Hp), dtype=torch.float32, device="cuda")
+    tok = torch.from_numpy(tokens).cuda()
+    fi = torch.from_numpy(frame_idx).cuda()
+    out = torch.empty((N, S, V), dtype=torch.float32, device="cuda")
+    hqs = []
+    for s in range(S):
+        r = Bd.qlstm_step(dd.pred_emb_q, dd.pred_emb_act, hq, c, dd.pred_lstm,
+                          x_row_idx=tok[:, s].contiguous())
+        hq, c = r["hq"], r["c"]
+        out[:, s] = Bd.qjoint_logprobs(e_dev, fi[:, s].contiguous(), hq, dd.pred_lstm.hid_act,
+                                       dd.pred_proj, dd.z_act, dd.joint_out)
+        hqs.append(hq)
+    return out, torch.stack(hqs, dim=1)
+
+
+def test_config2_reduced_all_rows(Bd):
+    dw = synth.decoder(seed=2, V=64, E=32, Hp=64, D=32, Hs=32, Ht=32)
+    N, S, T, B = 48, 20, 20, 3
+    encq_act = O.act_symmetric(1.0, 4)
+    frames = synth.enc_frames(2, T, B, 64)
+    proj = synth._linear(synth.Stream(2), "enc.proj", 32, 64)
+    e = O.linear(O.Linear(proj), O.quantize(frames.astype(np.float32).reshape(T * B, 64), encq_act), encq_act)
+    toks = np.concatenate([np.zeros((N, 1), np.int32), synth.labels(2, N, S - 1, 64)], axis=1)
+    fi = (np.arange(S, dtype=np.int32)[None, :] * B + (np.arange(N, dtype=np.int32)[:, None] % B)).astype(np.int32)
+    want, hq_w, c_w, p_w = O.pred_joint_forced(O.Decoder(dw), e, fi, toks, want_state=True)
+    dd = Bd.Decoder(dw)
+    got, hq_g = pred_joint_gpu(Bd, dd, torch.from_numpy(e).cuda(), fi, toks)
+    np.testing.assert_array_equal(gpu_codes(hq_g.reshape(N * S, -1), 64, encq_act).reshape(N, S, 64), hq_w)
+    assert np.abs(got.cpu().numpy() - want).max() <= LP_ATOL
+
+
+def test_config2_full_size_sampled_rows(Bd):
+    # 256 hypothesis rows x 300 steps; vocabulary 1024, embedding 256, prediction LSTM 1024,
+    # joint 1280 -> 256 -> 1024.  The oracle recomputes 3 of the 256 rows (rows are independent).
+    dw = synth.decoder(seed=2)
+    B, W, T, S = 16, 16, 300, 300
+    N = B * W
+    act = O.act_symmetric(1.0, 4)
+    frames = synth.enc_frames(2, T, B, 1280)
+    proj = synth._linear(synth.Stream(2), "enc.proj", 256, 1280)
+    dproj = Bd.DeviceLinear(proj)
+    fq = Bd.quantize_pack_int4(torch.from_numpy(frames).cuda().reshape(T * B, 1280), to_act(act))
+    e_dev = Bd.q4_linear_forward(fq, to_act(act), dproj)
+    toks = np.concatenate([np.zeros((N, 1), np.int32), synth.labels(2, N, S - 1, 1024)], axis=1)
+    fi = (np.arange(S, dtype=np.int32)[None, :] * B + (np.arange(N, dtype=np.int32)[:, None] // W)).astype(np.int32)
+    dd = Bd.Decoder(dw)
+    got, hq_g = pred_joint_gpu(Bd, dd, e_dev, fi, toks)
+    rows = [0, 117, 255]
+    e = e_dev.cpu().numpy()
+    # the projected frames themselves: bit-exact against the oracle on the frames those rows use
+    used = np.unique(fi[rows])
+    e_ref = O.linear(O.Linear(proj), O.quantize(frames.astype(np.float32).reshape(T * B, 1280)[used], act), act)
+    np.testing.assert_array_equal(e[used], e_ref)
+    want, hq_w, _, _ = O.pred_joint_forced(O.Decoder(dw), e, fi[rows], toks[rows], want_state=True)
+    np.testing.assert_array_equal(gpu_codes(hq_g[rows].reshape(len(rows) * S, -1), 1024, act).reshape(len(rows), S, 1024), hq_w)
+    assert np.abs(got[rows].cpu().numpy() - want).max() <= LP_ATOL
+
+
+def run_search(Bd, dw, e, utts=None):
+    dd = Bd.Decoder(dw)
+    T, B, D = e.shape
+    tokens, lens, scores = dd.decode(torch.from_numpy(e).cuda())
+    torch.cuda.synchronize()
+    assert dd.tensors["status"].item() == 0
+    ref = O.alsd(O.Decoder(dw), e, utts=utts)
+    return dd, tokens.cpu().numpy(), lens.cpu().numpy(), scores.cpu().numpy(), ref
+
+
+def compare_search(dd, tokens, lens, scores, ref, utts, T, U, W, min_same=0.99):
+    IT = T + U
+    bp_parent = dd.tensors["bp_parent"].cpu().numpy()[:IT]
+    bp_token = dd.tensors["bp_token"].cpu().numpy()[:IT]
+    bp_score = dd.tensors["bp_score"].cpu().numpy()[:IT]
+    same_top = 0
+    same_trace = 0
+    for i, b in enumerate(utts):
+        n = int(ref["len"][i])
+        top_ok = lens[b] == n and (tokens[b, :n] == ref["tokens"][i, :n]).all()
+        same_top += bool(top_ok)
+        if top_ok:
+            assert abs(scores[b] - ref["score"][i]) <= 1e-3
+        # whole trajectory: every iteration's beam (parent, token) and scores
+        tr_ok = True
+        for it in range(IT):
+            ns = int(ref["n_slots"][i, it])
+            gp, gt = bp_parent[it, b], bp_token[it, b]
+            if (gp >= 0).sum() != ns or (gp[:ns] != ref["parent"][i, it, :ns]).any() or \
+                    (gt[:ns] != ref["token"][i, it, :ns]).any():
+                tr_ok = False
+                break
+            assert np.abs(bp_score[it, b, :ns] - ref["tscore"][i, it, :ns]).max() <= 1e-3
+        same_trace += tr_ok
+    frac = same_top / len(utts)
+    assert frac >= min_same, f"top hypothesis identical on {frac:.3f} of utterances"
+    return frac, same_trace / len(utts)
+
+
+def test_search_tiny_unpruned_equals_oracle(Bd):
+    # V=32, beam 16 over a tiny net: exercises merging, finished list, empty beams
+    dw = synth.decoder(seed=31, V=32, E=32, Hp=32, D=32, Hs=32, Ht=32, tgt_layers=2, U_max=3, W=16)
+    e = synth.Stream(4).normal("e", (4, 5, 32)).astype(np.float32)
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e)
+    frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(5)), 4, 3, 16, min_same=1.0)
+    assert tr == 1.0
+    fin_n = dd.tensors["fin_n"].cpu().numpy()
+    np.testing.assert_array_equal(fin_n, ref["finals_n"])
+    fs = dd.tensors["fin_score"].cpu().numpy()
+    for b in range(5):
+        assert np.abs(fs[b, :fin_n[b]] - ref["finals_score"][b, :fin_n[b]]).max() <= 1e-3
+
+
+@pytest.mark.parametrize("W", [1, 4, 16])
+def test_search_beam_widths(Bd, W):
+    dw = synth.decoder(seed=41, V=64, E=32, Hp=64, D=32, Hs=32, Ht=64, tgt_layers=2, U_max=8, W=W)
+    e = synth.Stream(5).normal("e", (16, 8, 32)).astype(np.float32)
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e)
+    compare_search(dd, tokens, lens, scores, ref, list(range(8)), 16, 8, W, min_same=1.0)
+
+
+def test_search_parity_suite_256_utterances(Bd):
+    # reduced-dimension end-to-end suite: encoder on the GPU, then the fused search; the
+    # top hypothesis must be identical on >= 99 % of the utterances.
+    enc_w, dw = synth.parity_suite()
+    T, B = enc_w["T"], enc_w["B"]
+    got_enc = Bd.Encoder(enc_w["enc"]).forward(torch.from_numpy(enc_w["features"]).cuda())
+    e_ref = O.encoder_forward(enc_w["enc"], enc_w["features"])["e"]
+    np.testing.assert_array_equal(got_enc["e"].cpu().numpy(), e_ref)
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e_ref)
+    frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(B)), T, dw.U_max, dw.W)
+    print(f"parity suite: top identical {frac:.4f}, whole trajectory identical {tr:.4f}")
+    assert tr >= 0.95
+
+
+def config3_inputs(Bd, T, B):
+    act = O.act_symmetric(1.0, 4)
+    frames = synth.enc_frames(3, T, B, 1280)
+    proj = synth._linear(synth.Stream(3), "enc.proj", 256, 1280)
+    fq = Bd.quantize_pack_int4(torch.from_numpy(frames).cuda().reshape(T * B, 1280), to_act(act))
+    return Bd.q4_linear_forward(fq, to_act(act), Bd.DeviceLinear(proj)).reshape(T, B, 256)
+
+
+def test_config3_full_size_sampled_utterances(Bd):
+    # beam 16, 16 utterances, target LM 2x2048, source LM 1024, vocabulary 1024: the launch
+    # shapes of the full workload (256 hypothesis rows).  The oracle decodes 2 of the 16
+    # utterances over the first 24 frames with a label budget of 8 (about a minute of CPU);
+    # the GPU runs exactly that setting on all 16.
+    dw = synth.decoder(seed=3, U_max=8)
+    T, B = 24, 16
+    e = config3_inputs(Bd, 300, B)[:T].contiguous().cpu().numpy()
+    utts = [1, 14]
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e, utts=utts)
+    compare_search(dd, tokens, lens, scores, ref, utts, T, 8, 16, min_same=1.0)
+
+
+def test_config3_full_length_invariants(Bd):
+    # T=300, U_max=150 (450 iterations): properties that hold at any size.
+    dw = synth.decoder(seed=3, U_max=150)
+    T, B, W, U = 300, 16, 16, 150
+    e = config3_inputs(Bd, T, B)
+    dd = Bd.Decoder(dw)
+    tokens, lens, scores = dd.decode(e)
+    torch.cuda.synchronize()
+    assert dd.tensors["status"].item() == 0
+    IT = T + U
+    par = dd.tensors["bp_parent"].cpu().numpy()[:IT]
+    tok = dd.tensors["bp_token"].cpu().numpy()[:IT]
+    sc = dd.tensors["bp_score"].cpu().numpy()[:IT]
+    for b in range(B):
+        t = np.zeros(1, np.int64)
+        u = np.zeros(1, np.int64)
+        strings = [()]
+        for it in range(IT):
+            n = int((par[it, b] >= 0).sum())
+            assert (par[it, b, :n] >= 0).all() and (par[it, b, n:] < 0).all()     # slots are packed
+            assert (np.diff(sc[it, b, :n]) <= 0).all()                            # rank order
+            p, k = par[it, b, :n], tok[it, b, :n]
+            assert (p < len(strings)).all() and (k >= 0).all() and (k < 1024).all()
+            t, u = t[p] + (k == 0), u[p] + (k > 0)
+            assert ((t + u) == it + 1).all() and (t < T).all() and (u <= U).all()
+            strings = [strings[pp] + ((int(kk),) if kk > 0 else ()) for pp, kk in zip(p, k)]
+            assert len(set(strings)) == n                                         # merged: distinct
+    fin_n = dd.tensors["fin_n"].cpu().numpy()
+    fs = dd.tensors["fin_score"].cpu().numpy()
+    lens_h, tok_h, sc_h = lens.cpu().numpy(), tokens.cpu().numpy(), scores.cpu().numpy()
+    for b in range(B):
+        assert 1 <= fin_n[b] <= W
+        assert (np.diff(fs[b, :fin_n[b]]) <= 0).all()
+        assert sc_h[b] == fs[b, 0] and 0 <= lens_h[b] <= U
+        assert (tok_h[b, :lens_h[b]] > 0).all() and (tok_h[b, lens_h[b]:] == 0).all()

@@ -28,9 +28,11 @@ def step_case(Bd, lw, x_act, hid, xq, hq, c):
     H = c.shape[1]
     np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), want["acc_ih"])     # bit-exact
     np.testing.assert_array_equal(got["acc_hh"].cpu().numpy(), want["acc_hh"])
-    assert_close(got["c"].cpu().numpy(), want["c"], "cell state")
-    assert_close(got["h"].cpu().numpy(), want["h"], "cell output")
-    return assert_codes_match(gpu_codes(got["hq"], H, hid), want["hq"], want["h"], hid, "hq")
+    # the float stages are a fixed fp32 operation sequence on both sides: bit-exact
+    np.testing.assert_array_equal(got["c"].cpu().numpy(), want["c"])
+    np.testing.assert_array_equal(got["h"].cpu().numpy(), want["h"])
+    np.testing.assert_array_equal(gpu_codes(got["hq"], H, hid), want["hq"])
+    return 0
 
 
 def test_config0_teacher_forced_every_step(Bd):
@@ -49,7 +51,7 @@ def test_config0_teacher_forced_every_step(Bd):
         s = O.lstm_step(L, xq[t], x_act, hq, c, hid)          # oracle state feeds the next step
         hq, c = s["hq"], s["c"]
     np.testing.assert_array_equal(hq, ref["yq"][49])
-    assert ties <= 2
+    assert ties == 0
 
 
 @pytest.mark.parametrize("N,K,H,xb,hb,signed", [(70, 200, 96, 4, 4, True), (5, 32, 32, 4, 4, False),
@@ -86,7 +88,7 @@ def test_step_embedding_lookup(Bd):
                         Bd.DeviceLstm(lw), x_row_idx=torch.from_numpy(tok).cuda(), want_dbg=True)
     want = O.lstm_step(O.Lstm([lw]), O.quantize(emb[tok], a), a, hq, c, hid)
     np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), want["acc_ih"])
-    assert_codes_match(gpu_codes(got["hq"], H, hid), want["hq"], want["h"], hid)
+    np.testing.assert_array_equal(gpu_codes(got["hq"], H, hid), want["hq"])
 
 
 def layer_case(Bd, T, B, K, H, dirs, xb=4, hb=4, ob=None, seed=0, x_clip=3.0, max_off=1e-4):
@@ -109,34 +111,19 @@ def layer_case(Bd, T, B, K, H, dirs, xb=4, hb=4, ob=None, seed=0, x_clip=3.0, ma
     # input accumulators depend on the input only: bit-exact over the whole sequence
     np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), ref["acc_ih"])
     yq = gpu_codes(got["yq"], dirs * H, out).reshape(T, B, dirs * H)
-    diff = np.abs(yq.astype(np.int32) - ref["yq"])
-    # free-running: almost all codes identical, none off by more than one step
-    assert (diff > 1).mean() <= max_off, (diff > 1).mean()
-    assert (diff > 0).mean() <= 5e-3, (diff > 0).mean()
-    # recurrent accumulators are exact wherever the previous step's codes agreed
-    hh = got["acc_hh"].cpu().numpy()
-    for d in range(dirs):
-        order = list(range(T)) if d == 0 else list(range(T - 1, -1, -1))
-        ok = np.ones(B, bool)
-        for i, t in enumerate(order):
-            np.testing.assert_array_equal(hh[t, ok, d], ref["acc_hh"][t, ok, d])
-            if hb == ob:
-                ok &= (diff[t, :, d * H:(d + 1) * H] == 0).all(axis=1)
-            else:
-                break
-    c_n = got["c_n"].cpu().numpy()
-    clean = (diff == 0).all(axis=(0, 2))
-    if clean.any():
-        assert_close(c_n[:, clean], ref["c_n"][:, clean], "final cell state")
-        hqn = gpu_codes(got["hq_n"].reshape(dirs * B, -1), H, hid).reshape(dirs, B, H)
-        last = np.stack([ref["hq_hid"][T - 1, :, :H]] + ([ref["hq_hid"][0, :, H:]] if dirs == 2 else []))
-        assert (np.abs(hqn[:, clean] - last[:, clean]) <= 1).all()
-    return diff
+    # free-running over the whole sequence and still bit-exact: codes, accumulators, states
+    np.testing.assert_array_equal(yq, ref["yq"])
+    np.testing.assert_array_equal(got["acc_hh"].cpu().numpy(), ref["acc_hh"])
+    np.testing.assert_array_equal(got["c_n"].cpu().numpy(), ref["c_n"])
+    hqn = gpu_codes(got["hq_n"].reshape(dirs * B, -1), H, hid).reshape(dirs, B, H)
+    last = np.stack([ref["hq_hid"][T - 1, :, :H]] + ([ref["hq_hid"][0, :, H:]] if dirs == 2 else []))
+    np.testing.assert_array_equal(hqn, last)
+    return np.abs(yq.astype(np.int32) - ref["yq"])
 
 
 def test_config0_layer_forward(Bd):
     diff = layer_case(Bd, T=50, B=4, K=64, H=128, dirs=1, seed=0)
-    assert (diff > 0).sum() <= 8
+    assert (diff > 0).sum() == 0
 
 
 @pytest.mark.parametrize("T,B,K,H,dirs,xb,hb,ob", [(9, 3, 48, 32, 2, 4, 4, 4), (20, 70, 240, 64, 2, 8, 8, 4),
@@ -163,8 +150,7 @@ def test_layer_per_sequence_input_scale(Bd):
                                  [Bd.DeviceLstm(lw) for lw in w["layers"]],
                                  x_scale_b=torch.from_numpy(sc).cuda())
     yq = gpu_codes(got["yq"], 2 * H, hid).reshape(T, B, 2 * H)
-    assert (np.abs(yq - ref["yq"]) > 1).mean() <= 1e-4
-    assert (yq != ref["yq"]).mean() <= 1e-2
+    np.testing.assert_array_equal(yq, ref["yq"])
 
 
 def encoder_case(Bd, enc_w, feats, utts=None):
@@ -175,21 +161,12 @@ def encoder_case(Bd, enc_w, feats, utts=None):
     sel = list(range(B)) if utts is None else utts
     ref = O.encoder_forward(E, feats[:, sel, :], want_layers=True)
     H2 = 2 * enc_w["H"]
-    worst = 0.0
     for l, yq in enumerate(got["layers"]):
         a = dev.out_acts[l]
         g = gpu_codes(yq, H2, a).reshape(T, B, H2)[:, sel]
-        d = np.abs(g.astype(np.int32) - ref["layers"][l]["yq"])
-        worst = max(worst, float((d > 1).mean()))
-        assert (d > 1).mean() <= 1e-4, (l, (d > 1).mean())
-    e = got["e"].cpu().numpy()[:, sel]
-    # projected frames: compare where the last layer's codes agree exactly (else the
-    # difference is one quantization step times a weight, not an arithmetic error)
-    g = gpu_codes(got["yq"], H2, dev.out_acts[-1]).reshape(T, B, H2)[:, sel]
-    same = (g == ref["yq"]).all(axis=2)
-    assert same.mean() > 0.5
-    assert_close(e[same], ref["e"][same], "encoder projection")
-    return worst
+        np.testing.assert_array_equal(g, ref["layers"][l]["yq"], err_msg=f"layer {l}")
+    np.testing.assert_array_equal(got["e"].cpu().numpy()[:, sel], ref["e"])
+    return 0.0
 
 
 def test_encoder_reduced(Bd):
