@@ -1,0 +1,466 @@
+#!/usr/bin/env python
+"""Benchmark of the INT4 RNN-T hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input: feature
+prologue, input quantization, six bidirectional quantized LSTM layers, projection,
+then alignment-length synchronous beam search (width 16) with density-ratio LM fusion
+and the trace-back.  Default workload: the end-to-end configuration (64 utterances of
+10 s, first encoder layer and joint output layer at 8 bit, everything else at 4 bit).
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead, on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+TAG_NAMES = {1: "quantize", 2: "enc_input_gemm", 3: "enc_recurrent_step", 4: "linear",
+             5: "pred_lstm", 6: "pred_proj", 7: "src_lstm", 8: "src_head", 9: "tgt_lstm_l1",
+             10: "tgt_lstm_l2", 11: "tgt_head", 12: "joint", 13: "beam_select", 14: "other"}
+
+WORKLOADS = {
+    # name: (B, T100 or T, U_max, first-layer bits, joint-out bits, has encoder, has decoder)
+    "cfg4_end_to_end": dict(B=64, T=500, U_max=250, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
+    "cfg1_encoder": dict(B=32, T=500, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
+    "cfg3_beam": dict(B=16, T=300, U_max=150, l1_bits=4, out_bits=4, enc=False, dec=True, seed=3),
+}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-i", str(gpu_index), "-lms", "200"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            busy = [v for v in sm if v >= 0.5 * max(sm)] or sm
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------ oracle arm
+def oracle_sample(wl_name: str, cores: int, frames: int = 8):
+    """The CPU oracle on a bounded sample of the workload: `cores` utterances cut to the first
+    `frames` encoder frames (2*frames log-mel frames), label budget frames/2, all layers at
+    full width.  Returns (seconds, audio_seconds, description)."""
+    from oracle import oracle as O
+    from paper_2206_07882_b200 import synth
+    wl = WORKLOADS[wl_name]
+    n = max(1, cores)
+    seed = wl["seed"]
+    t0 = time.perf_counter()
+    e = None
+    if wl["enc"]:
+        enc_w = synth.encoder(seed, T=frames, B=n, first_layer_bits=wl["l1_bits"], in_max=wl["l1_bits"] == 8,
+                              features=False)
+        if wl_name.startswith("cfg4"):
+            mel = synth.logmel(seed, n, 2 * frames, 40)
+            feats = np.stack([O.features(mel[b]) for b in range(n)], axis=1).astype(np.float16)
+        else:
+            feats = synth.Stream(seed).normal("features", (frames, n, 240)).astype(np.float16)
+        e = O.encoder_forward(enc_w["enc"], feats, n_threads=n)["e"]
+    if wl["dec"]:
+        u = max(1, frames // 2)
+        dw = synth.decoder(3, out_bits=wl["out_bits"], U_max=u)
+        if e is None:
+            act = O.act_symmetric(1.0, 4)
+            fr = synth.enc_frames(seed, frames, n, 1280).astype(np.float32)
+            proj = synth._linear(synth.Stream(seed), "enc.proj", 256, 1280)
+            e = O.linear(O.Linear(proj), O.quantize(fr.reshape(frames * n, 1280), act), act).reshape(frames, n, 256)
+        O.alsd(O.Decoder(dw), e, trace=False, n_threads=n)
+    dt = time.perf_counter() - t0
+    audio = n * frames * 0.02
+    what = (f"{n} utterances x first {frames} encoder frames ({audio:.2f} s of audio), label budget "
+            f"{max(1, frames // 2)}, full layer widths, one utterance per thread")
+    return dt, audio, what
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = min(os.cpu_count() or 1, 8)
+    from oracle import oracle as O
+    O.build()
+    times = []
+    what = ""
+    audio = 1.0
+    for i in range(args.warmup + args.steps):
+        dt, audio, what = oracle_sample(args.workload, cores, frames=args.ref_frames)
+        if i >= args.warmup:
+            times.append(dt)
+    t = sum(times) / len(times)
+    rtf = t / audio
+    line = {"impl": "reference", "metric": "end_to_end_rtf", "value": rtf, "unit": "s/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "int4",
+            "data": "synthetic", "config": {"workload": args.workload, "sample": what},
+            "cpu_baseline": {"value": rtf, "unit": "s/s", "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": rtf, "unit": "s/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------ GPU arm
+class Job:
+    """Holds device weights and buffers of one workload and runs whole steps."""
+
+    def __init__(self, wl_name: str, rank: int):
+        import torch
+        from paper_2206_07882_b200 import binding as Bd
+        from paper_2206_07882_b200 import synth
+        self.torch, self.Bd = torch, Bd
+        wl = self.wl = WORKLOADS[wl_name]
+        self.name = wl_name
+        B, T = wl["B"], wl["T"]
+        seed = wl["seed"] + 1000 * rank           # every rank gets its own utterances
+        self.enc = self.dec = None
+        self.host_in = None
+        if wl["enc"]:
+            enc_w = synth.encoder(wl["seed"], T=T, B=B, first_layer_bits=wl["l1_bits"],
+                                  in_max=wl["l1_bits"] == 8, features=False)
+            self.enc = Bd.Encoder(enc_w["enc"])
+            if wl_name.startswith("cfg4"):
+                self.host_in = torch.from_numpy(synth.logmel(seed, B, 2 * T, 40)).pin_memory()
+            else:
+                self.host_in = torch.from_numpy(
+                    synth.Stream(seed).normal("features", (T, B, 240)).astype(np.float16)).pin_memory()
+        if wl["dec"]:
+            dw = synth.decoder(3, out_bits=wl["out_bits"], U_max=wl["U_max"])
+            self.dec = Bd.Decoder(dw)
+            self.dec.alloc_state(B, 16, T + wl["U_max"])
+            if not wl["enc"]:
+                self.host_in = torch.from_numpy(synth.enc_frames(seed, T, B, 1280)).pin_memory()
+                self.frame_act = Bd.q4_act_symmetric(1.0, 4)
+                self.frame_proj = Bd.DeviceLinear(synth._linear(synth.Stream(wl["seed"]), "enc.proj", 256, 1280))
+        self.dev_in = self.host_in.cuda()
+        self.ev = {}
+
+    def h2d_bytes(self):
+        return self.host_in.numel() * self.host_in.element_size()
+
+    def step(self, x, mark=None):
+        """One pass over device-resident input x.  mark(name) records phase boundaries."""
+        Bd, wl = self.Bd, self.wl
+        B, T = wl["B"], wl["T"]
+        res = None
+        if mark:
+            mark("start")
+        if self.enc is not None:
+            feats = Bd.q4_feature_prologue(x) if self.name.startswith("cfg4") else x
+            r = self.enc.forward(feats)
+            e = r["e"]
+            res = r["yq"]
+        else:
+            fq = Bd.quantize_pack_int4(x.reshape(T * B, 1280), self.frame_act)
+            e = Bd.q4_linear_forward(fq, self.frame_act, self.frame_proj).reshape(T, B, 256)
+        if mark:
+            mark("encoded")
+        if self.dec is not None:
+            res = self.dec.decode(e, u_max=wl["U_max"], W=16)
+        if mark:
+            mark("decoded")
+        return res
+
+    def result_to_host(self, res):
+        if isinstance(res, tuple):
+            out = [t.cpu() for t in res]
+            return sum(t.numel() * t.element_size() for t in out)
+        # encoder-only workload: the result is the packed last-layer codes; read a checksum row
+        o = res[-1].cpu()
+        return o.numel() * o.element_size()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4_end_to_end", choices=sorted(WORKLOADS))
+    ap.add_argument("--ref-frames", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2206_07882_b200 import binding as Bd
+    lib = Bd.lib()
+    job = Job(args.workload, rank)
+    wl = job.wl
+    B, T, U = wl["B"], wl["T"], wl["U_max"]
+    iters = T + U if wl["dec"] else 0
+    W = max(args.warmup, 3)
+    K = args.steps
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(W):
+        job.step(job.dev_in)
+    barrier()
+
+    # ---- per-kernel shares: one extra untimed step with every launch bracketed by events
+    import ctypes as C
+    shares = {}
+    n_launch_step = 0
+    if rank == 0:
+        cap = 40000
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(2 * cap)]
+        for ev in evs:
+            ev.record()                      # materialise the handles
+        torch.cuda.synchronize()
+        start = (C.c_void_p * cap)(*[ev.cuda_event for ev in evs[:cap]])
+        stop = (C.c_void_p * cap)(*[ev.cuda_event for ev in evs[cap:]])
+        tags = (C.c_int32 * cap)()
+        lib.q4_timing_set(C.c_uint32(0xFFFFFFFF), start, stop, tags, C.c_int32(cap))
+        l0 = Bd.launch_count()
+        job.step(job.dev_in)
+        torch.cuda.synchronize()
+        n_launch_step = Bd.launch_count() - l0
+        n = lib.q4_timing_count()
+        lib.q4_timing_set(C.c_uint32(0), None, None, None, C.c_int32(0))
+        tot = {}
+        cnt = {}
+        for i in range(n):
+            ms = evs[i].elapsed_time(evs[cap + i])
+            tot[tags[i]] = tot.get(tags[i], 0.0) + ms
+            cnt[tags[i]] = cnt.get(tags[i], 0) + 1
+        allms = sum(tot.values()) or 1.0
+        shares = {TAG_NAMES.get(t, str(t)): {"launches": cnt[t], "ms": round(tot[t], 3),
+                                             "share": round(tot[t] / allms, 4)} for t in sorted(tot)}
+    barrier()
+
+    # ---- timed region 1: inputs resident in HBM; the dominant kernel's launches carry events
+    dom_tag = None
+    if rank == 0 and shares:
+        dom_name = max(shares, key=lambda k: shares[k]["ms"])
+        dom_tag = [t for t, nme in TAG_NAMES.items() if nme == dom_name][0]
+        dcap = (shares[dom_name]["launches"] + 8) * K
+        devs = [torch.cuda.Event(enable_timing=True) for _ in range(2 * dcap)]
+        for ev in devs:
+            ev.record()
+        torch.cuda.synchronize()
+        dstart = (C.c_void_p * dcap)(*[ev.cuda_event for ev in devs[:dcap]])
+        dstop = (C.c_void_p * dcap)(*[ev.cuda_event for ev in devs[dcap:]])
+        dtags = (C.c_int32 * dcap)()
+        lib.q4_timing_set(C.c_uint32(1 << dom_tag), dstart, dstop, dtags, C.c_int32(dcap))
+    sampler = ClockSampler(local) if rank == 0 else None
+    marks = []
+
+    def mark(name):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        marks.append((name, ev))
+
+    barrier()
+    l0 = Bd.launch_count()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_stop = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for _ in range(K):
+        job.step(job.dev_in, mark)
+    t_stop.record()
+    barrier()
+    launches = Bd.launch_count() - l0
+    clocks = sampler.stop() if sampler else None
+    ms_total = t_start.elapsed_time(t_stop)
+    dom_ms = None
+    dom_n = 0
+    if dom_tag is not None:
+        dom_n = lib.q4_timing_count()
+        lib.q4_timing_set(C.c_uint32(0), None, None, None, C.c_int32(0))
+        dom_ms = sum(devs[i].elapsed_time(devs[dcap + i]) for i in range(dom_n)) / max(dom_n, 1)
+    enc_ms = dec_ms = 0.0
+    for i in range(0, len(marks), 3):
+        enc_ms += marks[i][1].elapsed_time(marks[i + 1][1])
+        dec_ms += marks[i + 1][1].elapsed_time(marks[i + 2][1])
+    enc_ms /= K
+    dec_ms /= K
+
+    # ---- timed region 2: end to end through the public API with host buffers
+    barrier()
+    e_start = torch.cuda.Event(enable_timing=True)
+    e_stop = torch.cuda.Event(enable_timing=True)
+    d2h = 0
+    e_start.record()
+    for _ in range(K):
+        x = job.host_in.to("cuda", non_blocking=True)
+        res = job.step(x)
+        d2h = job.result_to_host(res)
+    e_stop.record()
+    barrier()
+    ms_e2e = e_start.elapsed_time(e_stop)
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = t.tolist()
+    ms_step = ms_total / K
+    audio_s = world * B * T * 0.02
+    rtf = (ms_step / 1e3) / audio_s
+    rtf_e2e = (ms_e2e / K / 1e3) / audio_s
+
+    if rank == 0:
+        pk = peaks()
+        line = {"metric": "end_to_end_rtf", "value": rtf, "unit": "s/s", "n_gpus": world, "steps": K,
+                "warmup": W, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+                "vs_baseline": None, "dtype": "int4/int8 codes, int32 accumulate, fp32 gates",
+                "data": "synthetic",
+                "config": {"workload": args.workload, "utterances_per_gpu": B, "frames": T,
+                           "beam": 16 if wl["dec"] else 0, "label_budget": U, "search_iterations": iters,
+                           "l2": "weights (59 MB) and activations exceed no cache assumption: each "
+                                 "step streams >1 GB of accumulators and state; no flush needed"},
+                "parts": {"encoder_ms": enc_ms, "decode_ms": dec_ms,
+                          "encoder_frames_per_s": (B * T / (enc_ms / 1e3)) if wl["enc"] and enc_ms else None,
+                          "beam_hyps_per_s": (B * 16 * iters / (dec_ms / 1e3)) if wl["dec"] and dec_ms else None},
+                "e2e": {"value": rtf_e2e, "unit": "s/s", "h2d_bytes_per_step": job.h2d_bytes(),
+                        "d2h_bytes_per_step": d2h},
+                "gpu_launches": launches, "launches_per_step": n_launch_step, "kernels": shares,
+                "clocks": clocks, "peaks": pk,
+                "paper_context": {"rtf_int4_simulated": 0.065, "speedup_fp16_to_int4_simulated": 3.4,
+                                  "note": "simulated accelerator, 1 utterance of 152 frames, beam 16"}}
+        line["roofline"] = roofline(job, dom_tag, dom_ms, dom_n, pk) if dom_tag is not None else None
+        if not args.no_cpu_baseline:
+            from oracle import oracle as O
+            O.build()
+            cores = min(os.cpu_count() or 1, 8)
+            dt, audio, what = oracle_sample(args.workload, cores, frames=args.ref_frames)
+            line["cpu_baseline"] = {"value": dt / audio, "unit": "s/s", "cores": cores, "kind": "oracle",
+                                    "sample": what, "seconds": dt}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def roofline(job, tag, ms, n, pk):
+    """Roofline entry of the dominant kernel.  Algorithmic work per launch: the weight bytes
+    the kernel must read once plus per-row state traffic, and 2*rows*J*K integer ops."""
+    name = TAG_NAMES[tag]
+    wl = job.wl
+    N = wl["B"] * 16
+    int8_peak = 2.0 * pk["bf16_tflops_sustained"]          # dense int8 : bf16 = 2 : 1
+    out = {"kernel": name, "launches_timed": n, "avg_ms": ms, "traffic": None}
+
+    def lstm_work(l, rows, kx):
+        H = l.H
+        wbytes = l.w_ih.q.numel() + l.w_hh.q.numel() + 2 * 4 * 4 * H + 4 * 4 * H
+        per_row = kx * l.w_ih.bits // 8 + H * l.w_hh.bits // 8 * 2 + H * 4 * 2
+        ops = 2.0 * rows * 4 * H * (l.w_ih.k_pad + H)
+        return wbytes + rows * per_row, ops
+
+    if tag in (5, 7, 9, 10):
+        d = job.dec
+        l, kx = {5: (d.pred_lstm, 256), 7: (d.src.lstm[0], 256), 9: (d.tgt.lstm[0], 256),
+                 10: (d.tgt.lstm[-1], d.tgt.lstm[0].H)}[tag]
+        bytes_, ops = lstm_work(l, N, kx)
+    elif tag == 3:
+        l = job.enc.layers[1][0]
+        Bn = wl["B"]
+        H = l.H
+        bytes_ = 2 * (l.w_hh.q.numel() + Bn * 4 * H * 4 + Bn * H * 4 * 2 + Bn * H)
+        ops = 2 * 2.0 * Bn * 4 * H * H
+    elif tag == 2:
+        l = job.enc.layers[1][0]
+        M = wl["B"] * wl["T"]
+        bytes_ = M * l.w_ih.k_pad // 2 + l.w_ih.q.numel() + M * 4 * l.H * 4
+        ops = 2.0 * M * 4 * l.H * l.w_ih.k_pad
+    else:
+        out.update(bound="hbm", achieved=None, peak=pk["hbm_gbs"], unit="GB/s", frac=None)
+        return out
+    t_hbm = bytes_ / (pk["hbm_gbs"] * 1e9)
+    t_tensor = ops / (int8_peak * 1e12)
+    sec = ms / 1e3
+    out.update(algorithmic_bytes=bytes_, algorithmic_ops=ops,
+               hbm={"achieved": bytes_ / sec / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                    "frac": bytes_ / sec / 1e9 / pk["hbm_gbs"]},
+               tensor={"achieved": ops / sec / 1e12, "peak": int8_peak, "unit": "TOP/s (int8, 2x measured bf16)",
+                       "frac": ops / sec / 1e12 / int8_peak})
+    if t_tensor > t_hbm:
+        out.update(bound="tensor", achieved=ops / sec / 1e12, peak=int8_peak, unit="TFLOP/s",
+                   frac=ops / sec / 1e12 / int8_peak)
+    else:
+        out.update(bound="hbm", achieved=bytes_ / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s",
+                   frac=bytes_ / sec / 1e9 / pk["hbm_gbs"])
+    out["peak_source"] = pk["source"]
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -268,6 +268,18 @@ int q4_poll_status(const int32_t* device_status, q4_stream stream);
 int q4_version(void);
 int64_t q4_launch_count(void);
 
+/* Optional timing of the library's own launches with CUDA events lent by the caller (host
+ * arrays of cudaEvent_t, `capacity` entries each).  Every launch whose tag bit is set in
+ * tag_mask records start_events[i] before and stop_events[i] after itself on the stream it
+ * is launched on, and writes its tag to tags_out[i]; q4_timing_count() returns how many
+ * pairs were used.  tag_mask 0 switches timing off (the default).  Tags: 1 quantize, 2
+ * encoder input GEMM, 3 encoder recurrent step, 4 linear, 5 prediction LSTM, 6 prediction
+ * projection, 7 source-LM LSTM, 8 source-LM head, 9 target-LM layer 1, 10 target-LM layer 2,
+ * 11 target-LM head, 12 joint, 13 beam selection, 14 other. */
+int q4_timing_set(uint32_t tag_mask, void** start_events, void** stop_events, int32_t* tags_out,
+                  int32_t capacity);
+int q4_timing_count(void);
+
 #ifdef __cplusplus
 }
 #endif

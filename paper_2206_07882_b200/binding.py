@@ -72,7 +72,7 @@ class BeamStateS(C.Structure):
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
-           "q4_poll_status", "q4_version", "q4_launch_count"]
+           "q4_poll_status", "q4_version", "q4_launch_count", "q4_timing_set", "q4_timing_count"]
 
 _lib = None
 

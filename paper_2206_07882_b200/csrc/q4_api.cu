@@ -74,6 +74,15 @@ GemmArgs gemm_args(const void* x, long long x_stride, const int32_t* x_idx, cons
 extern "C" {
 
 int q4_version(void) { return 1; }
+
+int q4_timing_set(uint32_t tag_mask, void** start_events, void** stop_events, int32_t* tags_out,
+                  int32_t capacity) {
+  if (tag_mask != 0 && (!start_events || !stop_events || !tags_out || capacity <= 0)) return Q4_ERR_NULL;
+  timing_set(tag_mask, reinterpret_cast<cudaEvent_t*>(start_events),
+             reinterpret_cast<cudaEvent_t*>(stop_events), tags_out, tag_mask ? capacity : 0);
+  return Q4_OK;
+}
+int q4_timing_count(void) { return timing_count(); }
 int64_t q4_launch_count(void) { return g_launches; }
 
 int q4_act_symmetric(float alpha, int32_t bits, q4_act* out) {
@@ -143,8 +152,9 @@ int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k
                        const q4_act* act, int32_t mode, int32_t n_groups,
                        const float* per_row_scale, void* q_out, float* group_scale_out,
                        q4_stream stream) {
-  if (!x || !q_out || !act) return Q4_ERR_NULL;
+  if (!act) return Q4_ERR_NULL;
   if (rows < 0 || k <= 0 || k_pad < k) return Q4_ERR_DIM;
+  if (rows > 0 && (!x || !q_out)) return Q4_ERR_NULL;
   if (k_pad % 32 != 0 || !aligned16(q_out)) return Q4_ERR_ALIGN;
   if (act->bits != 4 && act->bits != 8) return Q4_ERR_BITS;
   if (mode < 0 || mode > 2) return Q4_ERR_UNSUPPORTED;
@@ -159,6 +169,7 @@ int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k
     if (mode == 2 && !per_row_scale) return Q4_ERR_NULL;
   }
   if (rows == 0) return Q4_OK;
+  TagScope tag(TAG_QUANT);
   Q4_TRY(launch_quantize(x, x_is_fp16 != 0, rows, k, k_pad, a, mode, n_groups, per_row_scale,
                          static_cast<uint8_t*>(q_out), group_scale_out, S(stream)));
   return Q4_OK;
@@ -175,6 +186,7 @@ int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_m
   GemmArgs g = gemm_args(xq, row_bytes(w->k_pad, w->bits), nullptr, *x_act, M, *w, bias, out,
                          w->rows, nullptr);
   g.dbg_acc = dbg_acc;
+  TagScope tag(TAG_LINEAR);
   Q4_TRY(launch_gemm(g, w->bits, EPI_F32, S(stream)));
   return Q4_OK;
 }
@@ -241,6 +253,7 @@ int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, co
   a.dbg_ih = dbg_acc_ih;
   a.dbg_hh = dbg_acc_hh;
   a.dbg_stride = 4LL * H;
+  TagScope tag(TAG_PRED_LSTM);
   Q4_TRY(launch_lstm(args, 1, w_ih->bits, w_hh->bits, S(stream)));
   return Q4_OK;
 }
@@ -284,6 +297,7 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
   for (int d = 0; d < dirs; ++d) {
     GemmArgs g = gemm_args(xq, xb, nullptr, *x_act, (int)TB, w_ih[d], nullptr,
                            acc_ih + (size_t)d * TB * G, G, nullptr);
+    TagScope tag(TAG_ENC_GEMM);
     Q4_TRY(launch_gemm(g, w_ih[d].bits, EPI_I32, s));
   }
   Q4_TRY(cudaMemsetAsync(hbuf, 0, (size_t)dirs * 2 * B * H, s));
@@ -314,6 +328,7 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
       if (dbg_acc_hh) a.dbg_hh = dbg_acc_hh + ((size_t)t * B * dirs + d) * G;
       a.dbg_stride = (long long)dirs * G;
     }
+    TagScope tag(TAG_ENC_STEP);
     Q4_TRY(launch_lstm(args, dirs, w_ih[0].bits, w_hh[0].bits, s));
   }
   for (int d = 0; d < dirs; ++d) {
@@ -346,6 +361,7 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
   if (workspace_bytes < q4_workspace_bytes(Q4_WS_JOINT, dims, 2)) return Q4_ERR_WORKSPACE;
   if (N == 0) return Q4_OK;
   cudaStream_t s = S(stream);
+  TagScope tag(TAG_JOINT);
   float* p = static_cast<float*>(workspace);
   uint8_t* zq = static_cast<uint8_t*>(workspace) + align_up((size_t)N * D * sizeof(float));
   GemmArgs g1 = gemm_args(pq, row_bytes(w_pred->k_pad, w_pred->bits), nullptr, *p_act, N, *w_pred,
@@ -363,6 +379,7 @@ int q4_feature_prologue(const float* mel, int32_t B, int32_t T100, int32_t M, vo
                         q4_stream stream) {
   if (!mel || !out_fp16) return Q4_ERR_NULL;
   if (B <= 0 || T100 < 2 || M <= 0) return Q4_ERR_DIM;
+  TagScope tag(TAG_MISC);
   Q4_TRY(launch_features(mel, B, T100, M, out_fp16, S(stream)));
   return Q4_OK;
 }
@@ -390,9 +407,10 @@ int q4_beam_init(q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters, q4
 
 // One network's pending advance for all slots: LSTM layers reading the parent's state row and
 // writing the fresh row, then the projection(s).
-static int advance_lstm(const q4_lstm& L, const void* x, long long x_stride, const int32_t* x_idx,
-                        const q4_act& x_act, void* hq, float* c, const q4_beam_state& st, int N,
-                        cudaStream_t s) {
+static int advance_lstm(int tag_id, const q4_lstm& L, const void* x, long long x_stride,
+                        const int32_t* x_idx, const q4_act& x_act, void* hq, float* c,
+                        const q4_beam_state& st, int N, cudaStream_t s) {
+  TagScope tag(tag_id);
   LstmArgs2 args;
   memset(&args, 0, sizeof(args));
   LstmArgs& a = args.d[0];
@@ -472,10 +490,11 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   // 1. pending advances -------------------------------------------------------------
   {  // prediction network: embedding row -> LSTM -> projection to D
     const q4_lstm& L = m.pred_lstm;
-    Q4_CHECK(advance_lstm(L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), st.adv_tok,
+    Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), st.adv_tok,
                           m.pred_emb_act, st.pred_hq, st.pred_c, st, N, s));
     GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), st.adv_dst,
                            L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, st.adv_dst);
+    TagScope tag(TAG_PRED_PROJ);
     Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
   }
   for (int which = 0; which < 2; ++which) {
@@ -485,14 +504,14 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     float* lp = which == 0 ? st.src_lp : st.tgt_lp;
     uint8_t* bq = which == 0 ? bq_src : bq_tgt;
     const q4_lstm& L0 = lm.lstm[0];
-    Q4_CHECK(advance_lstm(L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), st.adv_tok,
+    Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), st.adv_tok,
                           lm.emb_act, hq0, c0, st, N, s));
     const void* top = hq0;
     const q4_lstm* last = &L0;
     if (lm.n_layers == 2) {
       if (which == 0) return Q4_ERR_UNSUPPORTED;  // the state block holds one source-LM layer
       const q4_lstm& L1 = lm.lstm[1];
-      Q4_CHECK(advance_lstm(L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), st.adv_dst,
+      Q4_CHECK(advance_lstm(TAG_TGT_L2, L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), st.adv_dst,
                             L0.hid_act, st.tgt_hq[1], st.tgt_c[1], st, N, s));
       top = st.tgt_hq[1];
       last = &L1;
@@ -501,6 +520,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
                             last->hid_act, N, lm.bott.w, lm.bott.bias, bq,
                             row_bytes(D, lm.bott_act.bits), nullptr);
     gb.out_act = lm.bott_act;
+    TagScope tag(which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD);
     Q4_TRY(launch_gemm(gb, lm.bott.w.bits, EPI_QUANT, s));
     GemmArgs go = gemm_args(bq, row_bytes(D, lm.bott_act.bits), nullptr, lm.bott_act, N, lm.out.w,
                             lm.out.bias, lp, V, st.adv_dst);
@@ -509,6 +529,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   }
 
   // 2. joint network for every live slot at its frame -----------------------------------
+  TagScope tag_joint(TAG_JOINT);
   Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, zq, live, s));
   GemmArgs gj = gemm_args(zq, row_bytes(D, m.z_act.bits), live, m.z_act, N, m.joint_out.w,
                           m.joint_out.bias, logits, V, nullptr);
@@ -530,6 +551,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   sel.lambda_t = lambda_t;
   sel.lambda_s = lambda_s;
   sel.rho = rho;
+  TagScope tag_sel(TAG_SELECT);
   Q4_TRY(launch_beam_select(sel, s));
   return Q4_OK;
 }

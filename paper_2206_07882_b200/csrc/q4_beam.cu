@@ -238,7 +238,9 @@ cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     configured = smem;
   }
+  timing_begin(s);
   k_beam_select<<<a.B, SEL_NT, smem, s>>>(a);
+  timing_end(s);
   ++g_launches;
   return cudaGetLastError();
 }

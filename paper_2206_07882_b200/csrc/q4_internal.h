@@ -29,6 +29,22 @@ cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters,
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s);
 
+// Launch-site tags for the optional event timing hook (q4_timing_set).
+enum { TAG_NONE = 0, TAG_QUANT = 1, TAG_ENC_GEMM = 2, TAG_ENC_STEP = 3, TAG_LINEAR = 4,
+       TAG_PRED_LSTM = 5, TAG_PRED_PROJ = 6, TAG_SRC_LSTM = 7, TAG_SRC_HEAD = 8, TAG_TGT_L1 = 9,
+       TAG_TGT_L2 = 10, TAG_TGT_HEAD = 11, TAG_JOINT = 12, TAG_SELECT = 13, TAG_MISC = 14,
+       TAG_COUNT = 15 };
+extern int g_tag;   // tag of the launches being issued
+struct TagScope {
+  int prev;
+  explicit TagScope(int t) : prev(g_tag) { g_tag = t; }
+  ~TagScope() { g_tag = prev; }
+};
+void timing_begin(cudaStream_t s);
+void timing_end(cudaStream_t s);
+void timing_set(uint32_t mask, cudaEvent_t* start, cudaEvent_t* stop, int32_t* tags, int cap);
+int timing_count();
+
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 }  // namespace q4

@@ -7,6 +7,44 @@
 namespace q4 {
 
 int64_t g_launches = 0;
+int g_tag = TAG_NONE;
+
+// Optional event timing of tagged launches: the caller lends pairs of CUDA events; every
+// launch whose tag is enabled records one pair on its own stream.  Off by default.
+struct Timing {
+  uint32_t mask = 0;
+  cudaEvent_t* start = nullptr;
+  cudaEvent_t* stop = nullptr;
+  int32_t* tags = nullptr;
+  int cap = 0, n = 0;
+  bool open = false;
+} g_timing;
+
+void timing_begin(cudaStream_t s) {
+  Timing& t = g_timing;
+  t.open = false;
+  if (!(t.mask >> g_tag & 1u) || t.n >= t.cap) return;
+  cudaEventRecord(t.start[t.n], s);
+  t.open = true;
+}
+void timing_end(cudaStream_t s) {
+  Timing& t = g_timing;
+  if (!t.open) return;
+  cudaEventRecord(t.stop[t.n], s);
+  t.tags[t.n] = g_tag;
+  ++t.n;
+  t.open = false;
+}
+void timing_set(uint32_t mask, cudaEvent_t* start, cudaEvent_t* stop, int32_t* tags, int cap) {
+  g_timing.mask = mask;
+  g_timing.start = start;
+  g_timing.stop = stop;
+  g_timing.tags = tags;
+  g_timing.cap = cap;
+  g_timing.n = 0;
+  g_timing.open = false;
+}
+int timing_count() { return g_timing.n; }
 
 // =====================================================================================
 // Integer tile GEMM: acc[m, j] = sum_k W[j,k] * (x[m,k] - z).  64 x 64 outputs per CTA,
@@ -140,7 +178,9 @@ cudaError_t launch_gemm(const GemmArgs& a, int bits, int epi, cudaStream_t s) {
   dim3 grid((a.M + TILE - 1) / TILE, (a.J + TILE - 1) / TILE);
 #define Q4_GEMM_CASE(B_, E_)                           \
   if (bits == B_ && epi == E_) {                       \
+    timing_begin(s);                                   \
     k_gemm<B_, E_><<<grid, NT, 0, s>>>(a);             \
+    timing_end(s);                                     \
     ++g_launches;                                      \
     return cudaGetLastError();                         \
   }
@@ -352,7 +392,9 @@ cudaError_t launch_lstm(const LstmArgs2& a, int dirs, int x_bits, int h_bits, cu
   dim3 grid((a0.N + TILE - 1) / TILE, (a0.H + 15) / 16, dirs);
 #define Q4_LSTM_CASE(X_, H_)                    \
   if (x_bits == X_ && h_bits == H_) {           \
+    timing_begin(s);                            \
     k_lstm<X_, H_><<<grid, NT, 0, s>>>(a);      \
+    timing_end(s);                              \
     ++g_launches;                               \
     return cudaGetLastError();                  \
   }
@@ -407,7 +449,9 @@ __global__ void __launch_bounds__(256) k_logsoftmax(const float* in, float* out,
 cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long long stride,
                               const int32_t* idx, cudaStream_t s) {
   if (rows <= 0) return cudaSuccess;
+  timing_begin(s);
   k_logsoftmax<<<rows, 256, 0, s>>>(in, out, V, stride, idx);
+  timing_end(s);
   ++g_launches;
   return cudaGetLastError();
 }
@@ -451,8 +495,10 @@ cudaError_t launch_joint_z(const float* e, const int32_t* frame_idx, const int32
                            const q4_act& za, uint8_t* zq, int32_t* live_out, cudaStream_t s) {
   if (N <= 0) return cudaSuccess;
   const long long total = (long long)N * (D / 2);
+  timing_begin(s);
   k_joint_z<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(e, frame_idx, t_arr, B, W, p, p_idx, N,
                                                             D, za, zq, live_out);
+  timing_end(s);
   ++g_launches;
   return cudaGetLastError();
 }
@@ -542,10 +588,12 @@ cudaError_t launch_quantize(const void* x, bool fp16, long long rows, int k, int
   }
   const long long total = rows * (k_pad >> 3);
   const unsigned blocks = (unsigned)((total + 255) / 256);
+  timing_begin(s);
   if (fp16)
     k_quantize<true><<<blocks, 256, 0, s>>>(x, rows, k, k_pad, a, mode, n_groups, sv, out);
   else
     k_quantize<false><<<blocks, 256, 0, s>>>(x, rows, k, k_pad, a, mode, n_groups, sv, out);
+  timing_end(s);
   ++g_launches;
   return cudaGetLastError();
 }
@@ -583,7 +631,9 @@ __global__ void __launch_bounds__(256) k_features(const float* mel, int B, int T
 cudaError_t launch_features(const float* mel, int B, int T100, int M, void* out, cudaStream_t s) {
   const long long total = (long long)B * T100 * M;
   if (total <= 0) return cudaSuccess;
+  timing_begin(s);
   k_features<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(mel, B, T100, M, (__half*)out);
+  timing_end(s);
   ++g_launches;
   return cudaGetLastError();
 }

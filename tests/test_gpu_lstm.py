@@ -59,7 +59,7 @@ def test_config0_teacher_forced_every_step(Bd):
                                                  (64, 64, 32, 8, 4, True), (1, 1280, 640, 4, 4, True)])
 def test_step_shapes_and_formats(Bd, N, K, H, xb, hb, signed):
     st = synth.Stream(100 + N)
-    lw = synth._lstm(st, "l", K, H, 4, bias_std=0.2, hid_bits=hb)
+    lw = synth._lstm(st, "l", K, H, 4, bias_std=0.2, hid_alpha=0.95, hid_bits=hb)
     if xb == 8:
         lw.w_ih = synth._qmat(st, "w8", 4 * H, K, 8)
     if hb == 8:
