@@ -100,7 +100,10 @@ int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k
  *   hq_n [dirs, B, H] codes (hid_act) and c_n [dirs, B, H] fp32 receive the final states
  *   (nullable).  dbg_acc_ih / dbg_acc_hh [T, B, dirs, 4H] int32 (nullable) receive the raw
  *   accumulators for parity checks.  h0 = c0 = 0.
- *   workspace: q4_workspace_bytes(Q4_WS_LSTM_LAYER, {T,B,dirs,H}) bytes, scratch.
+ *   workspace: scratch of q4_workspace_bytes(Q4_WS_LSTM_LAYER, {T,B,dirs,H}) bytes (DP4A input
+ *   projection) or q4_workspace_bytes(Q4_WS_LSTM_LAYER, {T,B,dirs,H,kx_pad}) bytes (adds room for
+ *   int8 operand copies, which selects the tensor-core input projection when T*B >= 128).
+ *   Its first 4 bytes are a status word for q4_poll_status (bounded device waits).
  */
 int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scale_b, int32_t T,
                         int32_t B, int32_t dirs, const q4_mat* w_ih, const q4_mat* w_hh,
@@ -255,7 +258,7 @@ int q4_traceback(const q4_beam_state* state, int32_t B, int32_t W, int32_t n_ite
 int q4_feature_prologue(const float* mel, int32_t B, int32_t T100, int32_t M, void* out_fp16,
                         q4_stream stream);
 
-#define Q4_WS_LSTM_LAYER 1 /* dims = {T, B, dirs, H} */
+#define Q4_WS_LSTM_LAYER 1 /* dims = {T, B, dirs, H} or {T, B, dirs, H, kx_pad} */
 #define Q4_WS_JOINT 2      /* dims = {N, D} */
 #define Q4_WS_BEAM 3       /* dims = {B, W, V, D} */
 size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims);

@@ -222,7 +222,7 @@ class DeviceLinear:
 def qlstm_layer_forward(xq: torch.Tensor, x_act: Act, T: int, B: int, layers: Sequence[DeviceLstm],
                         out_act: Optional[Act] = None, x_scale_b: Optional[torch.Tensor] = None,
                         want_state: bool = False, want_dbg: bool = False,
-                        workspace: Optional[torch.Tensor] = None):
+                        workspace: Optional[torch.Tensor] = None, tensor_cores: bool = True):
     """xq [T*B, kx_pad*bits/8] codes.  Returns dict(yq [, hq_n, c_n, acc_ih, acc_hh])."""
     _need_cuda()
     dirs, H = len(layers), layers[0].H
@@ -230,10 +230,10 @@ def qlstm_layer_forward(xq: torch.Tensor, x_act: Act, T: int, B: int, layers: Se
     out_act = out_act or hid_act
     dev = xq.device
     yq = torch.empty((T * B, dirs * H * out_act.bits // 8), dtype=torch.uint8, device=dev)
-    need = workspace_bytes(WS_LSTM_LAYER, [T, B, dirs, H])
+    need = workspace_bytes(WS_LSTM_LAYER, [T, B, dirs, H] + ([layers[0].w_ih.k_pad] if tensor_cores else []))
     if workspace is None or workspace.numel() < need:
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
-    r = {"yq": yq}
+    r = {"yq": yq, "workspace": workspace}
     if want_state:
         r["hq_n"] = torch.empty((dirs, B, H * hid_act.bits // 8), dtype=torch.uint8, device=dev)
         r["c_n"] = torch.empty((dirs, B, H), dtype=torch.float32, device=dev)
@@ -268,6 +268,11 @@ def qlstm_step(xq: torch.Tensor, x_act: Act, hq_in: torch.Tensor, c_in: torch.Te
                           _p(r["hq"]), _p(r["c"]), _p(r["h"]), _p(r.get("acc_ih")),
                           _p(r.get("acc_hh")), _stream()), "qlstm_step")
     return r
+
+
+def q4_poll_status(status: torch.Tensor) -> int:
+    """Synchronise the stream and return the device status word (0 = ok)."""
+    return int(lib().q4_poll_status(_p(status), _stream()))
 
 
 def q4_linear_forward(xq: torch.Tensor, x_act: Act, lin: DeviceLinear, want_acc: bool = False):
@@ -341,7 +346,8 @@ class Encoder:
             xq = quantize_pack_int4(x2, self.in_act)
         x_act = self.in_act
         H = self.layers[0][0].H
-        need = workspace_bytes(WS_LSTM_LAYER, [T, B, 2, H])
+        kmax = max(dirs[0].w_ih.k_pad for dirs in self.layers)
+        need = workspace_bytes(WS_LSTM_LAYER, [T, B, 2, H, kmax])
         if self.ws is None or self.ws.numel() < need:
             self.ws = torch.empty(need, dtype=torch.uint8, device=features.device)
         outs = []

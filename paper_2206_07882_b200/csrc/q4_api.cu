@@ -122,10 +122,15 @@ size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims) {
   if (!dims) return 0;
   if (call_id == Q4_WS_LSTM_LAYER && ndims >= 4) {
     const size_t T = dims[0], B = dims[1], D = dims[2], H = dims[3];
-    size_t n = 0;
+    const size_t K = ndims >= 5 ? dims[4] : 0;
+    size_t n = 256;                                      // status word
     n += align_up(D * T * B * 4 * H * sizeof(int32_t));  // input accumulators
     n += align_up(D * 2 * B * H);                        // recurrent codes, double buffered
     n += align_up(D * B * H * sizeof(float));            // cell state
+    if (K > 0) {                                         // int8 operands of the tensor-core GEMM
+      n += align_up(T * B * K);
+      n += align_up(D * 4 * H * K);
+    }
     return n;
   }
   if (call_id == Q4_WS_JOINT && ndims >= 2) {
@@ -277,28 +282,49 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
   Q4_CHECK(check_act(out_act));
   if (!out_act->is_signed) return Q4_ERR_UNSUPPORTED;
   if (!aligned16(xq) || !aligned16(yq) || !aligned16(workspace)) return Q4_ERR_ALIGN;
-  const int32_t dims[4] = {T, B, dirs, H};
+  const int32_t dims[5] = {T, B, dirs, H, w_ih[0].k_pad};
   if (workspace_bytes < q4_workspace_bytes(Q4_WS_LSTM_LAYER, dims, 4)) return Q4_ERR_WORKSPACE;
+  const long long TB = (long long)T * B;
+  // tensor-core input projection when the caller's workspace has room for the int8 operands
+  const bool use_mma = TB >= 128 && workspace_bytes >= q4_workspace_bytes(Q4_WS_LSTM_LAYER, dims, 5);
 
   cudaStream_t s = S(stream);
-  const long long TB = (long long)T * B;
   const int G = 4 * H;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int32_t* status = reinterpret_cast<int32_t*>(ws);
+  ws += 256;
+  Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
   int32_t* acc_ih = reinterpret_cast<int32_t*>(ws);
   ws += align_up((size_t)dirs * TB * G * sizeof(int32_t));
   uint8_t* hbuf = ws;  // [dirs][2][B*H bytes]
   ws += align_up((size_t)dirs * 2 * B * H);
   float* cbuf = reinterpret_cast<float*>(ws);  // [dirs][B][H]
+  ws += align_up((size_t)dirs * B * H * sizeof(float));
+  const int Kx = w_ih[0].k_pad;
+  int8_t* x8 = reinterpret_cast<int8_t*>(ws);
+  int8_t* w8 = x8 + align_up((size_t)TB * Kx);
   const long long hb = row_bytes(H, hid_act->bits);
   const long long yb = row_bytes(dirs * H, out_act->bits);
   const long long xb = row_bytes(w_ih[0].k_pad, w_ih[0].bits);
 
   // time-parallel input projections for all frames
+  if (use_mma) {
+    TagScope tag(TAG_QUANT);
+    Q4_TRY(launch_unpack_rows(xq, xb, nullptr, *x_act, Kx, (int)TB, x8, Kx, 0, (int)TB, s));
+    for (int d = 0; d < dirs; ++d)
+      Q4_TRY(launch_prepare_w(w_ih[d], 0, w8 + (size_t)d * G * Kx, Kx, 0, s));
+  }
   for (int d = 0; d < dirs; ++d) {
-    GemmArgs g = gemm_args(xq, xb, nullptr, *x_act, (int)TB, w_ih[d], nullptr,
-                           acc_ih + (size_t)d * TB * G, G, nullptr);
     TagScope tag(TAG_ENC_GEMM);
-    Q4_TRY(launch_gemm(g, w_ih[d].bits, EPI_I32, s));
+    if (use_mma) {
+      Q4_TRY(launch_mma_gemm(x8, Kx, (int)TB, w8 + (size_t)d * G * Kx, Kx, G, Kx, EPI_I32,
+                             acc_ih + (size_t)d * TB * G, G, nullptr, nullptr, nullptr, 0.0f, nullptr,
+                             status, s));
+    } else {
+      GemmArgs g = gemm_args(xq, xb, nullptr, *x_act, (int)TB, w_ih[d], nullptr,
+                             acc_ih + (size_t)d * TB * G, G, nullptr);
+      Q4_TRY(launch_gemm(g, w_ih[d].bits, EPI_I32, s));
+    }
   }
   Q4_TRY(cudaMemsetAsync(hbuf, 0, (size_t)dirs * 2 * B * H, s));
   Q4_TRY(cudaMemsetAsync(cbuf, 0, (size_t)dirs * B * H * sizeof(float), s));

@@ -45,6 +45,49 @@ void timing_end(cudaStream_t s);
 void timing_set(uint32_t mask, cudaEvent_t* start, cudaEvent_t* stop, int32_t* tags, int cap);
 int timing_count();
 
+// ---- tensor-core path (q4_mma.cu)
+struct MmaLstmArgs {
+  int32_t N, H, Kx_pad;
+  const int32_t* acc_pre;   // optional precomputed input accumulators [row, 4H] in 4*cell+gate order
+  long long acc_pre_ld;
+  const float* sc_ih;       // per weight row, 4*cell+gate order
+  const float* sc_hh;
+  const float* bias;
+  float x_scale;
+  const float* x_scale_vec;
+  int32_t x_scale_mod;
+  q4_act hid_act, out_act;
+  const int32_t* src_row;   // state row read by launch row n (nullptr = n, negative = zero state)
+  const int32_t* dst_row;   // state row written (nullptr = n, negative = row inactive)
+  const float* c_in;
+  float* c_out;
+  uint8_t* hq_out;          // packed recurrent codes at dst row (nullable)
+  long long hq_ld;
+  int8_t* h8_out;           // int8 recurrent codes at launch row n (nullable)
+  long long h8_ld;
+  uint8_t* yq_out;          // packed out_act codes at launch row n (nullable)
+  long long yq_ld;
+  float* h_f32;
+  int32_t* dbg_ih;          // optional [n, 4H] gate-major
+  int32_t* dbg_hh;
+  long long dbg_ld;
+  int32_t* status;
+};
+enum { EPI_QUANT8 = 3 };    // re-quantize and store (code - zero_point) as int8, one per byte
+cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
+                               const q4_act& act, int k_pad, int n_rows, int8_t* dst,
+                               long long dst_stride, int col0, int n_rows_pad, cudaStream_t s);
+cudaError_t launch_prepare_w(const q4_mat& w, int interleave, int8_t* dst, long long dst_stride,
+                             int col0, cudaStream_t s);
+cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s);
+cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const int8_t* w8,
+                            long long w_pitch, int J, int K, int epi, void* out, long long ldo,
+                            const int32_t* out_idx, const float* w_scale, const float* bias,
+                            float x_scale, const q4_act* out_act, int32_t* status, cudaStream_t s);
+cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa_pitch,
+                            const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
+                            const int8_t* hw, long long hw_pitch, cudaStream_t s);
+
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 }  // namespace q4

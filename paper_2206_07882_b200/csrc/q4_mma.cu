@@ -1,0 +1,561 @@
+// Tensor-core path (sm_100a): TMA-fed tcgen05 kind::i8 GEMMs with int32 accumulators in
+// tensor memory.  Activations are the M operand (128 rows per tile), weight rows the N
+// operand, both K-major int8 in shared memory under the 128-byte swizzle.
+//   k_mma_gemm : D[128 x 256] tiles, epilogues: store int32 / de-quantize+bias / re-quantize.
+//   k_mma_lstm : D_ih, D_hh[128 x 128] tiles (32 cells x 4 gates, gate-interleaved weight
+//                rows) with the whole LSTM cell update fused into the epilogue.
+// Warp roles per CTA: epilogue warps (one TMEM lane quarter each), one TMA producer thread,
+// one MMA issuer thread.  4-bit codes are unpacked to int8 once per call by k_unpack_rows /
+// k_prepare_w before they meet the tensor cores.
+#include <string.h>
+
+#include "q4_internal.h"
+#include "q4_mma.cuh"
+
+namespace q4 {
+
+constexpr int BM = 128;          // activation rows per tile
+constexpr int BK = 128;          // K bytes per pipeline stage (one swizzle row)
+constexpr int GEMM_BN = 256;     // weight rows per tile, plain GEMM
+constexpr int GEMM_STAGES = 4;
+constexpr int LSTM_BN = 128;     // weight rows per tile, LSTM (32 cells x 4 gates)
+constexpr int LSTM_STAGES = 3;
+constexpr int LSTM_EPI_WARPS = 8;
+
+// ------------------------------------------------------------------ operand preparation
+// Gather + unpack activation rows to int8: dst[n, col0 + k] = code(src[idx[n], k]) - zero_point.
+__global__ void __launch_bounds__(256) k_unpack_rows(const uint8_t* src, long long src_stride,
+                                                     const int32_t* idx, int bits, int is_signed,
+                                                     int zp, int k_pad, int n_rows, int8_t* dst,
+                                                     long long dst_stride, int col0, int n_rows_pad) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = k_pad >> 5;  // 32 elements per thread
+  if (i >= (long long)n_rows_pad * per_row) return;
+  const int n = (int)(i / per_row), k = (int)(i % per_row) * 32;
+  uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
+  int r = -1;
+  if (n < n_rows) r = idx ? idx[n] : n;
+  if (r >= 0) {
+    const uint8_t* p = src + (long long)r * src_stride;
+    if (bits == 4) {
+      const uint4 v = *reinterpret_cast<const uint4*>(p + (k >> 1));
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      uint32_t o[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        // natural element order: byte b of the output word holds element 4*word + b
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          int a = (w[j] >> (4 * e)) & 0xF, c = (w[j] >> (4 * (e + 4))) & 0xF;
+          if (is_signed) {
+            a = (a ^ 8) - 8;
+            c = (c ^ 8) - 8;
+          } else {
+            a -= zp;
+            c -= zp;
+          }
+          lo |= (uint32_t)(a & 0xFF) << (8 * e);
+          hi |= (uint32_t)(c & 0xFF) << (8 * e);
+        }
+        o[2 * j] = lo;
+        o[2 * j + 1] = hi;
+      }
+      o0 = make_uint4(o[0], o[1], o[2], o[3]);
+      o1 = make_uint4(o[4], o[5], o[6], o[7]);
+    } else {
+      o0 = *reinterpret_cast<const uint4*>(p + k);
+      o1 = *reinterpret_cast<const uint4*>(p + k + 16);
+    }
+  }
+  uint4* d = reinterpret_cast<uint4*>(dst + (long long)n * dst_stride + col0 + k);
+  d[0] = o0;
+  d[1] = o1;
+}
+
+cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
+                               const q4_act& act, int k_pad, int n_rows, int8_t* dst,
+                               long long dst_stride, int col0, int n_rows_pad, cudaStream_t s) {
+  const long long total = (long long)n_rows_pad * (k_pad >> 5);
+  if (total <= 0) return cudaSuccess;
+  timing_begin(s);
+  k_unpack_rows<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
+      static_cast<const uint8_t*>(src), src_stride, idx, act.bits, act.is_signed, act.zero_point, k_pad,
+      n_rows, dst, dst_stride, col0, n_rows_pad);
+  timing_end(s);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
+// Weight preparation: unpack to int8; with `interleave` the 4H rows (gate-major i,f,g,o) are
+// reordered to row 4*cell + gate so that one thread of the epilogue owns all gates of a cell.
+__global__ void __launch_bounds__(256) k_prepare_w(const uint8_t* src, int bits, int rows, int k_pad,
+                                                   int interleave, int8_t* dst, long long dst_stride,
+                                                   int col0) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = k_pad >> 3;
+  if (i >= (long long)rows * per_row) return;
+  const int r = (int)(i / per_row), k = (int)(i % per_row) * 8;
+  int ro = r;
+  if (interleave) {
+    const int H = rows >> 2;
+    ro = 4 * (r % H) + r / H;
+  }
+  uint2 o;
+  if (bits == 4) {
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(src + (long long)r * (k_pad >> 1) + (k >> 1));
+    uint32_t lo = 0, hi = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int a = (((w >> (4 * e)) & 0xF) ^ 8) - 8, c = (((w >> (4 * (e + 4))) & 0xF) ^ 8) - 8;
+      lo |= (uint32_t)(a & 0xFF) << (8 * e);
+      hi |= (uint32_t)(c & 0xFF) << (8 * e);
+    }
+    o = make_uint2(lo, hi);
+  } else {
+    o = *reinterpret_cast<const uint2*>(src + (long long)r * k_pad + k);
+  }
+  *reinterpret_cast<uint2*>(dst + (long long)ro * dst_stride + col0 + k) = o;
+}
+__global__ void k_prepare_vec(const float* src, int rows, int interleave, float* dst) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows) return;
+  int ro = r;
+  if (interleave) {
+    const int H = rows >> 2;
+    ro = 4 * (r % H) + r / H;
+  }
+  dst[ro] = src ? src[r] : 0.0f;
+}
+
+cudaError_t launch_prepare_w(const q4_mat& w, int interleave, int8_t* dst, long long dst_stride,
+                             int col0, cudaStream_t s) {
+  const long long total = (long long)w.rows * (w.k_pad >> 3);
+  timing_begin(s);
+  k_prepare_w<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(static_cast<const uint8_t*>(w.q), w.bits,
+                                                              w.rows, w.k_pad, interleave, dst,
+                                                              dst_stride, col0);
+  timing_end(s);
+  ++g_launches;
+  return cudaGetLastError();
+}
+cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s) {
+  k_prepare_vec<<<(rows + 255) / 256, 256, 0, s>>>(src, rows, interleave, dst);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ tensor maps (host)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// int8 matrix [rows, k] with row pitch `pitch` bytes; box = 128 bytes of K x box_rows rows.
+bool make_tmap_i8(CUtensorMap* m, const void* base, uint64_t k, uint64_t rows, uint64_t pitch,
+                  uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) || (pitch & 15u)) return false;
+  const cuuint64_t dims[2] = {k, rows};
+  const cuuint64_t strides[1] = {pitch};
+  const cuuint32_t box[2] = {BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__device__ __forceinline__ void flag_timeout(int32_t* status) {
+  if (status) atomicExch(status, Q4_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------ plain GEMM
+struct MmaGemmArgs {
+  int M, J, K, epi;
+  void* out;
+  long long ldo;            // elements (int32 / float) or bytes (codes) between output rows
+  const int32_t* out_idx;   // output row of activation row m (nullptr = m, negative = skip)
+  const float* w_scale;
+  const float* bias;
+  float x_scale;
+  q4_act out_act;
+  int32_t* status;
+};
+
+__global__ void __launch_bounds__(192, 1)
+k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b,
+           const MmaGemmArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr int A_BYTES = BM * BK, B_BYTES = GEMM_BN * BK, STAGE = A_BYTES + B_BYTES;
+  __shared__ uint64_t full[GEMM_STAGES], empty[GEMM_STAGES], acc_full;
+  __shared__ uint32_t tmem_base_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * GEMM_BN;
+  const int nk = (a.K + BK - 1) / BK;
+
+  if (tid == 0) {
+    for (int s = 0; s < GEMM_STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(&acc_full, 1);
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 5) tmem_alloc(&tmem_base_s, GEMM_BN);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_s;
+
+  if (warp == 4 && lane == 0) {
+    prefetch_tmap(&tma_a);
+    prefetch_tmap(&tma_b);
+    bool ok = true;
+    for (int i = 0; i < nk && ok; ++i) {
+      const int s = i % GEMM_STAGES;
+      if (i >= GEMM_STAGES) ok = mbar_wait(&empty[s], ((i / GEMM_STAGES) - 1) & 1);
+      if (!ok) break;
+      mbar_expect_tx(&full[s], STAGE);
+      tma_load_2d(smem + s * STAGE, &tma_a, i * BK, m0, &full[s]);
+      tma_load_2d(smem + s * STAGE + A_BYTES, &tma_b, i * BK, n0, &full[s]);
+    }
+    if (!ok) flag_timeout(a.status);
+  } else if (warp == 5 && lane == 0) {
+    const uint32_t idesc = umma_idesc_i8(BM, GEMM_BN);
+    bool ok = true;
+    for (int i = 0; i < nk && ok; ++i) {
+      const int s = i % GEMM_STAGES;
+      ok = mbar_wait(&full[s], (i / GEMM_STAGES) & 1);
+      if (!ok) break;
+      tc_fence_after();
+      const uint64_t da = umma_desc_sw128(smem_u32(smem + s * STAGE));
+      const uint64_t db = umma_desc_sw128(smem_u32(smem + s * STAGE + A_BYTES));
+#pragma unroll
+      for (int kk = 0; kk < BK / 32; ++kk) umma_i8(tmem, da + 2 * kk, db + 2 * kk, idesc, (i | kk) != 0);
+      umma_commit(&empty[s]);
+    }
+    umma_commit(&acc_full);
+    if (!ok) flag_timeout(a.status);
+  } else if (warp < 4) {
+    const bool ok = mbar_wait(&acc_full, 0);
+    tc_fence_after();
+    if (!ok && lane == 0) flag_timeout(a.status);
+    const int mi = m0 + warp * 32 + lane;
+    int m = -1;
+    if (mi < a.M) m = a.out_idx ? a.out_idx[mi] : mi;
+    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+    for (int c0 = 0; c0 < GEMM_BN; c0 += 32) {
+      int r[32];
+      tmem_ld32(taddr + c0, r);
+      tmem_ld_wait();
+      const int j0 = n0 + c0;
+      if (!ok || m < 0 || j0 >= a.J) continue;
+      if (a.epi == EPI_I32) {
+        int32_t* o = reinterpret_cast<int32_t*>(a.out) + (long long)m * a.ldo + j0;
+        if (j0 + 32 <= a.J) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) *reinterpret_cast<int4*>(o + i) = make_int4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+        } else {
+          for (int i = 0; i < 32 && j0 + i < a.J; ++i) o[i] = r[i];
+        }
+      } else {
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int j = min(j0 + i, a.J - 1);
+          v[i] = __fmaf_rn((float)r[i], __fmul_rn(a.x_scale, __ldg(a.w_scale + j)), a.bias ? __ldg(a.bias + j) : 0.0f);
+        }
+        if (a.epi == EPI_F32) {
+          float* o = reinterpret_cast<float*>(a.out) + (long long)m * a.ldo + j0;
+          if (j0 + 32 <= a.J) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(o + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+          } else {
+            for (int i = 0; i < 32 && j0 + i < a.J; ++i) o[i] = v[i];
+          }
+        } else {  // EPI_QUANT / EPI_QUANT8 (J a multiple of 32)
+          const int lo = act_lo(a.out_act), hi = act_hi(a.out_act);
+          uint8_t* o = reinterpret_cast<uint8_t*>(a.out) + (long long)m * a.ldo;
+          if (a.epi == EPI_QUANT8) {
+            uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              w[i >> 2] |= (uint32_t)((quantize1(v[i], a.out_act.inv_scale, a.out_act.zero_point, lo, hi) -
+                                       a.out_act.zero_point) & 0xFF) << (8 * (i & 3));
+            *reinterpret_cast<uint4*>(o + j0) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(o + j0 + 16) = make_uint4(w[4], w[5], w[6], w[7]);
+          } else if (a.out_act.bits == 4) {
+            uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              w[i >> 3] |= (uint32_t)(quantize1(v[i], a.out_act.inv_scale, a.out_act.zero_point, lo, hi) & 0xF) << (4 * (i & 7));
+            *reinterpret_cast<uint4*>(o + (j0 >> 1)) = make_uint4(w[0], w[1], w[2], w[3]);
+          } else {
+            uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              w[i >> 2] |= (uint32_t)(quantize1(v[i], a.out_act.inv_scale, a.out_act.zero_point, lo, hi) & 0xFF) << (8 * (i & 3));
+            *reinterpret_cast<uint4*>(o + j0) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(o + j0 + 16) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, GEMM_BN);
+}
+
+// x8: int8 activations [M, K] (pitch x_pitch), w8: int8 weights [J, K] (pitch w_pitch).
+cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const int8_t* w8,
+                            long long w_pitch, int J, int K, int epi, void* out, long long ldo,
+                            const int32_t* out_idx, const float* w_scale, const float* bias,
+                            float x_scale, const q4_act* out_act, int32_t* status, cudaStream_t s) {
+  if (M <= 0 || J <= 0) return cudaSuccess;
+  CUtensorMap ta, tb;
+  if (!make_tmap_i8(&ta, x8, K, M, x_pitch, BM) || !make_tmap_i8(&tb, w8, K, J, w_pitch, GEMM_BN))
+    return cudaErrorInvalidValue;
+  MmaGemmArgs a;
+  memset(&a, 0, sizeof(a));
+  a.M = M;
+  a.J = J;
+  a.K = K;
+  a.epi = epi;
+  a.out = out;
+  a.ldo = ldo;
+  a.out_idx = out_idx;
+  a.w_scale = w_scale;
+  a.bias = bias;
+  a.x_scale = x_scale;
+  if (out_act) a.out_act = *out_act;
+  a.status = status;
+  const size_t smem = (size_t)GEMM_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_mma_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid((M + BM - 1) / BM, (J + GEMM_BN - 1) / GEMM_BN);
+  timing_begin(s);
+  k_mma_gemm<<<grid, 192, smem, s>>>(ta, tb, a);
+  timing_end(s);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ fused LSTM step
+__global__ void __launch_bounds__(32 * (LSTM_EPI_WARPS + 2), 2)
+k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ CUtensorMap tma_xw,
+           const __grid_constant__ CUtensorMap tma_ha, const __grid_constant__ CUtensorMap tma_hw,
+           const MmaLstmArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr int A_BYTES = BM * BK, B_BYTES = LSTM_BN * BK, STAGE = A_BYTES + B_BYTES;
+  constexpr int TCOLS = 2 * LSTM_BN;
+  __shared__ uint64_t full[LSTM_STAGES], empty[LSTM_STAGES], acc_full;
+  __shared__ uint32_t tmem_base_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * LSTM_BN;
+  const int nkx = a.acc_pre ? 0 : (a.Kx_pad + BK - 1) / BK;
+  const int nkh = (a.H + BK - 1) / BK;
+  const int nk = nkx + nkh;
+
+  if (tid == 0) {
+    for (int s = 0; s < LSTM_STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(&acc_full, 1);
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == LSTM_EPI_WARPS + 1) tmem_alloc(&tmem_base_s, TCOLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_s;
+
+  if (warp == LSTM_EPI_WARPS && lane == 0) {
+    bool ok = true;
+    for (int i = 0; i < nk && ok; ++i) {
+      const int s = i % LSTM_STAGES;
+      if (i >= LSTM_STAGES) ok = mbar_wait(&empty[s], ((i / LSTM_STAGES) - 1) & 1);
+      if (!ok) break;
+      mbar_expect_tx(&full[s], STAGE);
+      if (i < nkx) {
+        tma_load_2d(smem + s * STAGE, &tma_xa, i * BK, m0, &full[s]);
+        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_xw, i * BK, n0, &full[s]);
+      } else {
+        tma_load_2d(smem + s * STAGE, &tma_ha, (i - nkx) * BK, m0, &full[s]);
+        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_hw, (i - nkx) * BK, n0, &full[s]);
+      }
+    }
+    if (!ok) flag_timeout(a.status);
+  } else if (warp == LSTM_EPI_WARPS + 1 && lane == 0) {
+    const uint32_t idesc = umma_idesc_i8(BM, LSTM_BN);
+    bool ok = true;
+    for (int i = 0; i < nk && ok; ++i) {
+      const int s = i % LSTM_STAGES;
+      ok = mbar_wait(&full[s], (i / LSTM_STAGES) & 1);
+      if (!ok) break;
+      tc_fence_after();
+      const uint64_t da = umma_desc_sw128(smem_u32(smem + s * STAGE));
+      const uint64_t db = umma_desc_sw128(smem_u32(smem + s * STAGE + A_BYTES));
+      const bool xpart = i < nkx;
+      const uint32_t d = tmem + (xpart ? 0 : LSTM_BN);
+      const int first = xpart ? 0 : nkx;
+#pragma unroll
+      for (int kk = 0; kk < BK / 32; ++kk) umma_i8(d, da + 2 * kk, db + 2 * kk, idesc, (i != first) || kk != 0);
+      umma_commit(&empty[s]);
+    }
+    umma_commit(&acc_full);
+    if (!ok) flag_timeout(a.status);
+  } else if (warp < LSTM_EPI_WARPS) {
+    const int q = warp & 3, hf = warp >> 2;
+    const int rt = q * 32 + lane;            // row within the tile
+    const int n = m0 + rt;                   // row of this launch
+    int src = -1, dst = -1;
+    if (n < a.N) {
+      dst = a.dst_row ? a.dst_row[n] : n;
+      src = a.src_row ? a.src_row[n] : n;
+    }
+    const bool ok = mbar_wait(&acc_full, 0);
+    tc_fence_after();
+    if (!ok && lane == 0) flag_timeout(a.status);
+    const bool live = ok && dst >= 0;
+    const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
+    const int H = a.H;
+    const float sx = (live && a.x_scale_vec) ? a.x_scale_vec[n % a.x_scale_mod] : a.x_scale;
+    const float sh = a.hid_act.scale;
+    const int hlo = act_lo(a.hid_act), hhi = act_hi(a.hid_act);
+    const int ylo = act_lo(a.out_act), yhi = act_hi(a.out_act);
+    constexpr int CELLS_PER_HALF = LSTM_BN / 4 / 2;   // 16
+#pragma unroll 1
+    for (int ch = 0; ch < CELLS_PER_HALF / 4; ++ch) {
+      const int ct = hf * CELLS_PER_HALF + ch * 4;     // first cell of the chunk within the tile
+      const int cell0 = (n0 >> 2) + ct;
+      int ih[16], hh[16];
+      if (nkx > 0) {
+        tmem_ld16(taddr + 4 * ct, ih);
+      }
+      tmem_ld16(taddr + LSTM_BN + 4 * ct, hh);
+      tmem_ld_wait();
+      if (!live || cell0 >= H) continue;
+      if (nkx == 0) {
+        const int4* p = reinterpret_cast<const int4*>(a.acc_pre + (long long)n * a.acc_pre_ld + 4 * cell0);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int4 v = p[c];
+          ih[4 * c] = v.x;
+          ih[4 * c + 1] = v.y;
+          ih[4 * c + 2] = v.z;
+          ih[4 * c + 3] = v.w;
+        }
+      }
+      float4 cprev = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (src >= 0) cprev = *reinterpret_cast<const float4*>(a.c_in + (long long)src * H + cell0);
+      const float cp[4] = {cprev.x, cprev.y, cprev.z, cprev.w};
+      float cn[4], hn[4];
+      int qh[4], qy[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int cell = cell0 + c;
+        const float4 s_ih = __ldg(reinterpret_cast<const float4*>(a.sc_ih) + cell);
+        const float4 s_hh = __ldg(reinterpret_cast<const float4*>(a.sc_hh) + cell);
+        const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias) + cell);
+        const float pi = __fmaf_rn((float)hh[4 * c + 0], __fmul_rn(sh, s_hh.x), __fmaf_rn((float)ih[4 * c + 0], __fmul_rn(sx, s_ih.x), bb.x));
+        const float pf = __fmaf_rn((float)hh[4 * c + 1], __fmul_rn(sh, s_hh.y), __fmaf_rn((float)ih[4 * c + 1], __fmul_rn(sx, s_ih.y), bb.y));
+        const float pg = __fmaf_rn((float)hh[4 * c + 2], __fmul_rn(sh, s_hh.z), __fmaf_rn((float)ih[4 * c + 2], __fmul_rn(sx, s_ih.z), bb.z));
+        const float po = __fmaf_rn((float)hh[4 * c + 3], __fmul_rn(sh, s_hh.w), __fmaf_rn((float)ih[4 * c + 3], __fmul_rn(sx, s_ih.w), bb.w));
+        const float ig = sigmoid_fixed(pi), fg = sigmoid_fixed(pf), gg = tanh_fixed(pg), og = sigmoid_fixed(po);
+        cn[c] = __fmaf_rn(fg, cp[c], __fmul_rn(ig, gg));
+        hn[c] = __fmul_rn(og, tanh_fixed(cn[c]));
+        qh[c] = quantize1(hn[c], a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
+        qy[c] = quantize1(hn[c], a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
+        if (a.dbg_ih) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            a.dbg_ih[(long long)n * a.dbg_ld + g * H + cell] = ih[4 * c + g];
+            a.dbg_hh[(long long)n * a.dbg_ld + g * H + cell] = hh[4 * c + g];
+          }
+        }
+      }
+      *reinterpret_cast<float4*>(a.c_out + (long long)dst * H + cell0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
+      if (a.h_f32) *reinterpret_cast<float4*>(a.h_f32 + (long long)n * H + cell0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+      if (a.hq_out) {
+        if (a.hid_act.bits == 4)
+          *reinterpret_cast<uint16_t*>(a.hq_out + (long long)dst * a.hq_ld + (cell0 >> 1)) =
+              (uint16_t)((qh[0] & 0xF) | ((qh[1] & 0xF) << 4) | ((qh[2] & 0xF) << 8) | ((qh[3] & 0xF) << 12));
+        else
+          *reinterpret_cast<uint32_t*>(a.hq_out + (long long)dst * a.hq_ld + cell0) =
+              (uint32_t)(qh[0] & 0xFF) | ((uint32_t)(qh[1] & 0xFF) << 8) | ((uint32_t)(qh[2] & 0xFF) << 16) | ((uint32_t)(qh[3] & 0xFF) << 24);
+      }
+      if (a.h8_out)
+        *reinterpret_cast<uint32_t*>(a.h8_out + (long long)n * a.h8_ld + cell0) =
+            (uint32_t)(qh[0] & 0xFF) | ((uint32_t)(qh[1] & 0xFF) << 8) | ((uint32_t)(qh[2] & 0xFF) << 16) | ((uint32_t)(qh[3] & 0xFF) << 24);
+      if (a.yq_out) {
+        if (a.out_act.bits == 4)
+          *reinterpret_cast<uint16_t*>(a.yq_out + (long long)n * a.yq_ld + (cell0 >> 1)) =
+              (uint16_t)((qy[0] & 0xF) | ((qy[1] & 0xF) << 4) | ((qy[2] & 0xF) << 8) | ((qy[3] & 0xF) << 12));
+        else
+          *reinterpret_cast<uint32_t*>(a.yq_out + (long long)n * a.yq_ld + cell0) =
+              (uint32_t)(qy[0] & 0xFF) | ((uint32_t)(qy[1] & 0xFF) << 8) | ((uint32_t)(qy[2] & 0xFF) << 16) | ((uint32_t)(qy[3] & 0xFF) << 24);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == LSTM_EPI_WARPS + 1) tmem_dealloc(tmem, TCOLS);
+}
+
+// Operands: xa int8 [rows_pad, Kx_pad] (ignored with acc_pre), xw int8 [4H, Kx_pad] interleaved,
+// ha int8 [rows_pad, H], hw int8 [4H, H] interleaved.  rows_pad = N rounded up to 128.
+cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa_pitch,
+                            const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
+                            const int8_t* hw, long long hw_pitch, cudaStream_t s) {
+  if (a.N <= 0) return cudaSuccess;
+  const int rows_pad = (a.N + BM - 1) / BM * BM;
+  CUtensorMap txa, txw, tha, thw;
+  if (!make_tmap_i8(&tha, ha, a.H, rows_pad, ha_pitch, BM) || !make_tmap_i8(&thw, hw, a.H, 4 * a.H, hw_pitch, LSTM_BN))
+    return cudaErrorInvalidValue;
+  if (a.acc_pre) {
+    txa = tha;
+    txw = thw;
+  } else if (!make_tmap_i8(&txa, xa, a.Kx_pad, rows_pad, xa_pitch, BM) ||
+             !make_tmap_i8(&txw, xw, a.Kx_pad, 4 * a.H, xw_pitch, LSTM_BN)) {
+    return cudaErrorInvalidValue;
+  }
+  const size_t smem = (size_t)LSTM_STAGES * (BM * BK + LSTM_BN * BK) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_mma_lstm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid(rows_pad / BM, (4 * a.H + LSTM_BN - 1) / LSTM_BN);
+  timing_begin(s);
+  k_mma_lstm<<<grid, 32 * (LSTM_EPI_WARPS + 2), smem, s>>>(txa, txw, tha, thw, a);
+  timing_end(s);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
+}  // namespace q4

@@ -108,8 +108,13 @@ def layer_case(Bd, T, B, K, H, dirs, xb=4, hb=4, ob=None, seed=0, x_clip=3.0, ma
     layers = [Bd.DeviceLstm(lw) for lw in w["layers"]]
     got = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), x_act), to_act(x_act), T, B, layers,
                                  to_act(out), want_state=True, want_dbg=True)
+    assert Bd.q4_poll_status(got["workspace"]) == 0          # no bounded wait expired
     # input accumulators depend on the input only: bit-exact over the whole sequence
     np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), ref["acc_ih"])
+    if T * B >= 128:                                         # tensor-core and DP4A projections agree
+        alt = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), x_act), to_act(x_act), T, B, layers,
+                                     to_act(out), want_dbg=True, tensor_cores=False)
+        assert torch.equal(alt["acc_ih"], got["acc_ih"]) and torch.equal(alt["yq"], got["yq"])
     yq = gpu_codes(got["yq"], dirs * H, out).reshape(T, B, dirs * H)
     # free-running over the whole sequence and still bit-exact: codes, accumulators, states
     np.testing.assert_array_equal(yq, ref["yq"])
