@@ -178,7 +178,16 @@ typedef struct {
   q4_act z_act;
   q4_linear joint_out; /* D -> V */
   q4_lm src, tgt;
+  void* prepared; /* NULL, or the buffer filled by q4_prepare_model (tensor-core operands) */
 } q4_model;
+
+/* Optional one-time weight preparation for the tensor-core search path (weights are
+ * quantized once, activations at every step: Section 3.2).  Writes int8, gate-interleaved
+ * copies of the step weights into `buffer` (device, q4_prepared_bytes(model) bytes, owned by
+ * the caller, must outlive the model's use) and sets model->prepared.  With prepared == NULL
+ * the search uses the DP4A kernels on the packed weights. */
+size_t q4_prepared_bytes(const q4_model* model);
+int q4_prepare_model(q4_model* model, void* buffer, size_t bytes, q4_stream stream);
 
 /*
  * Caller-owned search state for B utterances x W beam slots.  R = B * 2W "state rows" hold
@@ -237,7 +246,9 @@ int q4_beam_init(q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters, q4
  *      W best others (score descending, then parent slot, then token) become the next beam.
  * e [T, B, D] fp32 projected encoder frames.  `iter` counts from 0; hypotheses in the beam
  * entering iteration `iter` satisfy t + u = iter.  mode: 0 (the only one implemented).
- * workspace: q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D}).
+ * workspace: q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D}), or, to enable the tensor-core path
+ * (needs model->prepared and B*W >= 128), q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D, E_pad, Hp,
+ * Hs, Ht}).  A bounded device wait that expires sets state->status to Q4_ERR_TIMEOUT.
  */
 int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float* e, int32_t B,
                         int32_t T, int32_t W, int32_t iter, int32_t u_max, float lambda_t,
@@ -260,7 +271,7 @@ int q4_feature_prologue(const float* mel, int32_t B, int32_t T100, int32_t M, vo
 
 #define Q4_WS_LSTM_LAYER 1 /* dims = {T, B, dirs, H} or {T, B, dirs, H, kx_pad} */
 #define Q4_WS_JOINT 2      /* dims = {N, D} */
-#define Q4_WS_BEAM 3       /* dims = {B, W, V, D} */
+#define Q4_WS_BEAM 3       /* dims = {B, W, V, D} or {B, W, V, D, E_pad, Hp, Hs, Ht} */
 size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims);
 
 /* Synchronise `stream`, read the device status word and return 0 or the error it holds. */

@@ -54,7 +54,8 @@ class LmS(C.Structure):
 class ModelS(C.Structure):
     _fields_ = [("V", C.c_int32), ("E", C.c_int32), ("D", C.c_int32), ("pred_emb_q", C.c_void_p),
                 ("pred_emb_act", Act), ("pred_lstm", LstmS), ("pred_proj", LinearS),
-                ("z_act", Act), ("joint_out", LinearS), ("src", LmS), ("tgt", LmS)]
+                ("z_act", Act), ("joint_out", LinearS), ("src", LmS), ("tgt", LmS),
+                ("prepared", C.c_void_p)]
 
 
 class BeamStateS(C.Structure):
@@ -72,7 +73,7 @@ class BeamStateS(C.Structure):
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
-           "q4_poll_status", "q4_version", "q4_launch_count", "q4_timing_set", "q4_timing_count"]
+           "q4_poll_status", "q4_version", "q4_launch_count", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model"]
 
 _lib = None
 
@@ -87,6 +88,7 @@ def lib() -> C.CDLL:
         _lib = C.CDLL(LIB_PATH)
         _lib.q4_workspace_bytes.restype = C.c_size_t
         _lib.q4_launch_count.restype = C.c_int64
+        _lib.q4_prepared_bytes.restype = C.c_size_t
     return _lib
 
 
@@ -389,9 +391,10 @@ class Decoder:
     """Device copy of prediction network, joint network and both fusion LMs, the search
     state, and the iteration loop (one library call per search iteration)."""
 
-    def __init__(self, dw, device="cuda"):
+    def __init__(self, dw, device="cuda", tensor_cores: bool = True):
         self.dw = dw
         self.device = device
+        self.tensor_cores = tensor_cores
         self.V, self.E = dw.pred.emb.shape
         self.pred_emb_act = q4_act_symmetric(dw.pred.emb_alpha, 4)
         emb = torch.from_numpy(np.ascontiguousarray(dw.pred.emb, dtype=np.float32)).to(device)
@@ -408,7 +411,18 @@ class Decoder:
         m.pred_lstm, m.pred_proj = self.pred_lstm.c(), self.pred_proj.c()
         m.z_act, m.joint_out = self.z_act, self.joint_out.c()
         m.src, m.tgt = self.src.c(), self.tgt.c()
+        m.prepared = None
+        self.prepared = None
+        if tensor_cores:
+            self.q4_prepare_model()
         self.state = None
+
+    def q4_prepare_model(self):
+        """One-time int8 / gate-interleaved copies of the step weights for the tensor cores."""
+        n = int(lib().q4_prepared_bytes(C.byref(self.model)))
+        self.prepared = torch.empty(n, dtype=torch.uint8, device=self.device)
+        _chk(lib().q4_prepare_model(C.byref(self.model), _p(self.prepared), C.c_size_t(n), _stream()),
+             "q4_prepare_model")
 
     def step_weight_bytes(self) -> int:
         return (self.pred_lstm.nbytes() + self.pred_proj.nbytes() + self.joint_out.nbytes() +
@@ -445,8 +459,10 @@ class Decoder:
         s.tgt_hq[0], s.tgt_hq[1] = t["tgt_hq0"].data_ptr(), t["tgt_hq1"].data_ptr()
         s.tgt_c[0], s.tgt_c[1] = t["tgt_c0"].data_ptr(), t["tgt_c1"].data_ptr()
         self.B, self.W, self.n_iters = B, W, n_iters
-        self.ws = torch.empty(workspace_bytes(WS_BEAM, [B, W, self.V, self.D]), dtype=torch.uint8,
-                              device=dev)
+        dims = [B, W, self.V, self.D]
+        if self.tensor_cores:
+            dims += [self.pred_lstm.w_ih.k_pad, Hp, Hs, Ht]
+        self.ws = torch.empty(workspace_bytes(WS_BEAM, dims), dtype=torch.uint8, device=dev)
 
     def q4_beam_init(self):
         _chk(lib().q4_beam_init(C.byref(self.state), C.c_int32(self.B), C.c_int32(self.W),

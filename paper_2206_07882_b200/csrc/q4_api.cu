@@ -139,7 +139,16 @@ size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims) {
   }
   if (call_id == Q4_WS_BEAM && ndims >= 4) {
     const size_t N = (size_t)dims[0] * dims[1], V = dims[2], D = dims[3];
-    return align_up(N * D) * 3 + align_up(N * V * sizeof(float)) + align_up(N * sizeof(int32_t));
+    size_t n = align_up(N * D) * 3 + align_up(N * V * sizeof(float)) + align_up(N * sizeof(int32_t));
+    if (ndims >= 8) {  // int8 operand scratch of the tensor-core path
+      const size_t Np = (N + 127) / 128 * 128;
+      const size_t E = dims[4], Hp = dims[5], Hs = dims[6], Ht = dims[7];
+      const size_t Hmax = Hp > Hs ? (Hp > Ht ? Hp : Ht) : (Hs > Ht ? Hs : Ht);
+      n += align_up(Np * E) + align_up(Np * Hmax);                       // gathered x / h operands
+      n += align_up(Np * Hp) + align_up(Np * Hs) + 2 * align_up(Np * Ht); // new cell outputs, int8
+      n += 3 * align_up(Np * D);                                         // bottleneck codes, z codes
+    }
+    return n;
   }
   return 0;
 }
@@ -393,7 +402,7 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
   GemmArgs g1 = gemm_args(pq, row_bytes(w_pred->k_pad, w_pred->bits), nullptr, *p_act, N, *w_pred,
                           b_pred, p, D, nullptr);
   Q4_TRY(launch_gemm(g1, w_pred->bits, EPI_F32, s));
-  Q4_TRY(launch_joint_z(e, frame_idx, nullptr, 1, 1, p, nullptr, N, D, *z_act, zq, nullptr, s));
+  Q4_TRY(launch_joint_z(e, frame_idx, nullptr, 1, 1, p, nullptr, N, D, *z_act, zq, nullptr, nullptr, s));
   GemmArgs g2 = gemm_args(zq, row_bytes(D, z_act->bits), nullptr, *z_act, N, *w_out, b_out, logp, V,
                           nullptr);
   Q4_TRY(launch_gemm(g2, w_out->bits, EPI_F32, s));
@@ -407,6 +416,96 @@ int q4_feature_prologue(const float* mel, int32_t B, int32_t T100, int32_t M, vo
   if (B <= 0 || T100 < 2 || M <= 0) return Q4_ERR_DIM;
   TagScope tag(TAG_MISC);
   Q4_TRY(launch_features(mel, B, T100, M, out_fp16, S(stream)));
+  return Q4_OK;
+}
+
+// ------------------------------------------------------------------------ prepared weights
+namespace {
+struct PrepLstm {
+  size_t xw, hw, sc_ih, sc_hh, bias;
+};
+struct PrepPlan {
+  PrepLstm lstm[4];   // prediction, source LM, target LM layer 1, target LM layer 2
+  size_t lin[6];      // pred_proj, src.bott, src.out, tgt.bott, tgt.out, joint_out
+  size_t total;
+};
+const q4_lstm* model_lstm(const q4_model& m, int i) {
+  switch (i) {
+    case 0: return &m.pred_lstm;
+    case 1: return &m.src.lstm[0];
+    case 2: return &m.tgt.lstm[0];
+    default: return m.tgt.n_layers == 2 ? &m.tgt.lstm[1] : nullptr;
+  }
+}
+const q4_linear* model_linear(const q4_model& m, int i) {
+  switch (i) {
+    case 0: return &m.pred_proj;
+    case 1: return &m.src.bott;
+    case 2: return &m.src.out;
+    case 3: return &m.tgt.bott;
+    case 4: return &m.tgt.out;
+    default: return &m.joint_out;
+  }
+}
+PrepPlan plan_prepared(const q4_model& m) {
+  PrepPlan p;
+  memset(&p, 0, sizeof(p));
+  size_t o = 0;
+  for (int i = 0; i < 4; ++i) {
+    const q4_lstm* L = model_lstm(m, i);
+    if (!L) continue;
+    const size_t G = L->w_ih.rows;
+    p.lstm[i].xw = o;
+    o += align_up(G * L->w_ih.k_pad);
+    p.lstm[i].hw = o;
+    o += align_up(G * L->w_hh.k_pad);
+    p.lstm[i].sc_ih = o;
+    o += align_up(G * sizeof(float));
+    p.lstm[i].sc_hh = o;
+    o += align_up(G * sizeof(float));
+    p.lstm[i].bias = o;
+    o += align_up(G * sizeof(float));
+  }
+  for (int i = 0; i < 6; ++i) {
+    const q4_linear* L = model_linear(m, i);
+    p.lin[i] = o;
+    o += align_up((size_t)L->w.rows * L->w.k_pad);
+  }
+  p.total = o;
+  return p;
+}
+}  // namespace
+
+size_t q4_prepared_bytes(const q4_model* model) {
+  if (!model) return 0;
+  return plan_prepared(*model).total;
+}
+
+int q4_prepare_model(q4_model* model, void* buffer, size_t bytes, q4_stream stream) {
+  if (!model || !buffer) return Q4_ERR_NULL;
+  if (!aligned16(buffer)) return Q4_ERR_ALIGN;
+  const PrepPlan p = plan_prepared(*model);
+  if (bytes < p.total) return Q4_ERR_WORKSPACE;
+  cudaStream_t s = S(stream);
+  uint8_t* b = static_cast<uint8_t*>(buffer);
+  TagScope tag(TAG_MISC);
+  for (int i = 0; i < 4; ++i) {
+    const q4_lstm* L = model_lstm(*model, i);
+    if (!L) continue;
+    Q4_CHECK(check_mat(&L->w_ih, 0, 0));
+    Q4_CHECK(check_mat(&L->w_hh, 0, 0));
+    Q4_TRY(launch_prepare_w(L->w_ih, 1, reinterpret_cast<int8_t*>(b + p.lstm[i].xw), L->w_ih.k_pad, 0, s));
+    Q4_TRY(launch_prepare_w(L->w_hh, 1, reinterpret_cast<int8_t*>(b + p.lstm[i].hw), L->w_hh.k_pad, 0, s));
+    Q4_TRY(launch_prepare_vec(L->w_ih.scale, L->w_ih.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].sc_ih), s));
+    Q4_TRY(launch_prepare_vec(L->w_hh.scale, L->w_hh.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].sc_hh), s));
+    Q4_TRY(launch_prepare_vec(L->bias, L->w_ih.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].bias), s));
+  }
+  for (int i = 0; i < 6; ++i) {
+    const q4_linear* L = model_linear(*model, i);
+    Q4_CHECK(check_mat(&L->w, 0, 0));
+    Q4_TRY(launch_prepare_w(L->w, 0, reinterpret_cast<int8_t*>(b + p.lin[i]), L->w.k_pad, 0, s));
+  }
+  model->prepared = buffer;
   return Q4_OK;
 }
 
@@ -513,53 +612,175 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   ws += align_up((size_t)N * V * sizeof(float));
   int32_t* live = reinterpret_cast<int32_t*>(ws);
 
-  // 1. pending advances -------------------------------------------------------------
-  {  // prediction network: embedding row -> LSTM -> projection to D
-    const q4_lstm& L = m.pred_lstm;
-    Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), st.adv_tok,
-                          m.pred_emb_act, st.pred_hq, st.pred_c, st, N, s));
-    GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), st.adv_dst,
-                           L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, st.adv_dst);
-    TagScope tag(TAG_PRED_PROJ);
-    Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
-  }
-  for (int which = 0; which < 2; ++which) {
-    const q4_lm& lm = *lms[which];
-    void* hq0 = which == 0 ? st.src_hq : st.tgt_hq[0];
-    float* c0 = which == 0 ? st.src_c : st.tgt_c[0];
-    float* lp = which == 0 ? st.src_lp : st.tgt_lp;
-    uint8_t* bq = which == 0 ? bq_src : bq_tgt;
-    const q4_lstm& L0 = lm.lstm[0];
-    Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), st.adv_tok,
-                          lm.emb_act, hq0, c0, st, N, s));
-    const void* top = hq0;
-    const q4_lstm* last = &L0;
-    if (lm.n_layers == 2) {
-      if (which == 0) return Q4_ERR_UNSUPPORTED;  // the state block holds one source-LM layer
-      const q4_lstm& L1 = lm.lstm[1];
-      Q4_CHECK(advance_lstm(TAG_TGT_L2, L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), st.adv_dst,
-                            L0.hid_act, st.tgt_hq[1], st.tgt_c[1], st, N, s));
-      top = st.tgt_hq[1];
-      last = &L1;
-    }
-    GemmArgs gb = gemm_args(top, row_bytes(last->w_hh.k_pad, last->hid_act.bits), st.adv_dst,
-                            last->hid_act, N, lm.bott.w, lm.bott.bias, bq,
-                            row_bytes(D, lm.bott_act.bits), nullptr);
-    gb.out_act = lm.bott_act;
-    TagScope tag(which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD);
-    Q4_TRY(launch_gemm(gb, lm.bott.w.bits, EPI_QUANT, s));
-    GemmArgs go = gemm_args(bq, row_bytes(D, lm.bott_act.bits), nullptr, lm.bott_act, N, lm.out.w,
-                            lm.out.bias, lp, V, st.adv_dst);
-    Q4_TRY(launch_gemm(go, lm.out.w.bits, EPI_F32, s));
-    Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, st.adv_dst, s));
-  }
+  // tensor-core path: prepared int8 weights, enough rows to fill 128-row tiles, and room
+  // for the int8 operand scratch
+  const int Hp = m.pred_lstm.w_hh.k_pad, Hs = m.src.lstm[0].w_hh.k_pad, Ht = m.tgt.lstm[0].w_hh.k_pad;
+  const int Ep = m.pred_lstm.w_ih.k_pad;
+  const int32_t dims8[8] = {B, W, V, D, Ep, Hp, Hs, Ht};
+  const bool use_mma = m.prepared != nullptr && N >= 128 && m.src.n_layers == 1 &&
+                       m.src.lstm[0].w_ih.k_pad == Ep && m.tgt.lstm[0].w_ih.k_pad == Ep &&
+                       Hp % 128 == 0 && Hs % 128 == 0 && Ht % 128 == 0 && V % 32 == 0 &&
+                       workspace_bytes >= q4_workspace_bytes(Q4_WS_BEAM, dims8, 8);
+  if (use_mma) {
+    ws += align_up((size_t)N * sizeof(int32_t));
+    const size_t Np = ((size_t)N + 127) / 128 * 128;
+    const int Hmax = Hp > Hs ? (Hp > Ht ? Hp : Ht) : (Hs > Ht ? Hs : Ht);
+    int8_t* xa8 = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * Ep);
+    int8_t* ha8 = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * Hmax);
+    int8_t* pred_h8 = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * Hp);
+    int8_t* src_h8 = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * Hs);
+    int8_t* tgt_h8[2];
+    tgt_h8[0] = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * Ht);
+    tgt_h8[1] = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * Ht);
+    int8_t* bq8[2];
+    bq8[0] = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * D);
+    bq8[1] = reinterpret_cast<int8_t*>(ws);
+    ws += align_up(Np * D);
+    int8_t* z8 = reinterpret_cast<int8_t*>(ws);
+    const PrepPlan pp = plan_prepared(m);
+    const uint8_t* pb = static_cast<const uint8_t*>(m.prepared);
 
-  // 2. joint network for every live slot at its frame -----------------------------------
-  TagScope tag_joint(TAG_JOINT);
-  Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, zq, live, s));
-  GemmArgs gj = gemm_args(zq, row_bytes(D, m.z_act.bits), live, m.z_act, N, m.joint_out.w,
-                          m.joint_out.bias, logits, V, nullptr);
-  Q4_TRY(launch_gemm(gj, m.joint_out.w.bits, EPI_F32, s));
+    // one LSTM layer of one network for every pending slot
+    auto lstm_mma = [&](int tag_id, int li, const q4_lstm& L, const q4_act& x_act, const void* x_src,
+                        long long x_stride, const int32_t* x_idx, const int8_t* x_ready, void* hq,
+                        float* c, int8_t* h8) -> int {
+      TagScope tag(tag_id);
+      const int H = L.w_hh.k_pad, Kx = L.w_ih.k_pad;
+      const int8_t* xa = x_ready;
+      if (!xa) {
+        Q4_TRY(launch_unpack_rows(x_src, x_stride, x_idx, x_act, Kx, N, xa8, Kx, 0, (int)Np, s));
+        xa = xa8;
+      }
+      Q4_TRY(launch_unpack_rows(hq, row_bytes(H, L.hid_act.bits), st.adv_src, L.hid_act, H, N, ha8, H, 0,
+                                (int)Np, s));
+      MmaLstmArgs a;
+      memset(&a, 0, sizeof(a));
+      a.N = N;
+      a.H = H;
+      a.Kx_pad = Kx;
+      a.sc_ih = reinterpret_cast<const float*>(pb + pp.lstm[li].sc_ih);
+      a.sc_hh = reinterpret_cast<const float*>(pb + pp.lstm[li].sc_hh);
+      a.bias = reinterpret_cast<const float*>(pb + pp.lstm[li].bias);
+      a.x_scale = x_act.scale;
+      a.hid_act = L.hid_act;
+      a.out_act = L.hid_act;
+      a.src_row = st.adv_src;
+      a.dst_row = st.adv_dst;
+      a.c_in = c;
+      a.c_out = c;
+      a.hq_out = static_cast<uint8_t*>(hq);
+      a.hq_ld = row_bytes(H, L.hid_act.bits);
+      a.h8_out = h8;
+      a.h8_ld = H;
+      a.status = st.status;
+      Q4_TRY(launch_mma_lstm(a, xa, Kx, reinterpret_cast<const int8_t*>(pb + pp.lstm[li].xw), Kx, ha8, H,
+                             reinterpret_cast<const int8_t*>(pb + pp.lstm[li].hw), H, s));
+      return Q4_OK;
+    };
+    auto linear_mma = [&](int tag_id, int wi, const q4_linear& L, const int8_t* x8, float x_scale,
+                          int epi, void* out, long long ldo, const int32_t* out_idx,
+                          const q4_act* out_act) -> int {
+      TagScope tag(tag_id);
+      Q4_TRY(launch_mma_gemm(x8, L.w.k_pad, N, reinterpret_cast<const int8_t*>(pb + pp.lin[wi]), L.w.k_pad,
+                             L.w.rows, L.w.k_pad, epi, out, ldo, out_idx, L.w.scale, L.bias, x_scale, out_act,
+                             st.status, s));
+      return Q4_OK;
+    };
+
+    // 1. pending advances
+    Q4_CHECK(lstm_mma(TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, m.pred_emb_q,
+                      row_bytes(Ep, m.pred_lstm.w_ih.bits), st.adv_tok, nullptr, st.pred_hq, st.pred_c,
+                      pred_h8));
+    Q4_CHECK(linear_mma(TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
+                        st.pred_p, D, st.adv_dst, nullptr));
+    for (int which = 0; which < 2; ++which) {
+      const q4_lm& lm = *lms[which];
+      const q4_lstm& L0 = lm.lstm[0];
+      void* hq0 = which == 0 ? st.src_hq : st.tgt_hq[0];
+      float* c0 = which == 0 ? st.src_c : st.tgt_c[0];
+      int8_t* h8_0 = which == 0 ? src_h8 : tgt_h8[0];
+      float* lp = which == 0 ? st.src_lp : st.tgt_lp;
+      Q4_CHECK(lstm_mma(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, which == 0 ? 1 : 2, L0, lm.emb_act, lm.emb_q,
+                        row_bytes(Ep, L0.w_ih.bits), st.adv_tok, nullptr, hq0, c0, h8_0));
+      const int8_t* top8 = h8_0;
+      const q4_lstm* last = &L0;
+      if (lm.n_layers == 2) {
+        const q4_lstm& L1 = lm.lstm[1];
+        Q4_CHECK(lstm_mma(TAG_TGT_L2, 3, L1, L0.hid_act, nullptr, 0, nullptr, h8_0, st.tgt_hq[1],
+                          st.tgt_c[1], tgt_h8[1]));
+        top8 = tgt_h8[1];
+        last = &L1;
+      }
+      const int head_tag = which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD;
+      Q4_CHECK(linear_mma(head_tag, which == 0 ? 1 : 3, lm.bott, top8, last->hid_act.scale, EPI_QUANT8,
+                          bq8[which], D, nullptr, &lm.bott_act));
+      Q4_CHECK(linear_mma(head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
+                          V, st.adv_dst, nullptr));
+      TagScope tag(head_tag);
+      Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, st.adv_dst, s));
+    }
+    // 2. joint network for every live slot at its frame
+    {
+      TagScope tag(TAG_JOINT);
+      Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, s));
+    }
+    Q4_CHECK(linear_mma(TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr));
+  } else {
+    // 1. pending advances -------------------------------------------------------------
+    {  // prediction network: embedding row -> LSTM -> projection to D
+      const q4_lstm& L = m.pred_lstm;
+      Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), st.adv_tok,
+                            m.pred_emb_act, st.pred_hq, st.pred_c, st, N, s));
+      GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), st.adv_dst,
+                             L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, st.adv_dst);
+      TagScope tag(TAG_PRED_PROJ);
+      Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
+    }
+    for (int which = 0; which < 2; ++which) {
+      const q4_lm& lm = *lms[which];
+      void* hq0 = which == 0 ? st.src_hq : st.tgt_hq[0];
+      float* c0 = which == 0 ? st.src_c : st.tgt_c[0];
+      float* lp = which == 0 ? st.src_lp : st.tgt_lp;
+      uint8_t* bq = which == 0 ? bq_src : bq_tgt;
+      const q4_lstm& L0 = lm.lstm[0];
+      Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), st.adv_tok,
+                            lm.emb_act, hq0, c0, st, N, s));
+      const void* top = hq0;
+      const q4_lstm* last = &L0;
+      if (lm.n_layers == 2) {
+        if (which == 0) return Q4_ERR_UNSUPPORTED;  // the state block holds one source-LM layer
+        const q4_lstm& L1 = lm.lstm[1];
+        Q4_CHECK(advance_lstm(TAG_TGT_L2, L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), st.adv_dst,
+                              L0.hid_act, st.tgt_hq[1], st.tgt_c[1], st, N, s));
+        top = st.tgt_hq[1];
+        last = &L1;
+      }
+      GemmArgs gb = gemm_args(top, row_bytes(last->w_hh.k_pad, last->hid_act.bits), st.adv_dst,
+                              last->hid_act, N, lm.bott.w, lm.bott.bias, bq,
+                              row_bytes(D, lm.bott_act.bits), nullptr);
+      gb.out_act = lm.bott_act;
+      TagScope tag(which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD);
+      Q4_TRY(launch_gemm(gb, lm.bott.w.bits, EPI_QUANT, s));
+      GemmArgs go = gemm_args(bq, row_bytes(D, lm.bott_act.bits), nullptr, lm.bott_act, N, lm.out.w,
+                              lm.out.bias, lp, V, st.adv_dst);
+      Q4_TRY(launch_gemm(go, lm.out.w.bits, EPI_F32, s));
+      Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, st.adv_dst, s));
+    }
+
+    // 2. joint network for every live slot at its frame -----------------------------------
+    TagScope tag_joint(TAG_JOINT);
+    Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, zq, nullptr, live, s));
+    GemmArgs gj = gemm_args(zq, row_bytes(D, m.z_act.bits), live, m.z_act, N, m.joint_out.w,
+                            m.joint_out.bias, logits, V, nullptr);
+    Q4_TRY(launch_gemm(gj, m.joint_out.w.bits, EPI_F32, s));
+  }
 
   // 3. Eq. 1 proposals, merge, finished list, next beam --------------------------------
   BeamSelArgs sel;

@@ -10,7 +10,8 @@ cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long
                               const int32_t* idx, cudaStream_t s);
 cudaError_t launch_joint_z(const float* e, const int32_t* frame_idx, const int32_t* t_arr, int B,
                            int W, const float* p, const int32_t* p_idx, int N, int D,
-                           const q4_act& za, uint8_t* zq, int32_t* live_out, cudaStream_t s);
+                           const q4_act& za, uint8_t* zq, int8_t* z8, int32_t* live_out,
+                           cudaStream_t s);
 cudaError_t launch_quantize(const void* x, bool fp16, long long rows, int k, int k_pad,
                             const q4_act& a, int mode, int n_groups, const float* scale_vec,
                             uint8_t* out, float* group_scale_out, cudaStream_t s);

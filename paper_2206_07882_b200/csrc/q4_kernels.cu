@@ -466,7 +466,7 @@ cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long
 __global__ void __launch_bounds__(256) k_joint_z(const float* e, const int32_t* frame_idx,
                                                  const int32_t* t_arr, int B, int W, const float* p,
                                                  const int32_t* p_idx, int N, int D, q4_act za,
-                                                 uint8_t* zq, int32_t* live_out) {
+                                                 uint8_t* zq, int8_t* z8, int32_t* live_out) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int half = D >> 1;
   if (i >= (long long)N * half) return;
@@ -482,7 +482,9 @@ __global__ void __launch_bounds__(256) k_joint_z(const float* e, const int32_t* 
     q0 = quantize1(tanh_fixed(__fmul_rn(ev.x, pv.x)), za.inv_scale, za.zero_point, lo, hi);
     q1 = quantize1(tanh_fixed(__fmul_rn(ev.y, pv.y)), za.inv_scale, za.zero_point, lo, hi);
   }
-  if (za.bits == 4) {
+  if (z8) {   // one code per byte, ready for the tensor-core GEMM
+    *reinterpret_cast<uint16_t*>(z8 + (long long)n * D + d) = (uint16_t)((q0 & 0xFF) | ((q1 & 0xFF) << 8));
+  } else if (za.bits == 4) {
     zq[(long long)n * half + (d >> 1)] = (uint8_t)((q0 & 0xF) | ((q1 & 0xF) << 4));
   } else {
     *reinterpret_cast<uint16_t*>(zq + (long long)n * D + d) = (uint16_t)((q0 & 0xFF) | ((q1 & 0xFF) << 8));
@@ -492,12 +494,13 @@ __global__ void __launch_bounds__(256) k_joint_z(const float* e, const int32_t* 
 
 cudaError_t launch_joint_z(const float* e, const int32_t* frame_idx, const int32_t* t_arr, int B,
                            int W, const float* p, const int32_t* p_idx, int N, int D,
-                           const q4_act& za, uint8_t* zq, int32_t* live_out, cudaStream_t s) {
+                           const q4_act& za, uint8_t* zq, int8_t* z8, int32_t* live_out,
+                           cudaStream_t s) {
   if (N <= 0) return cudaSuccess;
   const long long total = (long long)N * (D / 2);
   timing_begin(s);
   k_joint_z<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(e, frame_idx, t_arr, B, W, p, p_idx, N,
-                                                            D, za, zq, live_out);
+                                                            D, za, zq, z8, live_out);
   timing_end(s);
   ++g_launches;
   return cudaGetLastError();

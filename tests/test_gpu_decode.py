@@ -102,8 +102,8 @@ def test_config2_full_size_sampled_rows(Bd):
     assert np.abs(got[rows].cpu().numpy() - want).max() <= LP_ATOL
 
 
-def run_search(Bd, dw, e, utts=None):
-    dd = Bd.Decoder(dw)
+def run_search(Bd, dw, e, utts=None, tensor_cores=True):
+    dd = Bd.Decoder(dw, tensor_cores=tensor_cores)
     T, B, D = e.shape
     tokens, lens, scores = dd.decode(torch.from_numpy(e).cuda())
     torch.cuda.synchronize()
@@ -198,6 +198,18 @@ def test_config3_full_size_sampled_utterances(Bd):
     utts = [1, 14]
     dd, tokens, lens, scores, ref = run_search(Bd, dw, e, utts=utts)
     compare_search(dd, tokens, lens, scores, ref, utts, T, 8, 16, min_same=1.0)
+
+
+def test_tensor_core_and_dp4a_search_paths_agree(Bd):
+    # 8 utterances x 16 slots = 128 rows: enough for the tensor-core path; both paths must give
+    # identical beams (same integer accumulators, same fp32 operation sequence).
+    dw = synth.decoder(seed=51, V=64, E=32, Hp=128, D=32, Hs=128, Ht=256, tgt_layers=2, U_max=10, W=16)
+    e = synth.Stream(6).normal("e", (20, 8, 32)).astype(np.float32)
+    a = run_search(Bd, dw, e, tensor_cores=True)
+    b = run_search(Bd, dw, e, tensor_cores=False)
+    for k in ("bp_parent", "bp_token", "bp_score", "fin_score", "fin_n"):
+        assert torch.equal(a[0].tensors[k][:30], b[0].tensors[k][:30]), k
+    compare_search(a[0], a[1], a[2], a[3], a[4], list(range(8)), 20, 10, 16, min_same=1.0)
 
 
 def test_config3_full_length_invariants(Bd):
