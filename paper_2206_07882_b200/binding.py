@@ -500,3 +500,26 @@ class Decoder:
         for it in range(n_iters):
             self.dr_fusion_beam_step(e, T, it, u_max)
         return self.q4_traceback(n_iters, u_max)
+
+
+class GraphedStep:
+    """Replays one whole pass (any callable that only enqueues library calls on the current
+    stream) as a CUDA graph: the pass is run eagerly once (so that every kernel attribute is
+    configured), captured once, then replayed.  The callable must read its input from the
+    static tensors it closes over; results are the tensors it returned during capture."""
+
+    def __init__(self, fn):
+        self.fn = fn
+        self.graph = None
+        self.result = None
+
+    def __call__(self):
+        if self.graph is None:
+            self.fn()                                   # eager warm-up
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self.result = self.fn()
+            self.graph = g
+        self.graph.replay()
+        return self.result
