@@ -174,7 +174,8 @@ class Job:
         wl = self.wl = WORKLOADS[wl_name]
         self.name = wl_name
         B, T = wl["B"], wl["T"]
-        seed = wl["seed"] + 1000 * rank           # every rank gets its own utterances
+        from paper_2206_07882_b200 import sharding
+        seed = sharding.rank_seed(wl["seed"], rank)    # every rank gets its own utterances
         self.enc = self.dec = None
         self.host_in = None
         if wl["enc"]:
@@ -367,14 +368,12 @@ def main():
         enc_ms, dec_ms = e_ms * scale, d_ms * scale
     barrier()
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = t.tolist()
+    from paper_2206_07882_b200 import sharding
+    ms_total = sharding.job_time_ms(ms_total, "cuda")       # max over ranks
+    ms_e2e = sharding.job_time_ms(ms_e2e, "cuda")
     ms_step = ms_total / K
-    audio_s = world * B * T * 0.02
-    rtf = (ms_step / 1e3) / audio_s
-    rtf_e2e = (ms_e2e / K / 1e3) / audio_s
+    rtf = sharding.aggregate_rtf(ms_step, B, T * 0.02, world, "cuda")
+    rtf_e2e = sharding.aggregate_rtf(ms_e2e / K, B, T * 0.02, world, "cuda")
 
     if rank == 0:
         pk = peaks()
