@@ -147,6 +147,25 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
                     const q4_mat* w_out, const float* b_out, float* logp, void* workspace,
                     size_t workspace_bytes, q4_stream stream);
 
+/*
+ * qjoint_logprobs_static — qjoint_logprobs for callers that cannot allocate device memory when
+ * they call (a latency-critical decoding thread that must not wait on the allocator, a host
+ * that forbids allocations after start-up, a process in which another thread is capturing a
+ * stream).  The paper has no counterpart: this is the same computation with the workspace
+ * replaced by a fixed array inside the library's device image, so the call allocates nothing.
+ *   Limit: N * D <= 65536 (D = w_pred->rows), about 320 KB of device memory that every GPU
+ *   loading the library keeps until the process exits; larger problems get Q4_ERR_WORKSPACE.
+ *   The first call on each device looks up the array's device address (with that device
+ *   current); make that first call before starting any stream capture.
+ *   All calls on a device share the one array: calls that overlap on the GPU (different
+ *   streams) race with each other; calls on one stream are ordered and safe.  Nothing in the
+ *   array needs clearing, each call overwrites what it reads.
+ */
+int qjoint_logprobs_static(const float* e, const int32_t* frame_idx, const void* pq,
+                           const q4_act* p_act, int32_t N, const q4_mat* w_pred,
+                           const float* b_pred, const q4_act* z_act, const q4_mat* w_out,
+                           const float* b_out, float* logp, q4_stream stream);
+
 /* One LSTM layer / linear layer inside a model description. */
 typedef struct {
   q4_mat w_ih, w_hh;

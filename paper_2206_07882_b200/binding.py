@@ -73,7 +73,7 @@ class BeamStateS(C.Structure):
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
-           "q4_poll_status", "q4_version", "q4_launch_count", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model"]
+           "q4_poll_status", "q4_version", "q4_launch_count", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static"]
 
 _lib = None
 
@@ -304,6 +304,20 @@ def qjoint_logprobs(e: torch.Tensor, frame_idx: torch.Tensor, pq: torch.Tensor, 
                                C.byref(wp), _p(proj.bias), C.byref(z_act), C.byref(wo), _p(out.bias),
                                _p(logp), _p(workspace), C.c_size_t(workspace.numel()), _stream()),
          "qjoint_logprobs")
+    return logp
+
+
+def qjoint_logprobs_static(e: torch.Tensor, frame_idx: torch.Tensor, pq: torch.Tensor, p_act: Act,
+                           proj: DeviceLinear, z_act: Act, out: DeviceLinear, logp: torch.Tensor):
+    """Joint network without a caller workspace and without any allocation: the output tensor
+    is passed in and the scratch is the library's built-in array (N * D <= 65536).  For callers
+    that must not allocate at call time; overlapping calls on one GPU share that array."""
+    _need_cuda()
+    wp, wo = proj.w.c(), out.w.c()
+    _chk(lib().qjoint_logprobs_static(_p(e), _p(frame_idx), _p(pq), C.byref(p_act),
+                                      C.c_int32(pq.shape[0]), C.byref(wp), _p(proj.bias),
+                                      C.byref(z_act), C.byref(wo), _p(out.bias), _p(logp), _stream()),
+         "qjoint_logprobs_static")
     return logp
 
 
