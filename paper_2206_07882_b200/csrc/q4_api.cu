@@ -130,6 +130,8 @@ size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims) {
     if (K > 0) {                                         // int8 operands of the tensor-core GEMM
       n += align_up(T * B * K);
       n += align_up(D * 4 * H * K);
+      n += align_up(D * 4 * H * H);                      // resident recurrent weights, int8
+      n += 3 * align_up(D * 4 * H * sizeof(float));      // row scales and bias, cell-major
     }
     return n;
   }
@@ -312,6 +314,12 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
   const int Kx = w_ih[0].k_pad;
   int8_t* x8 = reinterpret_cast<int8_t*>(ws);
   int8_t* w8 = x8 + align_up((size_t)TB * Kx);
+  int8_t* whh8 = w8 + align_up((size_t)dirs * G * Kx);
+  float* vec_ih = reinterpret_cast<float*>(whh8 + align_up((size_t)dirs * G * H));
+  float* vec_hh = vec_ih + align_up((size_t)dirs * G * sizeof(float)) / sizeof(float);
+  float* vec_b = vec_hh + align_up((size_t)dirs * G * sizeof(float)) / sizeof(float);
+  // persistent recurrence: needs the tensor-core projection (cell-major accumulators)
+  const bool persistent = use_mma && enc_recurrent_supported(H, B, dirs);
   const long long hb = row_bytes(H, hid_act->bits);
   const long long yb = row_bytes(dirs * H, out_act->bits);
   const long long xb = row_bytes(w_ih[0].k_pad, w_ih[0].bits);
@@ -321,7 +329,15 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
     TagScope tag(TAG_QUANT);
     Q4_TRY(launch_unpack_rows(xq, xb, nullptr, *x_act, Kx, (int)TB, x8, Kx, 0, (int)TB, s));
     for (int d = 0; d < dirs; ++d)
-      Q4_TRY(launch_prepare_w(w_ih[d], 0, w8 + (size_t)d * G * Kx, Kx, 0, s));
+      Q4_TRY(launch_prepare_w(w_ih[d], persistent ? 1 : 0, w8 + (size_t)d * G * Kx, Kx, 0, s));
+    if (persistent) {
+      for (int d = 0; d < dirs; ++d) {
+        Q4_TRY(launch_prepare_w(w_hh[d], 1, whh8 + (size_t)d * G * H, H, 0, s));
+        Q4_TRY(launch_prepare_vec(w_ih[d].scale, G, 1, vec_ih + (size_t)d * G, s));
+        Q4_TRY(launch_prepare_vec(w_hh[d].scale, G, 1, vec_hh + (size_t)d * G, s));
+        Q4_TRY(launch_prepare_vec(bias ? bias[d] : nullptr, G, 1, vec_b + (size_t)d * G, s));
+      }
+    }
   }
   for (int d = 0; d < dirs; ++d) {
     TagScope tag(TAG_ENC_GEMM);
@@ -334,6 +350,37 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
                              acc_ih + (size_t)d * TB * G, G, nullptr);
       Q4_TRY(launch_gemm(g, w_ih[d].bits, EPI_I32, s));
     }
+  }
+  if (persistent) {
+    EncRecArgs ra;
+    memset(&ra, 0, sizeof(ra));
+    ra.T = T;
+    ra.B = B;
+    ra.H = H;
+    ra.dirs = dirs;
+    ra.x_scale = x_act->scale;
+    ra.x_scale_b = x_scale_b;
+    ra.hid_act = *hid_act;
+    ra.out_act = *out_act;
+    ra.yq_ld = yb;
+    ra.dbg_ld = (long long)dirs * G;
+    for (int d = 0; d < dirs; ++d) {
+      EncRecDir& D = ra.d[d];
+      D.w_hh = whh8 + (size_t)d * G * H;
+      D.sc_ih = vec_ih + (size_t)d * G;
+      D.sc_hh = vec_hh + (size_t)d * G;
+      D.bias = vec_b + (size_t)d * G;
+      D.acc_pre = acc_ih + (size_t)d * TB * G;
+      D.yq = static_cast<uint8_t*>(yq) + row_bytes(d * H, out_act->bits);
+      D.dbg_ih = dbg_acc_ih ? dbg_acc_ih + (size_t)d * G : nullptr;
+      D.dbg_hh = dbg_acc_hh ? dbg_acc_hh + (size_t)d * G : nullptr;
+      D.hq_n = hq_n ? static_cast<uint8_t*>(hq_n) + (size_t)d * B * hb : nullptr;
+      D.c_n = c_n ? c_n + (size_t)d * B * H : nullptr;
+    }
+    if ((dbg_acc_ih == nullptr) != (dbg_acc_hh == nullptr)) return Q4_ERR_NULL;
+    TagScope tag(TAG_ENC_STEP);
+    Q4_TRY(launch_enc_recurrent(ra, s));
+    return Q4_OK;
   }
   Q4_TRY(cudaMemsetAsync(hbuf, 0, (size_t)dirs * 2 * B * H, s));
   Q4_TRY(cudaMemsetAsync(cbuf, 0, (size_t)dirs * B * H * sizeof(float), s));

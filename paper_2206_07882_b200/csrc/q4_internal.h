@@ -89,6 +89,31 @@ cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa
                             const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
                             const int8_t* hw, long long hw_pitch, cudaStream_t s);
 
+// ---- persistent encoder recurrence (q4_recurrent.cu)
+struct EncRecDir {
+  const int8_t* w_hh;       // int8 [4H, H], rows in 4*cell+gate order
+  const float* sc_ih;       // [4H] in the same order
+  const float* sc_hh;
+  const float* bias;
+  const int32_t* acc_pre;   // input accumulators [T*B, 4H], columns in 4*cell+gate order
+  uint8_t* yq;              // layer output codes, already offset to this direction's columns
+  int32_t* dbg_ih;          // optional [T, B, dirs, 4H] gate-major, offset to this direction
+  int32_t* dbg_hh;
+  uint8_t* hq_n;            // optional final codes [B, H], this direction
+  float* c_n;               // optional final cell state [B, H], this direction
+};
+struct EncRecArgs {
+  EncRecDir d[2];
+  int32_t T, B, H, dirs, n_groups;
+  float x_scale;
+  const float* x_scale_b;
+  q4_act hid_act, out_act;
+  long long yq_ld;          // bytes per (t, b) output row
+  long long dbg_ld;         // elements per (t, b) debug row
+};
+bool enc_recurrent_supported(int H, int B, int dirs);
+cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s);
+
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 }  // namespace q4
