@@ -245,6 +245,13 @@ typedef struct {
   int32_t* fin_slot;  /* its slot in the beam entering that iteration */
   int32_t* fin_n;     /* [B] */
   int32_t* status;    /* [1] device status word, 0 = ok */
+  /* Optional concurrency (host handles, all NULL = everything on the call's stream): two more
+   * cudaStream_t and three cudaEvent_t (created without timing) owned by the caller.  The step
+   * then runs the prediction/joint chain and the source-LM chain on the auxiliary streams,
+   * forked from and joined back into the call's stream, so the call's stream still orders
+   * the whole step. */
+  void* aux_stream[2];
+  void* aux_event[3];
 } q4_beam_state;
 
 /* Reset `state` for a new batch: slot 0 of every utterance holds the empty hypothesis with

@@ -67,7 +67,8 @@ class BeamStateS(C.Structure):
                 ("adv_src", C.c_void_p), ("adv_dst", C.c_void_p), ("adv_tok", C.c_void_p),
                 ("bp_parent", C.c_void_p), ("bp_token", C.c_void_p), ("bp_score", C.c_void_p),
                 ("fin_score", C.c_void_p), ("fin_iter", C.c_void_p), ("fin_slot", C.c_void_p),
-                ("fin_n", C.c_void_p), ("status", C.c_void_p)]
+                ("fin_n", C.c_void_p), ("status", C.c_void_p),
+                ("aux_stream", C.c_void_p * 2), ("aux_event", C.c_void_p * 3)]
 
 
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
@@ -405,10 +406,11 @@ class Decoder:
     """Device copy of prediction network, joint network and both fusion LMs, the search
     state, and the iteration loop (one library call per search iteration)."""
 
-    def __init__(self, dw, device="cuda", tensor_cores: bool = True):
+    def __init__(self, dw, device="cuda", tensor_cores: bool = True, concurrent: bool = True):
         self.dw = dw
         self.device = device
         self.tensor_cores = tensor_cores
+        self.concurrent = concurrent and tensor_cores
         self.V, self.E = dw.pred.emb.shape
         self.pred_emb_act = q4_act_symmetric(dw.pred.emb_alpha, 4)
         emb = torch.from_numpy(np.ascontiguousarray(dw.pred.emb, dtype=np.float32)).to(device)
@@ -472,6 +474,16 @@ class Decoder:
             setattr(s, name, t[name].data_ptr())
         s.tgt_hq[0], s.tgt_hq[1] = t["tgt_hq0"].data_ptr(), t["tgt_hq1"].data_ptr()
         s.tgt_c[0], s.tgt_c[1] = t["tgt_c0"].data_ptr(), t["tgt_c1"].data_ptr()
+        if self.concurrent:
+            # two more streams and three untimed events lent to the library for fork / join
+            self._aux_streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
+            self._aux_events = [torch.cuda.Event() for _ in range(3)]
+            for ev in self._aux_events:
+                ev.record()
+            for i in range(2):
+                s.aux_stream[i] = self._aux_streams[i].cuda_stream
+            for i in range(3):
+                s.aux_event[i] = self._aux_events[i].cuda_event
         self.B, self.W, self.n_iters = B, W, n_iters
         dims = [B, W, self.V, self.D]
         if self.tensor_cores:

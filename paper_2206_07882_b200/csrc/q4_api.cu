@@ -142,11 +142,13 @@ size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims) {
   if (call_id == Q4_WS_BEAM && ndims >= 4) {
     const size_t N = (size_t)dims[0] * dims[1], V = dims[2], D = dims[3];
     size_t n = align_up(N * D) * 3 + align_up(N * V * sizeof(float)) + align_up(N * sizeof(int32_t));
+    n += 3 * align_up(N * sizeof(int32_t)) + 256;   // compacted pending advances + their count
     if (ndims >= 8) {  // int8 operand scratch of the tensor-core path
       const size_t Np = (N + 127) / 128 * 128;
       const size_t E = dims[4], Hp = dims[5], Hs = dims[6], Ht = dims[7];
       const size_t Hmax = Hp > Hs ? (Hp > Ht ? Hp : Ht) : (Hs > Ht ? Hs : Ht);
-      n += align_up(Np * E) + align_up(Np * Hmax);                       // gathered x / h operands
+      n += 3 * align_up(Np * E) + align_up(Np * Hp) + align_up(Np * Hs) + 2 * align_up(Np * Ht);  // gathered x / h operands
+      (void)Hmax;
       n += align_up(Np * Hp) + align_up(Np * Hs) + 2 * align_up(Np * Ht); // new cell outputs, int8
       n += 3 * align_up(Np * D);                                         // bottleneck codes, z codes
     }
@@ -344,7 +346,7 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
     if (use_mma) {
       Q4_TRY(launch_mma_gemm(x8, Kx, (int)TB, w8 + (size_t)d * G * Kx, Kx, G, Kx, EPI_I32,
                              acc_ih + (size_t)d * TB * G, G, nullptr, nullptr, nullptr, 0.0f, nullptr,
-                             status, s));
+                             status, nullptr, s));
     } else {
       GemmArgs g = gemm_args(xq, xb, nullptr, *x_act, (int)TB, w_ih[d], nullptr,
                              acc_ih + (size_t)d * TB * G, G, nullptr);
@@ -658,7 +660,24 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   float* logits = reinterpret_cast<float*>(ws);
   ws += align_up((size_t)N * V * sizeof(float));
   int32_t* live = reinterpret_cast<int32_t*>(ws);
+  ws += align_up((size_t)N * sizeof(int32_t));
+  int32_t* c_src = reinterpret_cast<int32_t*>(ws);
+  ws += align_up((size_t)N * sizeof(int32_t));
+  int32_t* c_dst = reinterpret_cast<int32_t*>(ws);
+  ws += align_up((size_t)N * sizeof(int32_t));
+  int32_t* c_tok = reinterpret_cast<int32_t*>(ws);
+  ws += align_up((size_t)N * sizeof(int32_t));
+  int32_t* n_active = reinterpret_cast<int32_t*>(ws);
+  ws += 256;
+  {  // list the slots with a pending advance first: the advance kernels then skip empty tiles
+    TagScope tag(TAG_MISC);
+    Q4_TRY(launch_compact(st, N, c_src, c_dst, c_tok, n_active, s));
+  }
 
+  q4_beam_state cst = st;   // same state, pending advances in compacted order
+  cst.adv_src = c_src;
+  cst.adv_dst = c_dst;
+  cst.adv_tok = c_tok;
   // tensor-core path: prepared int8 weights, enough rows to fill 128-row tiles, and room
   // for the int8 operand scratch
   const int Hp = m.pred_lstm.w_hh.k_pad, Hs = m.src.lstm[0].w_hh.k_pad, Ht = m.tgt.lstm[0].w_hh.k_pad;
@@ -669,13 +688,20 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
                        Hp % 128 == 0 && Hs % 128 == 0 && Ht % 128 == 0 && V % 32 == 0 &&
                        workspace_bytes >= q4_workspace_bytes(Q4_WS_BEAM, dims8, 8);
   if (use_mma) {
-    ws += align_up((size_t)N * sizeof(int32_t));
     const size_t Np = ((size_t)N + 127) / 128 * 128;
     const int Hmax = Hp > Hs ? (Hp > Ht ? Hp : Ht) : (Hs > Ht ? Hs : Ht);
-    int8_t* xa8 = reinterpret_cast<int8_t*>(ws);
-    ws += align_up(Np * Ep);
-    int8_t* ha8 = reinterpret_cast<int8_t*>(ws);
-    ws += align_up(Np * Hmax);
+    (void)Hmax;
+    int8_t* xa8[3];   // embedding rows of the pending symbols: prediction, source LM, target LM
+    for (int i = 0; i < 3; ++i) {
+      xa8[i] = reinterpret_cast<int8_t*>(ws);
+      ws += align_up(Np * Ep);
+    }
+    int8_t* ha8[4];   // previous cell outputs: prediction, source LM, target LM layers 1 and 2
+    const int hdim[4] = {Hp, Hs, Ht, Ht};
+    for (int i = 0; i < 4; ++i) {
+      ha8[i] = reinterpret_cast<int8_t*>(ws);
+      ws += align_up(Np * (size_t)hdim[i]);
+    }
     int8_t* pred_h8 = reinterpret_cast<int8_t*>(ws);
     ws += align_up(Np * Hp);
     int8_t* src_h8 = reinterpret_cast<int8_t*>(ws);
@@ -695,18 +721,57 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     const uint8_t* pb = static_cast<const uint8_t*>(m.prepared);
 
     // one LSTM layer of one network for every pending slot
-    auto lstm_mma = [&](int tag_id, int li, const q4_lstm& L, const q4_act& x_act, const void* x_src,
-                        long long x_stride, const int32_t* x_idx, const int8_t* x_ready, void* hq,
-                        float* c, int8_t* h8) -> int {
+    // all gathers of the iteration in one launch: embedding rows by pending symbol, previous
+    // cell-output codes by parent state row, unpacked to int8 operand rows
+    {
+      UnpackJobs uj;
+      memset(&uj, 0, sizeof(uj));
+      auto add = [&](const void* src, long long stride, const int32_t* idx, const q4_act& act, int k_pad,
+                     int8_t* dst) {
+        UnpackJob& j = uj.job[uj.n_jobs++];
+        j.src = static_cast<const uint8_t*>(src);
+        j.src_stride = stride;
+        j.idx = idx;
+        j.bits = act.bits;
+        j.is_signed = act.is_signed;
+        j.zp = act.zero_point;
+        j.k_pad = k_pad;
+        j.dst = dst;
+        j.dst_stride = k_pad;
+      };
+      add(m.pred_emb_q, row_bytes(Ep, m.pred_lstm.w_ih.bits), cst.adv_tok, m.pred_emb_act, Ep, xa8[0]);
+      add(m.src.emb_q, row_bytes(Ep, m.src.lstm[0].w_ih.bits), cst.adv_tok, m.src.emb_act, Ep, xa8[1]);
+      add(m.tgt.emb_q, row_bytes(Ep, m.tgt.lstm[0].w_ih.bits), cst.adv_tok, m.tgt.emb_act, Ep, xa8[2]);
+      add(st.pred_hq, row_bytes(Hp, m.pred_lstm.hid_act.bits), cst.adv_src, m.pred_lstm.hid_act, Hp, ha8[0]);
+      add(st.src_hq, row_bytes(Hs, m.src.lstm[0].hid_act.bits), cst.adv_src, m.src.lstm[0].hid_act, Hs, ha8[1]);
+      add(st.tgt_hq[0], row_bytes(Ht, m.tgt.lstm[0].hid_act.bits), cst.adv_src, m.tgt.lstm[0].hid_act, Ht, ha8[2]);
+      if (m.tgt.n_layers == 2)
+        add(st.tgt_hq[1], row_bytes(Ht, m.tgt.lstm[1].hid_act.bits), cst.adv_src, m.tgt.lstm[1].hid_act, Ht, ha8[3]);
+      uj.n_rows = N;
+      uj.n_rows_pad = (int)Np;
+      uj.zero_tail = 0;   // rows beyond the pending advances feed tiles whose results are dropped
+      uj.n_active = n_active;
+      TagScope tag(TAG_MISC);
+      Q4_TRY(launch_unpack_multi(uj, s));
+    }
+    // the three networks are independent until the selection: with two lent streams the
+    // prediction/joint chain and the source-LM chain run beside the target-LM chain
+    cudaStream_t sp = s, ss = s;
+    const bool forked = st.aux_stream[0] && st.aux_stream[1] && st.aux_event[0] && st.aux_event[1] &&
+                        st.aux_event[2];
+    if (forked) {
+      sp = reinterpret_cast<cudaStream_t>(st.aux_stream[0]);
+      ss = reinterpret_cast<cudaStream_t>(st.aux_stream[1]);
+      cudaEvent_t fork = reinterpret_cast<cudaEvent_t>(st.aux_event[0]);
+      Q4_TRY(cudaEventRecord(fork, s));
+      Q4_TRY(cudaStreamWaitEvent(sp, fork, 0));
+      Q4_TRY(cudaStreamWaitEvent(ss, fork, 0));
+    }
+    // one LSTM layer of one network for every pending slot
+    auto lstm_mma = [&](cudaStream_t s, int tag_id, int li, const q4_lstm& L, const q4_act& x_act,
+                        const int8_t* xa, const int8_t* ha, void* hq, float* c, int8_t* h8) -> int {
       TagScope tag(tag_id);
       const int H = L.w_hh.k_pad, Kx = L.w_ih.k_pad;
-      const int8_t* xa = x_ready;
-      if (!xa) {
-        Q4_TRY(launch_unpack_rows(x_src, x_stride, x_idx, x_act, Kx, N, xa8, Kx, 0, (int)Np, s));
-        xa = xa8;
-      }
-      Q4_TRY(launch_unpack_rows(hq, row_bytes(H, L.hid_act.bits), st.adv_src, L.hid_act, H, N, ha8, H, 0,
-                                (int)Np, s));
       MmaLstmArgs a;
       memset(&a, 0, sizeof(a));
       a.N = N;
@@ -718,8 +783,8 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       a.x_scale = x_act.scale;
       a.hid_act = L.hid_act;
       a.out_act = L.hid_act;
-      a.src_row = st.adv_src;
-      a.dst_row = st.adv_dst;
+      a.src_row = cst.adv_src;
+      a.dst_row = cst.adv_dst;
       a.c_in = c;
       a.c_out = c;
       a.hq_out = static_cast<uint8_t*>(hq);
@@ -727,66 +792,78 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       a.h8_out = h8;
       a.h8_ld = H;
       a.status = st.status;
-      Q4_TRY(launch_mma_lstm(a, xa, Kx, reinterpret_cast<const int8_t*>(pb + pp.lstm[li].xw), Kx, ha8, H,
+      a.n_active = n_active;
+      Q4_TRY(launch_mma_lstm(a, xa, Kx, reinterpret_cast<const int8_t*>(pb + pp.lstm[li].xw), Kx, ha, H,
                              reinterpret_cast<const int8_t*>(pb + pp.lstm[li].hw), H, s));
       return Q4_OK;
     };
-    auto linear_mma = [&](int tag_id, int wi, const q4_linear& L, const int8_t* x8, float x_scale,
-                          int epi, void* out, long long ldo, const int32_t* out_idx,
-                          const q4_act* out_act) -> int {
+    auto linear_mma = [&](cudaStream_t s, int tag_id, int wi, const q4_linear& L, const int8_t* x8,
+                          float x_scale, int epi, void* out, long long ldo, const int32_t* out_idx,
+                          const q4_act* out_act, const int32_t* rows_active) -> int {
       TagScope tag(tag_id);
       Q4_TRY(launch_mma_gemm(x8, L.w.k_pad, N, reinterpret_cast<const int8_t*>(pb + pp.lin[wi]), L.w.k_pad,
                              L.w.rows, L.w.k_pad, epi, out, ldo, out_idx, L.w.scale, L.bias, x_scale, out_act,
-                             st.status, s));
+                             st.status, rows_active, s));
       return Q4_OK;
     };
 
-    // 1. pending advances
-    Q4_CHECK(lstm_mma(TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, m.pred_emb_q,
-                      row_bytes(Ep, m.pred_lstm.w_ih.bits), st.adv_tok, nullptr, st.pred_hq, st.pred_c,
-                      pred_h8));
-    Q4_CHECK(linear_mma(TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
-                        st.pred_p, D, st.adv_dst, nullptr));
+    // 1a. prediction network, then the joint network for every live slot (stream sp)
+    Q4_CHECK(lstm_mma(sp, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
+                      st.pred_c, pred_h8));
+    Q4_CHECK(linear_mma(sp, TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
+                        st.pred_p, D, cst.adv_dst, nullptr, n_active));
+    {
+      TagScope tag(TAG_JOINT);
+      Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, sp));
+    }
+    Q4_CHECK(linear_mma(sp, TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr,
+                        nullptr));
+    // 1b. source LM (stream ss) and target LM (the call's stream)
     for (int which = 0; which < 2; ++which) {
       const q4_lm& lm = *lms[which];
+      cudaStream_t sl = which == 0 ? ss : s;
       const q4_lstm& L0 = lm.lstm[0];
       void* hq0 = which == 0 ? st.src_hq : st.tgt_hq[0];
       float* c0 = which == 0 ? st.src_c : st.tgt_c[0];
       int8_t* h8_0 = which == 0 ? src_h8 : tgt_h8[0];
       float* lp = which == 0 ? st.src_lp : st.tgt_lp;
-      Q4_CHECK(lstm_mma(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, which == 0 ? 1 : 2, L0, lm.emb_act, lm.emb_q,
-                        row_bytes(Ep, L0.w_ih.bits), st.adv_tok, nullptr, hq0, c0, h8_0));
+      Q4_CHECK(lstm_mma(sl, which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, which == 0 ? 1 : 2, L0, lm.emb_act,
+                        xa8[which + 1], ha8[which + 1], hq0, c0, h8_0));
       const int8_t* top8 = h8_0;
       const q4_lstm* last = &L0;
       if (lm.n_layers == 2) {
         const q4_lstm& L1 = lm.lstm[1];
-        Q4_CHECK(lstm_mma(TAG_TGT_L2, 3, L1, L0.hid_act, nullptr, 0, nullptr, h8_0, st.tgt_hq[1],
-                          st.tgt_c[1], tgt_h8[1]));
+        Q4_CHECK(lstm_mma(sl, TAG_TGT_L2, 3, L1, L0.hid_act, h8_0, ha8[3], st.tgt_hq[1], st.tgt_c[1],
+                          tgt_h8[1]));
         top8 = tgt_h8[1];
         last = &L1;
       }
       const int head_tag = which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD;
-      Q4_CHECK(linear_mma(head_tag, which == 0 ? 1 : 3, lm.bott, top8, last->hid_act.scale, EPI_QUANT8,
-                          bq8[which], D, nullptr, &lm.bott_act));
-      Q4_CHECK(linear_mma(head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
-                          V, st.adv_dst, nullptr));
-      TagScope tag(head_tag);
-      Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, st.adv_dst, s));
+      Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 1 : 3, lm.bott, top8, last->hid_act.scale, EPI_QUANT8,
+                          bq8[which], D, nullptr, &lm.bott_act, n_active));
+      Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
+                          V, cst.adv_dst, nullptr, n_active));
     }
-    // 2. joint network for every live slot at its frame
-    {
-      TagScope tag(TAG_JOINT);
-      Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, s));
+    if (forked) {   // join: the call's stream waits for both side chains
+      cudaEvent_t j0 = reinterpret_cast<cudaEvent_t>(st.aux_event[1]);
+      cudaEvent_t j1 = reinterpret_cast<cudaEvent_t>(st.aux_event[2]);
+      Q4_TRY(cudaEventRecord(j0, sp));
+      Q4_TRY(cudaEventRecord(j1, ss));
+      Q4_TRY(cudaStreamWaitEvent(s, j0, 0));
+      Q4_TRY(cudaStreamWaitEvent(s, j1, 0));
     }
-    Q4_CHECK(linear_mma(TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr));
+    {  // log-softmax of both LMs' new rows in one launch
+      TagScope tag(TAG_TGT_HEAD);
+      Q4_TRY(launch_logsoftmax(st.src_lp, st.src_lp, N, V, V, cst.adv_dst, s, st.tgt_lp));
+    }
   } else {
     // 1. pending advances -------------------------------------------------------------
     {  // prediction network: embedding row -> LSTM -> projection to D
       const q4_lstm& L = m.pred_lstm;
-      Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), st.adv_tok,
-                            m.pred_emb_act, st.pred_hq, st.pred_c, st, N, s));
-      GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), st.adv_dst,
-                             L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, st.adv_dst);
+      Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), cst.adv_tok,
+                            m.pred_emb_act, st.pred_hq, st.pred_c, cst, N, s));
+      GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), cst.adv_dst,
+                             L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, cst.adv_dst);
       TagScope tag(TAG_PRED_PROJ);
       Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
     }
@@ -797,28 +874,28 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       float* lp = which == 0 ? st.src_lp : st.tgt_lp;
       uint8_t* bq = which == 0 ? bq_src : bq_tgt;
       const q4_lstm& L0 = lm.lstm[0];
-      Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), st.adv_tok,
-                            lm.emb_act, hq0, c0, st, N, s));
+      Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), cst.adv_tok,
+                            lm.emb_act, hq0, c0, cst, N, s));
       const void* top = hq0;
       const q4_lstm* last = &L0;
       if (lm.n_layers == 2) {
         if (which == 0) return Q4_ERR_UNSUPPORTED;  // the state block holds one source-LM layer
         const q4_lstm& L1 = lm.lstm[1];
-        Q4_CHECK(advance_lstm(TAG_TGT_L2, L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), st.adv_dst,
-                              L0.hid_act, st.tgt_hq[1], st.tgt_c[1], st, N, s));
+        Q4_CHECK(advance_lstm(TAG_TGT_L2, L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), cst.adv_dst,
+                              L0.hid_act, st.tgt_hq[1], st.tgt_c[1], cst, N, s));
         top = st.tgt_hq[1];
         last = &L1;
       }
-      GemmArgs gb = gemm_args(top, row_bytes(last->w_hh.k_pad, last->hid_act.bits), st.adv_dst,
+      GemmArgs gb = gemm_args(top, row_bytes(last->w_hh.k_pad, last->hid_act.bits), cst.adv_dst,
                               last->hid_act, N, lm.bott.w, lm.bott.bias, bq,
                               row_bytes(D, lm.bott_act.bits), nullptr);
       gb.out_act = lm.bott_act;
       TagScope tag(which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD);
       Q4_TRY(launch_gemm(gb, lm.bott.w.bits, EPI_QUANT, s));
       GemmArgs go = gemm_args(bq, row_bytes(D, lm.bott_act.bits), nullptr, lm.bott_act, N, lm.out.w,
-                              lm.out.bias, lp, V, st.adv_dst);
+                              lm.out.bias, lp, V, cst.adv_dst);
       Q4_TRY(launch_gemm(go, lm.out.w.bits, EPI_F32, s));
-      Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, st.adv_dst, s));
+      Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, cst.adv_dst, s));
     }
 
     // 2. joint network for every live slot at its frame -----------------------------------

@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
   __shared__ float s_score[MAXW];
   __shared__ int s_t[MAXW], s_u[MAXW], s_row[MAXW], s_last[MAXW];
   __shared__ uint64_t s_hash[MAXW], s_prev[MAXW];
-  __shared__ uint64_t red[2][SEL_NT / 32];
+  __shared__ uint64_t slot_top[MAXW][MAXW];   // per slot: its W best proposals, best first (0 = none)
   __shared__ int win_idx[MAXW];
   __shared__ float win_score[MAXW];
   __shared__ int n_win_s;
@@ -66,9 +66,10 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     s_hash[tid] = st.hash[o];
     s_prev[tid] = st.prev_hash[o];
   }
+  if (tid < MAXW * MAXW) slot_top[tid / MAXW][tid % MAXW] = 0ull;
   __syncthreads();
 
-  // ---- proposals: one warp per slot
+  // ---- proposals: one warp per slot; the row of logits is read once and kept in registers
   for (int w = warp; w < W; w += SEL_NT / 32) {
     float* cw = cand + (size_t)w * V;
     const int row = s_row[w];
@@ -77,31 +78,70 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
       continue;
     }
     const float* x = a.logits + (size_t)(base + w) * V;
-    float m = NEG;
-    for (int k = lane; k < V; k += 32) m = fmaxf(m, x[k]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float s = 0.0f;
-    for (int k = lane; k < V; k += 32) s += expf(x[k] - m);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    const float lse = m + logf(s);
-    const double S = (double)s_score[w];
-    const bool labels = s_u[w] < a.u_max;
     const float* lt = a.tgt_lp + (size_t)row * V;
     const float* ls = a.src_lp + (size_t)row * V;
-    for (int k = lane; k < V; k += 32) {
-      const float lp = x[k] - lse;
-      float v;
-      if (k == 0) {
-        v = (float)(S + (double)lp);
-      } else if (labels) {
-        v = (float)(S + (double)lp + (double)a.lambda_t * (double)lt[k] -
-                    (double)a.lambda_s * (double)ls[k] + (double)a.rho);
-      } else {
-        v = NEG;
+    const double S = (double)s_score[w];
+    const bool labels = s_u[w] < a.u_max;
+    for (int k0 = 0; k0 < V; k0 += 1024) {      // V <= 1024: a single trip
+      float xv[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int k = k0 + lane + 32 * i;
+        xv[i] = k < V ? x[k] : NEG;
       }
-      cw[k] = v;
+      if (k0 == 0 && V <= 1024) {
+        float m = NEG;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) m = fmaxf(m, xv[i]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        float sum = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sum += expf(xv[i] - m);   // exp(-inf) = 0 for the padding
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float lse = m + logf(sum);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int k = lane + 32 * i;
+          if (k >= V) continue;
+          const float lp = xv[i] - lse;
+          float v;
+          if (k == 0) {
+            v = (float)(S + (double)lp);
+          } else if (labels) {
+            v = (float)(S + (double)lp + (double)a.lambda_t * (double)lt[k] -
+                        (double)a.lambda_s * (double)ls[k] + (double)a.rho);
+          } else {
+            v = NEG;
+          }
+          cw[k] = v;
+        }
+      }
+    }
+    if (V > 1024) {   // general vocabulary size: three passes over the row
+      float m = NEG;
+      for (int k = lane; k < V; k += 32) m = fmaxf(m, x[k]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      float sum = 0.0f;
+      for (int k = lane; k < V; k += 32) sum += expf(x[k] - m);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float lse = m + logf(sum);
+      for (int k = lane; k < V; k += 32) {
+        const float lp = x[k] - lse;
+        float v;
+        if (k == 0) {
+          v = (float)(S + (double)lp);
+        } else if (labels) {
+          v = (float)(S + (double)lp + (double)a.lambda_t * (double)lt[k] -
+                      (double)a.lambda_s * (double)ls[k] + (double)a.rho);
+        } else {
+          v = NEG;
+        }
+        cw[k] = v;
+      }
     }
   }
   __syncthreads();
@@ -126,8 +166,10 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     int* fi = st.fin_iter + base;
     int* fl = st.fin_slot + base;
     int n = st.fin_n[b];
+    bool any = false;
     for (int w = 0; w < W; ++w) {
       if (s_row[w] < 0 || s_t[w] + 1 != a.T) continue;
+      any = true;
       const float S = cand[(size_t)w * V];
       cand[(size_t)w * V] = NEG;
       int pos = n;
@@ -144,53 +186,77 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
       fl[pos] = w;
       n = min(n + 1, W);
     }
-    st.fin_n[b] = n;
+    if (any) st.fin_n[b] = n;
   }
   __syncthreads();
 
-  // ---- the W best remaining proposals
-  const int total = W * V;
-  uint64_t best = 0;
-  for (int i = tid; i < total; i += SEL_NT) best = u64max(best, make_key(cand[i], (uint32_t)i));
-  int n_win = 0;
-  for (int r = 0; r < W; ++r) {
-    const uint64_t wm = warp_max_u64(best);
-    if (lane == 0) red[r & 1][warp] = wm;
-    __syncthreads();
-    uint64_t g = lane < SEL_NT / 32 ? red[r & 1][lane] : 0ull;
-    g = warp_max_u64(g);
-    const float sc = key_score(g);
-    if (!(sc > NEG)) break;
-    const uint32_t idx = ~(uint32_t)g;
-    if (tid == 0) {
-      win_idx[r] = (int)idx;
-      win_score[r] = sc;
+  // ---- the W best remaining proposals.  Stage 1: every slot's own W best (one warp per slot)
+  for (int w = warp; w < W; w += SEL_NT / 32) {
+    if (s_row[w] < 0) continue;
+    float* cw = cand + (size_t)w * V;
+    const uint32_t off = (uint32_t)w * (uint32_t)V;
+    uint64_t best = 0;
+    for (int k = lane; k < V; k += 32) best = u64max(best, make_key(cw[k], off + (uint32_t)k));
+    for (int r = 0; r < W; ++r) {
+      const uint64_t g = warp_max_u64(best);
+      if (!(key_score(g) > NEG)) break;
+      if (lane == 0) slot_top[w][r] = g;
+      const int k = (int)(~(uint32_t)g - off);
+      if ((k & 31) == lane) {
+        cw[k] = NEG;
+        best = 0;
+        for (int kk = lane; kk < V; kk += 32) best = u64max(best, make_key(cw[kk], off + (uint32_t)kk));
+      }
     }
-    if ((int)(idx % SEL_NT) == tid) {
-      cand[idx] = NEG;
-      best = 0;
-      for (int i = tid; i < total; i += SEL_NT) best = u64max(best, make_key(cand[i], (uint32_t)i));
-    }
-    n_win = r + 1;
   }
-  if (tid == 0) n_win_s = n_win;
   __syncthreads();
+  // Stage 2: the W best of the (at most W*W) survivors, one warp, eight keys per lane
+  if (warp == 0) {
+    uint64_t mine[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) mine[i] = slot_top[lane >> 1][(lane & 1) * 8 + i];
+    int n_win = 0;
+    for (int r = 0; r < W; ++r) {
+      uint64_t lb = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) lb = u64max(lb, mine[i]);
+      const uint64_t g = warp_max_u64(lb);
+      if (g == 0ull) break;
+      if (lane == 0) {
+        win_idx[r] = (int)(~(uint32_t)g);
+        win_score[r] = key_score(g);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (mine[i] == g) mine[i] = 0ull;
+      n_win = r + 1;
+    }
+    if (lane == 0) n_win_s = n_win;
+    __syncwarp();
 
-  // ---- next beam, state rows, back-pointers
-  if (tid == 0) {
-    const int nw = n_win_s;
+    // ---- next beam, state rows, back-pointers: lane s writes slot s
+    const int nw = n_win;
     const int row0 = b * 2 * W;
     uint32_t used = 0;
     for (int w = 0; w < W; ++w)
       if (s_row[w] >= 0) used |= 1u << (s_row[w] - row0);
-    for (int s = 0; s < W; ++s) {
+    const uint32_t free_mask = ~used & (W >= 16 ? 0xFFFFFFFFu : ((1u << (2 * W)) - 1u));
+    const int s = lane;
+    int idx = 0, w = 0, k = 0;
+    bool is_label = false;
+    if (s < nw) {
+      idx = win_idx[s];
+      w = idx / V;
+      k = idx % V;
+      is_label = k != 0;
+    }
+    const unsigned lab = __ballot_sync(0xffffffffu, is_label);
+    if (s < W) {
       const int o = base + s;
       const size_t hist = ((size_t)a.iter * a.B + b) * W + s;
       if (s < nw) {
-        const int idx = win_idx[s];
-        const int w = idx / V, k = idx % V;
         st.score[o] = win_score[s];
-        if (k == 0) {
+        if (!is_label) {
           st.t[o] = s_t[w] + 1;
           st.u[o] = s_u[w];
           st.hash[o] = s_hash[w];
@@ -201,8 +267,10 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
           st.adv_dst[o] = -1;
           st.adv_tok[o] = -1;
         } else {
-          const int f = __ffs((int)~used) - 1;
-          used |= 1u << f;
+          // the j-th label extension (in slot order) takes the j-th state row not used by the
+          // beam that is being replaced
+          const int j = __popc(lab & ((1u << s) - 1u));
+          const int f = (int)__fns(free_mask, 0, j + 1);
           st.t[o] = s_t[w];
           st.u[o] = s_u[w] + 1;
           st.hash[o] = hash_mix(s_hash[w], (uint32_t)k);
@@ -240,6 +308,59 @@ cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s) {
   }
   timing_begin(s);
   k_beam_select<<<a.B, SEL_NT, smem, s>>>(a);
+  timing_end(s);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
+// Compaction of the pending network advances: slots whose adv_dst >= 0 are listed first, in
+// slot order, so that the advance kernels touch only tiles with work (most extensions of a
+// beam are blanks, which advance nothing).  One CTA; deterministic order.
+__global__ void __launch_bounds__(1024) k_compact(const int32_t* adv_src, const int32_t* adv_dst,
+                                                  const int32_t* adv_tok, int N, int32_t* c_src,
+                                                  int32_t* c_dst, int32_t* c_tok, int32_t* n_active) {
+  __shared__ int wsum[32];
+  __shared__ int base_s;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) base_s = 0;
+  __syncthreads();
+  for (int n0 = 0; n0 < N; n0 += 1024) {
+    const int n = n0 + tid;
+    const bool f = n < N && adv_dst[n] >= 0;
+    const unsigned m = __ballot_sync(0xffffffffu, f);
+    const int within = __popc(m & ((1u << lane) - 1u));
+    if (lane == 0) wsum[warp] = __popc(m);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < 32; ++w) {
+      const int c = wsum[w];
+      if (w < warp) before += c;
+      total += c;
+    }
+    const int base = base_s;
+    if (f) {
+      const int a = base + before + within;
+      c_src[a] = adv_src[n];
+      c_dst[a] = adv_dst[n];
+      c_tok[a] = adv_tok[n];
+    }
+    __syncthreads();
+    if (tid == 0) base_s = base + total;
+    __syncthreads();
+  }
+  const int total = base_s;
+  for (int a = total + tid; a < N; a += 1024) {
+    c_src[a] = -1;
+    c_dst[a] = -1;
+    c_tok[a] = -1;
+  }
+  if (tid == 0) *n_active = total;
+}
+
+cudaError_t launch_compact(const q4_beam_state& st, int N, int32_t* c_src, int32_t* c_dst, int32_t* c_tok,
+                           int32_t* n_active, cudaStream_t s) {
+  timing_begin(s);
+  k_compact<<<1, 1024, 0, s>>>(st.adv_src, st.adv_dst, st.adv_tok, N, c_src, c_dst, c_tok, n_active);
   timing_end(s);
   ++g_launches;
   return cudaGetLastError();

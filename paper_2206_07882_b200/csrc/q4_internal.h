@@ -7,7 +7,7 @@ namespace q4 {
 cudaError_t launch_gemm(const GemmArgs& a, int bits, int epi, cudaStream_t s);
 cudaError_t launch_lstm(const LstmArgs2& a, int dirs, int x_bits, int h_bits, cudaStream_t s);
 cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long long stride,
-                              const int32_t* idx, cudaStream_t s);
+                              const int32_t* idx, cudaStream_t s, float* second = nullptr);
 cudaError_t launch_joint_z(const float* e, const int32_t* frame_idx, const int32_t* t_arr, int B,
                            int W, const float* p, const int32_t* p_idx, int N, int D,
                            const q4_act& za, uint8_t* zq, int8_t* z8, int32_t* live_out,
@@ -26,6 +26,8 @@ struct BeamSelArgs {
   float lambda_t, lambda_s, rho;
 };
 cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s);
+cudaError_t launch_compact(const q4_beam_state& st, int N, int32_t* c_src, int32_t* c_dst, int32_t* c_tok,
+                           int32_t* n_active, cudaStream_t s);
 cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters, cudaStream_t s);
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s);
@@ -73,18 +75,34 @@ struct MmaLstmArgs {
   int32_t* dbg_hh;
   long long dbg_ld;
   int32_t* status;
+  const int32_t* n_active;  // optional: rows >= *n_active carry no work (tiles beyond it exit at once)
 };
 enum { EPI_QUANT8 = 3 };    // re-quantize and store (code - zero_point) as int8, one per byte
 cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
                                const q4_act& act, int k_pad, int n_rows, int8_t* dst,
                                long long dst_stride, int col0, int n_rows_pad, cudaStream_t s);
+struct UnpackJob {
+  const uint8_t* src;       // packed code rows
+  long long src_stride;
+  const int32_t* idx;       // source row of launch row n (negative = zero row)
+  int32_t bits, is_signed, zp, k_pad;
+  int8_t* dst;              // int8 [n_rows_pad, k_pad], pitch dst_stride
+  long long dst_stride;
+};
+struct UnpackJobs {
+  UnpackJob job[8];
+  int32_t n_jobs, n_rows, n_rows_pad, zero_tail;
+  const int32_t* n_active;
+};
+cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s);
 cudaError_t launch_prepare_w(const q4_mat& w, int interleave, int8_t* dst, long long dst_stride,
                              int col0, cudaStream_t s);
 cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s);
 cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const int8_t* w8,
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
                             const int32_t* out_idx, const float* w_scale, const float* bias,
-                            float x_scale, const q4_act* out_act, int32_t* status, cudaStream_t s);
+                            float x_scale, const q4_act* out_act, int32_t* status,
+                            const int32_t* n_active, cudaStream_t s);
 cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa_pitch,
                             const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
                             const int8_t* hw, long long hw_pitch, cudaStream_t s);

@@ -430,12 +430,14 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* red) 
 }
 
 __global__ void __launch_bounds__(256) k_logsoftmax(const float* in, float* out, int V,
-                                                    long long stride, const int32_t* idx) {
+                                                    long long stride, const int32_t* idx,
+                                                    float* second) {
   __shared__ float red[32];
   const int r = idx ? idx[blockIdx.x] : (int)blockIdx.x;
   if (r < 0) return;
-  const float* x = in + (long long)r * stride;
-  float* y = out + (long long)r * stride;
+  // blockIdx.y == 1 treats a second matrix with the same row indices, in place
+  const float* x = (blockIdx.y ? second : in) + (long long)r * stride;
+  float* y = (blockIdx.y ? second : out) + (long long)r * stride;
   float m = -INFINITY;
   for (int v = threadIdx.x; v < V; v += blockDim.x) m = fmaxf(m, x[v]);
   m = block_reduce(m, true, red);
@@ -447,10 +449,10 @@ __global__ void __launch_bounds__(256) k_logsoftmax(const float* in, float* out,
 }
 
 cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long long stride,
-                              const int32_t* idx, cudaStream_t s) {
+                              const int32_t* idx, cudaStream_t s, float* second) {
   if (rows <= 0) return cudaSuccess;
   timing_begin(s);
-  k_logsoftmax<<<rows, 256, 0, s>>>(in, out, V, stride, idx);
+  k_logsoftmax<<<dim3(rows, second ? 2 : 1), 256, 0, s>>>(in, out, V, stride, idx, second);
   timing_end(s);
   ++g_launches;
   return cudaGetLastError();

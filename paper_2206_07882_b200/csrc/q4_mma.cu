@@ -87,6 +87,68 @@ cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int3
   return cudaGetLastError();
 }
 
+// Several gather+unpack jobs in one launch (blockIdx.y selects the job).
+__global__ void __launch_bounds__(256) k_unpack_multi(const UnpackJobs jobs) {
+  const UnpackJob& j = jobs.job[blockIdx.y];
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = j.k_pad >> 5;
+  if (i >= (long long)jobs.n_rows_pad * per_row) return;
+  const int n = (int)(i / per_row), k = (int)(i % per_row) * 32;
+  uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
+  int r = -1;
+  if (n < jobs.n_rows) r = j.idx ? j.idx[n] : n;
+  if (r >= 0) {
+    const uint8_t* p = j.src + (long long)r * j.src_stride;
+    if (j.bits == 4) {
+      const uint4 v = *reinterpret_cast<const uint4*>(p + (k >> 1));
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      uint32_t o[8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          int a = (w[q] >> (4 * e)) & 0xF, c = (w[q] >> (4 * (e + 4))) & 0xF;
+          if (j.is_signed) {
+            a = (a ^ 8) - 8;
+            c = (c ^ 8) - 8;
+          } else {
+            a -= j.zp;
+            c -= j.zp;
+          }
+          lo |= (uint32_t)(a & 0xFF) << (8 * e);
+          hi |= (uint32_t)(c & 0xFF) << (8 * e);
+        }
+        o[2 * q] = lo;
+        o[2 * q + 1] = hi;
+      }
+      o0 = make_uint4(o[0], o[1], o[2], o[3]);
+      o1 = make_uint4(o[4], o[5], o[6], o[7]);
+    } else {
+      o0 = *reinterpret_cast<const uint4*>(p + k);
+      o1 = *reinterpret_cast<const uint4*>(p + k + 16);
+    }
+  } else if (n >= jobs.n_rows || (jobs.n_active && n >= *jobs.n_active)) {
+    if (!jobs.zero_tail) return;   // rows without work need not be cleared every time
+  }
+  uint4* d = reinterpret_cast<uint4*>(j.dst + (long long)n * j.dst_stride + k);
+  d[0] = o0;
+  d[1] = o1;
+}
+
+cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s) {
+  if (jobs.n_jobs <= 0) return cudaSuccess;
+  int kmax = 0;
+  for (int i = 0; i < jobs.n_jobs; ++i) kmax = jobs.job[i].k_pad > kmax ? jobs.job[i].k_pad : kmax;
+  const long long total = (long long)jobs.n_rows_pad * (kmax >> 5);
+  dim3 grid((unsigned)((total + 255) / 256), jobs.n_jobs);
+  timing_begin(s);
+  k_unpack_multi<<<grid, 256, 0, s>>>(jobs);
+  timing_end(s);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
 // Weight preparation: unpack to int8; with `interleave` the 4H rows (gate-major i,f,g,o) are
 // reordered to row 4*cell + gate so that one thread of the epilogue owns all gates of a cell.
 __global__ void __launch_bounds__(256) k_prepare_w(const uint8_t* src, int bits, int rows, int k_pad,
@@ -194,6 +256,7 @@ struct MmaGemmArgs {
   float x_scale;
   q4_act out_act;
   int32_t* status;
+  const int32_t* n_active;
 };
 
 __global__ void __launch_bounds__(192, 1)
@@ -207,6 +270,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m0 = blockIdx.x * BM, n0 = blockIdx.y * GEMM_BN;
   const int nk = (a.K + BK - 1) / BK;
+  if (a.n_active && m0 >= *a.n_active) return;   // whole tile without work (uniform per CTA)
 
   if (tid == 0) {
     for (int s = 0; s < GEMM_STAGES; ++s) {
@@ -327,7 +391,8 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
 cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const int8_t* w8,
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
                             const int32_t* out_idx, const float* w_scale, const float* bias,
-                            float x_scale, const q4_act* out_act, int32_t* status, cudaStream_t s) {
+                            float x_scale, const q4_act* out_act, int32_t* status,
+                            const int32_t* n_active, cudaStream_t s) {
   if (M <= 0 || J <= 0) return cudaSuccess;
   CUtensorMap ta, tb;
   if (!make_tmap_i8(&ta, x8, K, M, x_pitch, BM) || !make_tmap_i8(&tb, w8, K, J, w_pitch, GEMM_BN))
@@ -346,6 +411,7 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
   a.x_scale = x_scale;
   if (out_act) a.out_act = *out_act;
   a.status = status;
+  a.n_active = n_active;
   const size_t smem = (size_t)GEMM_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
   static bool configured = false;
   if (!configured) {
@@ -377,6 +443,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
   const int nkx = a.acc_pre ? 0 : (a.Kx_pad + BK - 1) / BK;
   const int nkh = (a.H + BK - 1) / BK;
   const int nk = nkx + nkh;
+  if (a.n_active && m0 >= *a.n_active) return;   // whole tile without work (uniform per CTA)
 
   if (tid == 0) {
     for (int s = 0; s < LSTM_STAGES; ++s) {
