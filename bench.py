@@ -36,6 +36,9 @@ WORKLOADS = {
     "cfg4_end_to_end": dict(B=64, T=500, U_max=250, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
     "cfg1_encoder": dict(B=32, T=500, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
     "cfg3_beam": dict(B=16, T=300, U_max=150, l1_bits=4, out_bits=4, enc=False, dec=True, seed=3),
+    # reduced lengths of the same shapes, for profiler captures that must end by themselves
+    "prof_encoder": dict(B=32, T=250, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
+    "prof_end_to_end": dict(B=64, T=24, U_max=12, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
 }
 
 
@@ -434,11 +437,21 @@ def roofline(job, tag, ms, n, pk):
                  10: (d.tgt.lstm[-1], d.tgt.lstm[0].H)}[tag]
         bytes_, ops = lstm_work(l, N, kx)
     elif tag == 3:
+        # persistent recurrence: one launch = all T steps of a layer, both directions.  It must
+        # read the int32 input accumulators once, the recurrent weights once, and write the codes;
+        # its arithmetic is DP4A on the plain ALUs, so the ALU roofline applies.
         l = job.enc.layers[1][0]
-        Bn = wl["B"]
-        H = l.H
-        bytes_ = 2 * (l.w_hh.q.numel() + Bn * 4 * H * 4 + Bn * H * 4 * 2 + Bn * H)
-        ops = 2 * 2.0 * Bn * 4 * H * H
+        Bn, Tn, H = wl["B"], wl["T"], l.H
+        bytes_ = 2 * (4 * H * H + Tn * Bn * 4 * H * 4 + Tn * Bn * H // 2)
+        ops = 2 * 2.0 * Tn * Bn * 4 * H * H
+        dp4a_peak = 148 * 128 * 8 * 1.965e9 / 1e12       # SMs x lanes x ops per DP4A x clock
+        sec = ms / 1e3
+        out.update(bound="alu", achieved=ops / sec / 1e12, peak=dp4a_peak, unit="TOP/s (DP4A)",
+                   frac=ops / sec / 1e12 / dp4a_peak, algorithmic_bytes=bytes_, algorithmic_ops=ops,
+                   hbm={"achieved": bytes_ / sec / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                        "frac": bytes_ / sec / 1e9 / pk["hbm_gbs"]},
+                   peak_source="148 SMs x 128 lanes x 8 int-ops x 1.965 GHz (unit counts and max clock)")
+        return out
     elif tag == 2:
         l = job.enc.layers[1][0]
         M = wl["B"] * wl["T"]
