@@ -235,6 +235,12 @@ typedef struct {
   int32_t* adv_src;   /* pending network advance: state row to read (-1 = zero state) */
   int32_t* adv_dst;   /* row to write (-1 = nothing pending) */
   int32_t* adv_tok;   /* symbol to feed */
+  /* the pending advances again, compacted (only slots with adv_dst >= 0, any order), double
+   * buffered by iteration parity: entry a of list p is at [p * B*W + a], pend_n[p] entries */
+  int32_t* pend_src;  /* [2, B*W] */
+  int32_t* pend_dst;  /* [2, B*W] */
+  int32_t* pend_tok;  /* [2, B*W] */
+  int32_t* pend_n;    /* [2] */
   /* history [n_iters, B, W] */
   int32_t* bp_parent; /* slot in the previous beam, -1 = empty */
   int32_t* bp_token;  /* 0 = blank */

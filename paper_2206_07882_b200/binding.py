@@ -65,6 +65,8 @@ class BeamStateS(C.Structure):
                 ("score", C.c_void_p), ("t", C.c_void_p), ("u", C.c_void_p), ("hash", C.c_void_p),
                 ("prev_hash", C.c_void_p), ("last_tok", C.c_void_p), ("row", C.c_void_p),
                 ("adv_src", C.c_void_p), ("adv_dst", C.c_void_p), ("adv_tok", C.c_void_p),
+                ("pend_src", C.c_void_p), ("pend_dst", C.c_void_p), ("pend_tok", C.c_void_p),
+                ("pend_n", C.c_void_p),
                 ("bp_parent", C.c_void_p), ("bp_token", C.c_void_p), ("bp_score", C.c_void_p),
                 ("fin_score", C.c_void_p), ("fin_iter", C.c_void_p), ("fin_slot", C.c_void_p),
                 ("fin_n", C.c_void_p), ("status", C.c_void_p),
@@ -461,6 +463,8 @@ class Decoder:
             hash=z(N, torch.int64), prev_hash=z(N, torch.int64), last_tok=z(N, torch.int32),
             row=z(N, torch.int32), adv_src=z(N, torch.int32), adv_dst=z(N, torch.int32),
             adv_tok=z(N, torch.int32),
+            pend_src=z((2, N), torch.int32), pend_dst=z((2, N), torch.int32),
+            pend_tok=z((2, N), torch.int32), pend_n=z(2, torch.int32),
             bp_parent=z((max(n_iters, 1), B, W), torch.int32),
             bp_token=z((max(n_iters, 1), B, W), torch.int32),
             bp_score=z((max(n_iters, 1), B, W), torch.float32),
@@ -469,6 +473,7 @@ class Decoder:
         s = self.state = BeamStateS()
         for name in ("pred_hq", "pred_c", "pred_p", "src_hq", "src_c", "src_lp", "tgt_lp", "score",
                      "t", "u", "hash", "prev_hash", "last_tok", "row", "adv_src", "adv_dst", "adv_tok",
+                     "pend_src", "pend_dst", "pend_tok", "pend_n",
                      "bp_parent", "bp_token", "bp_score", "fin_score", "fin_iter", "fin_slot",
                      "fin_n", "status"):
             setattr(s, name, t[name].data_ptr())

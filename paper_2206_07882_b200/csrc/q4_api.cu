@@ -142,7 +142,6 @@ size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims) {
   if (call_id == Q4_WS_BEAM && ndims >= 4) {
     const size_t N = (size_t)dims[0] * dims[1], V = dims[2], D = dims[3];
     size_t n = align_up(N * D) * 3 + align_up(N * V * sizeof(float)) + align_up(N * sizeof(int32_t));
-    n += 3 * align_up(N * sizeof(int32_t)) + 256;   // compacted pending advances + their count
     if (ndims >= 8) {  // int8 operand scratch of the tensor-core path
       const size_t Np = (N + 127) / 128 * 128;
       const size_t E = dims[4], Hp = dims[5], Hs = dims[6], Ht = dims[7];
@@ -565,7 +564,8 @@ static int check_state(const q4_beam_state* st, int n_lm_layers) {
                        st->tgt_hq[0], st->tgt_c[0], st->tgt_lp, st->score, st->t, st->u, st->hash,
                        st->prev_hash, st->last_tok, st->row, st->adv_src, st->adv_dst, st->adv_tok,
                        st->bp_parent, st->bp_token, st->bp_score, st->fin_score, st->fin_iter,
-                       st->fin_slot, st->fin_n, st->status};
+                       st->fin_slot, st->fin_n, st->status, st->pend_src, st->pend_dst, st->pend_tok,
+                       st->pend_n};
   for (const void* p : req)
     if (!p) return Q4_ERR_NULL;
   if (n_lm_layers > 1 && (!st->tgt_hq[1] || !st->tgt_c[1])) return Q4_ERR_NULL;
@@ -583,7 +583,7 @@ int q4_beam_init(q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters, q4
 // writing the fresh row, then the projection(s).
 static int advance_lstm(int tag_id, const q4_lstm& L, const void* x, long long x_stride,
                         const int32_t* x_idx, const q4_act& x_act, void* hq, float* c,
-                        const q4_beam_state& st, int N, cudaStream_t s) {
+                        const q4_beam_state& st, int N, const int32_t* n_active, cudaStream_t s) {
   TagScope tag(tag_id);
   LstmArgs2 args;
   memset(&args, 0, sizeof(args));
@@ -603,6 +603,7 @@ static int advance_lstm(int tag_id, const q4_lstm& L, const void* x, long long x
   a.out_idx = st.adv_dst;
   a.c_out = c;
   a.dbg_stride = 4LL * H;
+  a.n_active = n_active;
   Q4_TRY(launch_lstm(args, 1, L.w_ih.bits, L.w_hh.bits, s));
   return Q4_OK;
 }
@@ -661,19 +662,12 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   ws += align_up((size_t)N * V * sizeof(float));
   int32_t* live = reinterpret_cast<int32_t*>(ws);
   ws += align_up((size_t)N * sizeof(int32_t));
-  int32_t* c_src = reinterpret_cast<int32_t*>(ws);
-  ws += align_up((size_t)N * sizeof(int32_t));
-  int32_t* c_dst = reinterpret_cast<int32_t*>(ws);
-  ws += align_up((size_t)N * sizeof(int32_t));
-  int32_t* c_tok = reinterpret_cast<int32_t*>(ws);
-  ws += align_up((size_t)N * sizeof(int32_t));
-  int32_t* n_active = reinterpret_cast<int32_t*>(ws);
-  ws += 256;
-  {  // list the slots with a pending advance first: the advance kernels then skip empty tiles
-    TagScope tag(TAG_MISC);
-    Q4_TRY(launch_compact(st, N, c_src, c_dst, c_tok, n_active, s));
-  }
-
+  // pending advances of this iteration, compacted by the previous selection (or the reset)
+  const int par = iter & 1;
+  int32_t* c_src = st.pend_src + (size_t)par * N;
+  int32_t* c_dst = st.pend_dst + (size_t)par * N;
+  int32_t* c_tok = st.pend_tok + (size_t)par * N;
+  const int32_t* n_active = st.pend_n + par;
   q4_beam_state cst = st;   // same state, pending advances in compacted order
   cst.adv_src = c_src;
   cst.adv_dst = c_dst;
@@ -854,16 +848,17 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     }
     {  // log-softmax of both LMs' new rows in one launch
       TagScope tag(TAG_TGT_HEAD);
-      Q4_TRY(launch_logsoftmax(st.src_lp, st.src_lp, N, V, V, cst.adv_dst, s, st.tgt_lp));
+      Q4_TRY(launch_logsoftmax(st.src_lp, st.src_lp, N, V, V, cst.adv_dst, s, st.tgt_lp, n_active));
     }
   } else {
     // 1. pending advances -------------------------------------------------------------
     {  // prediction network: embedding row -> LSTM -> projection to D
       const q4_lstm& L = m.pred_lstm;
       Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), cst.adv_tok,
-                            m.pred_emb_act, st.pred_hq, st.pred_c, cst, N, s));
+                            m.pred_emb_act, st.pred_hq, st.pred_c, cst, N, n_active, s));
       GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), cst.adv_dst,
                              L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, cst.adv_dst);
+      g.n_active = n_active;
       TagScope tag(TAG_PRED_PROJ);
       Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
     }
@@ -875,14 +870,14 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       uint8_t* bq = which == 0 ? bq_src : bq_tgt;
       const q4_lstm& L0 = lm.lstm[0];
       Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), cst.adv_tok,
-                            lm.emb_act, hq0, c0, cst, N, s));
+                            lm.emb_act, hq0, c0, cst, N, n_active, s));
       const void* top = hq0;
       const q4_lstm* last = &L0;
       if (lm.n_layers == 2) {
         if (which == 0) return Q4_ERR_UNSUPPORTED;  // the state block holds one source-LM layer
         const q4_lstm& L1 = lm.lstm[1];
         Q4_CHECK(advance_lstm(TAG_TGT_L2, L1, hq0, row_bytes(L0.w_hh.k_pad, L0.hid_act.bits), cst.adv_dst,
-                              L0.hid_act, st.tgt_hq[1], st.tgt_c[1], cst, N, s));
+                              L0.hid_act, st.tgt_hq[1], st.tgt_c[1], cst, N, n_active, s));
         top = st.tgt_hq[1];
         last = &L1;
       }
@@ -890,12 +885,14 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
                               last->hid_act, N, lm.bott.w, lm.bott.bias, bq,
                               row_bytes(D, lm.bott_act.bits), nullptr);
       gb.out_act = lm.bott_act;
+      gb.n_active = n_active;
       TagScope tag(which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD);
       Q4_TRY(launch_gemm(gb, lm.bott.w.bits, EPI_QUANT, s));
       GemmArgs go = gemm_args(bq, row_bytes(D, lm.bott_act.bits), nullptr, lm.bott_act, N, lm.out.w,
                               lm.out.bias, lp, V, cst.adv_dst);
+      go.n_active = n_active;
       Q4_TRY(launch_gemm(go, lm.out.w.bits, EPI_F32, s));
-      Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, cst.adv_dst, s));
+      Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, cst.adv_dst, s, nullptr, n_active));
     }
 
     // 2. joint network for every live slot at its frame -----------------------------------

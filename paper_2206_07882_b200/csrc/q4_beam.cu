@@ -39,22 +39,31 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
   return v;
 }
 
+// Largest key of this lane's strided share of a shared array, and warp-wide arg-max helpers.
+__device__ __forceinline__ uint64_t strided_max(const uint64_t* arr, int n, int lane) {
+  uint64_t m = 0;
+  for (int i = lane; i < n; i += 32) m = u64max(m, arr[i]);
+  return m;
+}
+
 __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ BeamSelArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* cand = reinterpret_cast<float*>(smem_raw);  // [W * V]
+  const int W = a.W, V = a.V;
+  float* cand = reinterpret_cast<float*>(smem_raw);                         // [W * V]
+  uint64_t* list = reinterpret_cast<uint64_t*>(cand + (size_t)W * V);       // survivors of the filter
   __shared__ float s_score[MAXW];
   __shared__ int s_t[MAXW], s_u[MAXW], s_row[MAXW], s_last[MAXW];
   __shared__ uint64_t s_hash[MAXW], s_prev[MAXW];
-  __shared__ uint64_t slot_top[MAXW][MAXW];   // per slot: its W best proposals, best first (0 = none)
+  __shared__ int list_n;
   __shared__ int win_idx[MAXW];
   __shared__ float win_score[MAXW];
-  __shared__ int n_win_s;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = blockIdx.x, W = a.W, V = a.V;
+  const int b = blockIdx.x;
   const int base = b * W;
   const q4_beam_state& st = a.st;
   const float NEG = -INFINITY;
+  const int N = a.B * W;
 
   if (tid < W) {
     const int o = base + tid;
@@ -66,7 +75,11 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     s_hash[tid] = st.hash[o];
     s_prev[tid] = st.prev_hash[o];
   }
-  if (tid < MAXW * MAXW) slot_top[tid / MAXW][tid % MAXW] = 0ull;
+  if (tid == 0) {
+    list_n = 0;
+    // the list of pending advances consumed by this iteration is free again
+    if (b == 0) st.pend_n[a.iter & 1] = 0;
+  }
   __syncthreads();
 
   // ---- proposals: one warp per slot; the row of logits is read once and kept in registers
@@ -81,45 +94,44 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     const float* lt = a.tgt_lp + (size_t)row * V;
     const float* ls = a.src_lp + (size_t)row * V;
     const double S = (double)s_score[w];
+    const double rho_d = (double)a.rho;
     const bool labels = s_u[w] < a.u_max;
-    for (int k0 = 0; k0 < V; k0 += 1024) {      // V <= 1024: a single trip
+    if (V <= 1024) {
       float xv[32];
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        const int k = k0 + lane + 32 * i;
+        const int k = lane + 32 * i;
         xv[i] = k < V ? x[k] : NEG;
       }
-      if (k0 == 0 && V <= 1024) {
-        float m = NEG;
+      float m = NEG;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) m = fmaxf(m, xv[i]);
+      for (int i = 0; i < 32; ++i) m = fmaxf(m, xv[i]);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        float sum = 0.0f;
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      float sum = 0.0f;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sum += expf(xv[i] - m);   // exp(-inf) = 0 for the padding
+      for (int i = 0; i < 32; ++i) sum += expf(xv[i] - m);   // exp(-inf) = 0 for the padding
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        const float lse = m + logf(sum);
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float lse = m + logf(sum);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int k = lane + 32 * i;
-          if (k >= V) continue;
-          const float lp = xv[i] - lse;
-          float v;
-          if (k == 0) {
-            v = (float)(S + (double)lp);
-          } else if (labels) {
-            v = (float)(S + (double)lp + (double)a.lambda_t * (double)lt[k] -
-                        (double)a.lambda_s * (double)ls[k] + (double)a.rho);
-          } else {
-            v = NEG;
-          }
-          cw[k] = v;
+      for (int i = 0; i < 32; ++i) {
+        const int k = lane + 32 * i;
+        if (k >= V) continue;
+        const float lp = xv[i] - lse;
+        float v;
+        if (k == 0) {
+          v = (float)(S + (double)lp);
+        } else if (labels) {
+          // label increment in fp32 (magnitude of tens), one double add onto the running score
+          const float inc = __fmaf_rn(a.lambda_t, lt[k], __fmaf_rn(-a.lambda_s, ls[k], lp));
+          v = (float)(S + (double)inc + rho_d);
+        } else {
+          v = NEG;
         }
+        cw[k] = v;
       }
-    }
-    if (V > 1024) {   // general vocabulary size: three passes over the row
+    } else {   // general vocabulary size: three passes over the row
       float m = NEG;
       for (int k = lane; k < V; k += 32) m = fmaxf(m, x[k]);
 #pragma unroll
@@ -135,8 +147,9 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
         if (k == 0) {
           v = (float)(S + (double)lp);
         } else if (labels) {
-          v = (float)(S + (double)lp + (double)a.lambda_t * (double)lt[k] -
-                      (double)a.lambda_s * (double)ls[k] + (double)a.rho);
+          // label increment in fp32 (magnitude of tens), one double add onto the running score
+          const float inc = __fmaf_rn(a.lambda_t, lt[k], __fmaf_rn(-a.lambda_s, ls[k], lp));
+          v = (float)(S + (double)inc + rho_d);
         } else {
           v = NEG;
         }
@@ -162,79 +175,89 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
 
   // ---- finished hypotheses: blank proposals that consume the last frame
   if (tid == 0) {
-    float* fs = st.fin_score + base;
-    int* fi = st.fin_iter + base;
-    int* fl = st.fin_slot + base;
-    int n = st.fin_n[b];
     bool any = false;
-    for (int w = 0; w < W; ++w) {
-      if (s_row[w] < 0 || s_t[w] + 1 != a.T) continue;
-      any = true;
-      const float S = cand[(size_t)w * V];
-      cand[(size_t)w * V] = NEG;
-      int pos = n;
-      while (pos > 0 && fs[pos - 1] < S) --pos;
-      if (pos >= W) continue;
-      const int last = min(n, W - 1);
-      for (int i = last; i > pos; --i) {
-        fs[i] = fs[i - 1];
-        fi[i] = fi[i - 1];
-        fl[i] = fl[i - 1];
+    for (int w = 0; w < W; ++w) any |= s_row[w] >= 0 && s_t[w] + 1 == a.T;
+    if (any) {
+      float* fs = st.fin_score + base;
+      int* fi = st.fin_iter + base;
+      int* fl = st.fin_slot + base;
+      int n = st.fin_n[b];
+      for (int w = 0; w < W; ++w) {
+        if (s_row[w] < 0 || s_t[w] + 1 != a.T) continue;
+        const float S = cand[(size_t)w * V];
+        cand[(size_t)w * V] = NEG;
+        int pos = n;
+        while (pos > 0 && fs[pos - 1] < S) --pos;
+        if (pos >= W) continue;
+        const int last = min(n, W - 1);
+        for (int i = last; i > pos; --i) {
+          fs[i] = fs[i - 1];
+          fi[i] = fi[i - 1];
+          fl[i] = fl[i - 1];
+        }
+        fs[pos] = S;
+        fi[pos] = a.iter;
+        fl[pos] = w;
+        n = min(n + 1, W);
       }
-      fs[pos] = S;
-      fi[pos] = a.iter;
-      fl[pos] = w;
-      n = min(n + 1, W);
+      st.fin_n[b] = n;
     }
-    if (any) st.fin_n[b] = n;
   }
   __syncthreads();
 
-  // ---- the W best remaining proposals.  Stage 1: every slot's own W best (one warp per slot)
-  for (int w = warp; w < W; w += SEL_NT / 32) {
-    if (s_row[w] < 0) continue;
-    float* cw = cand + (size_t)w * V;
-    const uint32_t off = (uint32_t)w * (uint32_t)V;
-    uint64_t best = 0;
-    for (int k = lane; k < V; k += 32) best = u64max(best, make_key(cw[k], off + (uint32_t)k));
-    for (int r = 0; r < W; ++r) {
-      const uint64_t g = warp_max_u64(best);
-      if (!(key_score(g) > NEG)) break;
-      if (lane == 0) slot_top[w][r] = g;
-      const int k = (int)(~(uint32_t)g - off);
-      if ((k & 31) == lane) {
-        cw[k] = NEG;
-        best = 0;
-        for (int kk = lane; kk < V; kk += 32) best = u64max(best, make_key(cw[kk], off + (uint32_t)kk));
+  // ---- the W best remaining proposals, by a threshold filter.
+  // (1) every thread's best proposal ("head") among its strided share of its slot; (2) the
+  // W-th best head, found bit by bit with block-wide counts, is a lower bound of the W-th best
+  // proposal, and only the threads owning the W best heads can hold anything at or above it;
+  // (3) those go to a short list; (4) each list entry's rank is counted in parallel.
+  uint64_t head = 0;
+  if (warp < W && s_row[warp] >= 0) {
+    const float* cw = cand + (size_t)warp * V;
+    const uint32_t off = (uint32_t)warp * (uint32_t)V;
+    for (int k = lane; k < V; k += 32) {
+      const float v = cw[k];
+      if (v > NEG) head = u64max(head, make_key(v, off + (uint32_t)k));
+    }
+  }
+  uint64_t th = 0;
+  for (int bit = 63; bit >= 0; --bit) {
+    const uint64_t c = th | (1ull << bit);
+    if (__syncthreads_count(head >= c) >= W) th = c;
+  }
+  // th = the W-th best head (0 if there are fewer than W heads: then everything valid passes)
+  const int cap = 16 * ((V + 31) / 32);
+  if (head != 0ull && head >= th) {
+    const float* cw = cand + (size_t)warp * V;
+    const uint32_t off = (uint32_t)warp * (uint32_t)V;
+    for (int k = lane; k < V; k += 32) {
+      const float v = cw[k];
+      if (!(v > NEG)) continue;
+      const uint64_t key = make_key(v, off + (uint32_t)k);
+      if (key >= th) {
+        const int p = atomicAdd(&list_n, 1);
+        if (p < cap) list[p] = key;
       }
     }
   }
   __syncthreads();
-  // Stage 2: the W best of the (at most W*W) survivors, one warp, eight keys per lane
+  {
+    const int ln = min(list_n, cap);
+    for (int i = tid; i < ln; i += SEL_NT) {
+      const uint64_t mine = list[i];
+      int rank = 0;
+      for (int j = 0; j < ln; ++j) rank += list[j] > mine;
+      if (rank < W) {
+        win_idx[rank] = (int)(~(uint32_t)mine);
+        win_score[rank] = key_score(mine);
+      }
+    }
+  }
+  __syncthreads();
+
   if (warp == 0) {
-    uint64_t mine[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) mine[i] = slot_top[lane >> 1][(lane & 1) * 8 + i];
-    int n_win = 0;
-    for (int r = 0; r < W; ++r) {
-      uint64_t lb = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) lb = u64max(lb, mine[i]);
-      const uint64_t g = warp_max_u64(lb);
-      if (g == 0ull) break;
-      if (lane == 0) {
-        win_idx[r] = (int)(~(uint32_t)g);
-        win_score[r] = key_score(g);
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        if (mine[i] == g) mine[i] = 0ull;
-      n_win = r + 1;
-    }
-    if (lane == 0) n_win_s = n_win;
-    __syncwarp();
+    const int n_win = min(min(list_n, cap), W);
 
-    // ---- next beam, state rows, back-pointers: lane s writes slot s
+    // ---- next beam, state rows, back-pointers, pending advances: lane s writes slot s
     const int nw = n_win;
     const int row0 = b * 2 * W;
     uint32_t used = 0;
@@ -251,6 +274,11 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
       is_label = k != 0;
     }
     const unsigned lab = __ballot_sync(0xffffffffu, is_label);
+    // reserve a range of the next iteration's pending list for this utterance's label extensions
+    int pbase = 0;
+    if (lane == 0 && lab != 0u) pbase = atomicAdd(st.pend_n + ((a.iter + 1) & 1), __popc(lab));
+    pbase = __shfl_sync(0xffffffffu, pbase, 0);
+    const size_t poff = (size_t)((a.iter + 1) & 1) * N;
     if (s < W) {
       const int o = base + s;
       const size_t hist = ((size_t)a.iter * a.B + b) * W + s;
@@ -280,6 +308,9 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
           st.adv_src[o] = s_row[w];
           st.adv_dst[o] = row0 + f;
           st.adv_tok[o] = k;
+          st.pend_src[poff + pbase + j] = s_row[w];
+          st.pend_dst[poff + pbase + j] = row0 + f;
+          st.pend_tok[poff + pbase + j] = k;
         }
         st.bp_parent[hist] = w;
         st.bp_token[hist] = k;
@@ -298,7 +329,7 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
 }
 
 cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s) {
-  const size_t smem = (size_t)a.W * a.V * sizeof(float);
+  const size_t smem = (size_t)a.W * a.V * sizeof(float) + (size_t)16 * ((a.V + 31) / 32) * sizeof(uint64_t);
   static size_t configured = 0;
   if (smem > configured) {
     cudaError_t e = cudaFuncSetAttribute(k_beam_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -308,59 +339,6 @@ cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s) {
   }
   timing_begin(s);
   k_beam_select<<<a.B, SEL_NT, smem, s>>>(a);
-  timing_end(s);
-  ++g_launches;
-  return cudaGetLastError();
-}
-
-// Compaction of the pending network advances: slots whose adv_dst >= 0 are listed first, in
-// slot order, so that the advance kernels touch only tiles with work (most extensions of a
-// beam are blanks, which advance nothing).  One CTA; deterministic order.
-__global__ void __launch_bounds__(1024) k_compact(const int32_t* adv_src, const int32_t* adv_dst,
-                                                  const int32_t* adv_tok, int N, int32_t* c_src,
-                                                  int32_t* c_dst, int32_t* c_tok, int32_t* n_active) {
-  __shared__ int wsum[32];
-  __shared__ int base_s;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) base_s = 0;
-  __syncthreads();
-  for (int n0 = 0; n0 < N; n0 += 1024) {
-    const int n = n0 + tid;
-    const bool f = n < N && adv_dst[n] >= 0;
-    const unsigned m = __ballot_sync(0xffffffffu, f);
-    const int within = __popc(m & ((1u << lane) - 1u));
-    if (lane == 0) wsum[warp] = __popc(m);
-    __syncthreads();
-    int before = 0, total = 0;
-    for (int w = 0; w < 32; ++w) {
-      const int c = wsum[w];
-      if (w < warp) before += c;
-      total += c;
-    }
-    const int base = base_s;
-    if (f) {
-      const int a = base + before + within;
-      c_src[a] = adv_src[n];
-      c_dst[a] = adv_dst[n];
-      c_tok[a] = adv_tok[n];
-    }
-    __syncthreads();
-    if (tid == 0) base_s = base + total;
-    __syncthreads();
-  }
-  const int total = base_s;
-  for (int a = total + tid; a < N; a += 1024) {
-    c_src[a] = -1;
-    c_dst[a] = -1;
-    c_tok[a] = -1;
-  }
-  if (tid == 0) *n_active = total;
-}
-
-cudaError_t launch_compact(const q4_beam_state& st, int N, int32_t* c_src, int32_t* c_dst, int32_t* c_tok,
-                           int32_t* n_active, cudaStream_t s) {
-  timing_begin(s);
-  k_compact<<<1, 1024, 0, s>>>(st.adv_src, st.adv_dst, st.adv_tok, N, c_src, c_dst, c_tok, n_active);
   timing_end(s);
   ++g_launches;
   return cudaGetLastError();
@@ -385,7 +363,16 @@ __global__ void k_beam_init(q4_beam_state st, int B, int W) {
   st.fin_score[o] = -INFINITY;
   st.fin_iter[o] = 0;
   st.fin_slot[o] = 0;
-  if (s == 0) st.fin_n[b] = 0;
+  if (s == 0) {
+    st.fin_n[b] = 0;
+    st.pend_src[b] = -1;               // pending list of iteration 0: every utterance's root,
+    st.pend_dst[b] = b * 2 * W;        // fed the start symbol from the zero state
+    st.pend_tok[b] = 0;
+  }
+  if (o == 0) {
+    st.pend_n[0] = B;
+    st.pend_n[1] = 0;
+  }
 }
 
 cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters, cudaStream_t s) {

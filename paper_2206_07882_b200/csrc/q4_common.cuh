@@ -130,6 +130,7 @@ struct GemmArgs {
   const int32_t* out_idx;   // output row of x row m (nullptr = m; negative = skip)
   int32_t* dbg_acc;         // optional raw accumulators [M, J]
   q4_act out_act;           // EPI_QUANT
+  const int32_t* n_active;  // optional device count: rows >= *n_active carry no work
 };
 
 struct LstmArgs {
@@ -159,6 +160,7 @@ struct LstmArgs {
   int32_t* dbg_ih;          // optional, row n at n*dbg_stride
   int32_t* dbg_hh;
   long long dbg_stride;
+  const int32_t* n_active;  // optional device count: rows >= *n_active carry no work
 };
 struct LstmArgs2 {
   LstmArgs d[2];

@@ -7,7 +7,8 @@ namespace q4 {
 cudaError_t launch_gemm(const GemmArgs& a, int bits, int epi, cudaStream_t s);
 cudaError_t launch_lstm(const LstmArgs2& a, int dirs, int x_bits, int h_bits, cudaStream_t s);
 cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long long stride,
-                              const int32_t* idx, cudaStream_t s, float* second = nullptr);
+                              const int32_t* idx, cudaStream_t s, float* second = nullptr,
+                              const int32_t* n_active = nullptr);
 cudaError_t launch_joint_z(const float* e, const int32_t* frame_idx, const int32_t* t_arr, int B,
                            int W, const float* p, const int32_t* p_idx, int N, int D,
                            const q4_act& za, uint8_t* zq, int8_t* z8, int32_t* live_out,
@@ -26,8 +27,6 @@ struct BeamSelArgs {
   float lambda_t, lambda_s, rho;
 };
 cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s);
-cudaError_t launch_compact(const q4_beam_state& st, int N, int32_t* c_src, int32_t* c_dst, int32_t* c_tok,
-                           int32_t* n_active, cudaStream_t s);
 cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters, cudaStream_t s);
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s);

@@ -66,7 +66,7 @@ __global__ void __launch_bounds__(NT) k_gemm(const __grid_constant__ GemmArgs a)
     const int m = m0 + tid;
     const uint8_t* p = nullptr;
     int o = -1;
-    if (m < a.M) {
+    if (m < a.M && !(a.n_active && m >= *a.n_active)) {
       o = a.out_idx ? a.out_idx[m] : m;
       const int r = a.x.idx ? a.x.idx[m] : m;
       if (o >= 0 && r >= 0) p = a.x.base + (long long)r * a.x.stride;
@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
     const int n = n0 + tid;
     int hi = -1, oi = -1;
     const uint8_t* p = nullptr;
-    if (n < a.N) {
+    if (n < a.N && !(a.n_active && n >= *a.n_active)) {
       oi = a.out_idx ? a.out_idx[n] : n;
       if (oi >= 0) {
         hi = a.hin.idx ? a.hin.idx[n] : n;
@@ -431,8 +431,9 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* red) 
 
 __global__ void __launch_bounds__(256) k_logsoftmax(const float* in, float* out, int V,
                                                     long long stride, const int32_t* idx,
-                                                    float* second) {
+                                                    float* second, const int32_t* n_active) {
   __shared__ float red[32];
+  if (n_active && (int)blockIdx.x >= *n_active) return;
   const int r = idx ? idx[blockIdx.x] : (int)blockIdx.x;
   if (r < 0) return;
   // blockIdx.y == 1 treats a second matrix with the same row indices, in place
@@ -449,10 +450,11 @@ __global__ void __launch_bounds__(256) k_logsoftmax(const float* in, float* out,
 }
 
 cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long long stride,
-                              const int32_t* idx, cudaStream_t s, float* second) {
+                              const int32_t* idx, cudaStream_t s, float* second,
+                              const int32_t* n_active) {
   if (rows <= 0) return cudaSuccess;
   timing_begin(s);
-  k_logsoftmax<<<dim3(rows, second ? 2 : 1), 256, 0, s>>>(in, out, V, stride, idx, second);
+  k_logsoftmax<<<dim3(rows, second ? 2 : 1), 256, 0, s>>>(in, out, V, stride, idx, second, n_active);
   timing_end(s);
   ++g_launches;
   return cudaGetLastError();

@@ -96,7 +96,8 @@ __global__ void __launch_bounds__(256) k_unpack_multi(const UnpackJobs jobs) {
   const int n = (int)(i / per_row), k = (int)(i % per_row) * 32;
   uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
   int r = -1;
-  if (n < jobs.n_rows) r = j.idx ? j.idx[n] : n;
+  const bool has_work = n < jobs.n_rows && !(jobs.n_active && n >= *jobs.n_active);
+  if (has_work) r = j.idx ? j.idx[n] : n;
   if (r >= 0) {
     const uint8_t* p = j.src + (long long)r * j.src_stride;
     if (j.bits == 4) {
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(256) k_unpack_multi(const UnpackJobs jobs) {
       o0 = *reinterpret_cast<const uint4*>(p + k);
       o1 = *reinterpret_cast<const uint4*>(p + k + 16);
     }
-  } else if (n >= jobs.n_rows || (jobs.n_active && n >= *jobs.n_active)) {
+  } else if (!has_work) {
     if (!jobs.zero_tail) return;   // rows without work need not be cleared every time
   }
   uint4* d = reinterpret_cast<uint4*>(j.dst + (long long)n * j.dst_stride + k);
@@ -267,6 +268,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
   constexpr int A_BYTES = BM * BK, B_BYTES = GEMM_BN * BK, STAGE = A_BYTES + B_BYTES;
   __shared__ uint64_t full[GEMM_STAGES], empty[GEMM_STAGES], acc_full;
   __shared__ uint32_t tmem_base_s;
+  __shared__ float s_sc[GEMM_BN], s_bi[GEMM_BN];   // de-quantization constants of this tile's columns
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m0 = blockIdx.x * BM, n0 = blockIdx.y * GEMM_BN;
   const int nk = (a.K + BK - 1) / BK;
@@ -317,12 +319,20 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
     umma_commit(&acc_full);
     if (!ok) flag_timeout(a.status);
   } else if (warp < 4) {
+    if (a.epi != EPI_I32) {   // stage scale * row scale and bias while the MMAs run
+      for (int c = tid; c < GEMM_BN; c += 128) {
+        const int j = min(n0 + c, a.J - 1);
+        s_sc[c] = __fmul_rn(a.x_scale, __ldg(a.w_scale + j));
+        s_bi[c] = a.bias ? __ldg(a.bias + j) : 0.0f;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
     const bool ok = mbar_wait(&acc_full, 0);
     tc_fence_after();
     if (!ok && lane == 0) flag_timeout(a.status);
     const int mi = m0 + warp * 32 + lane;
     int m = -1;
-    if (mi < a.M) m = a.out_idx ? a.out_idx[mi] : mi;
+    if (mi < a.M && !(a.n_active && mi >= *a.n_active)) m = a.out_idx ? a.out_idx[mi] : mi;
     const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
     for (int c0 = 0; c0 < GEMM_BN; c0 += 32) {
       int r[32];
@@ -341,10 +351,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
       } else {
         float v[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int j = min(j0 + i, a.J - 1);
-          v[i] = __fmaf_rn((float)r[i], __fmul_rn(a.x_scale, __ldg(a.w_scale + j)), a.bias ? __ldg(a.bias + j) : 0.0f);
-        }
+        for (int i = 0; i < 32; ++i) v[i] = __fmaf_rn((float)r[i], s_sc[c0 + i], s_bi[c0 + i]);
         if (a.epi == EPI_F32) {
           float* o = reinterpret_cast<float*>(a.out) + (long long)m * a.ldo + j0;
           if (j0 + 32 <= a.J) {
@@ -500,7 +507,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
     const int rt = q * 32 + lane;            // row within the tile
     const int n = m0 + rt;                   // row of this launch
     int src = -1, dst = -1;
-    if (n < a.N) {
+    if (n < a.N && !(a.n_active && n >= *a.n_active)) {
       dst = a.dst_row ? a.dst_row[n] : n;
       src = a.src_row ? a.src_row[n] : n;
     }
