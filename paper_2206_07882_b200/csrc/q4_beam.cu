@@ -97,11 +97,14 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     const double rho_d = (double)a.rho;
     const bool labels = s_u[w] < a.u_max;
     if (V <= 1024) {
-      float xv[32];
+      // one round trip to memory: logits and both LM rows are requested together
+      float xv[32], ltv[32], lsv[32];
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
         const int k = lane + 32 * i;
         xv[i] = k < V ? x[k] : NEG;
+        ltv[i] = (k < V && labels) ? lt[k] : 0.0f;
+        lsv[i] = (k < V && labels) ? ls[k] : 0.0f;
       }
       float m = NEG;
 #pragma unroll
@@ -124,7 +127,7 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
           v = (float)(S + (double)lp);
         } else if (labels) {
           // label increment in fp32 (magnitude of tens), one double add onto the running score
-          const float inc = __fmaf_rn(a.lambda_t, lt[k], __fmaf_rn(-a.lambda_s, ls[k], lp));
+          const float inc = __fmaf_rn(a.lambda_t, ltv[i], __fmaf_rn(-a.lambda_s, lsv[i], lp));
           v = (float)(S + (double)inc + rho_d);
         } else {
           v = NEG;
@@ -219,10 +222,17 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
       if (v > NEG) head = u64max(head, make_key(v, off + (uint32_t)k));
     }
   }
+  // score bits first (32 counts); the index bits matter only if equal scores straddle the bound
   uint64_t th = 0;
-  for (int bit = 63; bit >= 0; --bit) {
+  for (int bit = 63; bit >= 32; --bit) {
     const uint64_t c = th | (1ull << bit);
     if (__syncthreads_count(head >= c) >= W) th = c;
+  }
+  if (__syncthreads_count(head >= th) > W) {
+    for (int bit = 31; bit >= 0; --bit) {
+      const uint64_t c = th | (1ull << bit);
+      if (__syncthreads_count(head >= c) >= W) th = c;
+    }
   }
   // th = the W-th best head (0 if there are fewer than W heads: then everything valid passes)
   const int cap = 16 * ((V + 31) / 32);
