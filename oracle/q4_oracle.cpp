@@ -211,6 +211,26 @@ float orc_tanh(float x) {
   const float t = (1.0f - e) / (1.0f + e);
   return std::copysign(t, x);
 }
+// LSTM cell update in fp32 with three divisions: the products i*g and o*tanh(c) are each
+// formed as one quotient,
+//   i*g = sign(g) (1 - eg) / ((1 + ei)(1 + eg)),   f = 1 / (1 + ef),
+//   c   = fma(f, c_prev, i*g),
+//   h   = sign(c) (1 - ec) / ((1 + eo)(1 + ec)),
+// with ei = exp(-i_pre), ef = exp(-f_pre), eo = exp(-o_pre) (arguments clamped to [-86, 86]),
+// eg = exp(-2 min(|g_pre|, 43)), ec = exp(-2 min(|c|, 43)).  Mathematically this is
+// sigmoid(i) tanh(g), sigmoid(f), sigmoid(o) tanh(c).
+void orc_cell(float pi, float pf, float pg, float po, float c_prev, float* c_out, float* h_out) {
+  const float ei = orc_exp(-std::fmin(std::fmax(pi, -86.0f), 86.0f));
+  const float ef = orc_exp(-std::fmin(std::fmax(pf, -86.0f), 86.0f));
+  const float eo = orc_exp(-std::fmin(std::fmax(po, -86.0f), 86.0f));
+  const float eg = orc_exp(-2.0f * std::fmin(std::fabs(pg), 43.0f));
+  const float ig = std::copysign((1.0f - eg) / ((1.0f + ei) * (1.0f + eg)), pg);
+  const float f = 1.0f / (1.0f + ef);
+  const float c = std::fmaf(f, c_prev, ig);
+  const float ec = orc_exp(-2.0f * std::fmin(std::fabs(c), 43.0f));
+  *c_out = c;
+  *h_out = std::copysign((1.0f - ec) / ((1.0f + eo) * (1.0f + ec)), c);
+}
 void orc_activations(const float* x, int64_t n, float* ex, float* sg, float* th) {
   for (int64_t i = 0; i < n; ++i) {
     if (ex) ex[i] = orc_exp(x[i]);
@@ -243,7 +263,7 @@ void orc_lstm_step(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act,
                    int32_t* acc_ih_out, int32_t* acc_hh_out, float* gates_out) {
   const int32_t H = L->H, K = L->K, G = 4 * H;
   std::vector<int32_t> a_ih(G), a_hh(G);
-  std::vector<float> act(G);
+  std::vector<float> pre(G);
   for (int32_t n = 0; n < N; ++n) {
     orc_int_matmul(L->w_ih, G, K, xq + (int64_t)n * K, x_act->zero_point, 1, a_ih.data());
     orc_int_matmul(L->w_hh, G, H, hq_in + (int64_t)n * H, hid_act->zero_point, 1, a_hh.data());
@@ -251,22 +271,21 @@ void orc_lstm_step(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act,
     const float s_h = hid_act->scale;
     for (int32_t j = 0; j < G; ++j) {
       // de-quantize: each accumulator times (activation scale * row scale), plus bias
-      float pre = std::fmaf((float)a_ih[j], s_x * L->s_wih[j], L->bias ? L->bias[j] : 0.0f);
-      pre = std::fmaf((float)a_hh[j], s_h * L->s_whh[j], pre);
-      act[j] = (j >= 2 * H && j < 3 * H) ? orc_tanh(pre) : orc_sigmoid(pre);
+      float v = std::fmaf((float)a_ih[j], s_x * L->s_wih[j], L->bias ? L->bias[j] : 0.0f);
+      pre[j] = std::fmaf((float)a_hh[j], s_h * L->s_whh[j], v);
     }
     for (int32_t u = 0; u < H; ++u) {
-      const float i = act[u], f = act[H + u], g = act[2 * H + u], o = act[3 * H + u];
-      const float c = std::fmaf(f, c_in[(int64_t)n * H + u], i * g);
-      const float h = o * orc_tanh(c);
+      float c, h;
+      orc_cell(pre[u], pre[H + u], pre[2 * H + u], pre[3 * H + u], c_in[(int64_t)n * H + u], &c, &h);
       c_out[(int64_t)n * H + u] = c;
       if (h_out) h_out[(int64_t)n * H + u] = h;
       hq_out[(int64_t)n * H + u] = (int16_t)quantize_one(h, *hid_act);
     }
     if (acc_ih_out) std::memcpy(acc_ih_out + (int64_t)n * G, a_ih.data(), G * sizeof(int32_t));
     if (acc_hh_out) std::memcpy(acc_hh_out + (int64_t)n * G, a_hh.data(), G * sizeof(int32_t));
-    if (gates_out)
-      for (int32_t j = 0; j < G; ++j) gates_out[(int64_t)n * G + j] = act[j];
+    if (gates_out)   // diagnostic: the four gate activations by themselves
+      for (int32_t j = 0; j < G; ++j)
+        gates_out[(int64_t)n * G + j] = (j >= 2 * H && j < 3 * H) ? orc_tanh(pre[j]) : orc_sigmoid(pre[j]);
   }
 }
 

@@ -114,6 +114,24 @@ __device__ __forceinline__ float tanh_fixed(float x) {
   return copysignf(t, x);
 }
 
+// LSTM cell update with three divisions (i*g and o*tanh(c) are one quotient each):
+//   i*g = sign(g)(1 - eg) / ((1 + ei)(1 + eg)),  f = 1 / (1 + ef),  c = fma(f, c_prev, i*g),
+//   h = sign(c)(1 - ec) / ((1 + eo)(1 + ec)),
+//   ei, ef, eo = exp(-pre) with pre clamped to [-86, 86]; eg, ec = exp(-2 min(|.|, 43)).
+__device__ __forceinline__ void cell_fixed(float pi, float pf, float pg, float po, float c_prev,
+                                           float& c, float& h) {
+  const float ei = exp_fixed(-fminf(fmaxf(pi, -86.0f), 86.0f));
+  const float ef = exp_fixed(-fminf(fmaxf(pf, -86.0f), 86.0f));
+  const float eo = exp_fixed(-fminf(fmaxf(po, -86.0f), 86.0f));
+  const float eg = exp_fixed(__fmul_rn(-2.0f, fminf(fabsf(pg), 43.0f)));
+  const float ig = copysignf(
+      __fdiv_rn(__fsub_rn(1.0f, eg), __fmul_rn(__fadd_rn(1.0f, ei), __fadd_rn(1.0f, eg))), pg);
+  const float f = __fdiv_rn(1.0f, __fadd_rn(1.0f, ef));
+  c = __fmaf_rn(f, c_prev, ig);
+  const float ec = exp_fixed(__fmul_rn(-2.0f, fminf(fabsf(c), 43.0f)));
+  h = copysignf(__fdiv_rn(__fsub_rn(1.0f, ec), __fmul_rn(__fadd_rn(1.0f, eo), __fadd_rn(1.0f, ec))), c);
+}
+
 // ---- argument blocks of the tile kernels -------------------------------------------
 enum { EPI_I32 = 0, EPI_F32 = 1, EPI_QUANT = 2 };
 

@@ -359,11 +359,9 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
         if (a.dbg_hh) a.dbg_hh[(long long)n * a.dbg_stride + j] = acc[r][cc][g];
         g4[g] = __fmaf_rn((float)acc[r][cc][g], __fmul_rn(sh, a.s_whh[j]), pre[r][cc][g]);
       }
-      const float ig = sigmoid_fixed(g4[0]), fg = sigmoid_fixed(g4[1]);
-      const float gg = tanh_fixed(g4[2]), og = sigmoid_fixed(g4[3]);
       const float cprev = hi >= 0 ? a.c_in[(long long)hi * H + cell] : 0.0f;
-      const float c = __fmaf_rn(fg, cprev, __fmul_rn(ig, gg));
-      const float h = __fmul_rn(og, tanh_fixed(c));
+      float c, h;
+      cell_fixed(g4[0], g4[1], g4[2], g4[3], cprev, c, h);
       a.c_out[(long long)oi * H + cell] = c;
       if (a.h_f32) a.h_f32[(long long)n * H + cell] = h;
       q[cc] = quantize1(h, a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);

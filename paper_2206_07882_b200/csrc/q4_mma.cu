@@ -559,9 +559,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
         const float pf = __fmaf_rn((float)hh[4 * c + 1], __fmul_rn(sh, s_hh.y), __fmaf_rn((float)ih[4 * c + 1], __fmul_rn(sx, s_ih.y), bb.y));
         const float pg = __fmaf_rn((float)hh[4 * c + 2], __fmul_rn(sh, s_hh.z), __fmaf_rn((float)ih[4 * c + 2], __fmul_rn(sx, s_ih.z), bb.z));
         const float po = __fmaf_rn((float)hh[4 * c + 3], __fmul_rn(sh, s_hh.w), __fmaf_rn((float)ih[4 * c + 3], __fmul_rn(sx, s_ih.w), bb.w));
-        const float ig = sigmoid_fixed(pi), fg = sigmoid_fixed(pf), gg = tanh_fixed(pg), og = sigmoid_fixed(po);
-        cn[c] = __fmaf_rn(fg, cp[c], __fmul_rn(ig, gg));
-        hn[c] = __fmul_rn(og, tanh_fixed(cn[c]));
+        cell_fixed(pi, pf, pg, po, cp[c], cn[c], hn[c]);
         qh[c] = quantize1(hn[c], a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
         qy[c] = quantize1(hn[c], a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
         if (a.dbg_ih) {

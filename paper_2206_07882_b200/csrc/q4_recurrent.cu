@@ -180,9 +180,8 @@ k_enc_recurrent(const EncRecArgs a) {
         const float pf = __fmaf_rn((float)hh[1], __fmul_rn(sh, s_hh.y), __fmaf_rn((float)pre[j].y, __fmul_rn(sx[j], s_ih.y), bb.y));
         const float pg = __fmaf_rn((float)hh[2], __fmul_rn(sh, s_hh.z), __fmaf_rn((float)pre[j].z, __fmul_rn(sx[j], s_ih.z), bb.z));
         const float po = __fmaf_rn((float)hh[3], __fmul_rn(sh, s_hh.w), __fmaf_rn((float)pre[j].w, __fmul_rn(sx[j], s_ih.w), bb.w));
-        const float ig = sigmoid_fixed(pi), fg = sigmoid_fixed(pf), gg = tanh_fixed(pg), og = sigmoid_fixed(po);
-        c_state[j] = __fmaf_rn(fg, c_state[j], __fmul_rn(ig, gg));
-        const float hval = __fmul_rn(og, tanh_fixed(c_state[j]));
+        float hval;
+        cell_fixed(pi, pf, pg, po, c_state[j], c_state[j], hval);
         q = quantize1(hval, a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
         q2 = quantize1(hval, a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
         last_q[j] = q;
