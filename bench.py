@@ -380,6 +380,14 @@ def main():
             ev.record()
             marks.append(ev)
 
+        # per-kernel durations are taken with the three search chains serialised on one stream
+        # (auxiliary streams withdrawn for these passes), so that an event pair brackets one
+        # kernel running alone, as in the profiler's launch list
+        saved_aux = None
+        if job.dec is not None and job.dec.state is not None:
+            st = job.dec.state
+            saved_aux = (st.aux_stream[0], st.aux_stream[1])
+            st.aux_stream[0], st.aux_stream[1] = None, None
         tot, cnt = {}, {}
         for _ in range(K):
             lib.q4_timing_set(C.c_uint32(0xFFFFFFFF), start, stop, tags, C.c_int32(cap))
@@ -393,6 +401,8 @@ def main():
                 ms = evs[i].elapsed_time(evs[cap + i])
                 tot[tags[i]] = tot.get(tags[i], 0.0) + ms
                 cnt[tags[i]] = cnt.get(tags[i], 0) + 1
+        if saved_aux is not None:
+            job.dec.state.aux_stream[0], job.dec.state.aux_stream[1] = saved_aux
         allms = sum(tot.values()) or 1.0
         shares = {TAG_NAMES.get(t, str(t)): {"launches": cnt[t] // K, "ms": round(tot[t] / K, 3),
                                              "avg_us": round(1e3 * tot[t] / cnt[t], 2),
@@ -433,9 +443,9 @@ def main():
                                   "note": "simulated accelerator, 1 utterance of 152 frames, beam 16"}}
         line["roofline"] = roofline(job, dom_tag, dom_ms, dom_n, pk) if dom_tag is not None else None
         if line["roofline"] is not None:
-            line["roofline"]["timing"] = ("CUDA events around every launch of this kernel in eager passes of "
-                                          "the same step; the headline region replays a CUDA graph, inside "
-                                          "which single launches cannot be bracketed")
+            line["roofline"]["timing"] = ("CUDA events around every launch of this kernel in eager, single-stream "
+                                          "passes of the same step; the headline region replays CUDA graphs, "
+                                          "inside which single launches cannot be bracketed")
         if not args.no_cpu_baseline:
             from oracle import oracle as O
             O.build()

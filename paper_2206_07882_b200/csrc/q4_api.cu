@@ -801,6 +801,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       return Q4_OK;
     };
 
+    const bool fused_head = D == 256;   // the fused LM head kernel is built for a 256-wide bottleneck
     // 1a. prediction network, then the joint network for every live slot (stream sp)
     Q4_CHECK(lstm_mma(sp, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
                       st.pred_c, pred_h8));
@@ -833,10 +834,33 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
         last = &L1;
       }
       const int head_tag = which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD;
-      Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 1 : 3, lm.bott, top8, last->hid_act.scale, EPI_QUANT8,
-                          bq8[which], D, nullptr, &lm.bott_act, n_active));
-      Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
-                          V, cst.adv_dst, nullptr, n_active));
+      if (fused_head) {
+        // bottleneck, re-quantization, output layer and log-softmax in one kernel
+        TagScope tag(head_tag);
+        LmHeadArgs ha;
+        memset(&ha, 0, sizeof(ha));
+        ha.N = N;
+        ha.H = last->w_hh.k_pad;
+        ha.V = V;
+        ha.x_scale = last->hid_act.scale;
+        ha.sc_bott = lm.bott.w.scale;
+        ha.b_bott = lm.bott.bias;
+        ha.bott_act = lm.bott_act;
+        ha.q_scale = lm.bott_act.scale;
+        ha.sc_out = lm.out.w.scale;
+        ha.b_out = lm.out.bias;
+        ha.lp = lp;
+        ha.dst_row = cst.adv_dst;
+        ha.n_active = n_active;
+        ha.status = st.status;
+        Q4_TRY(launch_mma_lmhead(ha, top8, ha.H, reinterpret_cast<const int8_t*>(pb + pp.lin[which == 0 ? 1 : 3]),
+                                 reinterpret_cast<const int8_t*>(pb + pp.lin[which == 0 ? 2 : 4]), sl));
+      } else {
+        Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 1 : 3, lm.bott, top8, last->hid_act.scale, EPI_QUANT8,
+                            bq8[which], D, nullptr, &lm.bott_act, n_active));
+        Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
+                            V, cst.adv_dst, nullptr, n_active));
+      }
     }
     if (forked) {   // join: the call's stream waits for both side chains
       cudaEvent_t j0 = reinterpret_cast<cudaEvent_t>(st.aux_event[1]);
@@ -846,7 +870,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       Q4_TRY(cudaStreamWaitEvent(s, j0, 0));
       Q4_TRY(cudaStreamWaitEvent(s, j1, 0));
     }
-    {  // log-softmax of both LMs' new rows in one launch
+    if (!fused_head) {  // log-softmax of both LMs' new rows in one launch
       TagScope tag(TAG_TGT_HEAD);
       Q4_TRY(launch_logsoftmax(st.src_lp, st.src_lp, N, V, V, cst.adv_dst, s, st.tgt_lp, n_active));
     }

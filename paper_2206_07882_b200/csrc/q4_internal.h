@@ -76,6 +76,22 @@ struct MmaLstmArgs {
   int32_t* status;
   const int32_t* n_active;  // optional: rows >= *n_active carry no work (tiles beyond it exit at once)
 };
+struct LmHeadArgs {
+  int32_t N, H, V;            // launch rows, LSTM width (K of the bottleneck), vocabulary
+  float x_scale;              // scale of the cell-output codes feeding the bottleneck
+  const float* sc_bott;       // [256] bottleneck row scales
+  const float* b_bott;        // [256] bias (nullable)
+  q4_act bott_act;            // quantizer of the bottleneck output
+  float q_scale;              // = bott_act.scale
+  const float* sc_out;        // [V] output-layer row scales
+  const float* b_out;         // [V] bias (nullable)
+  float* lp;                  // [*, V] log-probabilities, row dst_row[n]
+  const int32_t* dst_row;     // nullptr = n, negative = skip
+  const int32_t* n_active;
+  int32_t* status;
+};
+cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h_pitch, const int8_t* wb8,
+                              const int8_t* wo8, cudaStream_t s);
 enum { EPI_QUANT8 = 3 };    // re-quantize and store (code - zero_point) as int8, one per byte
 cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
                                const q4_act& act, int k_pad, int n_rows, int8_t* dst,
