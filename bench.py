@@ -274,6 +274,8 @@ def main():
     ap.add_argument("--workload", default="cfg4_end_to_end", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-frames", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-dependent-launch", action="store_true",
+                    help="launch the beam step's kernels in plain stream order")
     ap.add_argument("--eager", action="store_true",
                     help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
@@ -296,6 +298,9 @@ def main():
 
     from paper_2206_07882_b200 import binding as Bd
     lib = Bd.lib()
+    if args.no_dependent_launch:
+        from paper_2206_07882_b200 import binding as _Bd
+        _Bd.dependent_launch_set(False)
     job = Job(args.workload, rank)
     wl = job.wl
     B, T, U = wl["B"], wl["T"], wl["U_max"]

@@ -314,6 +314,13 @@ int q4_poll_status(const int32_t* device_status, q4_stream stream);
 int q4_version(void);
 int64_t q4_launch_count(void);
 
+/* dr_fusion_beam_step launches consecutive kernels of one stream as programmatic dependents
+ * (each kernel sets itself up while its predecessor drains and waits for the predecessor's
+ * completion before it reads anything).  enabled = 0 switches this off (plain stream order),
+ * non-zero switches it on (the default).  Returns the previous setting.  Results do not depend
+ * on it.  Not an operation of the paper. */
+int q4_dependent_launch_set(int32_t enabled);
+
 /* Optional timing of the library's own launches with CUDA events lent by the caller (host
  * arrays of cudaEvent_t, `capacity` entries each).  Every launch whose tag bit is set in
  * tag_mask records start_events[i] before and stop_events[i] after itself on the stream it

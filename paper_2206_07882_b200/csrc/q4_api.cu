@@ -84,6 +84,11 @@ int q4_timing_set(uint32_t tag_mask, void** start_events, void** stop_events, in
 }
 int q4_timing_count(void) { return timing_count(); }
 int64_t q4_launch_count(void) { return g_launches; }
+int q4_dependent_launch_set(int32_t enabled) {
+  const int prev = g_dependent_launch;
+  g_dependent_launch = enabled ? 1 : 0;
+  return prev;
+}
 
 int q4_act_symmetric(float alpha, int32_t bits, q4_act* out) {
   if (!out) return Q4_ERR_NULL;
@@ -746,7 +751,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       uj.zero_tail = 0;   // rows beyond the pending advances feed tiles whose results are dropped
       uj.n_active = n_active;
       TagScope tag(TAG_MISC);
-      Q4_TRY(launch_unpack_multi(uj, s));
+      Q4_TRY(launch_unpack_multi(uj, s, true));
     }
     // the three networks are independent until the selection: with two lent streams the
     // prediction/joint chain and the source-LM chain run beside the target-LM chain
@@ -762,7 +767,9 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       Q4_TRY(cudaStreamWaitEvent(ss, fork, 0));
     }
     // one LSTM layer of one network for every pending slot
-    auto lstm_mma = [&](cudaStream_t s, int tag_id, int li, const q4_lstm& L, const q4_act& x_act,
+    // `dep`: the previous launch on the same stream is a kernel of this library, so this one may
+    // be launched as its programmatic dependent
+    auto lstm_mma = [&](cudaStream_t s, bool dep, int tag_id, int li, const q4_lstm& L, const q4_act& x_act,
                         const int8_t* xa, const int8_t* ha, void* hq, float* c, int8_t* h8) -> int {
       TagScope tag(tag_id);
       const int H = L.w_hh.k_pad, Kx = L.w_ih.k_pad;
@@ -788,30 +795,30 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       a.status = st.status;
       a.n_active = n_active;
       Q4_TRY(launch_mma_lstm(a, xa, Kx, reinterpret_cast<const int8_t*>(pb + pp.lstm[li].xw), Kx, ha, H,
-                             reinterpret_cast<const int8_t*>(pb + pp.lstm[li].hw), H, s));
+                             reinterpret_cast<const int8_t*>(pb + pp.lstm[li].hw), H, s, dep));
       return Q4_OK;
     };
-    auto linear_mma = [&](cudaStream_t s, int tag_id, int wi, const q4_linear& L, const int8_t* x8,
+    auto linear_mma = [&](cudaStream_t s, bool dep, int tag_id, int wi, const q4_linear& L, const int8_t* x8,
                           float x_scale, int epi, void* out, long long ldo, const int32_t* out_idx,
                           const q4_act* out_act, const int32_t* rows_active) -> int {
       TagScope tag(tag_id);
       Q4_TRY(launch_mma_gemm(x8, L.w.k_pad, N, reinterpret_cast<const int8_t*>(pb + pp.lin[wi]), L.w.k_pad,
                              L.w.rows, L.w.k_pad, epi, out, ldo, out_idx, L.w.scale, L.bias, x_scale, out_act,
-                             st.status, rows_active, s));
+                             st.status, rows_active, s, dep));
       return Q4_OK;
     };
 
     const bool fused_head = D == 256;   // the fused LM head kernel is built for a 256-wide bottleneck
     // 1a. prediction network, then the joint network for every live slot (stream sp)
-    Q4_CHECK(lstm_mma(sp, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
+    Q4_CHECK(lstm_mma(sp, !forked, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
                       st.pred_c, pred_h8));
-    Q4_CHECK(linear_mma(sp, TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
+    Q4_CHECK(linear_mma(sp, true, TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
                         st.pred_p, D, cst.adv_dst, nullptr, n_active));
     {
       TagScope tag(TAG_JOINT);
-      Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, sp));
+      Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, sp, true));
     }
-    Q4_CHECK(linear_mma(sp, TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr,
+    Q4_CHECK(linear_mma(sp, true, TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr,
                         nullptr));
     // 1b. source LM (stream ss) and target LM (the call's stream)
     for (int which = 0; which < 2; ++which) {
@@ -822,13 +829,13 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       float* c0 = which == 0 ? st.src_c : st.tgt_c[0];
       int8_t* h8_0 = which == 0 ? src_h8 : tgt_h8[0];
       float* lp = which == 0 ? st.src_lp : st.tgt_lp;
-      Q4_CHECK(lstm_mma(sl, which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, which == 0 ? 1 : 2, L0, lm.emb_act,
+      Q4_CHECK(lstm_mma(sl, which == 1 || !forked, which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, which == 0 ? 1 : 2, L0, lm.emb_act,
                         xa8[which + 1], ha8[which + 1], hq0, c0, h8_0));
       const int8_t* top8 = h8_0;
       const q4_lstm* last = &L0;
       if (lm.n_layers == 2) {
         const q4_lstm& L1 = lm.lstm[1];
-        Q4_CHECK(lstm_mma(sl, TAG_TGT_L2, 3, L1, L0.hid_act, h8_0, ha8[3], st.tgt_hq[1], st.tgt_c[1],
+        Q4_CHECK(lstm_mma(sl, true, TAG_TGT_L2, 3, L1, L0.hid_act, h8_0, ha8[3], st.tgt_hq[1], st.tgt_c[1],
                           tgt_h8[1]));
         top8 = tgt_h8[1];
         last = &L1;
@@ -854,11 +861,11 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
         ha.n_active = n_active;
         ha.status = st.status;
         Q4_TRY(launch_mma_lmhead(ha, top8, ha.H, reinterpret_cast<const int8_t*>(pb + pp.lin[which == 0 ? 1 : 3]),
-                                 reinterpret_cast<const int8_t*>(pb + pp.lin[which == 0 ? 2 : 4]), sl));
+                                 reinterpret_cast<const int8_t*>(pb + pp.lin[which == 0 ? 2 : 4]), sl, true));
       } else {
-        Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 1 : 3, lm.bott, top8, last->hid_act.scale, EPI_QUANT8,
+        Q4_CHECK(linear_mma(sl, true, head_tag, which == 0 ? 1 : 3, lm.bott, top8, last->hid_act.scale, EPI_QUANT8,
                             bq8[which], D, nullptr, &lm.bott_act, n_active));
-        Q4_CHECK(linear_mma(sl, head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
+        Q4_CHECK(linear_mma(sl, true, head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
                             V, cst.adv_dst, nullptr, n_active));
       }
     }

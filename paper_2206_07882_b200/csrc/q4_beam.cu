@@ -263,6 +263,7 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     }
   }
   __syncthreads();
+  pdl_trigger();   // only the bookkeeping is left: the next kernel of the stream may set itself up
 
   if (warp == 0) {
     const int n_win = min(min(list_n, cap), W);

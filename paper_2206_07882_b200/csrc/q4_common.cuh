@@ -9,6 +9,15 @@
 
 namespace q4 {
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
+// start while its predecessor in the stream is still running; pdl_wait() returns once that
+// predecessor has completed and its writes are visible (at once when the launch carries no such
+// attribute), pdl_trigger() lets the successor's CTAs be scheduled once every CTA of this grid
+// has called it or exited.  Nothing produced by an earlier kernel is read before pdl_wait().
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+
 constexpr int TILE = 64;        // rows of each operand per CTA tile
 constexpr int KC = 128;         // K elements staged per chunk
 constexpr int PITCH = KC + 16;  // shared-memory row pitch in bytes (16 B aligned, conflict-free)

@@ -12,7 +12,7 @@ cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long
 cudaError_t launch_joint_z(const float* e, const int32_t* frame_idx, const int32_t* t_arr, int B,
                            int W, const float* p, const int32_t* p_idx, int N, int D,
                            const q4_act& za, uint8_t* zq, int8_t* z8, int32_t* live_out,
-                           cudaStream_t s);
+                           cudaStream_t s, bool dependent = false);
 cudaError_t launch_quantize(const void* x, bool fp16, long long rows, int k, int k_pad,
                             const q4_act& a, int mode, int n_groups, const float* scale_vec,
                             uint8_t* out, float* group_scale_out, cudaStream_t s);
@@ -91,7 +91,7 @@ struct LmHeadArgs {
   int32_t* status;
 };
 cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h_pitch, const int8_t* wb8,
-                              const int8_t* wo8, cudaStream_t s);
+                              const int8_t* wo8, cudaStream_t s, bool dependent = false);
 enum { EPI_QUANT8 = 3 };    // re-quantize and store (code - zero_point) as int8, one per byte
 cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
                                const q4_act& act, int k_pad, int n_rows, int8_t* dst,
@@ -109,7 +109,7 @@ struct UnpackJobs {
   int32_t n_jobs, n_rows, n_rows_pad, zero_tail;
   const int32_t* n_active;
 };
-cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s);
+cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s, bool dependent = false);
 cudaError_t launch_prepare_w(const q4_mat& w, int interleave, int8_t* dst, long long dst_stride,
                              int col0, cudaStream_t s);
 cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s);
@@ -117,10 +117,10 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
                             const int32_t* out_idx, const float* w_scale, const float* bias,
                             float x_scale, const q4_act* out_act, int32_t* status,
-                            const int32_t* n_active, cudaStream_t s);
+                            const int32_t* n_active, cudaStream_t s, bool dependent = false);
 cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa_pitch,
                             const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
-                            const int8_t* hw, long long hw_pitch, cudaStream_t s);
+                            const int8_t* hw, long long hw_pitch, cudaStream_t s, bool dependent = false);
 
 // ---- persistent encoder recurrence (q4_recurrent.cu)
 struct EncRecDir {
@@ -148,5 +148,36 @@ bool enc_recurrent_supported(int H, int B, int dirs);
 cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s);
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+// Kernel launch with optional attributes: `dependent` asks for programmatic stream
+// serialization (the kernel calls pdl_wait() before it touches its inputs), cluster_x > 1 for a
+// thread-block cluster along x.
+extern int g_dependent_launch;   // 0 switches the attribute off everywhere
+template <typename... KA, typename... A>
+inline cudaError_t launch_ex(void (*kern)(KA...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                             bool dependent, unsigned cluster_x, A&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[2];
+  unsigned n = 0;
+  if (cluster_x > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = cluster_x;
+    at[n].val.clusterDim.y = 1;
+    at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (dependent && g_dependent_launch) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<A&&>(args)...);
+}
 
 }  // namespace q4

@@ -8,6 +8,7 @@ namespace q4 {
 
 int64_t g_launches = 0;
 int g_tag = TAG_NONE;
+int g_dependent_launch = 1;
 
 // Optional event timing of tagged launches: the caller lends pairs of CUDA events; every
 // launch whose tag is enabled records one pair on its own stream.  Off by default.
@@ -469,6 +470,8 @@ __global__ void __launch_bounds__(256) k_joint_z(const float* e, const int32_t* 
                                                  const int32_t* t_arr, int B, int W, const float* p,
                                                  const int32_t* p_idx, int N, int D, q4_act za,
                                                  uint8_t* zq, int8_t* z8, int32_t* live_out) {
+  pdl_trigger();
+  pdl_wait();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int half = D >> 1;
   if (i >= (long long)N * half) return;
@@ -497,15 +500,15 @@ __global__ void __launch_bounds__(256) k_joint_z(const float* e, const int32_t* 
 cudaError_t launch_joint_z(const float* e, const int32_t* frame_idx, const int32_t* t_arr, int B,
                            int W, const float* p, const int32_t* p_idx, int N, int D,
                            const q4_act& za, uint8_t* zq, int8_t* z8, int32_t* live_out,
-                           cudaStream_t s) {
+                           cudaStream_t s, bool dependent) {
   if (N <= 0) return cudaSuccess;
   const long long total = (long long)N * (D / 2);
   timing_begin(s);
-  k_joint_z<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(e, frame_idx, t_arr, B, W, p, p_idx, N,
-                                                            D, za, zq, z8, live_out);
+  cudaError_t le = launch_ex(k_joint_z, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, dependent, 1, e,
+                             frame_idx, t_arr, B, W, p, p_idx, N, D, za, zq, z8, live_out);
   timing_end(s);
   ++g_launches;
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 // =====================================================================================

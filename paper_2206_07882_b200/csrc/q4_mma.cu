@@ -89,6 +89,8 @@ cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int3
 
 // Several gather+unpack jobs in one launch (blockIdx.y selects the job).
 __global__ void __launch_bounds__(256) k_unpack_multi(const UnpackJobs jobs) {
+  pdl_trigger();
+  pdl_wait();
   const UnpackJob& j = jobs.job[blockIdx.y];
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = j.k_pad >> 5;
@@ -137,17 +139,17 @@ __global__ void __launch_bounds__(256) k_unpack_multi(const UnpackJobs jobs) {
   d[1] = o1;
 }
 
-cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s) {
+cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s, bool dependent) {
   if (jobs.n_jobs <= 0) return cudaSuccess;
   int kmax = 0;
   for (int i = 0; i < jobs.n_jobs; ++i) kmax = jobs.job[i].k_pad > kmax ? jobs.job[i].k_pad : kmax;
   const long long total = (long long)jobs.n_rows_pad * (kmax >> 5);
   dim3 grid((unsigned)((total + 255) / 256), jobs.n_jobs);
   timing_begin(s);
-  k_unpack_multi<<<grid, 256, 0, s>>>(jobs);
+  cudaError_t e = launch_ex(k_unpack_multi, grid, dim3(256), 0, s, dependent, 1, jobs);
   timing_end(s);
   ++g_launches;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // Weight preparation: unpack to int8; with `interleave` the 4H rows (gate-major i,f,g,o) are
@@ -270,9 +272,8 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
   __shared__ uint32_t tmem_base_s;
   __shared__ float s_sc[GEMM_BN], s_bi[GEMM_BN];   // de-quantization constants of this tile's columns
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * GEMM_BN;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * GEMM_BN;   // row tiles slowest: tiles with work are dispatched first
   const int nk = (a.K + BK - 1) / BK;
-  if (a.n_active && m0 >= *a.n_active) return;   // whole tile without work (uniform per CTA)
 
   if (tid == 0) {
     for (int s = 0; s < GEMM_STAGES; ++s) {
@@ -284,14 +285,20 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
     fence_proxy_async();
   }
   if (warp == 5) tmem_alloc(&tmem_base_s, GEMM_BN);
+  if (warp == 4 && lane == 0) {
+    prefetch_tmap(&tma_a);
+    prefetch_tmap(&tma_b);
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
+  pdl_wait();   // everything above overlaps the tail of the previous kernel of the stream
+  const bool has_work = !(a.n_active && m0 >= *a.n_active);   // uniform per CTA
 
-  if (warp == 4 && lane == 0) {
-    prefetch_tmap(&tma_a);
-    prefetch_tmap(&tma_b);
+  if (!has_work) {
+    // whole tile without work
+  } else if (warp == 4 && lane == 0) {
     bool ok = true;
     for (int i = 0; i < nk && ok; ++i) {
       const int s = i % GEMM_STAGES;
@@ -301,6 +308,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
       tma_load_2d(smem + s * STAGE, &tma_a, i * BK, m0, &full[s]);
       tma_load_2d(smem + s * STAGE + A_BYTES, &tma_b, i * BK, n0, &full[s]);
     }
+    pdl_trigger();
     if (!ok) flag_timeout(a.status);
   } else if (warp == 5 && lane == 0) {
     const uint32_t idesc = umma_idesc_i8(BM, GEMM_BN);
@@ -317,6 +325,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
       umma_commit(&empty[s]);
     }
     umma_commit(&acc_full);
+    pdl_trigger();
     if (!ok) flag_timeout(a.status);
   } else if (warp < 4) {
     if (a.epi != EPI_I32) {   // stage scale * row scale and bias while the MMAs run
@@ -329,6 +338,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
     }
     const bool ok = mbar_wait(&acc_full, 0);
     tc_fence_after();
+    pdl_trigger();   // the main loop is over: the next kernel may set itself up
     if (!ok && lane == 0) flag_timeout(a.status);
     const int mi = m0 + warp * 32 + lane;
     int m = -1;
@@ -388,6 +398,8 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
         }
       }
     }
+  } else {
+    pdl_trigger();   // idle lanes of the producer and issuer warps
   }
   tc_fence_before();
   __syncthreads();
@@ -399,7 +411,7 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
                             const int32_t* out_idx, const float* w_scale, const float* bias,
                             float x_scale, const q4_act* out_act, int32_t* status,
-                            const int32_t* n_active, cudaStream_t s) {
+                            const int32_t* n_active, cudaStream_t s, bool dependent) {
   if (M <= 0 || J <= 0) return cudaSuccess;
   CUtensorMap ta, tb;
   if (!make_tmap_i8(&ta, x8, K, M, x_pitch, BM) || !make_tmap_i8(&tb, w8, K, J, w_pitch, GEMM_BN))
@@ -426,12 +438,12 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid((M + BM - 1) / BM, (J + GEMM_BN - 1) / GEMM_BN);
+  dim3 grid((J + GEMM_BN - 1) / GEMM_BN, (M + BM - 1) / BM);
   timing_begin(s);
-  k_mma_gemm<<<grid, 192, smem, s>>>(ta, tb, a);
+  cudaError_t le = launch_ex(k_mma_gemm, grid, dim3(192), smem, s, dependent, 1, ta, tb, a);
   timing_end(s);
   ++g_launches;
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 // ------------------------------------------------------------------ fused LM head
@@ -470,10 +482,9 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
   __shared__ float red_m[4][BM], red_s[4][BM];
   __shared__ float part_m[HEAD_MAX_BLOCKS][BM], part_s[HEAD_MAX_BLOCKS][BM];   // filled by every CTA of the cluster
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int m0 = blockIdx.x * BM;
-  const int nb = blockIdx.y;                    // my block of output columns = my cluster rank
-  const int nblk = gridDim.y;
-  if (a.n_active && m0 >= *a.n_active) return;  // whole row tile without work: the whole cluster leaves
+  const int m0 = blockIdx.y * BM;
+  const int nb = blockIdx.x;                    // my block of output columns = my cluster rank
+  const int nblk = gridDim.x;
   const int nk1 = (a.H + BK - 1) / BK;
   const int nloads = nk1 + 2;
 
@@ -493,6 +504,11 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
+  pdl_wait();   // everything above overlaps the tail of the previous kernel of the stream
+  if (a.n_active && m0 >= *a.n_active) {   // whole row tile without work: the whole cluster leaves
+    if (warp == HEAD_EPI_WARPS + 1) tmem_dealloc(tmem, 512);
+    return;
+  }
   cl_barrier();   // every CTA of the cluster is running before anyone stores into a peer's shared memory
 
   if (warp == HEAD_EPI_WARPS && lane == 0) {
@@ -513,6 +529,7 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
         tma_load_2d(smem + s * STAGE + A_BYTES, &tma_wo, (i - nk1) * BK, nb * HEAD_D, &full[s]);
       }
     }
+    pdl_trigger();
     if (!ok) flag_timeout(a.status);
   } else if (warp == HEAD_EPI_WARPS + 1 && lane == 0) {
     // ---- MMA issuer
@@ -545,6 +562,7 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
       umma_commit(&empty[s]);
     }
     umma_commit(&acc2_full);
+    pdl_trigger();
     if (!ok) flag_timeout(a.status);
   } else if (warp < HEAD_EPI_WARPS) {
     // ---- epilogue: warp = (lane quarter q, column share cs)
@@ -594,6 +612,7 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
     // my 64 logits of this block, kept in registers until the row's log-sum-exp is known
     if (ok) ok = mbar_wait(&acc2_full, 0);
     tc_fence_after();
+    pdl_trigger();   // both GEMMs are over: the next kernel may set itself up
     float v[64];
     float my_m = -INFINITY;
 #pragma unroll
@@ -649,7 +668,10 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
     if (!ok && lane == 0) flag_timeout(a.status);
   }
   __syncwarp();
-  if (warp >= HEAD_EPI_WARPS) cl_barrier();   // the producer and issuer warps join the cluster barrier too
+  if (warp >= HEAD_EPI_WARPS) {
+    pdl_trigger();
+    cl_barrier();
+  }   // the producer and issuer warps join the cluster barrier too
   tc_fence_before();
   __syncthreads();
   if (warp == HEAD_EPI_WARPS + 1) tmem_dealloc(tmem, 512);
@@ -657,7 +679,7 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
 }
 
 cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h_pitch, const int8_t* wb8,
-                              const int8_t* wo8, cudaStream_t s) {
+                              const int8_t* wo8, cudaStream_t s, bool dependent) {
   if (a.N <= 0) return cudaSuccess;
   const int rows_pad = (a.N + BM - 1) / BM * BM;
   const int nblk = (a.V + HEAD_D - 1) / HEAD_D;
@@ -673,20 +695,9 @@ cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(rows_pad / BM, nblk);
-  cfg.blockDim = dim3(HEAD_THREADS);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = s;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = 1;
-  at[0].val.clusterDim.y = nblk;
-  at[0].val.clusterDim.z = 1;
-  cfg.attrs = at;
-  cfg.numAttrs = 1;
   timing_begin(s);
-  cudaError_t e = cudaLaunchKernelEx(&cfg, k_mma_lmhead, th, tb, to, a);
+  cudaError_t e = launch_ex(k_mma_lmhead, dim3(nblk, rows_pad / BM), dim3(HEAD_THREADS), smem, s, dependent,
+                            (unsigned)nblk, th, tb, to, a);
   timing_end(s);
   ++g_launches;
   return e != cudaSuccess ? e : cudaGetLastError();
@@ -704,11 +715,10 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
   __shared__ uint64_t full[LSTM_STAGES], empty[LSTM_STAGES], acc_full;
   __shared__ uint32_t tmem_base_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * LSTM_BN;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * LSTM_BN;   // row tiles slowest: tiles with work are dispatched first
   const int nkx = a.acc_pre ? 0 : (a.Kx_pad + BK - 1) / BK;
   const int nkh = (a.H + BK - 1) / BK;
   const int nk = nkx + nkh;
-  if (a.n_active && m0 >= *a.n_active) return;   // whole tile without work (uniform per CTA)
 
   if (tid == 0) {
     for (int s = 0; s < LSTM_STAGES; ++s) {
@@ -724,8 +734,12 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
+  pdl_wait();   // everything above overlaps the tail of the previous kernel of the stream
+  const bool has_work = !(a.n_active && m0 >= *a.n_active);   // uniform per CTA
 
-  if (warp == LSTM_EPI_WARPS && lane == 0) {
+  if (!has_work) {
+    // whole tile without work
+  } else if (warp == LSTM_EPI_WARPS && lane == 0) {
     bool ok = true;
     for (int i = 0; i < nk && ok; ++i) {
       const int s = i % LSTM_STAGES;
@@ -740,6 +754,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
         tma_load_2d(smem + s * STAGE + A_BYTES, &tma_hw, (i - nkx) * BK, n0, &full[s]);
       }
     }
+    pdl_trigger();
     if (!ok) flag_timeout(a.status);
   } else if (warp == LSTM_EPI_WARPS + 1 && lane == 0) {
     const uint32_t idesc = umma_idesc_i8(BM, LSTM_BN);
@@ -759,6 +774,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
       umma_commit(&empty[s]);
     }
     umma_commit(&acc_full);
+    pdl_trigger();
     if (!ok) flag_timeout(a.status);
   } else if (warp < LSTM_EPI_WARPS) {
     const int q = warp & 3, hf = warp >> 2;
@@ -771,6 +787,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
     }
     const bool ok = mbar_wait(&acc_full, 0);
     tc_fence_after();
+    pdl_trigger();   // the main loop is over: the next kernel may set itself up
     if (!ok && lane == 0) flag_timeout(a.status);
     const bool live = ok && dst >= 0;
     const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
@@ -850,6 +867,8 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
               (uint32_t)(qy[0] & 0xFF) | ((uint32_t)(qy[1] & 0xFF) << 8) | ((uint32_t)(qy[2] & 0xFF) << 16) | ((uint32_t)(qy[3] & 0xFF) << 24);
       }
     }
+  } else {
+    pdl_trigger();   // idle lanes of the producer and issuer warps
   }
   tc_fence_before();
   __syncthreads();
@@ -860,7 +879,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
 // ha int8 [rows_pad, H], hw int8 [4H, H] interleaved.  rows_pad = N rounded up to 128.
 cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa_pitch,
                             const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
-                            const int8_t* hw, long long hw_pitch, cudaStream_t s) {
+                            const int8_t* hw, long long hw_pitch, cudaStream_t s, bool dependent) {
   if (a.N <= 0) return cudaSuccess;
   const int rows_pad = (a.N + BM - 1) / BM * BM;
   CUtensorMap txa, txw, tha, thw;
@@ -880,12 +899,13 @@ cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid(rows_pad / BM, (4 * a.H + LSTM_BN - 1) / LSTM_BN);
+  dim3 grid((4 * a.H + LSTM_BN - 1) / LSTM_BN, rows_pad / BM);
   timing_begin(s);
-  k_mma_lstm<<<grid, 32 * (LSTM_EPI_WARPS + 2), smem, s>>>(txa, txw, tha, thw, a);
+  cudaError_t le = launch_ex(k_mma_lstm, grid, dim3(32 * (LSTM_EPI_WARPS + 2)), smem, s, dependent, 1, txa, txw,
+                             tha, thw, a);
   timing_end(s);
   ++g_launches;
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace q4
