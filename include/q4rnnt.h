@@ -321,6 +321,12 @@ int64_t q4_launch_count(void);
  * on it.  Not an operation of the paper. */
 int q4_dependent_launch_set(int32_t enabled);
 
+/* The beam selection first bounds the W-th best proposal from below by the smallest of 16
+ * group maxima and ranks the few proposals above that bound; if they overflow its short list
+ * it falls back to an exact bit-by-bit threshold search.  enabled != 0 makes every selection
+ * take the exact search (for tests; both give the same beam).  Returns the previous setting. */
+int q4_beam_select_exact_set(int32_t enabled);
+
 /* Optional timing of the library's own launches with CUDA events lent by the caller (host
  * arrays of cudaEvent_t, `capacity` entries each).  Every launch whose tag bit is set in
  * tag_mask records start_events[i] before and stop_events[i] after itself on the stream it

@@ -76,7 +76,7 @@ class BeamStateS(C.Structure):
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
-           "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static"]
+           "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_beam_select_exact_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static"]
 
 _lib = None
 
@@ -124,6 +124,11 @@ def launch_count() -> int:
 def dependent_launch_set(enabled: bool) -> bool:
     """Switch programmatic dependent launches of the beam step on or off; returns the previous setting."""
     return bool(lib().q4_dependent_launch_set(1 if enabled else 0))
+
+
+def beam_select_exact_set(enabled: bool) -> bool:
+    """Force the exact threshold search in every beam selection (tests); returns the previous setting."""
+    return bool(lib().q4_beam_select_exact_set(1 if enabled else 0))
 
 
 def workspace_bytes(call_id: int, dims: Sequence[int]) -> int:

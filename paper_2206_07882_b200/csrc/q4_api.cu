@@ -84,6 +84,13 @@ int q4_timing_set(uint32_t tag_mask, void** start_events, void** stop_events, in
 }
 int q4_timing_count(void) { return timing_count(); }
 int64_t q4_launch_count(void) { return g_launches; }
+static int g_select_exact = 0;
+static int select_exact_only() { return g_select_exact; }
+int q4_beam_select_exact_set(int32_t enabled) {
+  const int prev = g_select_exact;
+  g_select_exact = enabled ? 1 : 0;
+  return prev;
+}
 int q4_dependent_launch_set(int32_t enabled) {
   const int prev = g_dependent_launch;
   g_dependent_launch = enabled ? 1 : 0;
@@ -656,6 +663,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   cudaStream_t s = S(stream);
   const q4_beam_state& st = *state;
   const int N = B * W;
+  int joint_normalized = 0;   // the tensor-core joint kernel leaves log-probabilities, not logits
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   uint8_t* zq = ws;
   ws += align_up((size_t)N * D);
@@ -808,7 +816,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       return Q4_OK;
     };
 
-    const bool fused_head = D == 256;   // the fused LM head kernel is built for a 256-wide bottleneck
+    const bool fused_head = D == 256 && V <= 2048;   // the fused head kernel: 256-wide bottleneck, one cluster per row tile
     // 1a. prediction network, then the joint network for every live slot (stream sp)
     Q4_CHECK(lstm_mma(sp, !forked, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
                       st.pred_c, pred_h8));
@@ -818,8 +826,26 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       TagScope tag(TAG_JOINT);
       Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, sp, true));
     }
-    Q4_CHECK(linear_mma(sp, true, TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr,
-                        nullptr));
+    joint_normalized = fused_head ? 1 : 0;
+    if (fused_head) {
+      // output layer of the joint network with the log-softmax over the vocabulary in its epilogue
+      TagScope tag(TAG_JOINT);
+      LmHeadArgs ja;
+      memset(&ja, 0, sizeof(ja));
+      ja.N = N;
+      ja.H = 0;
+      ja.V = V;
+      ja.q_scale = m.z_act.scale;
+      ja.sc_out = m.joint_out.w.scale;
+      ja.b_out = m.joint_out.bias;
+      ja.lp = logits;
+      ja.dst_row = live;
+      ja.status = st.status;
+      Q4_TRY(launch_mma_lmhead(ja, z8, D, nullptr, reinterpret_cast<const int8_t*>(pb + pp.lin[5]), sp, true));
+    } else {
+      Q4_CHECK(linear_mma(sp, true, TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr,
+                          nullptr));
+    }
     // 1b. source LM (stream ss) and target LM (the call's stream)
     for (int which = 0; which < 2; ++which) {
       const q4_lm& lm = *lms[which];
@@ -950,8 +976,10 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   sel.lambda_t = lambda_t;
   sel.lambda_s = lambda_s;
   sel.rho = rho;
+  sel.exact_only = select_exact_only();
+  sel.normalized = joint_normalized;
   TagScope tag_sel(TAG_SELECT);
-  Q4_TRY(launch_beam_select(sel, s));
+  Q4_TRY(launch_beam_select(sel, s, use_mma));
   return Q4_OK;
 }
 

@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
   __shared__ int list_n;
   __shared__ int win_idx[MAXW];
   __shared__ float win_score[MAXW];
+  __shared__ float s_gmax[SEL_NT / 32][16];   // per warp: best label proposal of lanes g and g + 16
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.x;
@@ -64,7 +65,19 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
   const q4_beam_state& st = a.st;
   const float NEG = -INFINITY;
   const int N = a.B * W;
+  const bool fast = V <= 1024 && W <= SEL_NT / 32 && !a.exact_only;   // one warp per slot, row in registers
 
+  pdl_wait();
+  // the joint logits of slot `warp` do not depend on the beam state: request them first
+  float v[32];
+  if (fast && warp < W) {
+    const float* x = a.logits + (size_t)(base + warp) * V;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int k = lane + 32 * i;
+      v[i] = k < V ? x[k] : NEG;
+    }
+  }
   if (tid < W) {
     const int o = base + tid;
     s_row[tid] = st.row[o];
@@ -80,83 +93,126 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     // the list of pending advances consumed by this iteration is free again
     if (b == 0) st.pend_n[a.iter & 1] = 0;
   }
+  if (lane < 16) s_gmax[warp][lane] = NEG;
   __syncthreads();
 
-  // ---- proposals: one warp per slot; the row of logits is read once and kept in registers
-  for (int w = warp; w < W; w += SEL_NT / 32) {
-    float* cw = cand + (size_t)w * V;
-    const int row = s_row[w];
-    if (row < 0) {
-      for (int k = lane; k < V; k += 32) cw[k] = NEG;
-      continue;
-    }
-    const float* x = a.logits + (size_t)(base + w) * V;
-    const float* lt = a.tgt_lp + (size_t)row * V;
-    const float* ls = a.src_lp + (size_t)row * V;
-    const double S = (double)s_score[w];
-    const double rho_d = (double)a.rho;
-    const bool labels = s_u[w] < a.u_max;
-    if (V <= 1024) {
-      // one round trip to memory: logits and both LM rows are requested together
-      float xv[32], ltv[32], lsv[32];
+  // ---- proposals
+  uint32_t skip = 0;   // fast path: bit i = element lane + 32 i is not a label proposal that can win
+  if (fast) {
+    if (warp < W) {
+      const int w = warp;
+      float* cw = cand + (size_t)w * V;
+      const int row = s_row[w];
+      const bool labels = row >= 0 && s_u[w] < a.u_max;
+      if (row < 0) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const int k = lane + 32 * i;
-        xv[i] = k < V ? x[k] : NEG;
-        ltv[i] = (k < V && labels) ? lt[k] : 0.0f;
-        lsv[i] = (k < V && labels) ? ls[k] : 0.0f;
-      }
-      float m = NEG;
-#pragma unroll
-      for (int i = 0; i < 32; ++i) m = fmaxf(m, xv[i]);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      float sum = 0.0f;
-#pragma unroll
-      for (int i = 0; i < 32; ++i) sum += expf(xv[i] - m);   // exp(-inf) = 0 for the padding
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      const float lse = m + logf(sum);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const int k = lane + 32 * i;
-        if (k >= V) continue;
-        const float lp = xv[i] - lse;
-        float v;
-        if (k == 0) {
-          v = (float)(S + (double)lp);
-        } else if (labels) {
-          // label increment in fp32 (magnitude of tens), one double add onto the running score
-          const float inc = __fmaf_rn(a.lambda_t, ltv[i], __fmaf_rn(-a.lambda_s, lsv[i], lp));
-          v = (float)(S + (double)inc + rho_d);
-        } else {
-          v = NEG;
+        for (int i = 0; i < 32; ++i) {
+          const int k = lane + 32 * i;
+          if (k < V) cw[k] = NEG;
         }
-        cw[k] = v;
+        skip = 0xFFFFFFFFu;
+      } else {
+        // one round trip to memory for both LM rows
+        float ltv[32], lsv[32];
+        const float* lt = a.tgt_lp + (size_t)row * V;
+        const float* ls = a.src_lp + (size_t)row * V;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int k = lane + 32 * i;
+          ltv[i] = (k < V && labels) ? lt[k] : 0.0f;
+          lsv[i] = (k < V && labels) ? ls[k] : 0.0f;
+        }
+        const double S = (double)s_score[w];
+        const double S_rho = S + (double)a.rho;
+        float lse = 0.0f;       // the joint kernel may already have normalised its rows
+        if (!a.normalized) {
+          float m = NEG;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) m = fmaxf(m, v[i]);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+          float sum = 0.0f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sum += expf(v[i] - m);   // exp(-inf) = 0 for the padding
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+          lse = m + logf(sum);
+        }
+        // label proposals of this slot that the merge below folds into another slot's blank
+        for (int w1 = 0; w1 < W; ++w1)
+          if (s_row[w1] >= 0 && s_u[w1] == s_u[w] + 1 && s_prev[w1] == s_hash[w] && labels &&
+              (s_last[w1] & 31) == lane)
+            skip |= 1u << (s_last[w1] >> 5);
+        float best = NEG;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int k = lane + 32 * i;
+          const float lp = v[i] - lse;
+          float sc;
+          if (k >= V) {
+            sc = NEG;
+            skip |= 1u << i;
+          } else if (k == 0) {
+            sc = (float)(S + (double)lp);
+            skip |= 1u << i;          // the blank proposal is read back after merge and finished list
+          } else if (labels) {
+            // label increment in fp32 (magnitude of tens), one double add onto the running score
+            const float inc = __fmaf_rn(a.lambda_t, ltv[i], __fmaf_rn(-a.lambda_s, lsv[i], lp));
+            sc = (float)(S_rho + (double)inc);
+          } else {
+            sc = NEG;
+            skip |= 1u << i;
+          }
+          v[i] = sc;
+          if (k < V) cw[k] = sc;
+          if (!((skip >> i) & 1u)) best = fmaxf(best, sc);
+        }
+        best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, 16));
+        if (lane < 16) s_gmax[w][lane] = best;
       }
-    } else {   // general vocabulary size: three passes over the row
-      float m = NEG;
-      for (int k = lane; k < V; k += 32) m = fmaxf(m, x[k]);
+    } else {
+      skip = 0xFFFFFFFFu;
+    }
+  } else {
+    for (int w = warp; w < W; w += SEL_NT / 32) {
+      float* cw = cand + (size_t)w * V;
+      const int row = s_row[w];
+      if (row < 0) {
+        for (int k = lane; k < V; k += 32) cw[k] = NEG;
+        continue;
+      }
+      const float* x = a.logits + (size_t)(base + w) * V;
+      const float* lt = a.tgt_lp + (size_t)row * V;
+      const float* ls = a.src_lp + (size_t)row * V;
+      const double S = (double)s_score[w];
+      const double S_rho = S + (double)a.rho;
+      const bool labels = s_u[w] < a.u_max;
+      // general vocabulary size: three passes over the row
+      float lse = 0.0f;
+      if (!a.normalized) {
+        float m = NEG;
+        for (int k = lane; k < V; k += 32) m = fmaxf(m, x[k]);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      float sum = 0.0f;
-      for (int k = lane; k < V; k += 32) sum += expf(x[k] - m);
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        float sum = 0.0f;
+        for (int k = lane; k < V; k += 32) sum += expf(x[k] - m);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      const float lse = m + logf(sum);
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        lse = m + logf(sum);
+      }
       for (int k = lane; k < V; k += 32) {
         const float lp = x[k] - lse;
-        float v;
+        float sc;
         if (k == 0) {
-          v = (float)(S + (double)lp);
+          sc = (float)(S + (double)lp);
         } else if (labels) {
           // label increment in fp32 (magnitude of tens), one double add onto the running score
           const float inc = __fmaf_rn(a.lambda_t, lt[k], __fmaf_rn(-a.lambda_s, ls[k], lp));
-          v = (float)(S + (double)inc + rho_d);
+          sc = (float)(S_rho + (double)inc);
         } else {
-          v = NEG;
+          sc = NEG;
         }
-        cw[k] = v;
+        cw[k] = sc;
       }
     }
   }
@@ -173,6 +229,20 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
       cand[(size_t)w * V] = (float)(mx + log1p(exp(-fabs(x - y))));
       cand[(size_t)w2 * V + k] = NEG;
     }
+  }
+  // fast path: a lower bound of the W-th best proposal.  The label proposals are split into 16
+  // disjoint groups (by lane modulo 16); each group's best is a distinct proposal, so at least
+  // 16 >= W proposals reach the smallest of the 16 group maxima.  An empty group (no slot may
+  // emit labels) gives -inf: then only the at most W blank proposals exist and all pass.
+  float bound = NEG;
+  if (fast) {
+    float g = NEG;
+    if (lane < 16)
+      for (int w = 0; w < W; ++w) g = fmaxf(g, s_gmax[w][lane]);
+    g = __shfl_sync(0xffffffffu, g, lane & 15);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) g = fminf(g, __shfl_xor_sync(0xffffffffu, g, o));
+    bound = g;
   }
   __syncthreads();
 
@@ -208,48 +278,99 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
   }
   __syncthreads();
 
-  // ---- the W best remaining proposals, by a threshold filter.
-  // (1) every thread's best proposal ("head") among its strided share of its slot; (2) the
-  // W-th best head, found bit by bit with block-wide counts, is a lower bound of the W-th best
-  // proposal, and only the threads owning the W best heads can hold anything at or above it;
-  // (3) those go to a short list; (4) each list entry's rank is counted in parallel.
-  uint64_t head = 0;
-  if (warp < W && s_row[warp] >= 0) {
-    const float* cw = cand + (size_t)warp * V;
-    const uint32_t off = (uint32_t)warp * (uint32_t)V;
-    for (int k = lane; k < V; k += 32) {
-      const float v = cw[k];
-      if (v > NEG) head = u64max(head, make_key(v, off + (uint32_t)k));
+  // ---- the W best remaining proposals
+  const int cap = 16 * ((V + 31) / 32);
+  bool exact = !fast;
+  if (fast) {
+    // everything at or above the bound goes to the short list (label proposals from registers,
+    // the blank proposal from shared memory, where merge and finished list have updated it)
+    if (warp < W && s_row[warp] >= 0) {   // uniform per warp: one list reservation per warp
+      const uint32_t off = (uint32_t)warp * (uint32_t)V;
+      uint32_t hit = 0;
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (!((skip >> i) & 1u) && v[i] >= bound) hit |= 1u << i;
+      float vb = NEG;
+      if (lane == 0) {
+        vb = cand[(size_t)warp * V];
+        if (!(vb >= bound)) vb = NEG;
+      }
+      const int mine = __popc(hit) + (vb > NEG ? 1 : 0);
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      const int total = __shfl_sync(0xffffffffu, incl, 31);
+      int p0 = 0;
+      if (lane == 31 && total > 0) p0 = atomicAdd(&list_n, total);
+      p0 = __shfl_sync(0xffffffffu, p0, 31) + incl - mine;
+      if (vb > NEG) {
+        if (p0 < cap) list[p0] = make_key(vb, off);
+        ++p0;
+      }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {   // static register indices
+        if ((hit >> i) & 1u) {
+          if (p0 < cap) list[p0] = make_key(v[i], off + (uint32_t)(lane + 32 * i));
+          ++p0;
+        }
+      }
     }
+    __syncthreads();
+    exact = list_n > cap;     // the bound was too loose for the list: take the exact threshold instead
+    __syncthreads();
+    if (exact && tid == 0) list_n = 0;
+    if (exact) __syncthreads();
   }
-  // score bits first (32 counts); the index bits matter only if equal scores straddle the bound
-  uint64_t th = 0;
-  for (int bit = 63; bit >= 32; --bit) {
-    const uint64_t c = th | (1ull << bit);
-    if (__syncthreads_count(head >= c) >= W) th = c;
-  }
-  if (__syncthreads_count(head >= th) > W) {
-    for (int bit = 31; bit >= 0; --bit) {
+  if (exact) {
+    // Threshold filter.  (1) every thread's best proposal ("head") among its strided share of
+    // its slot; (2) the W-th best head, found bit by bit with block-wide counts, is a lower bound
+    // of the W-th best proposal, and only the threads owning the W best heads can hold anything
+    // at or above it; (3) those go to the short list.
+    uint64_t head = 0;
+    for (int w = warp; w < W; w += SEL_NT / 32) {
+      if (s_row[w] < 0) continue;
+      const float* cw = cand + (size_t)w * V;
+      const uint32_t off = (uint32_t)w * (uint32_t)V;
+      for (int k = lane; k < V; k += 32) {
+        const float x = cw[k];
+        if (x > NEG) head = u64max(head, make_key(x, off + (uint32_t)k));
+      }
+    }
+    // score bits first (32 counts); the index bits matter only if equal scores straddle the bound
+    uint64_t th = 0;
+    for (int bit = 63; bit >= 32; --bit) {
       const uint64_t c = th | (1ull << bit);
       if (__syncthreads_count(head >= c) >= W) th = c;
     }
-  }
-  // th = the W-th best head (0 if there are fewer than W heads: then everything valid passes)
-  const int cap = 16 * ((V + 31) / 32);
-  if (head != 0ull && head >= th) {
-    const float* cw = cand + (size_t)warp * V;
-    const uint32_t off = (uint32_t)warp * (uint32_t)V;
-    for (int k = lane; k < V; k += 32) {
-      const float v = cw[k];
-      if (!(v > NEG)) continue;
-      const uint64_t key = make_key(v, off + (uint32_t)k);
-      if (key >= th) {
-        const int p = atomicAdd(&list_n, 1);
-        if (p < cap) list[p] = key;
+    if (__syncthreads_count(head >= th) > W) {
+      for (int bit = 31; bit >= 0; --bit) {
+        const uint64_t c = th | (1ull << bit);
+        if (__syncthreads_count(head >= c) >= W) th = c;
       }
     }
+    // th = the W-th best head (0 if there are fewer than W heads: then everything valid passes)
+    if (head != 0ull && head >= th) {
+      for (int w = warp; w < W; w += SEL_NT / 32) {
+        if (s_row[w] < 0) continue;
+        const float* cw = cand + (size_t)w * V;
+        const uint32_t off = (uint32_t)w * (uint32_t)V;
+        for (int k = lane; k < V; k += 32) {
+          const float x = cw[k];
+          if (!(x > NEG)) continue;
+          const uint64_t key = make_key(x, off + (uint32_t)k);
+          if (key >= th) {
+            const int p = atomicAdd(&list_n, 1);
+            if (p < cap) list[p] = key;
+          }
+        }
+      }
+    }
+    __syncthreads();
   }
-  __syncthreads();
+  // each list entry's rank is counted in parallel
   {
     const int ln = min(list_n, cap);
     for (int i = tid; i < ln; i += SEL_NT) {
@@ -339,7 +460,7 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
   }
 }
 
-cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s) {
+cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s, bool dependent) {
   const size_t smem = (size_t)a.W * a.V * sizeof(float) + (size_t)16 * ((a.V + 31) / 32) * sizeof(uint64_t);
   static size_t configured = 0;
   if (smem > configured) {
@@ -349,10 +470,10 @@ cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s) {
     configured = smem;
   }
   timing_begin(s);
-  k_beam_select<<<a.B, SEL_NT, smem, s>>>(a);
+  cudaError_t le = launch_ex(k_beam_select, dim3(a.B), dim3(SEL_NT), smem, s, dependent, 1, a);
   timing_end(s);
   ++g_launches;
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 __global__ void k_beam_init(q4_beam_state st, int B, int W) {
@@ -393,9 +514,16 @@ cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters,
   return cudaGetLastError();
 }
 
-__global__ void k_traceback(q4_beam_state st, int B, int W, int n_iters, int u_max,
-                            int32_t* tokens, int32_t* lens, float* scores) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+// One warp per utterance.  The walk from the winning slot back to the root is a chain of
+// dependent look-ups; to keep it off the memory latency, the warp first copies the back-pointer
+// rows of 32 consecutive iterations into shared memory (one iteration per lane, all W slots),
+// then lane 0 follows the chain there.
+constexpr int TB_WARPS = 4;
+__global__ void __launch_bounds__(32 * TB_WARPS) k_traceback(q4_beam_state st, int B, int W, int n_iters, int u_max,
+                                                             int32_t* tokens, int32_t* lens, float* scores) {
+  __shared__ int s_par[TB_WARPS][32][MAXW], s_tok[TB_WARPS][32][MAXW];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x * TB_WARPS + warp;
   if (b >= B) return;
   int j, s;
   float sc;
@@ -414,26 +542,42 @@ __global__ void k_traceback(q4_beam_state st, int B, int W, int n_iters, int u_m
   }
   int32_t* out = tokens + (size_t)b * u_max;
   int len = 0;
-  while (j >= 0 && s >= 0) {
-    const size_t h = ((size_t)j * B + b) * W + s;
-    const int k = st.bp_token[h];
-    if (k > 0 && len < u_max) out[len++] = k;
-    s = st.bp_parent[h];
-    --j;
+  while (j >= 0 && s >= 0) {   // uniform across the warp
+    const int jl = j - lane;
+    if (jl >= 0) {
+      const size_t h = ((size_t)jl * B + b) * W;
+      for (int i = 0; i < W; ++i) {
+        s_par[warp][lane][i] = st.bp_parent[h + i];
+        s_tok[warp][lane][i] = st.bp_token[h + i];
+      }
+    }
+    __syncwarp();
+    if (lane == 0) {
+      for (int l = 0; l < 32 && j >= 0 && s >= 0; ++l, --j) {
+        const int k = s_tok[warp][l][s];
+        if (k > 0 && len < u_max) out[len++] = k;
+        s = s_par[warp][l][s];
+      }
+    }
+    j = __shfl_sync(0xffffffffu, j, 0);
+    s = __shfl_sync(0xffffffffu, s, 0);
+    __syncwarp();
   }
-  for (int i = 0; i < len / 2; ++i) {
-    const int32_t tmp = out[i];
-    out[i] = out[len - 1 - i];
-    out[len - 1 - i] = tmp;
+  if (lane == 0) {
+    for (int i = 0; i < len / 2; ++i) {
+      const int32_t tmp = out[i];
+      out[i] = out[len - 1 - i];
+      out[len - 1 - i] = tmp;
+    }
+    for (int i = len; i < u_max; ++i) out[i] = 0;
+    lens[b] = len;
+    scores[b] = sc;
   }
-  for (int i = len; i < u_max; ++i) out[i] = 0;
-  lens[b] = len;
-  scores[b] = sc;
 }
 
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s) {
-  k_traceback<<<(B + 63) / 64, 64, 0, s>>>(st, B, W, n_iters, u_max, tokens, lens, scores);
+  k_traceback<<<(B + TB_WARPS - 1) / TB_WARPS, 32 * TB_WARPS, 0, s>>>(st, B, W, n_iters, u_max, tokens, lens, scores);
   ++g_launches;
   return cudaGetLastError();
 }

@@ -25,8 +25,10 @@ struct BeamSelArgs {
   q4_beam_state st;
   int32_t B, T, W, V, iter, u_max;
   float lambda_t, lambda_s, rho;
+  int32_t normalized;       // 1 = `logits` already holds log-probabilities (rows sum to one)
+  int32_t exact_only;       // 1 = skip the register-resident fast filter (the exact threshold path alone)
 };
-cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s);
+cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s, bool dependent = false);
 cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters, cudaStream_t s);
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s);
@@ -77,7 +79,8 @@ struct MmaLstmArgs {
   const int32_t* n_active;  // optional: rows >= *n_active carry no work (tiles beyond it exit at once)
 };
 struct LmHeadArgs {
-  int32_t N, H, V;            // launch rows, LSTM width (K of the bottleneck), vocabulary
+  int32_t N, H, V;            // launch rows, LSTM width (K of the bottleneck; 0 = no bottleneck: the
+                              // operand h8 is [N, 256] and feeds the output layer directly), vocabulary
   float x_scale;              // scale of the cell-output codes feeding the bottleneck
   const float* sc_bott;       // [256] bottleneck row scales
   const float* b_bott;        // [256] bias (nullable)

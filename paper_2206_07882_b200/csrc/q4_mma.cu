@@ -447,19 +447,20 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
 }
 
 // ------------------------------------------------------------------ fused LM head
-// One launch per language model and iteration.  A cluster of ceil(V/256) CTAs serves one tile
-// of 128 rows; every CTA computes the bottleneck GEMM (H -> D = 256, cheap, int32 in TMEM),
-// de-quantizes + biases + re-quantizes it (asymmetric constants) straight into a swizzled
-// shared-memory operand tile, multiplies it with its own block of 256 output-layer rows, and
-// keeps its 256 logits per row in registers (64 per thread).  Row maxima and sums of the
-// blocks are exchanged through distributed shared memory, one cluster barrier later every
-// thread knows the row's log-sum-exp and stores log-probabilities: one global write, no
-// separate log-softmax pass.
+// One launch per language model (and one for the joint network's output layer) and iteration.
+// A cluster of ceil(V/NB) CTAs serves one tile of 128 rows; every CTA computes the bottleneck
+// GEMM (H -> D = 256, cheap, int32 in TMEM), de-quantizes + biases + re-quantizes it
+// (asymmetric constants) straight into a swizzled shared-memory operand tile, multiplies it
+// with its own block of NB output-layer rows, and keeps its NB logits per row in registers
+// (NB/4 per thread).  Row maxima and sums of the blocks are exchanged through distributed
+// shared memory, one cluster barrier later every thread knows the row's log-sum-exp and stores
+// log-probabilities: one global write, no separate log-softmax pass.  With H = 0 there is no
+// bottleneck: the 256-wide operand rows are read from memory (joint network).
 constexpr int HEAD_D = 256;
 constexpr int HEAD_STAGES = 3;
-constexpr int HEAD_EPI_WARPS = 16;           // four warps per TMEM lane quarter, 64 columns each
+constexpr int HEAD_EPI_WARPS = 16;           // four warps per TMEM lane quarter, NB/4 columns each
 constexpr int HEAD_THREADS = 32 * (HEAD_EPI_WARPS + 2);
-constexpr int HEAD_MAX_BLOCKS = 8;           // portable cluster size: V <= 2048
+constexpr int HEAD_MAX_BLOCKS = 8;           // portable cluster size: V <= 8 NB
 
 __device__ __forceinline__ void cl_barrier() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -470,15 +471,18 @@ __device__ __forceinline__ void cl_store_f32(const float* local, uint32_t rank, 
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
 
+template <int NB>
 __global__ void __launch_bounds__(HEAD_THREADS, 1)
 k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ CUtensorMap tma_wb,
              const __grid_constant__ CUtensorMap tma_wo, const LmHeadArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   constexpr int A_BYTES = BM * BK, B_BYTES = HEAD_D * BK, STAGE = A_BYTES + B_BYTES;
+  constexpr int B2_BYTES = NB * BK;            // one K chunk of my block of output-layer rows
+  constexpr int CPT = NB / 4;                  // logits per thread
   __shared__ uint64_t full[HEAD_STAGES], empty[HEAD_STAGES], acc1_full, a2_ready, acc2_full;
   __shared__ uint32_t tmem_base_s;
-  __shared__ float s_sc1[HEAD_D], s_b1[HEAD_D], s_sc2[HEAD_D], s_b2[HEAD_D];
+  __shared__ __align__(16) float s_sc1[HEAD_D], s_b1[HEAD_D], s_sc2[NB], s_b2[NB];
   __shared__ float red_m[4][BM], red_s[4][BM];
   __shared__ float part_m[HEAD_MAX_BLOCKS][BM], part_s[HEAD_MAX_BLOCKS][BM];   // filled by every CTA of the cluster
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -500,6 +504,17 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
     fence_proxy_async();
   }
   if (warp == HEAD_EPI_WARPS + 1) tmem_alloc(&tmem_base_s, 512);
+  if (warp < HEAD_EPI_WARPS) {   // de-quantization constants: weights only, nothing of the previous kernel
+    for (int c = tid; c < HEAD_D; c += 32 * HEAD_EPI_WARPS) {
+      s_sc1[c] = nk1 > 0 ? __fmul_rn(a.x_scale, __ldg(a.sc_bott + c)) : 0.0f;
+      s_b1[c] = (nk1 > 0 && a.b_bott) ? __ldg(a.b_bott + c) : 0.0f;
+    }
+    for (int c = tid; c < NB; c += 32 * HEAD_EPI_WARPS) {
+      const int j = min(nb * NB + c, a.V - 1);
+      s_sc2[c] = __fmul_rn(a.q_scale, __ldg(a.sc_out + j));
+      s_b2[c] = a.b_out ? __ldg(a.b_out + j) : 0.0f;
+    }
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -522,18 +537,23 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
         mbar_expect_tx(&full[s], STAGE);
         tma_load_2d(smem + s * STAGE, &tma_h, i * BK, m0, &full[s]);
         tma_load_2d(smem + s * STAGE + A_BYTES, &tma_wb, i * BK, 0, &full[s]);
-      } else {
+      } else if (nk1 > 0) {
         // only the weight half of the stage is loaded: the activation halves of stages 0 and 1
         // receive the re-quantized bottleneck codes from the epilogue warps
-        mbar_expect_tx(&full[s], B_BYTES);
-        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_wo, (i - nk1) * BK, nb * HEAD_D, &full[s]);
+        mbar_expect_tx(&full[s], B2_BYTES);
+        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_wo, (i - nk1) * BK, nb * NB, &full[s]);
+      } else {
+        // no bottleneck: the 256-wide operand rows come from memory (stage i holds chunk i)
+        mbar_expect_tx(&full[s], A_BYTES + B2_BYTES);
+        tma_load_2d(smem + s * STAGE, &tma_h, i * BK, m0, &full[s]);
+        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_wo, i * BK, nb * NB, &full[s]);
       }
     }
     pdl_trigger();
     if (!ok) flag_timeout(a.status);
   } else if (warp == HEAD_EPI_WARPS + 1 && lane == 0) {
     // ---- MMA issuer
-    const uint32_t idesc = umma_idesc_i8(BM, HEAD_D);
+    const uint32_t idesc1 = umma_idesc_i8(BM, HEAD_D), idesc2 = umma_idesc_i8(BM, NB);
     bool ok = true;
     for (int i = 0; i < nk1 && ok; ++i) {
       const int s = i % HEAD_STAGES;
@@ -543,11 +563,11 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
       const uint64_t da = umma_desc_sw128(smem_u32(smem + s * STAGE));
       const uint64_t db = umma_desc_sw128(smem_u32(smem + s * STAGE + A_BYTES));
 #pragma unroll
-      for (int kk = 0; kk < BK / 32; ++kk) umma_i8(tmem, da + 2 * kk, db + 2 * kk, idesc, (i | kk) != 0);
+      for (int kk = 0; kk < BK / 32; ++kk) umma_i8(tmem, da + 2 * kk, db + 2 * kk, idesc1, (i | kk) != 0);
       umma_commit(&empty[s]);
     }
     umma_commit(&acc1_full);
-    if (ok) ok = mbar_wait(&a2_ready, 0);
+    if (ok && nk1 > 0) ok = mbar_wait(&a2_ready, 0);
     tc_fence_after();
     for (int kc = 0; kc < 2 && ok; ++kc) {
       const int i = nk1 + kc;
@@ -555,10 +575,10 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
       ok = mbar_wait(&full[s], (i / HEAD_STAGES) & 1);
       if (!ok) break;
       tc_fence_after();
-      const uint64_t da = umma_desc_sw128(smem_u32(smem + kc * STAGE));      // bottleneck codes
+      const uint64_t da = umma_desc_sw128(smem_u32(smem + kc * STAGE));      // bottleneck codes / operand rows
       const uint64_t db = umma_desc_sw128(smem_u32(smem + s * STAGE + A_BYTES));
 #pragma unroll
-      for (int kk = 0; kk < BK / 32; ++kk) umma_i8(tmem + HEAD_D, da + 2 * kk, db + 2 * kk, idesc, (kc | kk) != 0);
+      for (int kk = 0; kk < BK / 32; ++kk) umma_i8(tmem + HEAD_D, da + 2 * kk, db + 2 * kk, idesc2, (kc | kk) != 0);
       umma_commit(&empty[s]);
     }
     umma_commit(&acc2_full);
@@ -571,66 +591,77 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
     const int n = m0 + rt;
     int dst = -1;
     if (n < a.N && !(a.n_active && n >= *a.n_active)) dst = a.dst_row ? a.dst_row[n] : n;
-    for (int c = tid; c < HEAD_D; c += 32 * HEAD_EPI_WARPS) {
-      s_sc1[c] = __fmul_rn(a.x_scale, __ldg(a.sc_bott + c));
-      s_b1[c] = a.b_bott ? __ldg(a.b_bott + c) : 0.0f;
-      const int j = min(nb * HEAD_D + c, a.V - 1);
-      s_sc2[c] = __fmul_rn(a.q_scale, __ldg(a.sc_out + j));
-      s_b2[c] = a.b_out ? __ldg(a.b_out + j) : 0.0f;
-    }
-    asm volatile("bar.sync 1, %0;" ::"n"(32 * HEAD_EPI_WARPS) : "memory");
-    bool ok = mbar_wait(&acc1_full, 0);
-    tc_fence_after();
+    bool ok = true;
     const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
-    const int lo = act_lo(a.bott_act), hi = act_hi(a.bott_act), zp = a.bott_act.zero_point;
-    // bottleneck codes of my row, columns [64 cs, 64 cs + 64), into the swizzled operand tiles
+    if (nk1 > 0) {
+      const int lo = act_lo(a.bott_act), hi = act_hi(a.bott_act), zp = a.bott_act.zero_point;
+      ok = mbar_wait(&acc1_full, 0);
+      tc_fence_after();
+      // bottleneck codes of my row, columns [64 cs, 64 cs + 64), into the swizzled operand tiles
 #pragma unroll 1
-    for (int ch = 0; ch < 2; ++ch) {
-      const int c0 = 64 * cs + 32 * ch;
-      int r[32];
-      tmem_ld32(taddr + c0, r);
-      tmem_ld_wait();
-      uint32_t w[8];
+      for (int ch = 0; ch < 2; ++ch) {
+        const int c0 = 64 * cs + 32 * ch;
+        int r[32];
+        tmem_ld32(taddr + c0, r);
+        tmem_ld_wait();
+        uint32_t w[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) w[i] = 0;
+        for (int i = 0; i < 8; ++i) w[i] = 0;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float v = __fmaf_rn((float)r[i], s_sc1[c0 + i], s_b1[c0 + i]);
-        const int code = quantize1(v, a.bott_act.inv_scale, zp, lo, hi) - zp;
-        w[i >> 2] |= (uint32_t)(code & 0xFF) << (8 * (i & 3));
+        for (int i = 0; i < 32; i += 4) {
+          const float4 sc = *reinterpret_cast<const float4*>(s_sc1 + c0 + i);
+          const float4 bi = *reinterpret_cast<const float4*>(s_b1 + c0 + i);
+          const float scv[4] = {sc.x, sc.y, sc.z, sc.w}, biv[4] = {bi.x, bi.y, bi.z, bi.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float x = __fmaf_rn((float)r[i + e], scv[e], biv[e]);
+            const int code = quantize1(x, a.bott_act.inv_scale, zp, lo, hi) - zp;
+            w[(i + e) >> 2] |= (uint32_t)(code & 0xFF) << (8 * ((i + e) & 3));
+          }
+        }
+        const int kc = c0 >> 7, kb = c0 & 127;            // operand chunk and byte within its 128-byte row
+        uint8_t* tile = smem + kc * STAGE + (rt >> 3) * 1024 + (rt & 7) * 128;
+        *reinterpret_cast<uint4*>(tile + ((((kb >> 4) + 0) ^ (rt & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(tile + ((((kb >> 4) + 1) ^ (rt & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
       }
-      const int kc = c0 >> 7, kb = c0 & 127;            // operand chunk and byte within its 128-byte row
-      uint8_t* tile = smem + kc * STAGE + (rt >> 3) * 1024 + (rt & 7) * 128;
-      *reinterpret_cast<uint4*>(tile + ((((kb >> 4) + 0) ^ (rt & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-      *reinterpret_cast<uint4*>(tile + ((((kb >> 4) + 1) ^ (rt & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+      fence_proxy_async();        // generic-proxy writes -> visible to the tensor core's async proxy
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&a2_ready);
     }
-    fence_proxy_async();        // generic-proxy writes -> visible to the tensor core's async proxy
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&a2_ready);
 
-    // my 64 logits of this block, kept in registers until the row's log-sum-exp is known
+    // my CPT logits of this block, kept in registers until the row's log-sum-exp is known
     if (ok) ok = mbar_wait(&acc2_full, 0);
     tc_fence_after();
     pdl_trigger();   // both GEMMs are over: the next kernel may set itself up
-    float v[64];
+    float v[CPT];
     float my_m = -INFINITY;
+    const int col0 = nb * NB + CPT * cs;       // first vocabulary entry of my share
 #pragma unroll
-    for (int ch = 0; ch < 2; ++ch) {
-      const int c0 = 64 * cs + 32 * ch;
+    for (int ch = 0; ch < CPT / 32; ++ch) {
+      const int c0 = CPT * cs + 32 * ch;
       int r[32];
       tmem_ld32(taddr + HEAD_D + c0, r);
       tmem_ld_wait();
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        v[32 * ch + i] = __fmaf_rn((float)r[i], s_sc2[c0 + i], s_b2[c0 + i]);
-        if (nb * HEAD_D + c0 + i < a.V) my_m = fmaxf(my_m, v[32 * ch + i]);
+      for (int i = 0; i < 32; i += 4) {
+        const float4 sc = *reinterpret_cast<const float4*>(s_sc2 + c0 + i);
+        const float4 bi = *reinterpret_cast<const float4*>(s_b2 + c0 + i);
+        v[32 * ch + i + 0] = __fmaf_rn((float)r[i + 0], sc.x, bi.x);
+        v[32 * ch + i + 1] = __fmaf_rn((float)r[i + 1], sc.y, bi.y);
+        v[32 * ch + i + 2] = __fmaf_rn((float)r[i + 2], sc.z, bi.z);
+        v[32 * ch + i + 3] = __fmaf_rn((float)r[i + 3], sc.w, bi.w);
       }
     }
+#pragma unroll
+    for (int i = 0; i < CPT; ++i)
+      if (col0 + i < a.V) my_m = fmaxf(my_m, v[i]);
+    // exponentials by the hardware base-2 unit: relative error near 1e-6, far inside what the
+    // log-sum-exp of a thousand terms needs
     float my_s = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 64; ++i)
-      if (nb * HEAD_D + 64 * cs + i < a.V) my_s += expf(v[i] - my_m);
+    for (int i = 0; i < CPT; ++i)
+      if (col0 + i < a.V) my_s += __expf(v[i] - my_m);
     red_m[cs][rt] = my_m;
     red_s[cs][rt] = my_s;
     asm volatile("bar.sync 1, %0;" ::"n"(32 * HEAD_EPI_WARPS) : "memory");
@@ -639,7 +670,7 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
       float ssum = 0.0f;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        if (red_s[i][rt] > 0.0f) ssum += red_s[i][rt] * expf(red_m[i][rt] - m);
+        if (red_s[i][rt] > 0.0f) ssum += red_s[i][rt] * __expf(red_m[i][rt] - m);
       for (int r = 0; r < nblk; ++r) {
         cl_store_f32(&part_m[nb][rt], (uint32_t)r, m);
         cl_store_f32(&part_s[nb][rt], (uint32_t)r, ssum);
@@ -650,28 +681,28 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
     for (int r = 0; r < nblk; ++r) m = fmaxf(m, part_m[r][rt]);
     float ssum = 0.0f;
     for (int r = 0; r < nblk; ++r)
-      if (part_s[r][rt] > 0.0f) ssum += part_s[r][rt] * expf(part_m[r][rt] - m);
+      if (part_s[r][rt] > 0.0f) ssum += part_s[r][rt] * __expf(part_m[r][rt] - m);
     const float lse = m + logf(ssum);
     if (dst >= 0 && ok) {
-      float* out = a.lp + (long long)dst * a.V + nb * HEAD_D + 64 * cs;
-      const int left = a.V - (nb * HEAD_D + 64 * cs);
-      if (left >= 64) {
+      float* out = a.lp + (long long)dst * a.V + col0;
+      const int left = a.V - col0;
+      if (left >= CPT) {
 #pragma unroll
-        for (int i = 0; i < 64; i += 4)
+        for (int i = 0; i < CPT; i += 4)
           *reinterpret_cast<float4*>(out + i) = make_float4(v[i] - lse, v[i + 1] - lse, v[i + 2] - lse, v[i + 3] - lse);
       } else {
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
+        for (int i = 0; i < CPT; ++i)
           if (i < left) out[i] = v[i] - lse;
       }
     }
     if (!ok && lane == 0) flag_timeout(a.status);
   }
   __syncwarp();
-  if (warp >= HEAD_EPI_WARPS) {
+  if (warp >= HEAD_EPI_WARPS) {   // the producer and issuer warps join the cluster barrier too
     pdl_trigger();
     cl_barrier();
-  }   // the producer and issuer warps join the cluster barrier too
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == HEAD_EPI_WARPS + 1) tmem_dealloc(tmem, 512);
@@ -682,22 +713,35 @@ cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h
                               const int8_t* wo8, cudaStream_t s, bool dependent) {
   if (a.N <= 0) return cudaSuccess;
   const int rows_pad = (a.N + BM - 1) / BM * BM;
-  const int nblk = (a.V + HEAD_D - 1) / HEAD_D;
+  const int NB = a.V <= 128 * HEAD_MAX_BLOCKS ? 128 : 256;   // the narrower block spreads a row over more CTAs
+  const int nblk = (a.V + NB - 1) / NB;
   if (nblk > HEAD_MAX_BLOCKS) return cudaErrorInvalidValue;
   CUtensorMap th, tb, to;
-  if (!make_tmap_i8(&th, h8, a.H, rows_pad, h_pitch, BM) || !make_tmap_i8(&tb, wb8, a.H, HEAD_D, a.H, HEAD_D) ||
-      !make_tmap_i8(&to, wo8, HEAD_D, a.V, HEAD_D, HEAD_D))
+  const int Ka = a.H > 0 ? a.H : HEAD_D;
+  if (!make_tmap_i8(&th, h8, Ka, rows_pad, h_pitch, BM) || !make_tmap_i8(&to, wo8, HEAD_D, a.V, HEAD_D, NB))
     return cudaErrorInvalidValue;
+  if (a.H > 0) {
+    if (!make_tmap_i8(&tb, wb8, a.H, HEAD_D, a.H, HEAD_D)) return cudaErrorInvalidValue;
+  } else {
+    tb = to;   // unused without a bottleneck
+  }
   const size_t smem = (size_t)HEAD_STAGES * (BM * BK + HEAD_D * BK) + 1024;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_mma_lmhead, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_mma_lmhead<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_mma_lmhead<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   timing_begin(s);
-  cudaError_t e = launch_ex(k_mma_lmhead, dim3(nblk, rows_pad / BM), dim3(HEAD_THREADS), smem, s, dependent,
-                            (unsigned)nblk, th, tb, to, a);
+  cudaError_t e;
+  if (NB == 128)
+    e = launch_ex(k_mma_lmhead<128>, dim3(nblk, rows_pad / BM), dim3(HEAD_THREADS), smem, s, dependent,
+                  (unsigned)nblk, th, tb, to, a);
+  else
+    e = launch_ex(k_mma_lmhead<256>, dim3(nblk, rows_pad / BM), dim3(HEAD_THREADS), smem, s, dependent,
+                  (unsigned)nblk, th, tb, to, a);
   timing_end(s);
   ++g_launches;
   return e != cudaSuccess ? e : cudaGetLastError();

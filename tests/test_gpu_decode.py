@@ -230,6 +230,31 @@ def test_fused_lm_head_small_search(Bd):
             np.testing.assert_allclose(np.exp(lp.astype(np.float64)).sum(1), 1.0, atol=1e-5)
 
 
+def test_selection_paths_and_launch_modes_agree(Bd):
+    # the bounded fast filter against the exact threshold search, and programmatic dependent
+    # launches against plain stream order: bit-identical beams and scores
+    dw = synth.decoder(seed=71, V=1024, E=32, Hp=128, D=256, Hs=128, Ht=256, tgt_layers=2, U_max=8, W=16)
+    e = synth.Stream(9).normal("e", (12, 8, 256)).astype(np.float32)
+    base = run_search(Bd, dw, e)
+    compare_search(base[0], base[1], base[2], base[3], base[4], list(range(8)), 12, 8, 16, min_same=1.0)
+    runs = []
+    prev = Bd.beam_select_exact_set(True)
+    try:
+        runs.append(run_search(Bd, dw, e))
+    finally:
+        Bd.beam_select_exact_set(prev)
+    prev = Bd.dependent_launch_set(False)
+    try:
+        runs.append(run_search(Bd, dw, e))
+    finally:
+        Bd.dependent_launch_set(prev)
+    for other in runs:
+        for k in ("bp_parent", "bp_token", "bp_score", "fin_n", "fin_score", "fin_iter", "fin_slot"):
+            assert torch.equal(base[0].tensors[k][:20], other[0].tensors[k][:20]), k
+        np.testing.assert_array_equal(base[1], other[1])
+        np.testing.assert_array_equal(base[3], other[3])
+
+
 def test_config3_full_length_invariants(Bd):
     # T=300, U_max=150 (450 iterations): properties that hold at any size.
     dw = synth.decoder(seed=3, U_max=150)
