@@ -150,11 +150,19 @@ def unpack4(b: np.ndarray, k: int, is_signed: bool) -> np.ndarray:
 
 
 def activations(x: np.ndarray):
-    """The oracle's fp32 exp, sigmoid and tanh on an array."""
+    """The oracle's fp32 2^x, sigmoid and tanh on an array."""
     x = _c(x, np.float32)
     ex, sg, th = np.empty_like(x), np.empty_like(x), np.empty_like(x)
     lib().orc_activations(_p(x), C.c_int64(x.size), _p(ex), _p(sg), _p(th))
     return ex, sg, th
+
+
+def cells(pre_i, pre_f, pre_g, pre_o, c_prev):
+    """The oracle's fp32 LSTM cell update on arrays of pre-activations: returns (c, h)."""
+    a = [_c(v, np.float32) for v in (pre_i, pre_f, pre_g, pre_o, c_prev)]
+    c, h = np.empty_like(a[0]), np.empty_like(a[0])
+    lib().orc_cells(*[_p(v) for v in a], C.c_int64(a[0].size), _p(c), _p(h))
+    return c, h
 
 
 def int_matmul(w: np.ndarray, xq: np.ndarray, zero_point: int = 0) -> np.ndarray:

@@ -171,9 +171,11 @@ void orc_linear(const OrcLinear* L, const int16_t* xq, const OrcAct* x_act, int3
 
 
 // ------------------------------------------------- fp32 activation functions
-// exp(x) for x in [-86, 88]: n = rne(x*log2(e)); r = x - n*ln2 (two-constant
-// reduction, fused multiply-adds); degree-7 Taylor polynomial in r by Horner's
-// rule with fused multiply-adds; scaling by 2^n through the exponent field.
+// 2^t for |t| <= 125 as a fixed sequence of fp32 operations: n = rne(t), obtained by adding
+// and subtracting 1.5 * 2^23; r = t - n (exact, |r| <= 1/2); p = 1 + r (c1 + r (c2 + ... +
+// r c6)) by Horner's rule with fused multiply-adds, c1..c6 being the interpolant of
+// (2^r - 1)/r at the six Chebyshev nodes of [-1/2, 1/2] rounded to fp32; scaling by 2^n
+// through the exponent field.
 static inline float f32_from_bits(uint32_t b) {
   float f;
   std::memcpy(&f, &b, 4);
@@ -184,56 +186,63 @@ static inline uint32_t bits_from_f32(float f) {
   std::memcpy(&b, &f, 4);
   return b;
 }
-float orc_exp(float x) {
-  x = std::fmin(std::fmax(x, -86.0f), 88.0f);
-  const float n = std::nearbyintf(x * 0x1.715476p+0f);
-  float r = std::fmaf(n, -0x1.62e400p-1f, x);
-  r = std::fmaf(n, -0x1.7f7d1cp-20f, r);
-  float p = 0x1.a01a02p-13f;               // 1/5040
-  p = std::fmaf(p, r, 0x1.6c16c2p-10f);    // 1/720
-  p = std::fmaf(p, r, 0x1.111112p-7f);     // 1/120
-  p = std::fmaf(p, r, 0x1.555556p-5f);     // 1/24
-  p = std::fmaf(p, r, 0x1.555556p-3f);     // 1/6
-  p = std::fmaf(p, r, 0.5f);
+float orc_exp2(float t) {
+  const float nf = t + 12582912.0f;
+  const float n = nf - 12582912.0f;
+  const float r = t - n;
+  float p = 0x1.44138ap-13f;
+  p = std::fmaf(p, r, 0x1.5f0890p-10f);
+  p = std::fmaf(p, r, 0x1.3b2a54p-7f);
+  p = std::fmaf(p, r, 0x1.c6af6cp-5f);
+  p = std::fmaf(p, r, 0x1.ebfbe0p-3f);
+  p = std::fmaf(p, r, 0x1.62e430p-1f);
   p = std::fmaf(p, r, 1.0f);
-  p = std::fmaf(p, r, 1.0f);
-  return f32_from_bits(bits_from_f32(p) + ((uint32_t)(int32_t)n << 23));
+  return f32_from_bits(bits_from_f32(p) + (bits_from_f32(nf) << 23));
 }
-// sigmoid(x) = 1 / (1 + exp(-x)), argument clamped to [-86, 86].
+static const float kNegLog2e = -0x1.715476p+0f;   // -log2(e) rounded to fp32
+// sigmoid(x) = 1 / (1 + 2^(-log2(e) x)), argument clamped to [-40, 40].
 float orc_sigmoid(float x) {
-  x = std::fmin(std::fmax(x, -86.0f), 86.0f);
-  return 1.0f / (1.0f + orc_exp(-x));
+  x = std::fmin(std::fmax(x, -40.0f), 40.0f);
+  return 1.0f / (1.0f + orc_exp2(x * kNegLog2e));
 }
-// tanh(x) = sign(x) * (1 - e) / (1 + e), e = exp(-2 min(|x|, 43)).
+// tanh(x) = sign(x) * (1 - e) * (1 / (1 + e)), e = 2^(-2 log2(e) min(|x|, 40)).
 float orc_tanh(float x) {
-  const float a = std::fmin(std::fabs(x), 43.0f);
-  const float e = orc_exp(-2.0f * a);
-  const float t = (1.0f - e) / (1.0f + e);
-  return std::copysign(t, x);
+  const float e = orc_exp2(std::fmin(std::fabs(x), 40.0f) * (2.0f * kNegLog2e));
+  const float rcp = 1.0f / (1.0f + e);
+  return std::copysign((1.0f - e) * rcp, x);
 }
-// LSTM cell update in fp32 with three divisions: the products i*g and o*tanh(c) are each
-// formed as one quotient,
-//   i*g = sign(g) (1 - eg) / ((1 + ei)(1 + eg)),   f = 1 / (1 + ef),
+// LSTM cell update in fp32 with two reciprocals.  With ei = 2^(-log2(e) i_pre) and likewise
+// ef, eo (arguments clamped to [-40, 40]), eg = 2^(-2 log2(e) min(|g_pre|, 40)):
+//   R   = 1 / (((1 + ei)(1 + eg))(1 + ef)),
+//   i*g = sign(g) ((1 - eg)(1 + ef)) R,     f = ((1 + ei)(1 + eg)) R,
 //   c   = fma(f, c_prev, i*g),
-//   h   = sign(c) (1 - ec) / ((1 + eo)(1 + ec)),
-// with ei = exp(-i_pre), ef = exp(-f_pre), eo = exp(-o_pre) (arguments clamped to [-86, 86]),
-// eg = exp(-2 min(|g_pre|, 43)), ec = exp(-2 min(|c|, 43)).  Mathematically this is
-// sigmoid(i) tanh(g), sigmoid(f), sigmoid(o) tanh(c).
+//   h   = sign(c) (1 - ec) (1 / ((1 + eo)(1 + ec))),   ec = 2^(-2 log2(e) min(|c|, 40)).
+// Mathematically this is sigmoid(i) tanh(g), sigmoid(f), sigmoid(o) tanh(c); every factor
+// lies in [1, 2^58], so no product overflows.
 void orc_cell(float pi, float pf, float pg, float po, float c_prev, float* c_out, float* h_out) {
-  const float ei = orc_exp(-std::fmin(std::fmax(pi, -86.0f), 86.0f));
-  const float ef = orc_exp(-std::fmin(std::fmax(pf, -86.0f), 86.0f));
-  const float eo = orc_exp(-std::fmin(std::fmax(po, -86.0f), 86.0f));
-  const float eg = orc_exp(-2.0f * std::fmin(std::fabs(pg), 43.0f));
-  const float ig = std::copysign((1.0f - eg) / ((1.0f + ei) * (1.0f + eg)), pg);
-  const float f = 1.0f / (1.0f + ef);
+  const float ei = orc_exp2(std::fmin(std::fmax(pi, -40.0f), 40.0f) * kNegLog2e);
+  const float ef = orc_exp2(std::fmin(std::fmax(pf, -40.0f), 40.0f) * kNegLog2e);
+  const float eo = orc_exp2(std::fmin(std::fmax(po, -40.0f), 40.0f) * kNegLog2e);
+  const float eg = orc_exp2(std::fmin(std::fabs(pg), 40.0f) * (2.0f * kNegLog2e));
+  const float ag = (1.0f + ei) * (1.0f + eg);
+  const float F = 1.0f + ef;
+  const float R = 1.0f / (ag * F);
+  const float ig = std::copysign(((1.0f - eg) * F) * R, pg);
+  const float f = ag * R;
   const float c = std::fmaf(f, c_prev, ig);
-  const float ec = orc_exp(-2.0f * std::fmin(std::fabs(c), 43.0f));
+  const float ec = orc_exp2(std::fmin(std::fabs(c), 40.0f) * (2.0f * kNegLog2e));
+  const float R2 = 1.0f / ((1.0f + eo) * (1.0f + ec));
   *c_out = c;
-  *h_out = std::copysign((1.0f - ec) / ((1.0f + eo) * (1.0f + ec)), c);
+  *h_out = std::copysign((1.0f - ec) * R2, c);
+}
+// orc_cell on arrays (for the tests that pin it to the textbook formulas).
+void orc_cells(const float* pre_i, const float* pre_f, const float* pre_g, const float* pre_o,
+               const float* c_prev, int64_t n, float* c_out, float* h_out) {
+  for (int64_t i = 0; i < n; ++i) orc_cell(pre_i[i], pre_f[i], pre_g[i], pre_o[i], c_prev[i], c_out + i, h_out + i);
 }
 void orc_activations(const float* x, int64_t n, float* ex, float* sg, float* th) {
   for (int64_t i = 0; i < n; ++i) {
-    if (ex) ex[i] = orc_exp(x[i]);
+    if (ex) ex[i] = orc_exp2(x[i]);
     if (sg) sg[i] = orc_sigmoid(x[i]);
     if (th) th[i] = orc_tanh(x[i]);
   }

@@ -90,55 +90,58 @@ __device__ __forceinline__ int act_hi(const q4_act& a) {
   return a.is_signed ? (1 << (a.bits - 1)) - 1 : (1 << a.bits) - 1;
 }
 
-// Gate non-linearities as a fixed sequence of IEEE fp32 operations (round-to-nearest
-// multiply / fused multiply-add / divide), so that the code a cell output quantizes to does
+// Gate non-linearities as a fixed sequence of IEEE fp32 operations (round-to-nearest add,
+// multiply, fused multiply-add, reciprocal), so that the code a cell output quantizes to does
 // not depend on a math library:
-//   exp(x), x clamped to [-86, 88]: n = rne(x * log2 e); r = x - n ln2 with ln2 split in two
-//   constants; 7th-degree Taylor polynomial in r (Horner); times 2^n via the exponent field.
-__device__ __forceinline__ float exp_fixed(float x) {
-  x = fminf(fmaxf(x, -86.0f), 88.0f);
-  const float n = rintf(__fmul_rn(x, 1.44269502162933349609375f));
-  float r = __fmaf_rn(n, -0.693145751953125f, x);
-  r = __fmaf_rn(n, -1.428606765330187045037746429443359375e-6f, r);
-  float p = 1.98412701138295233249664306640625e-4f;
-  p = __fmaf_rn(p, r, 1.388888922519981861114501953125e-3f);
-  p = __fmaf_rn(p, r, 8.3333335816860198974609375e-3f);
-  p = __fmaf_rn(p, r, 4.1666667908430099487304687500e-2f);
-  p = __fmaf_rn(p, r, 0.16666667163372039794921875f);
-  p = __fmaf_rn(p, r, 0.5f);
+//   2^t for |t| <= 125: n = rne(t) by adding and subtracting 1.5 * 2^23; r = t - n (exact,
+//   |r| <= 1/2); p = 1 + r (c1 + r (c2 + ... + r c6)) by Horner's rule with fused multiply-adds,
+//   c1..c6 fixed constants (interpolation of (2^r - 1)/r at the six Chebyshev nodes of
+//   [-1/2, 1/2], relative error below 1e-8); times 2^n by adding n to the exponent field.
+__device__ __forceinline__ float exp2_fixed(float t) {
+  const float nf = __fadd_rn(t, 12582912.0f);
+  const float r = __fsub_rn(t, __fsub_rn(nf, 12582912.0f));
+  float p = 0x1.44138ap-13f;
+  p = __fmaf_rn(p, r, 0x1.5f0890p-10f);
+  p = __fmaf_rn(p, r, 0x1.3b2a54p-7f);
+  p = __fmaf_rn(p, r, 0x1.c6af6cp-5f);
+  p = __fmaf_rn(p, r, 0x1.ebfbe0p-3f);
+  p = __fmaf_rn(p, r, 0x1.62e430p-1f);
   p = __fmaf_rn(p, r, 1.0f);
-  p = __fmaf_rn(p, r, 1.0f);
-  return __uint_as_float(__float_as_uint(p) + ((uint32_t)(int)n << 23));
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(nf) << 23));
 }
-//   sigmoid(x) = 1 / (1 + exp(-x)), x clamped to [-86, 86]
+constexpr float NEG_LOG2E = -0x1.715476p+0f;        // -log2(e) rounded to fp32
+constexpr float NEG_2LOG2E = -0x1.715476p+1f;       // twice that
+//   sigmoid(x) = 1 / (1 + 2^(-log2(e) x)), x clamped to [-40, 40]
 __device__ __forceinline__ float sigmoid_fixed(float x) {
-  x = fminf(fmaxf(x, -86.0f), 86.0f);
-  return __fdiv_rn(1.0f, __fadd_rn(1.0f, exp_fixed(-x)));
+  x = fminf(fmaxf(x, -40.0f), 40.0f);
+  return __frcp_rn(__fadd_rn(1.0f, exp2_fixed(__fmul_rn(x, NEG_LOG2E))));
 }
-//   tanh(x) = sign(x) (1 - e) / (1 + e), e = exp(-2 min(|x|, 43))
+//   tanh(x) = sign(x) (1 - e) * (1 / (1 + e)), e = 2^(-2 log2(e) min(|x|, 40))
 __device__ __forceinline__ float tanh_fixed(float x) {
-  const float a = fminf(fabsf(x), 43.0f);
-  const float e = exp_fixed(__fmul_rn(-2.0f, a));
-  const float t = __fdiv_rn(__fsub_rn(1.0f, e), __fadd_rn(1.0f, e));
-  return copysignf(t, x);
+  const float e = exp2_fixed(__fmul_rn(fminf(fabsf(x), 40.0f), NEG_2LOG2E));
+  return copysignf(__fmul_rn(__fsub_rn(1.0f, e), __frcp_rn(__fadd_rn(1.0f, e))), x);
 }
 
-// LSTM cell update with three divisions (i*g and o*tanh(c) are one quotient each):
-//   i*g = sign(g)(1 - eg) / ((1 + ei)(1 + eg)),  f = 1 / (1 + ef),  c = fma(f, c_prev, i*g),
-//   h = sign(c)(1 - ec) / ((1 + eo)(1 + ec)),
-//   ei, ef, eo = exp(-pre) with pre clamped to [-86, 86]; eg, ec = exp(-2 min(|.|, 43)).
+// LSTM cell update with two reciprocals:
+//   ei, ef, eo = 2^(-log2(e) pre), pre clamped to [-40, 40]; eg, ec = 2^(-2 log2(e) min(|.|, 40));
+//   R = 1 / (((1 + ei)(1 + eg))(1 + ef));  i*g = sign(g) ((1 - eg)(1 + ef)) R;  f = ((1 + ei)(1 + eg)) R;
+//   c = fma(f, c_prev, i*g);  h = sign(c) (1 - ec) * (1 / ((1 + eo)(1 + ec))).
+// Every factor lies in [1, 2^58], so no product overflows.
 __device__ __forceinline__ void cell_fixed(float pi, float pf, float pg, float po, float c_prev,
                                            float& c, float& h) {
-  const float ei = exp_fixed(-fminf(fmaxf(pi, -86.0f), 86.0f));
-  const float ef = exp_fixed(-fminf(fmaxf(pf, -86.0f), 86.0f));
-  const float eo = exp_fixed(-fminf(fmaxf(po, -86.0f), 86.0f));
-  const float eg = exp_fixed(__fmul_rn(-2.0f, fminf(fabsf(pg), 43.0f)));
-  const float ig = copysignf(
-      __fdiv_rn(__fsub_rn(1.0f, eg), __fmul_rn(__fadd_rn(1.0f, ei), __fadd_rn(1.0f, eg))), pg);
-  const float f = __fdiv_rn(1.0f, __fadd_rn(1.0f, ef));
+  const float ei = exp2_fixed(__fmul_rn(fminf(fmaxf(pi, -40.0f), 40.0f), NEG_LOG2E));
+  const float ef = exp2_fixed(__fmul_rn(fminf(fmaxf(pf, -40.0f), 40.0f), NEG_LOG2E));
+  const float eo = exp2_fixed(__fmul_rn(fminf(fmaxf(po, -40.0f), 40.0f), NEG_LOG2E));
+  const float eg = exp2_fixed(__fmul_rn(fminf(fabsf(pg), 40.0f), NEG_2LOG2E));
+  const float ag = __fmul_rn(__fadd_rn(1.0f, ei), __fadd_rn(1.0f, eg));
+  const float F = __fadd_rn(1.0f, ef);
+  const float R = __frcp_rn(__fmul_rn(ag, F));
+  const float ig = copysignf(__fmul_rn(__fmul_rn(__fsub_rn(1.0f, eg), F), R), pg);
+  const float f = __fmul_rn(ag, R);
   c = __fmaf_rn(f, c_prev, ig);
-  const float ec = exp_fixed(__fmul_rn(-2.0f, fminf(fabsf(c), 43.0f)));
-  h = copysignf(__fdiv_rn(__fsub_rn(1.0f, ec), __fmul_rn(__fadd_rn(1.0f, eo), __fadd_rn(1.0f, ec))), c);
+  const float ec = exp2_fixed(__fmul_rn(fminf(fabsf(c), 40.0f), NEG_2LOG2E));
+  const float R2 = __frcp_rn(__fmul_rn(__fadd_rn(1.0f, eo), __fadd_rn(1.0f, ec)));
+  h = copysignf(__fmul_rn(__fsub_rn(1.0f, ec), R2), c);
 }
 
 // ---- argument blocks of the tile kernels -------------------------------------------

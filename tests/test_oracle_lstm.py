@@ -229,6 +229,32 @@ def test_features_prologue_by_hand():
     np.testing.assert_allclose(out, want, atol=1e-6)
 
 
+def test_cell_update_against_textbook_formulas():
+    # c = sigmoid(f) c_prev + sigmoid(i) tanh(g), h = sigmoid(o) tanh(c) evaluated in double
+    st = synth.Stream(77)
+    n = 200000
+    pre = [st.normal(f"p{k}", (n,)).astype(np.float32) * np.float32(s) for k, s in enumerate((3, 3, 3, 3))]
+    cp = (st.normal("c", (n,)) * 2).astype(np.float32)
+    # extremes: saturated gates in every combination, huge cell state
+    ext = np.array([-1e4, -100.0, -41.0, -40.0, 0.0, 40.0, 41.0, 100.0, 1e4], dtype=np.float32)
+    gi, gf, gg, go = [v.ravel() for v in np.meshgrid(ext, ext, ext, ext)]
+    pre = [np.concatenate([p, e]) for p, e in zip(pre, (gi, gf, gg, go))]
+    cp = np.concatenate([cp, np.resize(np.array([-50.0, -1.0, 0.0, 1.0, 50.0], dtype=np.float32), gi.size)])
+    c, h = O.cells(pre[0], pre[1], pre[2], pre[3], cp)
+    assert np.isfinite(c).all() and np.isfinite(h).all()
+    d = [p.astype(np.float64) for p in pre]
+    sig = lambda v: 1 / (1 + np.exp(-np.clip(v, -700, 700)))
+    c_ref = sig(d[1]) * cp.astype(np.float64) + sig(d[0]) * np.tanh(d[2])
+    h_ref = sig(d[3]) * np.tanh(c_ref)
+    # a handful of fp32 roundings on f and i*g, the first scaled by |c_prev|
+    assert np.max(np.abs(c - c_ref) / np.maximum(1.0, np.abs(cp.astype(np.float64)))) < 4e-7
+    assert np.max(np.abs(h - h_ref)) < 4e-7
+    assert (np.abs(h) <= 1).all()
+    # a cell whose forget gate is open and input gate shut keeps its state exactly
+    c2, _ = O.cells(np.float32([-100.0]), np.float32([100.0]), np.float32([0.3]), np.float32([0.0]), np.float32([1.2345678]))
+    assert c2[0] == np.float32(1.2345678)
+
+
 def test_fp32_activation_functions_against_libm():
     # The gate non-linearities are fixed fp32 operation sequences (so that codes are
     # reproducible); here they are pinned to the real functions evaluated in double.
@@ -237,7 +263,13 @@ def test_fp32_activation_functions_against_libm():
     ex, sg, th = O.activations(x)
     xd = x.astype(np.float64)
     inr = np.abs(xd) <= 30
-    assert np.max(np.abs(ex[inr] / np.exp(xd[inr]) - 1)) < 2e-7
+    assert np.max(np.abs(ex[inr] / np.exp2(xd[inr]) - 1)) < 2e-7
+    # the power of two over its whole range, and exactly at the integers
+    t = np.linspace(-125, 125, 500001).astype(np.float32)
+    e2, _, _ = O.activations(t)
+    assert np.max(np.abs(e2 / np.exp2(t.astype(np.float64)) - 1)) < 2e-7
+    ti = np.arange(-125, 126).astype(np.float32)
+    np.testing.assert_array_equal(O.activations(ti)[0], np.exp2(ti.astype(np.float64)).astype(np.float32))
     assert np.max(np.abs(sg - 1 / (1 + np.exp(-np.clip(xd, -700, 700))))) < 2e-7
     assert np.max(np.abs(th - np.tanh(xd))) < 2e-7
     assert (sg >= 0).all() and (sg <= 1).all() and (np.abs(th) <= 1).all()
