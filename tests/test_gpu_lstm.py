@@ -132,7 +132,10 @@ def test_config0_layer_forward(Bd):
 
 
 @pytest.mark.parametrize("T,B,K,H,dirs,xb,hb,ob", [(9, 3, 48, 32, 2, 4, 4, 4), (20, 70, 240, 64, 2, 8, 8, 4),
-                                                   (12, 33, 128, 96, 1, 4, 4, 8), (7, 1, 1280, 160, 2, 4, 4, 4)])
+                                                   (12, 33, 128, 96, 1, 4, 4, 8), (7, 1, 1280, 160, 2, 4, 4, 4),
+                                                   # 64 and 60 sequences x 2 directions of 640 cells: groups of 16
+                                                   # sequences per cluster, full and ragged
+                                                   (6, 64, 64, 640, 2, 4, 4, 4), (5, 60, 32, 640, 2, 8, 8, 4)])
 def test_layer_shapes_directions_precisions(Bd, T, B, K, H, dirs, xb, hb, ob):
     layer_case(Bd, T, B, K, H, dirs, xb, hb, ob, seed=11)
 
