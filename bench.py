@@ -463,6 +463,15 @@ def main():
         dist.destroy_process_group()
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the captures summarised under
+# profiles/ (k_mma_lstm_prof_end_to_end.md, k_enc_recurrent_prof_encoder.md); to be reset to None
+# when those kernels change.
+NCU_TRAFFIC = {
+    "k_mma_lstm_tgt_l2": {"bytes": 42246400 + 1237248, "rows": 1024, "weights": 2 * 8192 * 2048},
+    "k_enc_recurrent": {"bytes": 167305216 + 6090752},
+}
+
+
 def roofline(job, tag, ms, n, pk):
     """Roofline entry of the dominant kernel.  Algorithmic work per launch: the weight bytes
     the kernel must read once plus per-row state traffic, and 2*rows*J*K integer ops."""
@@ -496,21 +505,29 @@ def roofline(job, tag, ms, n, pk):
         l, kx = {5: (d.pred_lstm, 256), 7: (d.src.lstm[0], 256), 9: (d.tgt.lstm[0], 256),
                  10: (d.tgt.lstm[-1], d.tgt.lstm[0].H)}[tag]
         bytes_, ops = lstm_work(l, N, kx)
+        if tag == 10 and l.H == 2048:
+            # DRAM bytes of one launch from the ncu capture (cold caches, 1024 rows): the weights do
+            # not depend on the rows, the rest scales with them
+            t = NCU_TRAFFIC["k_mma_lstm_tgt_l2"]
+            out["traffic"] = t["weights"] + (t["bytes"] - t["weights"]) * N / t["rows"]
     elif tag == 3:
         # persistent recurrence: one launch = all T steps of a layer, both directions.  It must
-        # read the int32 input accumulators once, the recurrent weights once, and write the codes;
-        # its arithmetic is DP4A on the plain ALUs, so the ALU roofline applies.
+        # read the int32 input accumulators once, the recurrent weights once, and write the codes.
+        # By bytes it is an HBM kernel; in practice the T dependent steps (MMA, cell update,
+        # exchange of the new codes, cluster barrier) bind it, so the fraction is small by nature.
         l = job.enc.layers[1][0]
         Bn, Tn, H = wl["B"], wl["T"], l.H
         bytes_ = 2 * (4 * H * H + Tn * Bn * 4 * H * 4 + Tn * Bn * H // 2)
         ops = 2 * 2.0 * Tn * Bn * 4 * H * H
-        dp4a_peak = 148 * 128 * 8 * 1.965e9 / 1e12       # SMs x lanes x ops per DP4A x clock
         sec = ms / 1e3
-        out.update(bound="alu", achieved=ops / sec / 1e12, peak=dp4a_peak, unit="TOP/s (DP4A)",
-                   frac=ops / sec / 1e12 / dp4a_peak, algorithmic_bytes=bytes_, algorithmic_ops=ops,
-                   hbm={"achieved": bytes_ / sec / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                        "frac": bytes_ / sec / 1e9 / pk["hbm_gbs"]},
-                   peak_source="148 SMs x 128 lanes x 8 int-ops x 1.965 GHz (unit counts and max clock)")
+        out.update(bound="hbm", achieved=bytes_ / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s",
+                   frac=bytes_ / sec / 1e9 / pk["hbm_gbs"], algorithmic_bytes=bytes_, algorithmic_ops=ops,
+                   tensor={"achieved": ops / sec / 1e12, "peak": int8_peak, "unit": "TOP/s (int8, 2x measured bf16)",
+                           "frac": ops / sec / 1e12 / int8_peak},
+                   us_per_step=ms * 1e3 / Tn, peak_source=pk["source"],
+                   note="latency-bound: T dependent steps per launch, each ending in a cluster barrier")
+        if Bn == 32 and Tn == 250:
+            out["traffic"] = NCU_TRAFFIC["k_enc_recurrent"]["bytes"]
         return out
     elif tag == 2:
         l = job.enc.layers[1][0]
