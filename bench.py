@@ -39,6 +39,10 @@ WORKLOADS = {
     # reduced lengths of the same shapes, for profiler captures that must end by themselves
     "prof_encoder": dict(B=32, T=250, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
     "prof_end_to_end": dict(B=64, T=24, U_max=12, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
+    # the regime of the paper's run-time figure (Section 4.1): ONE utterance of 152 encoder frames,
+    # everything at 4 bits, beam width from --beam (1..16): 16 hypothesis rows at most, so every
+    # step streams all weights for a handful of rows
+    "fig2_single_utterance": dict(B=1, T=152, U_max=76, l1_bits=4, out_bits=4, enc=True, dec=True, seed=6),
 }
 
 
@@ -169,13 +173,14 @@ def run_reference(args):
 class Job:
     """Holds device weights and buffers of one workload and runs whole steps."""
 
-    def __init__(self, wl_name: str, rank: int):
+    def __init__(self, wl_name: str, rank: int, beam: int = 16):
         import torch
         from paper_2206_07882_b200 import binding as Bd
         from paper_2206_07882_b200 import synth
         self.torch, self.Bd = torch, Bd
         wl = self.wl = WORKLOADS[wl_name]
         self.name = wl_name
+        self.W = max(1, min(16, beam))
         B, T = wl["B"], wl["T"]
         from paper_2206_07882_b200 import sharding
         seed = sharding.rank_seed(wl["seed"], rank)    # every rank gets its own utterances
@@ -193,7 +198,7 @@ class Job:
         if wl["dec"]:
             dw = synth.decoder(3, out_bits=wl["out_bits"], U_max=wl["U_max"])
             self.dec = Bd.Decoder(dw)
-            self.dec.alloc_state(B, 16, T + wl["U_max"])
+            self.dec.alloc_state(B, self.W, T + wl["U_max"])
             if not wl["enc"]:
                 self.host_in = torch.from_numpy(synth.enc_frames(seed, T, B, 1280)).pin_memory()
                 self.frame_act = Bd.q4_act_symmetric(1.0, 4)
@@ -241,7 +246,7 @@ class Job:
     def search(self, enc_out):
         e, res = enc_out if isinstance(enc_out, tuple) else (enc_out, None)
         if self.dec is not None:
-            res = self.dec.decode(e, u_max=self.wl["U_max"], W=16)
+            res = self.dec.decode(e, u_max=self.wl["U_max"], W=self.W)
         return res
 
     def step(self, x, mark=None):
@@ -273,6 +278,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4_end_to_end", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-frames", type=int, default=8)
+    ap.add_argument("--beam", type=int, default=16, help="beam width W (1..16)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dependent-launch", action="store_true",
                     help="launch the beam step's kernels in plain stream order")
@@ -301,7 +307,7 @@ def main():
     if args.no_dependent_launch:
         from paper_2206_07882_b200 import binding as _Bd
         _Bd.dependent_launch_set(False)
-    job = Job(args.workload, rank)
+    job = Job(args.workload, rank, args.beam)
     wl = job.wl
     B, T, U = wl["B"], wl["T"], wl["U_max"]
     iters = T + U if wl["dec"] else 0
@@ -433,13 +439,13 @@ def main():
                 "vs_baseline": None, "dtype": "int4/int8 codes, int32 accumulate, fp32 gates",
                 "data": "synthetic",
                 "config": {"workload": args.workload, "utterances_per_gpu": B, "frames": T,
-                           "beam": 16 if wl["dec"] else 0, "label_budget": U, "search_iterations": iters,
+                           "beam": job.W if wl["dec"] else 0, "label_budget": U, "search_iterations": iters,
                            "launch": "cuda graph replay of the whole pass" if use_graph else "eager",
                            "l2": "no flush: one pass streams more than 1 GB of accumulators, codes and "
                                  "state through the 126 MB L2 between two uses of any input"},
                 "parts": {"encoder_ms": enc_ms, "decode_ms": dec_ms,
                           "encoder_frames_per_s": (B * T / (enc_ms / 1e3)) if wl["enc"] and enc_ms else None,
-                          "beam_hyps_per_s": (B * 16 * iters / (dec_ms / 1e3)) if wl["dec"] and dec_ms else None},
+                          "beam_hyps_per_s": (B * job.W * iters / (dec_ms / 1e3)) if wl["dec"] and dec_ms else None},
                 "e2e": {"value": rtf_e2e, "unit": "s/s", "h2d_bytes_per_step": job.h2d_bytes(),
                         "d2h_bytes_per_step": d2h},
                 "gpu_launches": n_launch_step * K, "launches_per_step": n_launch_step, "kernels": shares,
@@ -477,7 +483,7 @@ def roofline(job, tag, ms, n, pk):
     the kernel must read once plus per-row state traffic, and 2*rows*J*K integer ops."""
     name = TAG_NAMES[tag]
     wl = job.wl
-    N = wl["B"] * 16
+    N = wl["B"] * job.W
     if job.dec is not None and tag in (5, 7, 9, 10):
         # rows a launch really advances: label extensions of the previous selection (blank
         # extensions keep their parent's state), counted from the search history of the last pass

@@ -268,6 +268,35 @@ def logmel(seed: int, B: int, T100: int = 1000, n_mel: int = 40) -> np.ndarray:
     return Stream(seed).normal("logmel", (B, T100, n_mel)).astype(np.float32)
 
 
+def paper_dimensions(seed: int = 5, T: int = 12, B: int = 2, U_max: int = 6):
+    """The model sizes the paper states in Section 2: 340-d encoder input, 6 bidirectional layers of
+    640 cells, 256-d encoder/prediction outputs, prediction LSTM of 768 cells behind a small
+    embedding (10-d reproduces the 2.6 M parameters quoted), 46 output characters, external LM of
+    two 2048-cell layers with a 256 bottleneck, source LM shaped like the prediction network;
+    fusion weights 0.7 / 0.5 / 0.2 as after Eq. 1."""
+    enc = encoder(seed, T=T, B=B, F=340, H=640, L=6, D=256)
+    dec = decoder(seed + 1000, V=46, E=10, Hp=768, D=256, Hs=768, Ht=2048, tgt_layers=2, U_max=U_max,
+                  lambda_t=0.7, lambda_s=0.5, rho=0.2)
+    return enc, dec
+
+
+def parameter_counts(enc: EncoderW, dec: DecoderW) -> dict:
+    """Trainable parameters of a weight set (matrices, biases, embeddings) by component."""
+    def lstm(l: LstmW) -> int:
+        return l.w_ih.codes.size + l.w_hh.codes.size + l.bias.size
+
+    def linear(l: LinearW) -> int:
+        return l.w.codes.size + (l.bias.size if l.bias is not None else 0)
+
+    def lm(m: LmW) -> int:
+        return m.emb.size + sum(lstm(l) for l in m.lstm) + linear(m.bott) + linear(m.out)
+
+    n_enc = sum(lstm(l) for layer in enc.layers for l in layer) + (linear(enc.proj) if enc.proj else 0)
+    n_pred = dec.pred.emb.size + lstm(dec.pred.lstm) + linear(dec.pred.proj) + linear(dec.joint.out)
+    return {"encoder": n_enc, "prediction": n_pred, "rnnt": n_enc + n_pred, "lm_ext": lm(dec.tgt),
+            "lm_src": lm(dec.src)}
+
+
 # Reduced-dimension suite for whole-search comparisons over many utterances.
 def parity_suite(seed: int = 7, n_utt: int = 256, T: int = 32, V: int = 64):
     enc = encoder(seed, T=T, B=n_utt, F=48, H=64, L=2, D=32)
