@@ -778,7 +778,8 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     // `dep`: the previous launch on the same stream is a kernel of this library, so this one may
     // be launched as its programmatic dependent
     auto lstm_mma = [&](cudaStream_t s, bool dep, int tag_id, int li, const q4_lstm& L, const q4_act& x_act,
-                        const int8_t* xa, const int8_t* ha, void* hq, float* c, int8_t* h8) -> int {
+                        const int8_t* xa, const int8_t* ha, void* hq, float* c, int8_t* h8, int h_first = 0,
+                        int trigger_early = 0) -> int {
       TagScope tag(tag_id);
       const int H = L.w_hh.k_pad, Kx = L.w_ih.k_pad;
       MmaLstmArgs a;
@@ -802,6 +803,8 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       a.h8_ld = H;
       a.status = st.status;
       a.n_active = n_active;
+      a.h_first = dep ? h_first : 0;
+      a.trigger_early = trigger_early;
       Q4_TRY(launch_mma_lstm(a, xa, Kx, reinterpret_cast<const int8_t*>(pb + pp.lstm[li].xw), Kx, ha, H,
                              reinterpret_cast<const int8_t*>(pb + pp.lstm[li].hw), H, s, dep));
       return Q4_OK;
@@ -856,13 +859,15 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       int8_t* h8_0 = which == 0 ? src_h8 : tgt_h8[0];
       float* lp = which == 0 ? st.src_lp : st.tgt_lp;
       Q4_CHECK(lstm_mma(sl, which == 1 || !forked, which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, which == 0 ? 1 : 2, L0, lm.emb_act,
-                        xa8[which + 1], ha8[which + 1], hq0, c0, h8_0));
+                        xa8[which + 1], ha8[which + 1], hq0, c0, h8_0, 0, lm.n_layers == 2 ? 1 : 0));
       const int8_t* top8 = h8_0;
       const q4_lstm* last = &L0;
       if (lm.n_layers == 2) {
         const q4_lstm& L1 = lm.lstm[1];
+        // layer 2 reads layer 1's output only as its input operand: its recurrent half starts
+        // while layer 1 is still in its cell update
         Q4_CHECK(lstm_mma(sl, true, TAG_TGT_L2, 3, L1, L0.hid_act, h8_0, ha8[3], st.tgt_hq[1], st.tgt_c[1],
-                          tgt_h8[1]));
+                          tgt_h8[1], 1, 0));
         top8 = tgt_h8[1];
         last = &L1;
       }

@@ -77,6 +77,9 @@ struct MmaLstmArgs {
   long long dbg_ld;
   int32_t* status;
   const int32_t* n_active;  // optional: rows >= *n_active carry no work (tiles beyond it exit at once)
+  int32_t h_first;          // 1: only the input operand comes from the previous kernel of the stream, so
+                            // the recurrent half of the K loop runs before waiting for that kernel
+  int32_t trigger_early;    // 1: let the next kernel of the stream start beside this one
 };
 struct LmHeadArgs {
   int32_t N, H, V;            // launch rows, LSTM width (K of the bottleneck; 0 = no bottleneck: the

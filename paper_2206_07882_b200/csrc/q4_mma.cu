@@ -778,24 +778,32 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
-  pdl_wait();   // everything above overlaps the tail of the previous kernel of the stream
+  // Everything above overlaps the tail of the previous kernel of the stream.  With h_first only
+  // the input operand is that kernel's output: the recurrent half of the K loop (operands from
+  // kernels further back, all complete) runs before the wait, the input half after it.
+  const bool h_first = a.h_first != 0 && nkx > 0;
+  if (!h_first) pdl_wait();
   const bool has_work = !(a.n_active && m0 >= *a.n_active);   // uniform per CTA
+  if (a.trigger_early) pdl_trigger();   // the successor has a half it can run beside this kernel
+  const int x_first = h_first ? nkh : 0, hh_first = h_first ? 0 : nkx;   // first chunk of each part
 
   if (!has_work) {
-    // whole tile without work
+    if (h_first) pdl_wait();   // whole tile without work; still ordered behind the previous kernel
   } else if (warp == LSTM_EPI_WARPS && lane == 0) {
     bool ok = true;
     for (int i = 0; i < nk && ok; ++i) {
       const int s = i % LSTM_STAGES;
       if (i >= LSTM_STAGES) ok = mbar_wait(&empty[s], ((i / LSTM_STAGES) - 1) & 1);
       if (!ok) break;
+      const bool xpart = h_first ? i >= nkh : i < nkx;
+      if (h_first && i == x_first) pdl_wait();
       mbar_expect_tx(&full[s], STAGE);
-      if (i < nkx) {
-        tma_load_2d(smem + s * STAGE, &tma_xa, i * BK, m0, &full[s]);
-        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_xw, i * BK, n0, &full[s]);
+      if (xpart) {
+        tma_load_2d(smem + s * STAGE, &tma_xa, (i - x_first) * BK, m0, &full[s]);
+        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_xw, (i - x_first) * BK, n0, &full[s]);
       } else {
-        tma_load_2d(smem + s * STAGE, &tma_ha, (i - nkx) * BK, m0, &full[s]);
-        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_hw, (i - nkx) * BK, n0, &full[s]);
+        tma_load_2d(smem + s * STAGE, &tma_ha, (i - hh_first) * BK, m0, &full[s]);
+        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_hw, (i - hh_first) * BK, n0, &full[s]);
       }
     }
     pdl_trigger();
@@ -810,9 +818,9 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
       tc_fence_after();
       const uint64_t da = umma_desc_sw128(smem_u32(smem + s * STAGE));
       const uint64_t db = umma_desc_sw128(smem_u32(smem + s * STAGE + A_BYTES));
-      const bool xpart = i < nkx;
+      const bool xpart = h_first ? i >= nkh : i < nkx;
       const uint32_t d = tmem + (xpart ? 0 : LSTM_BN);
-      const int first = xpart ? 0 : nkx;
+      const int first = xpart ? x_first : hh_first;
 #pragma unroll
       for (int kk = 0; kk < BK / 32; ++kk) umma_i8(d, da + 2 * kk, db + 2 * kk, idesc, (i != first) || kk != 0);
       umma_commit(&empty[s]);
@@ -831,6 +839,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
     }
     const bool ok = mbar_wait(&acc_full, 0);
     tc_fence_after();
+    if (h_first) pdl_wait();   // before the first global write of this thread
     pdl_trigger();   // the main loop is over: the next kernel may set itself up
     if (!ok && lane == 0) flag_timeout(a.status);
     const bool live = ok && dst >= 0;
