@@ -436,6 +436,33 @@ def alsd(dec: Decoder, e: np.ndarray, utts: Optional[Sequence[int]] = None, trac
     return r
 
 
+def tsd(dec: Decoder, e: np.ndarray, S_max: int, utts: Optional[Sequence[int]] = None, trace: bool = True,
+        n_threads: int = 8):
+    """Time-synchronous search, at most S_max labels per frame.  e [T,B,D].  Returns dict like alsd():
+    tokens, len, score, finals_* and, with trace, parent / token / tscore / u [n, T (S_max+1), W] and
+    n_slots [n, T (S_max+1)] (frame-close steps hold parent = first proposing slot, token = -1 - step)."""
+    e = _c(e, np.float32)
+    T, B, D = e.shape
+    utts = np.arange(B, dtype=np.int32) if utts is None else _c(utts, np.int32)
+    n = len(utts)
+    W, U = dec.c.W, dec.c.U_max
+    IT = T * (S_max + 1)
+    r = dict(tokens=np.zeros((n, max(U, 1)), np.int32), len=np.zeros(n, np.int32),
+             score=np.zeros(n, np.float32), finals_n=np.zeros(n, np.int32),
+             finals_tokens=np.zeros((n, W, max(U, 1)), np.int32),
+             finals_len=np.zeros((n, W), np.int32), finals_score=np.zeros((n, W), np.float32))
+    if trace:
+        r.update(parent=np.full((n, IT, W), -1, np.int32), token=np.zeros((n, IT, W), np.int32),
+                 tscore=np.zeros((n, IT, W), np.float32), u=np.zeros((n, IT, W), np.int32),
+                 n_slots=np.zeros((n, IT), np.int32))
+    lib().orc_tsd_batch(C.byref(dec.c), _p(e), C.c_int32(T), C.c_int32(B), C.c_int32(S_max), _p(utts),
+                        C.c_int32(n), _p(r["tokens"]), _p(r["len"]), _p(r["score"]), _p(r.get("parent")),
+                        _p(r.get("token")), _p(r.get("tscore")), _p(r.get("u")), _p(r.get("n_slots")),
+                        _p(r["finals_n"]), _p(r["finals_tokens"]), _p(r["finals_len"]),
+                        _p(r["finals_score"]), C.c_int32(n_threads))
+    return r
+
+
 def sequence_score(dec: Decoder, e_utt: np.ndarray, y: Sequence[int]):
     """Eq. 1 score of one label string via the transducer forward recursion."""
     e = _c(e_utt, np.float32)

@@ -758,6 +758,154 @@ void orc_alsd_batch(const OrcDecoder* Dc, const float* e, int32_t T, int32_t B,
   for (auto& th : pool) th.join();
 }
 
+// Time-synchronous beam search with the score of Eq. 1 for ONE utterance: all hypotheses of
+// the beam stand at the same frame t.  A frame takes S_max + 1 steps.  In step s every
+// hypothesis of the current set A proposes its blank (score + log P(blank)): the string moves
+// to the next frame and is collected in the set B, equal label strings merged by log-addition
+// (the entry keeps the provenance of its first insertion); while s < S_max and |y| < U_max it
+// also proposes every label k (score + log P(k) + lambda_t log P_tgt(k) - lambda_s log
+// P_src(k) + rho), and the W best label proposals (score descending, then parent slot, then
+// token) become the set A of step s + 1, still at frame t.  After step S_max the W best
+// entries of B (score descending, then insertion order) are the beam of frame t + 1.  The
+// entries of B after the last frame are the final hypotheses.  T (S_max + 1) steps in all.
+//
+// Trace arrays [T (S_max+1), W]: the set produced by each step.  For s < S_max: parent slot,
+// token (> 0), score, |y| of each new member of A.  For s = S_max (frame close): parent = the
+// slot the entry's blank was first proposed from, token = -1 - (step of that proposal within
+// the frame), score, |y|.
+void orc_tsd(const OrcDecoder* Dc, const float* e, int32_t T, int32_t S_max, int32_t* best_tokens,
+             int32_t* best_len, float* best_score, int32_t* trace_parent, int32_t* trace_token,
+             float* trace_score, int32_t* trace_u, int32_t* trace_n, int32_t* finals_n,
+             int32_t* finals_tokens, int32_t* finals_len, float* finals_score) {
+  const int32_t W = Dc->W, U_max = Dc->U_max, V = Dc->joint.out.J, D = Dc->joint.out.K;
+  struct Entry {
+    Hyp h;
+    int32_t org_step, org_slot;
+  };
+  std::vector<Hyp> A(1);
+  A[0].t = 0;
+  A[0].S = 0.0f;
+  pred_init(Dc->pred, A[0].pred);
+  lm_init(Dc->src, A[0].src);
+  lm_init(Dc->tgt, A[0].tgt);
+  pred_advance(Dc->pred, 0, A[0].pred);   // start symbol = 0
+  lm_advance(Dc->src, 0, A[0].src);
+  lm_advance(Dc->tgt, 0, A[0].tgt);
+  std::vector<Entry> Bset;
+  std::vector<float> lp(V);
+  int32_t it = 0;
+  for (int32_t t = 0; t < T; ++t) {
+    Bset.clear();
+    for (int32_t s = 0; s <= S_max; ++s, ++it) {
+      std::vector<Cand> labels;
+      for (int32_t w = 0; w < (int32_t)A.size(); ++w) {
+        const Hyp& h = A[w];
+        orc_joint(&Dc->joint, e + (int64_t)t * D, h.pred.p.data(), 1, lp.data(), nullptr, nullptr);
+        const float sb = (float)((double)h.S + (double)lp[0]);
+        bool merged = false;
+        for (Entry& b : Bset)
+          if (b.h.y == h.y) {
+            b.h.S = log_add(b.h.S, sb);
+            merged = true;
+            break;
+          }
+        if (!merged) {
+          Entry b{h, s, w};
+          b.h.S = sb;
+          b.h.t = t + 1;
+          Bset.push_back(std::move(b));
+        }
+        if (s < S_max && (int32_t)h.y.size() < U_max)
+          for (int32_t k = 1; k < V; ++k) {
+            const double sc = (double)h.S + (double)lp[k] + (double)Dc->lambda_t * (double)h.tgt.lp[k] -
+                              (double)Dc->lambda_s * (double)h.src.lp[k] + (double)Dc->rho;
+            labels.push_back({(float)sc, w, k, false});
+          }
+      }
+      std::vector<Hyp> next;
+      if (s < S_max) {
+        std::sort(labels.begin(), labels.end(), ranks_before);
+        if ((int32_t)labels.size() > W) labels.resize(W);
+        for (size_t i = 0; i < labels.size(); ++i) {
+          const Cand& c = labels[i];
+          Hyp h = A[c.parent];
+          h.S = c.S;
+          h.y.push_back(c.token);
+          pred_advance(Dc->pred, c.token, h.pred);
+          lm_advance(Dc->src, c.token, h.src);
+          lm_advance(Dc->tgt, c.token, h.tgt);
+          if (trace_parent) {
+            const int64_t o = (int64_t)it * W + (int64_t)i;
+            trace_parent[o] = c.parent;
+            trace_token[o] = c.token;
+            trace_score[o] = c.S;
+            trace_u[o] = (int32_t)h.y.size();
+          }
+          next.push_back(std::move(h));
+        }
+      } else {
+        std::vector<int32_t> idx(Bset.size());
+        for (size_t i = 0; i < idx.size(); ++i) idx[i] = (int32_t)i;
+        std::stable_sort(idx.begin(), idx.end(),
+                         [&](int32_t a, int32_t b) { return Bset[a].h.S > Bset[b].h.S; });
+        if ((int32_t)idx.size() > W) idx.resize(W);
+        for (size_t i = 0; i < idx.size(); ++i) {
+          const Entry& b = Bset[idx[i]];
+          if (trace_parent) {
+            const int64_t o = (int64_t)it * W + (int64_t)i;
+            trace_parent[o] = b.org_slot;
+            trace_token[o] = -1 - b.org_step;
+            trace_score[o] = b.h.S;
+            trace_u[o] = (int32_t)b.h.y.size();
+          }
+          next.push_back(b.h);
+        }
+      }
+      if (trace_n) trace_n[it] = (int32_t)next.size();
+      A.swap(next);
+    }
+  }
+  // A = the W best final hypotheses, best first
+  *best_len = A.empty() ? 0 : (int32_t)A[0].y.size();
+  *best_score = A.empty() ? 0.0f : A[0].S;
+  for (int32_t i = 0; i < *best_len && i < U_max; ++i) best_tokens[i] = A[0].y[i];
+  if (finals_n) *finals_n = (int32_t)A.size();
+  if (finals_tokens)
+    for (size_t f = 0; f < A.size(); ++f) {
+      finals_len[f] = (int32_t)A[f].y.size();
+      finals_score[f] = A[f].S;
+      for (size_t i = 0; i < A[f].y.size(); ++i) finals_tokens[f * U_max + i] = A[f].y[i];
+    }
+}
+
+void orc_tsd_batch(const OrcDecoder* Dc, const float* e, int32_t T, int32_t B, int32_t S_max,
+                   const int32_t* utts, int32_t n_utts, int32_t* best_tokens, int32_t* best_len,
+                   float* best_score, int32_t* trace_parent, int32_t* trace_token, float* trace_score,
+                   int32_t* trace_u, int32_t* trace_n, int32_t* finals_n, int32_t* finals_tokens,
+                   int32_t* finals_len, float* finals_score, int32_t n_threads) {
+  const int32_t D = Dc->joint.out.K, W = Dc->W, U = std::max(Dc->U_max, 1), IT = T * (S_max + 1);
+  n_threads = std::max(1, std::min(n_threads, n_utts));
+  std::vector<std::thread> pool;
+  for (int32_t w = 0; w < n_threads; ++w)
+    pool.emplace_back([=]() {
+      for (int32_t i = w; i < n_utts; i += n_threads) {
+        const int32_t b = utts[i];
+        std::vector<float> eu((size_t)T * D);
+        for (int32_t t = 0; t < T; ++t)
+          std::memcpy(&eu[(size_t)t * D], e + ((int64_t)t * B + b) * D, D * sizeof(float));
+        const int64_t o = (int64_t)i * IT * W;
+        orc_tsd(Dc, eu.data(), T, S_max, best_tokens + (int64_t)i * U, best_len + i, best_score + i,
+                trace_parent ? trace_parent + o : nullptr, trace_token ? trace_token + o : nullptr,
+                trace_score ? trace_score + o : nullptr, trace_u ? trace_u + o : nullptr,
+                trace_n ? trace_n + (int64_t)i * IT : nullptr, finals_n ? finals_n + i : nullptr,
+                finals_tokens ? finals_tokens + (int64_t)i * W * U : nullptr,
+                finals_tokens ? finals_len + (int64_t)i * W : nullptr,
+                finals_tokens ? finals_score + (int64_t)i * W : nullptr);
+      }
+    });
+  for (auto& th : pool) th.join();
+}
+
 // Score of ONE given label string under Eq. 1, with log P(y|x) from the
 // textbook transducer forward recursion over the (t,u) lattice:
 //   a(0,0)=0; a(t,u) = logadd(a(t-1,u)+blank(t-1,u), a(t,u-1)+label(t,u-1));

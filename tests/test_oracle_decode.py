@@ -254,3 +254,77 @@ def test_slot_order_does_not_matter():
     b = O.alsd(dec, e, utts=[4, 3, 2, 1, 0], n_threads=3)
     for k in ("tokens", "len", "score"):
         np.testing.assert_array_equal(a[k], b[k][::-1])
+
+
+# ---------------------------------------------------------------- time-synchronous search
+@pytest.mark.parametrize("T,U_max,seed", [(1, 2, 0), (2, 2, 1), (3, 2, 2), (3, 1, 3), (2, 3, 4)])
+def test_time_synchronous_unpruned_equals_brute_force_eq1(T, U_max, seed):
+    # beam >= number of label strings and as many labels per frame as the budget allows: nothing is
+    # pruned, every alignment is reachable, so every final score is Eq. 1 by the forward recursion
+    dw, dec = tiny_decoder(seed=30 + seed, U_max=U_max, W=16)
+    e = tiny_e(seed, T)
+    r = O.tsd(dec, e, S_max=U_max)
+    got = finals_dict(r)
+    strings = list(all_strings(3, U_max))
+    assert set(got) == set(strings)
+    for y in strings:
+        want = brute_force_score(dec, dw, e[:, 0, :], y)[0]
+        assert abs(got[y] - want) < 2e-5, (y, got[y], want)
+    # the two search orders agree when neither prunes
+    ref = finals_dict(O.alsd(dec, e))
+    for y in strings:
+        assert abs(got[y] - ref[y]) < 2e-5
+    best = max(strings, key=lambda y: got[y])
+    assert tuple(r["tokens"][0, :r["len"][0]].tolist()) == best
+    # finals are listed best first
+    fs = r["finals_score"][0, :r["finals_n"][0]]
+    assert (np.diff(fs) <= 0).all()
+
+
+def test_time_synchronous_label_limit_per_frame():
+    dw, dec = tiny_decoder(seed=52, V=4, U_max=3, W=16)
+    e = tiny_e(5, 2)
+    # no labels at all: the empty string, scored by the blanks alone
+    r0 = O.tsd(dec, e, S_max=0)
+    assert finals_dict(r0).keys() == {()}
+    assert abs(finals_dict(r0)[()] - brute_force_score(dec, dw, e[:, 0, :], ())[0]) < 2e-5
+    # one frame, one label per frame: strings of length <= 1, each with its single alignment
+    e1 = tiny_e(6, 1)
+    r1 = O.tsd(dec, e1, S_max=1)
+    got = finals_dict(r1)
+    assert set(got) == {(), (1,), (2,), (3,)}
+    for y in got:
+        assert abs(got[y] - brute_force_score(dec, dw, e1[:, 0, :], y)[0]) < 2e-5
+    # two frames, one label per frame: "ab" needs a at frame 0 and b at frame 1 -- one alignment of the
+    # three the lattice has, so its score stays below the full sum
+    r2 = O.tsd(dec, e, S_max=1)
+    got2 = finals_dict(r2)
+    full = brute_force_score(dec, dw, e[:, 0, :], (1, 2))[0]
+    assert (1, 2) in got2 and got2[(1, 2)] < full
+    assert max(len(y) for y in got2) == 2
+
+
+def test_time_synchronous_pruned_trace_invariants():
+    dw, dec = tiny_decoder(seed=61, V=6, U_max=5, W=3)
+    T, S = 6, 2
+    e = tiny_e(8, T)
+    r = O.tsd(dec, e, S_max=S)
+    par, tok, sc, u, ns = r["parent"][0], r["token"][0], r["tscore"][0], r["u"][0], r["n_slots"][0]
+    assert ns.shape == (T * (S + 1),) and (ns <= 3).all() and ns[-1] >= 1
+    for it in range(T * (S + 1)):
+        s = it % (S + 1)
+        n = ns[it]
+        prev_n = 1 if it == 0 else ns[it - 1]
+        prev_u = np.zeros(1, np.int32) if it == 0 else u[it - 1]
+        assert (np.diff(sc[it, :n]) <= 0).all()                      # ranked by score
+        if s < S:
+            assert ((tok[it, :n] >= 1) & (tok[it, :n] < 6)).all()
+            assert ((par[it, :n] >= 0) & (par[it, :n] < prev_n)).all()
+            assert (u[it, :n] == prev_u[par[it, :n]] + 1).all()
+            assert (u[it, :n] <= 5).all()
+        else:
+            org = -1 - tok[it, :n]
+            assert ((org >= 0) & (org <= S)).all()                   # the step the blank was proposed in
+            assert (par[it, :n] >= 0).all()
+    # the best final is the first slot of the last frame close
+    assert abs(r["score"][0] - sc[-1, 0]) == 0.0 and r["len"][0] == u[-1, 0]
