@@ -36,6 +36,10 @@ WORKLOADS = {
     "cfg4_end_to_end": dict(B=64, T=500, U_max=250, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
     "cfg1_encoder": dict(B=32, T=500, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
     "cfg3_beam": dict(B=16, T=300, U_max=150, l1_bits=4, out_bits=4, enc=False, dec=True, seed=3),
+    # the same beam workload driven time-synchronously (its wording): at most 2 labels per frame,
+    # 3 calls per frame, 900 calls
+    "cfg3_beam_time_synchronous": dict(B=16, T=300, U_max=150, l1_bits=4, out_bits=4, enc=False, dec=True,
+                                       seed=3, tsd=2),
     # reduced lengths of the same shapes, for profiler captures that must end by themselves
     "prof_encoder": dict(B=32, T=250, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
     "prof_end_to_end": dict(B=64, T=24, U_max=12, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
@@ -198,7 +202,10 @@ class Job:
         if wl["dec"]:
             dw = synth.decoder(3, out_bits=wl["out_bits"], U_max=wl["U_max"])
             self.dec = Bd.Decoder(dw)
-            self.dec.alloc_state(B, self.W, T + wl["U_max"])
+            if "tsd" in wl:
+                self.dec.alloc_state(B, self.W, T * (wl["tsd"] + 1), wl["tsd"])
+            else:
+                self.dec.alloc_state(B, self.W, T + wl["U_max"])
             if not wl["enc"]:
                 self.host_in = torch.from_numpy(synth.enc_frames(seed, T, B, 1280)).pin_memory()
                 self.frame_act = Bd.q4_act_symmetric(1.0, 4)
@@ -246,7 +253,10 @@ class Job:
     def search(self, enc_out):
         e, res = enc_out if isinstance(enc_out, tuple) else (enc_out, None)
         if self.dec is not None:
-            res = self.dec.decode(e, u_max=self.wl["U_max"], W=self.W)
+            if "tsd" in self.wl:
+                res = self.dec.decode_time_synchronous(e, self.wl["tsd"], u_max=self.wl["U_max"], W=self.W)
+            else:
+                res = self.dec.decode(e, u_max=self.wl["U_max"], W=self.W)
         return res
 
     def step(self, x, mark=None):
@@ -310,7 +320,7 @@ def main():
     job = Job(args.workload, rank, args.beam)
     wl = job.wl
     B, T, U = wl["B"], wl["T"], wl["U_max"]
-    iters = T + U if wl["dec"] else 0
+    iters = (T * (wl["tsd"] + 1) if "tsd" in wl else T + U) if wl["dec"] else 0
     W = max(args.warmup, 3)
     K = args.steps
     use_graph = not args.eager
@@ -487,7 +497,7 @@ def roofline(job, tag, ms, n, pk):
     if job.dec is not None and tag in (5, 7, 9, 10):
         # rows a launch really advances: label extensions of the previous selection (blank
         # extensions keep their parent's state), counted from the search history of the last pass
-        tok = job.dec.tensors["bp_token"][:wl["T"] + wl["U_max"]]
+        tok = job.dec.tensors["bp_token"][:(wl["T"] * (wl["tsd"] + 1) if "tsd" in wl else wl["T"] + wl["U_max"])]
         N = max(1.0, float((tok > 0).sum().item() + wl["B"]) / float(tok.shape[0]))
         out_rows = N
     else:

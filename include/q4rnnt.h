@@ -258,6 +258,21 @@ typedef struct {
    * the whole step. */
   void* aux_stream[2];
   void* aux_event[3];
+  /* Time-synchronous search only (modes 1 and 2 of dr_fusion_beam_step; leave zero / NULL for the
+   * alignment-length synchronous search).  tsd_smax: at most that many labels per frame (0..3).
+   * rows_per_utt: state rows per utterance; 0 means 2W; the time-synchronous search needs
+   * W (tsd_smax + 1) <= 64 of them (R = B * rows_per_utt then).  nb_*: the candidate set of the next
+   * frame, CB = W (tsd_smax + 1) entries per utterance [B, CB], nb_n [B] entries in use. */
+  int32_t tsd_smax;
+  int32_t rows_per_utt;
+  float* nb_score;
+  int32_t* nb_u;
+  int32_t* nb_last_tok;
+  int32_t* nb_row;
+  int32_t* nb_origin;      /* (step within the frame) << 8 | slot of the first proposal of the entry */
+  uint64_t* nb_hash;
+  uint64_t* nb_prev_hash;
+  int32_t* nb_n;
 } q4_beam_state;
 
 /* Reset `state` for a new batch: slot 0 of every utterance holds the empty hypothesis with
@@ -277,7 +292,17 @@ int q4_beam_init(q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters, q4
  *      proposals that consumed the last frame go to the finished list (best W kept); the
  *      W best others (score descending, then parent slot, then token) become the next beam.
  * e [T, B, D] fp32 projected encoder frames.  `iter` counts from 0; hypotheses in the beam
- * entering iteration `iter` satisfy t + u = iter.  mode: 0 (the only one implemented).
+ * entering iteration `iter` satisfy t + u = iter.
+ * mode 0: the search above (the paper's, Section 2), T + u_max iterations.
+ * modes 1 and 2: time-synchronous search over the same networks (the beam workload's wording):
+ * all hypotheses stand at frame t = iter / (S + 1), S = state->tsd_smax; a frame takes S + 1 calls.
+ * Call number s = iter % (S + 1) < S is mode 1: every blank proposal joins the candidate set of the
+ * next frame (equal label strings merged by log-addition, state->nb_*), and the W best label
+ * proposals become the hypotheses of the next call at the same frame.  Call s = S is mode 2: blanks
+ * join the candidate set, no labels are proposed, and the W best candidates (score descending, then
+ * order of insertion) open frame t + 1; after the last frame they are the finished list.
+ * T (S + 1) iterations.  History of a mode-2 call: bp_parent = slot that first proposed the entry,
+ * bp_token = -1 - (call number within the frame of that proposal).
  * workspace: q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D}), or, to enable the tensor-core path
  * (needs model->prepared and B*W >= 128), q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D, E_pad, Hp,
  * Hs, Ht}).  A bounded device wait that expires sets state->status to Q4_ERR_TIMEOUT.

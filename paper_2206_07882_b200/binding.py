@@ -70,7 +70,11 @@ class BeamStateS(C.Structure):
                 ("bp_parent", C.c_void_p), ("bp_token", C.c_void_p), ("bp_score", C.c_void_p),
                 ("fin_score", C.c_void_p), ("fin_iter", C.c_void_p), ("fin_slot", C.c_void_p),
                 ("fin_n", C.c_void_p), ("status", C.c_void_p),
-                ("aux_stream", C.c_void_p * 2), ("aux_event", C.c_void_p * 3)]
+                ("aux_stream", C.c_void_p * 2), ("aux_event", C.c_void_p * 3),
+                ("tsd_smax", C.c_int32), ("rows_per_utt", C.c_int32),
+                ("nb_score", C.c_void_p), ("nb_u", C.c_void_p), ("nb_last_tok", C.c_void_p),
+                ("nb_row", C.c_void_p), ("nb_origin", C.c_void_p), ("nb_hash", C.c_void_p),
+                ("nb_prev_hash", C.c_void_p), ("nb_n", C.c_void_p)]
 
 
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
@@ -444,6 +448,7 @@ class Decoder:
         if tensor_cores:
             self.q4_prepare_model()
         self.state = None
+        self.S_max = None
 
     def q4_prepare_model(self):
         """One-time int8 / gate-interleaved copies of the step weights for the tensor cores."""
@@ -456,9 +461,12 @@ class Decoder:
         return (self.pred_lstm.nbytes() + self.pred_proj.nbytes() + self.joint_out.nbytes() +
                 self.src.nbytes() - self.src.emb_q.numel() + self.tgt.nbytes() - self.tgt.emb_q.numel())
 
-    def alloc_state(self, B: int, W: int, n_iters: int):
+    def alloc_state(self, B: int, W: int, n_iters: int, S_max: Optional[int] = None):
+        """State for B utterances x W slots and n_iters calls; with S_max the layout of the
+        time-synchronous search (W (S_max + 1) state rows per utterance and its candidate set)."""
         dev = self.device
-        R, N = B * 2 * W, B * W
+        RW = 2 * W if S_max is None else max(2 * W, W * (S_max + 1))
+        R, N = B * RW, B * W
         Hp, Hs, Ht = self.pred_lstm.H, self.src.lstm[0].H, self.tgt.lstm[0].H
         z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
         t = self.tensors = dict(
@@ -489,6 +497,17 @@ class Decoder:
             setattr(s, name, t[name].data_ptr())
         s.tgt_hq[0], s.tgt_hq[1] = t["tgt_hq0"].data_ptr(), t["tgt_hq1"].data_ptr()
         s.tgt_c[0], s.tgt_c[1] = t["tgt_c0"].data_ptr(), t["tgt_c1"].data_ptr()
+        self.S_max = S_max
+        if S_max is not None:
+            CB = W * (S_max + 1)
+            t.update(nb_score=z((B, CB), torch.float32), nb_u=z((B, CB), torch.int32),
+                     nb_last_tok=z((B, CB), torch.int32), nb_row=z((B, CB), torch.int32),
+                     nb_origin=z((B, CB), torch.int32), nb_hash=z((B, CB), torch.int64),
+                     nb_prev_hash=z((B, CB), torch.int64), nb_n=z(B, torch.int32))
+            for name in ("nb_score", "nb_u", "nb_last_tok", "nb_row", "nb_origin", "nb_hash", "nb_prev_hash",
+                         "nb_n"):
+                setattr(s, name, t[name].data_ptr())
+            s.tsd_smax, s.rows_per_utt = S_max, RW
         if self.concurrent:
             # two more streams and three untimed events lent to the library for fork / join
             self._aux_streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
@@ -509,12 +528,12 @@ class Decoder:
         _chk(lib().q4_beam_init(C.byref(self.state), C.c_int32(self.B), C.c_int32(self.W),
                                 C.c_int32(self.n_iters), _stream()), "q4_beam_init")
 
-    def dr_fusion_beam_step(self, e: torch.Tensor, T: int, it: int, u_max: int):
+    def dr_fusion_beam_step(self, e: torch.Tensor, T: int, it: int, u_max: int, mode: int = 0):
         dw = self.dw
         _chk(lib().dr_fusion_beam_step(C.byref(self.model), C.byref(self.state), _p(e),
                                        C.c_int32(self.B), C.c_int32(T), C.c_int32(self.W),
                                        C.c_int32(it), C.c_int32(u_max), C.c_float(dw.lambda_t),
-                                       C.c_float(dw.lambda_s), C.c_float(dw.rho), C.c_int32(0),
+                                       C.c_float(dw.lambda_s), C.c_float(dw.rho), C.c_int32(mode),
                                        _p(self.ws), C.c_size_t(self.ws.numel()), _stream()),
              "dr_fusion_beam_step")
 
@@ -535,11 +554,27 @@ class Decoder:
         u_max = self.dw.U_max if u_max is None else u_max
         W = self.dw.W if W is None else W
         n_iters = T + u_max
-        if self.state is None or (self.B, self.W) != (B, W) or self.n_iters < n_iters:
+        if self.state is None or (self.B, self.W) != (B, W) or self.n_iters < n_iters or self.S_max is not None:
             self.alloc_state(B, W, n_iters)
         self.q4_beam_init()
         for it in range(n_iters):
             self.dr_fusion_beam_step(e, T, it, u_max)
+        return self.q4_traceback(n_iters, u_max)
+
+    def decode_time_synchronous(self, e: torch.Tensor, S_max: int, u_max: Optional[int] = None,
+                                W: Optional[int] = None):
+        """Time-synchronous search with at most S_max labels per frame: T (S_max + 1) calls of
+        dr_fusion_beam_step (mode 1, the last of every frame mode 2).  Returns like decode()."""
+        T, B, D = e.shape
+        u_max = self.dw.U_max if u_max is None else u_max
+        W = self.dw.W if W is None else W
+        n_iters = T * (S_max + 1)
+        if (self.state is None or (self.B, self.W) != (B, W) or self.n_iters < n_iters or
+                self.S_max != S_max):
+            self.alloc_state(B, W, n_iters, S_max)
+        self.q4_beam_init()
+        for it in range(n_iters):
+            self.dr_fusion_beam_step(e, T, it, u_max, mode=2 if it % (S_max + 1) == S_max else 1)
         return self.q4_traceback(n_iters, u_max)
 
 

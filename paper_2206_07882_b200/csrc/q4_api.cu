@@ -630,10 +630,22 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
                         float lambda_s, float rho, int32_t mode, void* workspace,
                         size_t workspace_bytes, q4_stream stream) {
   if (!model || !e || !workspace) return Q4_ERR_NULL;
-  if (mode != 0) return Q4_ERR_UNSUPPORTED;
+  if (mode < 0 || mode > 2) return Q4_ERR_UNSUPPORTED;
   if (B <= 0 || T <= 0 || W <= 0 || W > 16 || iter < 0 || u_max < 0) return Q4_ERR_DIM;
   const q4_model& m = *model;
   Q4_CHECK(check_state(state, m.tgt.n_layers));
+  if (mode != 0) {   // time-synchronous search: candidate set, enough state rows, call number matches
+    const q4_beam_state& ts = *state;
+    if (!ts.nb_score || !ts.nb_u || !ts.nb_last_tok || !ts.nb_row || !ts.nb_origin || !ts.nb_hash ||
+        !ts.nb_prev_hash || !ts.nb_n)
+      return Q4_ERR_NULL;
+    if (ts.tsd_smax < 0 || ts.tsd_smax > 3 || ts.rows_per_utt < W * (ts.tsd_smax + 1) || ts.rows_per_utt > 64)
+      return Q4_ERR_DIM;
+    const bool closing = iter % (ts.tsd_smax + 1) == ts.tsd_smax;
+    if (closing != (mode == 2) || iter / (ts.tsd_smax + 1) >= T) return Q4_ERR_DIM;
+  } else if (state->rows_per_utt != 0 && state->rows_per_utt < 2 * W) {
+    return Q4_ERR_DIM;
+  }
   const int V = m.V, D = m.D;
   if (V <= 1 || D <= 0 || D % 32 != 0 || m.E <= 0) return Q4_ERR_DIM;
   if (m.src.n_layers < 1 || m.src.n_layers > 2 || m.tgt.n_layers < 1 || m.tgt.n_layers > 2)
@@ -983,8 +995,12 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   sel.rho = rho;
   sel.exact_only = select_exact_only();
   sel.normalized = joint_normalized;
+  sel.mode = mode;
   TagScope tag_sel(TAG_SELECT);
-  Q4_TRY(launch_beam_select(sel, s, use_mma));
+  if (mode != 0)
+    Q4_TRY(launch_tsd_select(sel, s));
+  else
+    Q4_TRY(launch_beam_select(sel, s, use_mma));
   return Q4_OK;
 }
 

@@ -391,7 +391,7 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
 
     // ---- next beam, state rows, back-pointers, pending advances: lane s writes slot s
     const int nw = n_win;
-    const int row0 = b * 2 * W;
+    const int row0 = b * (st.rows_per_utt > 0 ? st.rows_per_utt : 2 * W);
     uint32_t used = 0;
     for (int w = 0; w < W; ++w)
       if (s_row[w] >= 0) used |= 1u << (s_row[w] - row0);
@@ -476,6 +476,377 @@ cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s, bool depend
   return le != cudaSuccess ? le : cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ time-synchronous search
+// One call of the time-synchronous search for one utterance per CTA (the networks and the joint
+// have already run for the hypotheses of the current set A, all at frame t).  Every live slot's
+// blank proposal joins the candidate set of the next frame (global arrays nb_*, at most
+// W (S+1) entries, equal label strings merged by log-addition in insertion order).  In an inner
+// call (mode 1) the W best label proposals (score, parent slot, token) become the next set A at
+// the same frame: fresh state rows, pending network advances, back-pointers, exactly like label
+// extensions of the alignment-length synchronous search.  In the frame-closing call (mode 2) no
+// label is proposed and the W best candidates (score, insertion order) open frame t + 1.
+constexpr int TSD_MAXC = 64;
+__global__ void __launch_bounds__(SEL_NT) k_tsd_select(const __grid_constant__ BeamSelArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int W = a.W, V = a.V;
+  float* cand = reinterpret_cast<float*>(smem_raw);                         // [W * V] label proposals
+  uint64_t* list = reinterpret_cast<uint64_t*>(cand + (size_t)W * V);
+  __shared__ float s_score[MAXW], s_blank[MAXW];
+  __shared__ int s_u[MAXW], s_row[MAXW], s_last[MAXW];
+  __shared__ uint64_t s_hash[MAXW], s_prev[MAXW];
+  __shared__ int list_n;
+  __shared__ int win_idx[MAXW];
+  __shared__ float win_score[MAXW];
+  __shared__ float c_score[TSD_MAXC];
+  __shared__ int c_u[TSD_MAXC], c_last[TSD_MAXC], c_row[TSD_MAXC], c_org[TSD_MAXC], c_n;
+  __shared__ uint64_t c_hash[TSD_MAXC], c_prev[TSD_MAXC];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.x;
+  const int base = b * W;
+  const q4_beam_state& st = a.st;
+  const float NEG = -INFINITY;
+  const int N = a.B * W;
+  const int S = st.tsd_smax;
+  const int CB = W * (S + 1);
+  const int step = a.iter % (S + 1), frame = a.iter / (S + 1);
+  const bool inner = a.mode == 1;
+  const int RW = st.rows_per_utt;
+
+  pdl_wait();
+  if (tid < W) {
+    const int o = base + tid;
+    s_row[tid] = st.row[o];
+    s_score[tid] = st.score[o];
+    s_u[tid] = st.u[o];
+    s_last[tid] = st.last_tok[o];
+    s_hash[tid] = st.hash[o];
+    s_prev[tid] = st.prev_hash[o];
+  }
+  const int cn0 = st.nb_n[b];
+  for (int j = tid; j < cn0; j += SEL_NT) {
+    const size_t o = (size_t)b * CB + j;
+    c_score[j] = st.nb_score[o];
+    c_u[j] = st.nb_u[o];
+    c_last[j] = st.nb_last_tok[o];
+    c_row[j] = st.nb_row[o];
+    c_org[j] = st.nb_origin[o];
+    c_hash[j] = st.nb_hash[o];
+    c_prev[j] = st.nb_prev_hash[o];
+  }
+  if (tid == 0) {
+    list_n = 0;
+    c_n = cn0;
+    if (b == 0) st.pend_n[a.iter & 1] = 0;   // the list consumed by this call is free again
+  }
+  __syncthreads();
+
+  // ---- proposals: one warp per slot at a time
+  for (int w = warp; w < W; w += SEL_NT / 32) {
+    float* cw = cand + (size_t)w * V;
+    const int row = s_row[w];
+    if (row < 0) {
+      for (int k = lane; k < V; k += 32) cw[k] = NEG;
+      if (lane == 0) s_blank[w] = NEG;
+      continue;
+    }
+    const float* x = a.logits + (size_t)(base + w) * V;
+    const float* lt = a.tgt_lp + (size_t)row * V;
+    const float* ls = a.src_lp + (size_t)row * V;
+    const double S_rho = (double)s_score[w] + (double)a.rho;
+    const bool labels = inner && s_u[w] < a.u_max;
+    float lse = 0.0f;
+    if (!a.normalized) {
+      float m = NEG;
+      for (int k = lane; k < V; k += 32) m = fmaxf(m, x[k]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      float sum = 0.0f;
+      for (int k = lane; k < V; k += 32) sum += expf(x[k] - m);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      lse = m + logf(sum);
+    }
+    for (int k = lane; k < V; k += 32) {
+      const float lp = x[k] - lse;
+      float sc = NEG;
+      if (k == 0) {
+        s_blank[w] = (float)((double)s_score[w] + (double)lp);
+      } else if (labels) {
+        const float inc = __fmaf_rn(a.lambda_t, lt[k], __fmaf_rn(-a.lambda_s, ls[k], lp));
+        sc = (float)(S_rho + (double)inc);
+      }
+      cw[k] = sc;
+    }
+  }
+  __syncthreads();
+
+  // ---- blanks join the candidate set, in slot order (warp 0; lanes search, lane 0 updates)
+  if (warp == 0) {
+    for (int w = 0; w < W; ++w) {
+      if (s_row[w] < 0) continue;             // uniform
+      const int n = c_n;
+      const uint64_t h = s_hash[w];
+      int found = -1;
+      for (int j0 = 0; j0 < n; j0 += 32) {
+        const int j = j0 + lane;
+        const unsigned m = __ballot_sync(0xffffffffu, j < n && c_hash[j] == h);
+        if (m) {
+          found = j0 + __ffs(m) - 1;
+          break;
+        }
+      }
+      if (lane == 0) {
+        if (found >= 0) {
+          const double x = (double)c_score[found], y = (double)s_blank[w];
+          c_score[found] = (float)(fmax(x, y) + log1p(exp(-fabs(x - y))));
+        } else if (n < TSD_MAXC && n < CB) {
+          c_score[n] = s_blank[w];
+          c_u[n] = s_u[w];
+          c_last[n] = s_last[w];
+          c_row[n] = s_row[w];
+          c_org[n] = (step << 8) | w;
+          c_hash[n] = h;
+          c_prev[n] = s_prev[w];
+          c_n = n + 1;
+        }
+      }
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+
+  if (inner) {
+    // ---- the W best label proposals: exact threshold search (see k_beam_select)
+    const int cap = 16 * ((V + 31) / 32);
+    uint64_t head = 0;
+    for (int w = warp; w < W; w += SEL_NT / 32) {
+      if (s_row[w] < 0) continue;
+      const float* cw = cand + (size_t)w * V;
+      const uint32_t off = (uint32_t)w * (uint32_t)V;
+      for (int k = lane; k < V; k += 32) {
+        const float x = cw[k];
+        if (x > NEG) head = u64max(head, make_key(x, off + (uint32_t)k));
+      }
+    }
+    uint64_t th = 0;
+    for (int bit = 63; bit >= 32; --bit) {
+      const uint64_t c = th | (1ull << bit);
+      if (__syncthreads_count(head >= c) >= W) th = c;
+    }
+    if (__syncthreads_count(head >= th) > W) {
+      for (int bit = 31; bit >= 0; --bit) {
+        const uint64_t c = th | (1ull << bit);
+        if (__syncthreads_count(head >= c) >= W) th = c;
+      }
+    }
+    if (head != 0ull && head >= th) {
+      for (int w = warp; w < W; w += SEL_NT / 32) {
+        if (s_row[w] < 0) continue;
+        const float* cw = cand + (size_t)w * V;
+        const uint32_t off = (uint32_t)w * (uint32_t)V;
+        for (int k = lane; k < V; k += 32) {
+          const float x = cw[k];
+          if (!(x > NEG)) continue;
+          const uint64_t key = make_key(x, off + (uint32_t)k);
+          if (key >= th) {
+            const int p = atomicAdd(&list_n, 1);
+            if (p < cap) list[p] = key;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    {
+      const int ln = min(list_n, cap);
+      for (int i = tid; i < ln; i += SEL_NT) {
+        const uint64_t mine = list[i];
+        int rank = 0;
+        for (int j = 0; j < ln; ++j) rank += list[j] > mine;
+        if (rank < W) {
+          win_idx[rank] = (int)(~(uint32_t)mine);
+          win_score[rank] = key_score(mine);
+        }
+      }
+    }
+    __syncthreads();
+    pdl_trigger();
+    if (warp == 0) {
+      const int nw = min(min(list_n, cap), W);
+      const int row0 = b * RW;
+      // rows in use: those of the current set and those the candidates refer to
+      uint64_t used = 0;
+      for (int w = 0; w < W; ++w)
+        if (s_row[w] >= 0) used |= 1ull << (s_row[w] - row0);
+      for (int j = 0; j < c_n; ++j) used |= 1ull << (c_row[j] - row0);
+      const uint64_t all = RW >= 64 ? ~0ull : ((1ull << RW) - 1ull);
+      uint64_t free_mask = ~used & all;
+      const int s = lane;
+      // the j-th winner takes the j-th free row
+      int f = -1;
+      {
+        uint64_t m = free_mask;
+        for (int j = 0; j <= s && j < nw; ++j) {
+          f = m ? __ffsll((long long)m) - 1 : -1;
+          m &= m - 1;
+        }
+      }
+      int pbase = 0;
+      if (lane == 0 && nw > 0) pbase = atomicAdd(st.pend_n + ((a.iter + 1) & 1), nw);
+      pbase = __shfl_sync(0xffffffffu, pbase, 0);
+      const size_t poff = (size_t)((a.iter + 1) & 1) * N;
+      if (s < W) {
+        const int o = base + s;
+        const size_t hist = ((size_t)a.iter * a.B + b) * W + s;
+        if (s < nw && f >= 0) {
+          const int idx = win_idx[s];
+          const int w = idx / V, k = idx % V;
+          st.score[o] = win_score[s];
+          st.t[o] = frame;
+          st.u[o] = s_u[w] + 1;
+          st.hash[o] = hash_mix(s_hash[w], (uint32_t)k);
+          st.prev_hash[o] = s_hash[w];
+          st.last_tok[o] = k;
+          st.row[o] = row0 + f;
+          st.adv_src[o] = s_row[w];
+          st.adv_dst[o] = row0 + f;
+          st.adv_tok[o] = k;
+          st.pend_src[poff + pbase + s] = s_row[w];
+          st.pend_dst[poff + pbase + s] = row0 + f;
+          st.pend_tok[poff + pbase + s] = k;
+          st.bp_parent[hist] = w;
+          st.bp_token[hist] = k;
+          st.bp_score[hist] = win_score[s];
+        } else {
+          st.row[o] = -1;
+          st.adv_src[o] = -1;
+          st.adv_dst[o] = -1;
+          st.adv_tok[o] = -1;
+          st.bp_parent[hist] = -1;
+          st.bp_token[hist] = 0;
+          st.bp_score[hist] = 0.0f;
+        }
+      }
+    }
+    // the candidate set goes back to memory
+    for (int j = tid; j < c_n; j += SEL_NT) {
+      const size_t o = (size_t)b * CB + j;
+      st.nb_score[o] = c_score[j];
+      st.nb_u[o] = c_u[j];
+      st.nb_last_tok[o] = c_last[j];
+      st.nb_row[o] = c_row[j];
+      st.nb_origin[o] = c_org[j];
+      st.nb_hash[o] = c_hash[j];
+      st.nb_prev_hash[o] = c_prev[j];
+    }
+    if (tid == 0) st.nb_n[b] = c_n;
+  } else {
+    // ---- frame close: the W best candidates (score descending, then insertion order)
+    pdl_trigger();
+    const int n = c_n;
+    const int nw = min(n, W);
+    if (tid < n) {
+      const float mine = c_score[tid];
+      int rank = 0;
+      for (int j = 0; j < n; ++j) rank += (c_score[j] > mine) || (c_score[j] == mine && j < tid);
+      if (rank < W) {
+        const int o = base + rank;
+        const size_t hist = ((size_t)a.iter * a.B + b) * W + rank;
+        st.score[o] = mine;
+        st.t[o] = frame + 1;
+        st.u[o] = c_u[tid];
+        st.hash[o] = c_hash[tid];
+        st.prev_hash[o] = c_prev[tid];
+        st.last_tok[o] = c_last[tid];
+        st.row[o] = c_row[tid];
+        st.adv_src[o] = -1;
+        st.adv_dst[o] = -1;
+        st.adv_tok[o] = -1;
+        st.bp_parent[hist] = c_org[tid] & 0xFF;
+        st.bp_token[hist] = -1 - (c_org[tid] >> 8);
+        st.bp_score[hist] = mine;
+        if (frame + 1 == a.T) {
+          st.fin_score[base + rank] = mine;
+          st.fin_iter[base + rank] = a.iter + 1;
+          st.fin_slot[base + rank] = rank;
+        }
+      }
+    }
+    if (tid >= nw && tid < W) {
+      const int o = base + tid;
+      const size_t hist = ((size_t)a.iter * a.B + b) * W + tid;
+      st.row[o] = -1;
+      st.adv_src[o] = -1;
+      st.adv_dst[o] = -1;
+      st.adv_tok[o] = -1;
+      st.bp_parent[hist] = -1;
+      st.bp_token[hist] = 0;
+      st.bp_score[hist] = 0.0f;
+    }
+    if (tid == 0) {
+      st.nb_n[b] = 0;
+      if (frame + 1 == a.T) st.fin_n[b] = nw;
+    }
+  }
+}
+
+cudaError_t launch_tsd_select(const BeamSelArgs& a, cudaStream_t s) {
+  const size_t smem = (size_t)a.W * a.V * sizeof(float) + (size_t)16 * ((a.V + 31) / 32) * sizeof(uint64_t);
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_tsd_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  timing_begin(s);
+  cudaError_t le = launch_ex(k_tsd_select, dim3(a.B), dim3(SEL_NT), smem, s, false, 1, a);
+  timing_end(s);
+  ++g_launches;
+  return le != cudaSuccess ? le : cudaGetLastError();
+}
+
+// Trace-back of the time-synchronous search: a frame-closing call points at the call of the same
+// frame whose blank created the entry; an inner call points at its parent slot of the call before.
+__global__ void k_traceback_tsd(q4_beam_state st, int B, int W, int n_iters, int u_max, int32_t* tokens,
+                                int32_t* lens, float* scores) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int S1 = st.tsd_smax + 1;
+  int j = -1, s = -1;
+  float sc = 0.0f;
+  if (st.fin_n[b] > 0) {
+    sc = st.fin_score[b * W];
+    j = st.fin_iter[b * W] - 1;
+    s = st.fin_slot[b * W];
+  } else if (n_iters > 0 && st.row[b * W] >= 0) {
+    sc = st.score[b * W];
+    j = n_iters - 1;
+    s = 0;
+  }
+  int32_t* out = tokens + (size_t)b * u_max;
+  int len = 0;
+  while (j >= 0 && s >= 0) {
+    const size_t h = ((size_t)j * B + b) * W + s;
+    const int k = st.bp_token[h];
+    const int par = st.bp_parent[h];
+    if (j % S1 == S1 - 1) {         // frame close: jump to the set the blank was proposed from
+      j = j - (S1 - 1) + (-1 - k) - 1;
+    } else {
+      if (k > 0 && len < u_max) out[len++] = k;
+      --j;
+    }
+    s = par;
+  }
+  for (int i = 0; i < len / 2; ++i) {
+    const int32_t tmp = out[i];
+    out[i] = out[len - 1 - i];
+    out[len - 1 - i] = tmp;
+  }
+  for (int i = len; i < u_max; ++i) out[i] = 0;
+  lens[b] = len;
+  scores[b] = sc;
+}
+
 __global__ void k_beam_init(q4_beam_state st, int B, int W) {
   const int o = blockIdx.x * blockDim.x + threadIdx.x;
   if (o == 0) st.status[0] = 0;
@@ -488,9 +859,10 @@ __global__ void k_beam_init(q4_beam_state st, int B, int W) {
   st.hash[o] = HASH0;
   st.prev_hash[o] = 0;
   st.last_tok[o] = 0;
-  st.row[o] = root ? b * 2 * W : -1;
+  const int RW = st.rows_per_utt > 0 ? st.rows_per_utt : 2 * W;
+  st.row[o] = root ? b * RW : -1;
   st.adv_src[o] = -1;                      // zero state
-  st.adv_dst[o] = root ? b * 2 * W : -1;
+  st.adv_dst[o] = root ? b * RW : -1;
   st.adv_tok[o] = root ? 0 : -1;           // start symbol
   st.fin_score[o] = -INFINITY;
   st.fin_iter[o] = 0;
@@ -498,7 +870,8 @@ __global__ void k_beam_init(q4_beam_state st, int B, int W) {
   if (s == 0) {
     st.fin_n[b] = 0;
     st.pend_src[b] = -1;               // pending list of iteration 0: every utterance's root,
-    st.pend_dst[b] = b * 2 * W;        // fed the start symbol from the zero state
+    st.pend_dst[b] = b * RW;           // fed the start symbol from the zero state
+    if (st.nb_n) st.nb_n[b] = 0;
     st.pend_tok[b] = 0;
   }
   if (o == 0) {
@@ -577,7 +950,10 @@ __global__ void __launch_bounds__(32 * TB_WARPS) k_traceback(q4_beam_state st, i
 
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s) {
-  k_traceback<<<(B + TB_WARPS - 1) / TB_WARPS, 32 * TB_WARPS, 0, s>>>(st, B, W, n_iters, u_max, tokens, lens, scores);
+  if (st.nb_score)   // the state of a time-synchronous search
+    k_traceback_tsd<<<(B + 63) / 64, 64, 0, s>>>(st, B, W, n_iters, u_max, tokens, lens, scores);
+  else
+    k_traceback<<<(B + TB_WARPS - 1) / TB_WARPS, 32 * TB_WARPS, 0, s>>>(st, B, W, n_iters, u_max, tokens, lens, scores);
   ++g_launches;
   return cudaGetLastError();
 }

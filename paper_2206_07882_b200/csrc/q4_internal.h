@@ -25,10 +25,12 @@ struct BeamSelArgs {
   q4_beam_state st;
   int32_t B, T, W, V, iter, u_max;
   float lambda_t, lambda_s, rho;
+  int32_t mode;             // 0 alignment-length synchronous; 1 / 2 time-synchronous inner call / frame close
   int32_t normalized;       // 1 = `logits` already holds log-probabilities (rows sum to one)
   int32_t exact_only;       // 1 = skip the register-resident fast filter (the exact threshold path alone)
 };
 cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s, bool dependent = false);
+cudaError_t launch_tsd_select(const BeamSelArgs& a, cudaStream_t s);
 cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters, cudaStream_t s);
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s);

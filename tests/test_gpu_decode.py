@@ -290,3 +290,86 @@ def test_config3_full_length_invariants(Bd):
         assert (np.diff(fs[b, :fin_n[b]]) <= 0).all()
         assert sc_h[b] == fs[b, 0] and 0 <= lens_h[b] <= U
         assert (tok_h[b, :lens_h[b]] > 0).all() and (tok_h[b, lens_h[b]:] == 0).all()
+
+
+def run_tsd(Bd, dw, e, S_max, utts=None, tensor_cores=True):
+    dd = Bd.Decoder(dw, tensor_cores=tensor_cores)
+    tokens, lens, scores = dd.decode_time_synchronous(torch.from_numpy(e).cuda(), S_max)
+    torch.cuda.synchronize()
+    assert dd.tensors["status"].item() == 0
+    ref = O.tsd(O.Decoder(dw), e, S_max, utts=utts)
+    return dd, tokens.cpu().numpy(), lens.cpu().numpy(), scores.cpu().numpy(), ref
+
+
+def compare_tsd(dd, tokens, lens, scores, ref, utts, T, S_max, W):
+    IT = T * (S_max + 1)
+    bp_parent = dd.tensors["bp_parent"].cpu().numpy()[:IT]
+    bp_token = dd.tensors["bp_token"].cpu().numpy()[:IT]
+    bp_score = dd.tensors["bp_score"].cpu().numpy()[:IT]
+    same = 0
+    for i, b in enumerate(utts):
+        n = int(ref["len"][i])
+        assert lens[b] == n and (tokens[b, :n] == ref["tokens"][i, :n]).all(), (b, tokens[b], ref["tokens"][i])
+        assert abs(scores[b] - ref["score"][i]) <= 1e-3
+        ok = True
+        for it in range(IT):
+            ns = int(ref["n_slots"][i, it])
+            gp, gt = bp_parent[it, b], bp_token[it, b]
+            if (gp >= 0).sum() != ns or (gp[:ns] != ref["parent"][i, it, :ns]).any() or \
+                    (gt[:ns] != ref["token"][i, it, :ns]).any():
+                ok = False
+                break
+            if ns:
+                assert np.abs(bp_score[it, b, :ns] - ref["tscore"][i, it, :ns]).max() <= 1e-3
+        same += ok
+    return same / len(utts)
+
+
+@pytest.mark.parametrize("S_max,W", [(0, 4), (1, 16), (2, 16), (3, 5)])
+def test_time_synchronous_search_small(Bd, S_max, W):
+    # every set of every call (parents, tokens, provenance of the frame-closing entries) as the oracle's
+    dw = synth.decoder(seed=81, V=64, E=32, Hp=64, D=32, Hs=32, Ht=64, tgt_layers=2, U_max=7, W=W)
+    e = synth.Stream(12).normal("e", (10, 6, 32)).astype(np.float32)
+    dd, tokens, lens, scores, ref = run_tsd(Bd, dw, e, S_max)
+    assert compare_tsd(dd, tokens, lens, scores, ref, list(range(6)), 10, S_max, W) == 1.0
+
+
+def test_time_synchronous_search_tensor_core_path(Bd):
+    # 8 utterances x 16 slots = 128 rows and a 256-wide bottleneck: tensor-core LSTMs and cluster heads
+    dw = synth.decoder(seed=83, V=128, E=32, Hp=128, D=256, Hs=128, Ht=256, tgt_layers=2, U_max=9, W=16)
+    e = synth.Stream(13).normal("e", (8, 8, 256)).astype(np.float32)
+    dd, tokens, lens, scores, ref = run_tsd(Bd, dw, e, 2)
+    assert compare_tsd(dd, tokens, lens, scores, ref, list(range(8)), 8, 2, 16) == 1.0
+    # the alignment-length synchronous search still runs on a decoder that has just done this one
+    t2, l2, s2 = dd.decode(torch.from_numpy(e).cuda())
+    r2 = O.alsd(O.Decoder(dw), e, trace=False)
+    for b in range(8):
+        n = int(r2["len"][b])
+        assert l2[b].item() == n and (t2[b, :n].cpu().numpy() == r2["tokens"][b, :n]).all()
+
+
+def test_config3_time_synchronous_full_size_sampled_utterances(Bd):
+    # the beam workload's sizes (target LM 2x2048, source LM 1024, vocabulary 1024, 16 utterances x 16
+    # slots), 8 frames x 3 calls, label budget 8; the oracle decodes 2 of the 16 utterances
+    dw = synth.decoder(seed=3, U_max=8)
+    T, B = 8, 16
+    e = config3_inputs(Bd, 300, B)[:T].contiguous().cpu().numpy()
+    utts = [2, 13]
+    dd, tokens, lens, scores, ref = run_tsd(Bd, dw, e, 2, utts=utts)
+    assert compare_tsd(dd, tokens, lens, scores, ref, utts, T, 2, 16) == 1.0
+
+
+def test_time_synchronous_mode_checks(Bd):
+    dw = synth.decoder(seed=81, V=64, E=32, Hp=64, D=32, Hs=32, Ht=64, tgt_layers=2, U_max=4, W=4)
+    dd = Bd.Decoder(dw)
+    e = torch.zeros((3, 2, 32), device="cuda")
+    dd.alloc_state(2, 4, 9)                      # layout of the alignment-length synchronous search
+    dd.q4_beam_init()
+    with pytest.raises(RuntimeError):            # no candidate set in this state
+        dd.dr_fusion_beam_step(e, 3, 0, 4, mode=1)
+    dd.alloc_state(2, 4, 9, S_max=2)
+    dd.q4_beam_init()
+    with pytest.raises(RuntimeError):            # call 0 of a frame is not the closing one
+        dd.dr_fusion_beam_step(e, 3, 0, 4, mode=2)
+    with pytest.raises(RuntimeError):            # beyond the last frame
+        dd.dr_fusion_beam_step(e, 3, 9, 4, mode=1)

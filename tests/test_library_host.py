@@ -37,7 +37,7 @@ def test_every_declared_symbol_is_exported(Bd):
 def test_struct_layouts_match_header_sizes(Bd):
     assert C.sizeof(Bd.Act) == 20 and C.sizeof(Bd.Mat) == 32
     assert C.sizeof(Bd.LstmS) == 2 * 32 + 8 + 20 + 4          # two mats, pointer, act, padding
-    assert C.sizeof(Bd.BeamStateS) == 38 * 8
+    assert C.sizeof(Bd.BeamStateS) == 47 * 8   # 38 pointers, two int32, 8 pointers of the candidate set
 
 
 def test_quantizer_constants_equal_oracle(Bd):
