@@ -676,6 +676,9 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   const q4_beam_state& st = *state;
   const int N = B * W;
   int joint_normalized = 0;   // the tensor-core joint kernel leaves log-probabilities, not logits
+  // the first call of a frame of the time-synchronous search follows a frame close, which creates
+  // no label extension: no network has anything to advance, only the joint runs
+  const bool nets = !(mode != 0 && iter > 0 && iter % (state->tsd_smax + 1) == 0);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   uint8_t* zq = ws;
   ws += align_up((size_t)N * D);
@@ -739,10 +742,9 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     const PrepPlan pp = plan_prepared(m);
     const uint8_t* pb = static_cast<const uint8_t*>(m.prepared);
 
-    // one LSTM layer of one network for every pending slot
     // all gathers of the iteration in one launch: embedding rows by pending symbol, previous
     // cell-output codes by parent state row, unpacked to int8 operand rows
-    {
+    if (nets) {
       UnpackJobs uj;
       memset(&uj, 0, sizeof(uj));
       auto add = [&](const void* src, long long stride, const int32_t* idx, const q4_act& act, int k_pad,
@@ -776,7 +778,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     // the three networks are independent until the selection: with two lent streams the
     // prediction/joint chain and the source-LM chain run beside the target-LM chain
     cudaStream_t sp = s, ss = s;
-    const bool forked = st.aux_stream[0] && st.aux_stream[1] && st.aux_event[0] && st.aux_event[1] &&
+    const bool forked = nets && st.aux_stream[0] && st.aux_stream[1] && st.aux_event[0] && st.aux_event[1] &&
                         st.aux_event[2];
     if (forked) {
       sp = reinterpret_cast<cudaStream_t>(st.aux_stream[0]);
@@ -833,10 +835,12 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
 
     const bool fused_head = D == 256 && V <= 2048;   // the fused head kernel: 256-wide bottleneck, one cluster per row tile
     // 1a. prediction network, then the joint network for every live slot (stream sp)
-    Q4_CHECK(lstm_mma(sp, !forked, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
-                      st.pred_c, pred_h8));
-    Q4_CHECK(linear_mma(sp, true, TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
-                        st.pred_p, D, cst.adv_dst, nullptr, n_active));
+    if (nets) {
+      Q4_CHECK(lstm_mma(sp, !forked, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
+                        st.pred_c, pred_h8));
+      Q4_CHECK(linear_mma(sp, true, TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
+                          st.pred_p, D, cst.adv_dst, nullptr, n_active));
+    }
     {
       TagScope tag(TAG_JOINT);
       Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, sp, true));
@@ -862,7 +866,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
                           nullptr));
     }
     // 1b. source LM (stream ss) and target LM (the call's stream)
-    for (int which = 0; which < 2; ++which) {
+    for (int which = 0; which < 2 && nets; ++which) {
       const q4_lm& lm = *lms[which];
       cudaStream_t sl = which == 0 ? ss : s;
       const q4_lstm& L0 = lm.lstm[0];
@@ -920,13 +924,13 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       Q4_TRY(cudaStreamWaitEvent(s, j0, 0));
       Q4_TRY(cudaStreamWaitEvent(s, j1, 0));
     }
-    if (!fused_head) {  // log-softmax of both LMs' new rows in one launch
+    if (!fused_head && nets) {  // log-softmax of both LMs' new rows in one launch
       TagScope tag(TAG_TGT_HEAD);
       Q4_TRY(launch_logsoftmax(st.src_lp, st.src_lp, N, V, V, cst.adv_dst, s, st.tgt_lp, n_active));
     }
   } else {
     // 1. pending advances -------------------------------------------------------------
-    {  // prediction network: embedding row -> LSTM -> projection to D
+    if (nets) {  // prediction network: embedding row -> LSTM -> projection to D
       const q4_lstm& L = m.pred_lstm;
       Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), cst.adv_tok,
                             m.pred_emb_act, st.pred_hq, st.pred_c, cst, N, n_active, s));
@@ -936,7 +940,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       TagScope tag(TAG_PRED_PROJ);
       Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
     }
-    for (int which = 0; which < 2; ++which) {
+    for (int which = 0; which < 2 && nets; ++which) {
       const q4_lm& lm = *lms[which];
       void* hq0 = which == 0 ? st.src_hq : st.tgt_hq[0];
       float* c0 = which == 0 ? st.src_c : st.tgt_c[0];
