@@ -304,8 +304,8 @@ int q4_beam_init(q4_beam_state* state, int32_t B, int32_t W, int32_t n_iters, q4
  * T (S + 1) iterations.  History of a mode-2 call: bp_parent = slot that first proposed the entry,
  * bp_token = -1 - (call number within the frame of that proposal).
  * workspace: q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D}), or, to enable the tensor-core path
- * (needs model->prepared and B*W >= 128), q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D, E_pad, Hp,
- * Hs, Ht}).  A bounded device wait that expires sets state->status to Q4_ERR_TIMEOUT.
+ * (needs model->prepared, LSTM widths that are multiples of 128 and V a multiple of 32),
+ * q4_workspace_bytes(Q4_WS_BEAM, {B, W, V, D, E_pad, Hp, Hs, Ht}).  A bounded device wait that expires sets state->status to Q4_ERR_TIMEOUT.
  */
 int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float* e, int32_t B,
                         int32_t T, int32_t W, int32_t iter, int32_t u_max, float lambda_t,

@@ -700,12 +700,13 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   cst.adv_src = c_src;
   cst.adv_dst = c_dst;
   cst.adv_tok = c_tok;
-  // tensor-core path: prepared int8 weights, enough rows to fill 128-row tiles, and room
-  // for the int8 operand scratch
+  // tensor-core path: prepared int8 weights and room for the int8 operand scratch.  It is taken
+  // for any number of rows: even 16 rows padded to one 128-row tile finish sooner than on the DP4A
+  // kernels (measured 3x on a single utterance), since the time goes to streaming the weights
   const int Hp = m.pred_lstm.w_hh.k_pad, Hs = m.src.lstm[0].w_hh.k_pad, Ht = m.tgt.lstm[0].w_hh.k_pad;
   const int Ep = m.pred_lstm.w_ih.k_pad;
   const int32_t dims8[8] = {B, W, V, D, Ep, Hp, Hs, Ht};
-  const bool use_mma = m.prepared != nullptr && N >= 128 && m.src.n_layers == 1 &&
+  const bool use_mma = m.prepared != nullptr && m.src.n_layers == 1 &&
                        m.src.lstm[0].w_ih.k_pad == Ep && m.tgt.lstm[0].w_ih.k_pad == Ep &&
                        Hp % 128 == 0 && Hs % 128 == 0 && Ht % 128 == 0 && V % 32 == 0 &&
                        workspace_bytes >= q4_workspace_bytes(Q4_WS_BEAM, dims8, 8);
