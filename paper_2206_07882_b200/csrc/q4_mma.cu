@@ -87,56 +87,63 @@ cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int3
   return cudaGetLastError();
 }
 
-// Several gather+unpack jobs in one launch (blockIdx.y selects the job).
+// Several gather+unpack jobs in one launch (blockIdx.y selects the job).  The grid is sized for
+// the SMs, not for the padded row count: each thread strides over the 32-element pieces of the
+// rows that carry work (their number is known on the device only).
 __global__ void __launch_bounds__(256) k_unpack_multi(const UnpackJobs jobs) {
   pdl_trigger();
   pdl_wait();
   const UnpackJob& j = jobs.job[blockIdx.y];
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = j.k_pad >> 5;
-  if (i >= (long long)jobs.n_rows_pad * per_row) return;
-  const int n = (int)(i / per_row), k = (int)(i % per_row) * 32;
-  uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
-  int r = -1;
-  const bool has_work = n < jobs.n_rows && !(jobs.n_active && n >= *jobs.n_active);
-  if (has_work) r = j.idx ? j.idx[n] : n;
-  if (r >= 0) {
-    const uint8_t* p = j.src + (long long)r * j.src_stride;
-    if (j.bits == 4) {
-      const uint4 v = *reinterpret_cast<const uint4*>(p + (k >> 1));
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-      uint32_t o[8];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t lo = 0, hi = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          int a = (w[q] >> (4 * e)) & 0xF, c = (w[q] >> (4 * (e + 4))) & 0xF;
-          if (j.is_signed) {
-            a = (a ^ 8) - 8;
-            c = (c ^ 8) - 8;
-          } else {
-            a -= j.zp;
-            c -= j.zp;
-          }
-          lo |= (uint32_t)(a & 0xFF) << (8 * e);
-          hi |= (uint32_t)(c & 0xFF) << (8 * e);
-        }
-        o[2 * q] = lo;
-        o[2 * q + 1] = hi;
-      }
-      o0 = make_uint4(o[0], o[1], o[2], o[3]);
-      o1 = make_uint4(o[4], o[5], o[6], o[7]);
-    } else {
-      o0 = *reinterpret_cast<const uint4*>(p + k);
-      o1 = *reinterpret_cast<const uint4*>(p + k + 16);
-    }
-  } else if (!has_work) {
-    if (!jobs.zero_tail) return;   // rows without work need not be cleared every time
+  int rows = jobs.n_rows_pad;
+  if (!jobs.zero_tail) {   // rows without work need not be cleared every time
+    rows = jobs.n_rows;
+    if (jobs.n_active) rows = min(rows, *jobs.n_active);
   }
-  uint4* d = reinterpret_cast<uint4*>(j.dst + (long long)n * j.dst_stride + k);
-  d[0] = o0;
-  d[1] = o1;
+  const long long total = (long long)rows * per_row;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int n = (int)(i / per_row), k = (int)(i % per_row) * 32;
+    uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
+    int r = -1;
+    const bool has_work = n < jobs.n_rows && !(jobs.n_active && n >= *jobs.n_active);
+    if (has_work) r = j.idx ? j.idx[n] : n;
+    if (r >= 0) {
+      const uint8_t* p = j.src + (long long)r * j.src_stride;
+      if (j.bits == 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p + (k >> 1));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t lo = 0, hi = 0;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            int a = (w[q] >> (4 * e)) & 0xF, c = (w[q] >> (4 * (e + 4))) & 0xF;
+            if (j.is_signed) {
+              a = (a ^ 8) - 8;
+              c = (c ^ 8) - 8;
+            } else {
+              a -= j.zp;
+              c -= j.zp;
+            }
+            lo |= (uint32_t)(a & 0xFF) << (8 * e);
+            hi |= (uint32_t)(c & 0xFF) << (8 * e);
+          }
+          o[2 * q] = lo;
+          o[2 * q + 1] = hi;
+        }
+        o0 = make_uint4(o[0], o[1], o[2], o[3]);
+        o1 = make_uint4(o[4], o[5], o[6], o[7]);
+      } else {
+        o0 = *reinterpret_cast<const uint4*>(p + k);
+        o1 = *reinterpret_cast<const uint4*>(p + k + 16);
+      }
+    }
+    uint4* d = reinterpret_cast<uint4*>(j.dst + (long long)n * j.dst_stride + k);
+    d[0] = o0;
+    d[1] = o1;
+  }
 }
 
 cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s, bool dependent) {
@@ -144,7 +151,10 @@ cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s, bool dep
   int kmax = 0;
   for (int i = 0; i < jobs.n_jobs; ++i) kmax = jobs.job[i].k_pad > kmax ? jobs.job[i].k_pad : kmax;
   const long long total = (long long)jobs.n_rows_pad * (kmax >> 5);
-  dim3 grid((unsigned)((total + 255) / 256), jobs.n_jobs);
+  long long blocks = (total + 255) / 256;
+  const long long cap = (2 * 148 + jobs.n_jobs - 1) / jobs.n_jobs;   // about two CTAs per SM in all
+  if (blocks > cap) blocks = cap;
+  dim3 grid((unsigned)blocks, jobs.n_jobs);
   timing_begin(s);
   cudaError_t e = launch_ex(k_unpack_multi, grid, dim3(256), 0, s, dependent, 1, jobs);
   timing_end(s);
