@@ -556,8 +556,13 @@ int q4_prepare_model(q4_model* model, void* buffer, size_t bytes, q4_stream stre
     Q4_CHECK(check_mat(&L->w_hh, 0, 0));
     Q4_TRY(launch_prepare_w(L->w_ih, 1, reinterpret_cast<int8_t*>(b + p.lstm[i].xw), L->w_ih.k_pad, 0, s));
     Q4_TRY(launch_prepare_w(L->w_hh, 1, reinterpret_cast<int8_t*>(b + p.lstm[i].hw), L->w_hh.k_pad, 0, s));
-    Q4_TRY(launch_prepare_vec(L->w_ih.scale, L->w_ih.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].sc_ih), s));
-    Q4_TRY(launch_prepare_vec(L->w_hh.scale, L->w_hh.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].sc_hh), s));
+    // de-quantization products of the search (input scale * row scale, hidden scale * row scale)
+    const q4_model& mm = *model;
+    const float xs = i == 0 ? mm.pred_emb_act.scale : i == 1 ? mm.src.emb_act.scale
+                     : i == 2 ? mm.tgt.emb_act.scale : mm.tgt.lstm[0].hid_act.scale;
+    Q4_TRY(launch_prepare_vec(L->w_ih.scale, L->w_ih.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].sc_ih), s, xs));
+    Q4_TRY(launch_prepare_vec(L->w_hh.scale, L->w_hh.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].sc_hh), s,
+                              L->hid_act.scale));
     Q4_TRY(launch_prepare_vec(L->bias, L->w_ih.rows, 1, reinterpret_cast<float*>(b + p.lstm[i].bias), s));
   }
   for (int i = 0; i < 6; ++i) {
@@ -818,6 +823,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       a.h8_ld = H;
       a.status = st.status;
       a.n_active = n_active;
+      a.premultiplied = 1;   // q4_prepare_model stored the products
       a.h_first = dep ? h_first : 0;
       a.trigger_early = trigger_early;
       Q4_TRY(launch_mma_lstm(a, xa, Kx, reinterpret_cast<const int8_t*>(pb + pp.lstm[li].xw), Kx, ha, H,

@@ -82,6 +82,7 @@ struct MmaLstmArgs {
   int32_t h_first;          // 1: only the input operand comes from the previous kernel of the stream, so
                             // the recurrent half of the K loop runs before waiting for that kernel
   int32_t trigger_early;    // 1: let the next kernel of the stream start beside this one
+  int32_t premultiplied;    // 1: sc_ih = x_scale * row scale and sc_hh = hidden scale * row scale already
 };
 struct LmHeadArgs {
   int32_t N, H, V;            // launch rows, LSTM width (K of the bottleneck; 0 = no bottleneck: the
@@ -120,7 +121,8 @@ struct UnpackJobs {
 cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s, bool dependent = false);
 cudaError_t launch_prepare_w(const q4_mat& w, int interleave, int8_t* dst, long long dst_stride,
                              int col0, cudaStream_t s);
-cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s);
+cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s,
+                               float mul = 1.0f);
 cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const int8_t* w8,
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
                             const int32_t* out_idx, const float* w_scale, const float* bias,

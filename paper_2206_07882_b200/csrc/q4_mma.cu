@@ -192,7 +192,7 @@ __global__ void __launch_bounds__(256) k_prepare_w(const uint8_t* src, int bits,
   }
   *reinterpret_cast<uint2*>(dst + (long long)ro * dst_stride + col0 + k) = o;
 }
-__global__ void k_prepare_vec(const float* src, int rows, int interleave, float* dst) {
+__global__ void k_prepare_vec(const float* src, int rows, int interleave, float* dst, float mul) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= rows) return;
   int ro = r;
@@ -200,7 +200,7 @@ __global__ void k_prepare_vec(const float* src, int rows, int interleave, float*
     const int H = rows >> 2;
     ro = 4 * (r % H) + r / H;
   }
-  dst[ro] = src ? src[r] : 0.0f;
+  dst[ro] = src ? __fmul_rn(mul, src[r]) : 0.0f;   // mul = 1 leaves the value as it is
 }
 
 cudaError_t launch_prepare_w(const q4_mat& w, int interleave, int8_t* dst, long long dst_stride,
@@ -214,8 +214,8 @@ cudaError_t launch_prepare_w(const q4_mat& w, int interleave, int8_t* dst, long 
   ++g_launches;
   return cudaGetLastError();
 }
-cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s) {
-  k_prepare_vec<<<(rows + 255) / 256, 256, 0, s>>>(src, rows, interleave, dst);
+cudaError_t launch_prepare_vec(const float* src, int rows, int interleave, float* dst, cudaStream_t s, float mul) {
+  k_prepare_vec<<<(rows + 255) / 256, 256, 0, s>>>(src, rows, interleave, dst, mul);
   ++g_launches;
   return cudaGetLastError();
 }
@@ -758,6 +758,12 @@ cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h
 }
 
 // ------------------------------------------------------------------ fused LSTM step
+// EXTRAS = false drops the second code (yq_out), the fp32 copy (h_f32) and the accumulator dumps
+// from the cell loop: the search needs none of them, and without their branches the four cells
+// of a thread are scheduled as one block.
+// PREMUL = true: sc_ih / sc_hh already hold (input scale * row scale) and (hidden scale * row
+// scale), the products the de-quantization needs (same fp32 multiplication, done once).
+template <bool EXTRAS, bool PREMUL>
 __global__ void __launch_bounds__(32 * (LSTM_EPI_WARPS + 2), 2)
 k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ CUtensorMap tma_xw,
            const __grid_constant__ CUtensorMap tma_ha, const __grid_constant__ CUtensorMap tma_hw,
@@ -893,14 +899,14 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
         const float4 s_ih = __ldg(reinterpret_cast<const float4*>(a.sc_ih) + cell);
         const float4 s_hh = __ldg(reinterpret_cast<const float4*>(a.sc_hh) + cell);
         const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias) + cell);
-        const float pi = __fmaf_rn((float)hh[4 * c + 0], __fmul_rn(sh, s_hh.x), __fmaf_rn((float)ih[4 * c + 0], __fmul_rn(sx, s_ih.x), bb.x));
-        const float pf = __fmaf_rn((float)hh[4 * c + 1], __fmul_rn(sh, s_hh.y), __fmaf_rn((float)ih[4 * c + 1], __fmul_rn(sx, s_ih.y), bb.y));
-        const float pg = __fmaf_rn((float)hh[4 * c + 2], __fmul_rn(sh, s_hh.z), __fmaf_rn((float)ih[4 * c + 2], __fmul_rn(sx, s_ih.z), bb.z));
-        const float po = __fmaf_rn((float)hh[4 * c + 3], __fmul_rn(sh, s_hh.w), __fmaf_rn((float)ih[4 * c + 3], __fmul_rn(sx, s_ih.w), bb.w));
+        const float pi = __fmaf_rn((float)hh[4 * c + 0], (PREMUL ? s_hh.x : __fmul_rn(sh, s_hh.x)), __fmaf_rn((float)ih[4 * c + 0], (PREMUL ? s_ih.x : __fmul_rn(sx, s_ih.x)), bb.x));
+        const float pf = __fmaf_rn((float)hh[4 * c + 1], (PREMUL ? s_hh.y : __fmul_rn(sh, s_hh.y)), __fmaf_rn((float)ih[4 * c + 1], (PREMUL ? s_ih.y : __fmul_rn(sx, s_ih.y)), bb.y));
+        const float pg = __fmaf_rn((float)hh[4 * c + 2], (PREMUL ? s_hh.z : __fmul_rn(sh, s_hh.z)), __fmaf_rn((float)ih[4 * c + 2], (PREMUL ? s_ih.z : __fmul_rn(sx, s_ih.z)), bb.z));
+        const float po = __fmaf_rn((float)hh[4 * c + 3], (PREMUL ? s_hh.w : __fmul_rn(sh, s_hh.w)), __fmaf_rn((float)ih[4 * c + 3], (PREMUL ? s_ih.w : __fmul_rn(sx, s_ih.w)), bb.w));
         cell_fixed(pi, pf, pg, po, cp[c], cn[c], hn[c]);
         qh[c] = quantize1(hn[c], a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
-        qy[c] = quantize1(hn[c], a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
-        if (a.dbg_ih) {
+        qy[c] = EXTRAS ? quantize1(hn[c], a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi) : 0;
+        if (EXTRAS && a.dbg_ih) {
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             a.dbg_ih[(long long)n * a.dbg_ld + g * H + cell] = ih[4 * c + g];
@@ -909,7 +915,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
         }
       }
       *reinterpret_cast<float4*>(a.c_out + (long long)dst * H + cell0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
-      if (a.h_f32) *reinterpret_cast<float4*>(a.h_f32 + (long long)n * H + cell0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+      if (EXTRAS && a.h_f32) *reinterpret_cast<float4*>(a.h_f32 + (long long)n * H + cell0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
       if (a.hq_out) {
         if (a.hid_act.bits == 4)
           *reinterpret_cast<uint16_t*>(a.hq_out + (long long)dst * a.hq_ld + (cell0 >> 1)) =
@@ -921,7 +927,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
       if (a.h8_out)
         *reinterpret_cast<uint32_t*>(a.h8_out + (long long)n * a.h8_ld + cell0) =
             (uint32_t)(qh[0] & 0xFF) | ((uint32_t)(qh[1] & 0xFF) << 8) | ((uint32_t)(qh[2] & 0xFF) << 16) | ((uint32_t)(qh[3] & 0xFF) << 24);
-      if (a.yq_out) {
+      if (EXTRAS && a.yq_out) {
         if (a.out_act.bits == 4)
           *reinterpret_cast<uint16_t*>(a.yq_out + (long long)n * a.yq_ld + (cell0 >> 1)) =
               (uint16_t)((qy[0] & 0xF) | ((qy[1] & 0xF) << 4) | ((qy[2] & 0xF) << 8) | ((qy[3] & 0xF) << 12));
@@ -958,14 +964,26 @@ cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa
   const size_t smem = (size_t)LSTM_STAGES * (BM * BK + LSTM_BN * BK) + 1024;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_mma_lstm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_mma_lstm<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_mma_lstm<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_mma_lstm<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   dim3 grid((4 * a.H + LSTM_BN - 1) / LSTM_BN, rows_pad / BM);
+  const bool extras = a.yq_out || a.h_f32 || a.dbg_ih;
+  if (a.premultiplied && (extras || a.x_scale_vec)) return cudaErrorInvalidValue;
+  const dim3 block(32 * (LSTM_EPI_WARPS + 2));
   timing_begin(s);
-  cudaError_t le = launch_ex(k_mma_lstm, grid, dim3(32 * (LSTM_EPI_WARPS + 2)), smem, s, dependent, 1, txa, txw,
-                             tha, thw, a);
+  cudaError_t le;
+  if (extras)
+    le = launch_ex(k_mma_lstm<true, false>, grid, block, smem, s, dependent, 1, txa, txw, tha, thw, a);
+  else if (a.premultiplied)
+    le = launch_ex(k_mma_lstm<false, true>, grid, block, smem, s, dependent, 1, txa, txw, tha, thw, a);
+  else
+    le = launch_ex(k_mma_lstm<false, false>, grid, block, smem, s, dependent, 1, txa, txw, tha, thw, a);
   timing_end(s);
   ++g_launches;
   return le != cudaSuccess ? le : cudaGetLastError();
