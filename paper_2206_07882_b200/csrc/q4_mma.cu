@@ -853,6 +853,16 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
       dst = a.dst_row ? a.dst_row[n] : n;
       src = a.src_row ? a.src_row[n] : n;
     }
+    // previous cell states of all my cells: requested before the main loop ends (they belong to
+    // rows no kernel of this iteration writes), so that their trip to memory costs the epilogue nothing
+    float4 cprev_all[LSTM_BN / 32];
+#pragma unroll
+    for (int ch = 0; ch < LSTM_BN / 32; ++ch) {
+      const int cell0 = (n0 >> 2) + hf * (LSTM_BN / 8) + ch * 4;
+      cprev_all[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (dst >= 0 && src >= 0 && cell0 < a.H)
+        cprev_all[ch] = *reinterpret_cast<const float4*>(a.c_in + (long long)src * a.H + cell0);
+    }
     const bool ok = mbar_wait(&acc_full, 0);
     tc_fence_after();
     if (h_first) pdl_wait();   // before the first global write of this thread
@@ -866,7 +876,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
     const int hlo = act_lo(a.hid_act), hhi = act_hi(a.hid_act);
     const int ylo = act_lo(a.out_act), yhi = act_hi(a.out_act);
     constexpr int CELLS_PER_HALF = LSTM_BN / 4 / 2;   // 16
-#pragma unroll 1
+#pragma unroll
     for (int ch = 0; ch < CELLS_PER_HALF / 4; ++ch) {
       const int ct = hf * CELLS_PER_HALF + ch * 4;     // first cell of the chunk within the tile
       const int cell0 = (n0 >> 2) + ct;
@@ -888,8 +898,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
           ih[4 * c + 3] = v.w;
         }
       }
-      float4 cprev = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (src >= 0) cprev = *reinterpret_cast<const float4*>(a.c_in + (long long)src * H + cell0);
+      const float4 cprev = cprev_all[ch];
       const float cp[4] = {cprev.x, cprev.y, cprev.z, cprev.w};
       float cn[4], hn[4];
       int qh[4], qy[4];
