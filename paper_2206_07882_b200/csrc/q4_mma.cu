@@ -876,6 +876,14 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
     const int hlo = act_lo(a.hid_act), hhi = act_hi(a.hid_act);
     const int ylo = act_lo(a.out_act), yhi = act_hi(a.out_act);
     constexpr int CELLS_PER_HALF = LSTM_BN / 4 / 2;   // 16
+    // Without the extras the codes of all 16 cells of a thread are kept and stored once: the rows
+    // of a warp's lanes lie far apart, so every store instruction touches 32 lines, and four small
+    // stores per output cost the load/store unit four times as much as one wide one.
+    const int cell_first = (n0 >> 2) + hf * CELLS_PER_HALF;
+    const bool combine = !EXTRAS && cell_first + CELLS_PER_HALF <= H;
+    uint32_t w8[CELLS_PER_HALF / 4];
+#pragma unroll
+    for (int ch = 0; ch < CELLS_PER_HALF / 4; ++ch) w8[ch] = 0;
 #pragma unroll
     for (int ch = 0; ch < CELLS_PER_HALF / 4; ++ch) {
       const int ct = hf * CELLS_PER_HALF + ch * 4;     // first cell of the chunk within the tile
@@ -925,6 +933,9 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
       }
       *reinterpret_cast<float4*>(a.c_out + (long long)dst * H + cell0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
       if (EXTRAS && a.h_f32) *reinterpret_cast<float4*>(a.h_f32 + (long long)n * H + cell0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+      w8[ch] = (uint32_t)(qh[0] & 0xFF) | ((uint32_t)(qh[1] & 0xFF) << 8) | ((uint32_t)(qh[2] & 0xFF) << 16) |
+               ((uint32_t)(qh[3] & 0xFF) << 24);
+      if (combine) continue;
       if (a.hq_out) {
         if (a.hid_act.bits == 4)
           *reinterpret_cast<uint16_t*>(a.hq_out + (long long)dst * a.hq_ld + (cell0 >> 1)) =
@@ -943,6 +954,24 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
         else
           *reinterpret_cast<uint32_t*>(a.yq_out + (long long)n * a.yq_ld + cell0) =
               (uint32_t)(qy[0] & 0xFF) | ((uint32_t)(qy[1] & 0xFF) << 8) | ((uint32_t)(qy[2] & 0xFF) << 16) | ((uint32_t)(qy[3] & 0xFF) << 24);
+      }
+    }
+    if (combine && live) {
+      static_assert(CELLS_PER_HALF == 16, "one uint4 of int8 codes per thread");
+      if (a.h8_out)
+        *reinterpret_cast<uint4*>(a.h8_out + (long long)n * a.h8_ld + cell_first) = make_uint4(w8[0], w8[1], w8[2], w8[3]);
+      if (a.hq_out) {
+        if (a.hid_act.bits == 4) {
+          uint32_t lo = 0, hi = 0;   // 16 nibbles, cell order
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            lo |= ((w8[0] >> (8 * c)) & 0xFu) << (4 * c) | ((w8[1] >> (8 * c)) & 0xFu) << (16 + 4 * c);
+            hi |= ((w8[2] >> (8 * c)) & 0xFu) << (4 * c) | ((w8[3] >> (8 * c)) & 0xFu) << (16 + 4 * c);
+          }
+          *reinterpret_cast<uint2*>(a.hq_out + (long long)dst * a.hq_ld + (cell_first >> 1)) = make_uint2(lo, hi);
+        } else {
+          *reinterpret_cast<uint4*>(a.hq_out + (long long)dst * a.hq_ld + cell_first) = make_uint4(w8[0], w8[1], w8[2], w8[3]);
+        }
       }
     }
   } else {
