@@ -856,12 +856,24 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
     // previous cell states of all my cells: requested before the main loop ends (they belong to
     // rows no kernel of this iteration writes), so that their trip to memory costs the epilogue nothing
     float4 cprev_all[LSTM_BN / 32];
+    // 16 cells = 64 contiguous bytes per row: two 256-bit accesses when the layout allows it
+    const bool wide = (n0 >> 2) + hf * (LSTM_BN / 8) + LSTM_BN / 8 <= a.H && (a.H & 7) == 0 &&
+                      ((reinterpret_cast<uintptr_t>(a.c_in) | reinterpret_cast<uintptr_t>(a.c_out)) & 31) == 0;
 #pragma unroll
-    for (int ch = 0; ch < LSTM_BN / 32; ++ch) {
-      const int cell0 = (n0 >> 2) + hf * (LSTM_BN / 8) + ch * 4;
-      cprev_all[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (dst >= 0 && src >= 0 && cell0 < a.H)
-        cprev_all[ch] = *reinterpret_cast<const float4*>(a.c_in + (long long)src * a.H + cell0);
+    for (int ch = 0; ch < LSTM_BN / 32; ++ch) cprev_all[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (wide) {
+      if (dst >= 0 && src >= 0) {
+        const float* cp0 = a.c_in + (long long)src * a.H + (n0 >> 2) + hf * (LSTM_BN / 8);
+        ld_global_v8(cp0, cprev_all[0], cprev_all[1]);
+        ld_global_v8(cp0 + 8, cprev_all[2], cprev_all[3]);
+      }
+    } else {
+#pragma unroll
+      for (int ch = 0; ch < LSTM_BN / 32; ++ch) {
+        const int cell0 = (n0 >> 2) + hf * (LSTM_BN / 8) + ch * 4;
+        if (dst >= 0 && src >= 0 && cell0 < a.H)
+          cprev_all[ch] = *reinterpret_cast<const float4*>(a.c_in + (long long)src * a.H + cell0);
+      }
     }
     const bool ok = mbar_wait(&acc_full, 0);
     tc_fence_after();
@@ -884,6 +896,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
     uint32_t w8[CELLS_PER_HALF / 4];
 #pragma unroll
     for (int ch = 0; ch < CELLS_PER_HALF / 4; ++ch) w8[ch] = 0;
+    float4 c_even = make_float4(0.f, 0.f, 0.f, 0.f);   // new cell states of the even chunk, stored with the odd one
 #pragma unroll
     for (int ch = 0; ch < CELLS_PER_HALF / 4; ++ch) {
       const int ct = hf * CELLS_PER_HALF + ch * 4;     // first cell of the chunk within the tile
@@ -931,7 +944,14 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
           }
         }
       }
-      *reinterpret_cast<float4*>(a.c_out + (long long)dst * H + cell0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
+      if (wide) {
+        if (ch & 1)
+          st_global_v8(a.c_out + (long long)dst * H + cell0 - 4, c_even, make_float4(cn[0], cn[1], cn[2], cn[3]));
+        else
+          c_even = make_float4(cn[0], cn[1], cn[2], cn[3]);
+      } else {
+        *reinterpret_cast<float4*>(a.c_out + (long long)dst * H + cell0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
+      }
       if (EXTRAS && a.h_f32) *reinterpret_cast<float4*>(a.h_f32 + (long long)n * H + cell0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
       w8[ch] = (uint32_t)(qh[0] & 0xFF) | ((uint32_t)(qh[1] & 0xFF) << 8) | ((uint32_t)(qh[2] & 0xFF) << 16) |
                ((uint32_t)(qh[3] & 0xFF) << 24);
