@@ -374,7 +374,12 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
         for (int i = 0; i < 32; ++i) v[i] = __fmaf_rn((float)r[i], s_sc[c0 + i], s_bi[c0 + i]);
         if (a.epi == EPI_F32) {
           float* o = reinterpret_cast<float*>(a.out) + (long long)m * a.ldo + j0;
-          if (j0 + 32 <= a.J) {
+          if (j0 + 32 <= a.J && (reinterpret_cast<uintptr_t>(o) & 31) == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8)
+              st_global_v8(o + i, make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]),
+                           make_float4(v[i + 4], v[i + 5], v[i + 6], v[i + 7]));
+          } else if (j0 + 32 <= a.J) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(o + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
           } else {
@@ -696,7 +701,12 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
     if (dst >= 0 && ok) {
       float* out = a.lp + (long long)dst * a.V + col0;
       const int left = a.V - col0;
-      if (left >= CPT) {
+      if (left >= CPT && (reinterpret_cast<uintptr_t>(out) & 31) == 0) {
+#pragma unroll
+        for (int i = 0; i < CPT; i += 8)   // rows of a warp's lanes are V floats apart: few, wide stores
+          st_global_v8(out + i, make_float4(v[i] - lse, v[i + 1] - lse, v[i + 2] - lse, v[i + 3] - lse),
+                       make_float4(v[i + 4] - lse, v[i + 5] - lse, v[i + 6] - lse, v[i + 7] - lse));
+      } else if (left >= CPT) {
 #pragma unroll
         for (int i = 0; i < CPT; i += 4)
           *reinterpret_cast<float4*>(out + i) = make_float4(v[i] - lse, v[i + 1] - lse, v[i + 2] - lse, v[i + 3] - lse);
