@@ -472,7 +472,7 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
 // log-probabilities: one global write, no separate log-softmax pass.  With H = 0 there is no
 // bottleneck: the 256-wide operand rows are read from memory (joint network).
 constexpr int HEAD_D = 256;
-constexpr int HEAD_STAGES = 3;
+constexpr int HEAD_STAGES = 4;
 constexpr int HEAD_EPI_WARPS = 16;           // four warps per TMEM lane quarter, NB/4 columns each
 constexpr int HEAD_THREADS = 32 * (HEAD_EPI_WARPS + 2);
 constexpr int HEAD_MAX_BLOCKS = 8;           // portable cluster size: V <= 8 NB
