@@ -500,6 +500,7 @@ __global__ void __launch_bounds__(SEL_NT) k_tsd_select(const __grid_constant__ B
   __shared__ float c_score[TSD_MAXC];
   __shared__ int c_u[TSD_MAXC], c_last[TSD_MAXC], c_row[TSD_MAXC], c_org[TSD_MAXC], c_n;
   __shared__ uint64_t c_hash[TSD_MAXC], c_prev[TSD_MAXC];
+  __shared__ float s_gmax[SEL_NT / 32][16];   // per warp: best label proposal of lanes g and g + 16
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.x;
@@ -512,6 +513,9 @@ __global__ void __launch_bounds__(SEL_NT) k_tsd_select(const __grid_constant__ B
   const int step = a.iter % (S + 1), frame = a.iter / (S + 1);
   const bool inner = a.mode == 1;
   const int RW = st.rows_per_utt;
+  // inner calls with a vocabulary of at most 1024: one warp per slot keeps its proposals in registers
+  // and the W best are found from a lower bound, as in k_beam_select
+  const bool fast = inner && V <= 1024 && W <= SEL_NT / 32 && !a.exact_only;
 
   pdl_wait();
   if (tid < W) {
@@ -539,9 +543,85 @@ __global__ void __launch_bounds__(SEL_NT) k_tsd_select(const __grid_constant__ B
     c_n = cn0;
     if (b == 0) st.pend_n[a.iter & 1] = 0;   // the list consumed by this call is free again
   }
+  if (lane < 16) s_gmax[warp][lane] = NEG;
   __syncthreads();
 
-  // ---- proposals: one warp per slot at a time
+  // ---- proposals
+  float v[32];
+  uint32_t skip = 0xFFFFFFFFu;   // fast path: bit i = element lane + 32 i is not a label proposal
+  if (!inner && a.normalized) {
+    // a frame close proposes blanks only, and the joint kernel has normalised its rows
+    if (tid < W)
+      s_blank[tid] = s_row[tid] >= 0
+                         ? (float)((double)s_score[tid] + (double)a.logits[(size_t)(base + tid) * V])
+                         : NEG;
+  } else if (fast) {
+    if (warp < W) {
+      const int w = warp;
+      float* cw = cand + (size_t)w * V;
+      const int row = s_row[w];
+      if (row < 0) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int k = lane + 32 * i;
+          if (k < V) cw[k] = NEG;
+        }
+        if (lane == 0) s_blank[w] = NEG;
+      } else {
+        const bool labels = s_u[w] < a.u_max;
+        const float* x = a.logits + (size_t)(base + w) * V;
+        const float* lt = a.tgt_lp + (size_t)row * V;
+        const float* ls = a.src_lp + (size_t)row * V;
+        float ltv[32], lsv[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int k = lane + 32 * i;
+          v[i] = k < V ? x[k] : NEG;
+          ltv[i] = (k < V && labels) ? lt[k] : 0.0f;
+          lsv[i] = (k < V && labels) ? ls[k] : 0.0f;
+        }
+        const double S_rho = (double)s_score[w] + (double)a.rho;
+        float lse = 0.0f;
+        if (!a.normalized) {
+          float m = NEG;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) m = fmaxf(m, v[i]);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+          float sum = 0.0f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sum += expf(v[i] - m);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+          lse = m + logf(sum);
+        }
+        skip = 0;
+        float best = NEG;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int k = lane + 32 * i;
+          const float lp = v[i] - lse;
+          float sc = NEG;
+          if (k >= V) {
+            skip |= 1u << i;
+          } else if (k == 0) {
+            s_blank[w] = (float)((double)s_score[w] + (double)lp);
+            skip |= 1u << i;
+          } else if (labels) {
+            const float inc = __fmaf_rn(a.lambda_t, ltv[i], __fmaf_rn(-a.lambda_s, lsv[i], lp));
+            sc = (float)(S_rho + (double)inc);
+            best = fmaxf(best, sc);
+          } else {
+            skip |= 1u << i;
+          }
+          v[i] = sc;
+          if (k < V) cw[k] = sc;
+        }
+        best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, 16));
+        if (lane < 16) s_gmax[w][lane] = best;
+      }
+    }
+  } else
   for (int w = warp; w < W; w += SEL_NT / 32) {
     float* cw = cand + (size_t)w * V;
     const int row = s_row[w];
@@ -614,12 +694,57 @@ __global__ void __launch_bounds__(SEL_NT) k_tsd_select(const __grid_constant__ B
       __syncwarp();
     }
   }
+  // lower bound of the W-th best label proposal: the smallest of the 16 group maxima (k_beam_select)
+  float bound = NEG;
+  if (fast) {
+    float g = NEG;
+    if (lane < 16)
+      for (int w = 0; w < W; ++w) g = fmaxf(g, s_gmax[w][lane]);
+    g = __shfl_sync(0xffffffffu, g, lane & 15);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) g = fminf(g, __shfl_xor_sync(0xffffffffu, g, o));
+    bound = g;
+  }
   __syncthreads();
 
   if (inner) {
-    // ---- the W best label proposals: exact threshold search (see k_beam_select)
     const int cap = 16 * ((V + 31) / 32);
+    bool exact = !fast;
+    if (fast) {
+      if (warp < W && s_row[warp] >= 0) {   // uniform per warp: one list reservation per warp
+        const uint32_t off = (uint32_t)warp * (uint32_t)V;
+        uint32_t hit = 0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (!((skip >> i) & 1u) && v[i] >= bound) hit |= 1u << i;
+        const int mine = __popc(hit);
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        int p0 = 0;
+        if (lane == 31 && total > 0) p0 = atomicAdd(&list_n, total);
+        p0 = __shfl_sync(0xffffffffu, p0, 31) + incl - mine;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {   // static register indices
+          if ((hit >> i) & 1u) {
+            if (p0 < cap) list[p0] = make_key(v[i], off + (uint32_t)(lane + 32 * i));
+            ++p0;
+          }
+        }
+      }
+      __syncthreads();
+      exact = list_n > cap;     // the bound was too loose for the list: take the exact threshold instead
+      __syncthreads();
+      if (exact && tid == 0) list_n = 0;
+      if (exact) __syncthreads();
+    }
+    // ---- otherwise the exact threshold search (see k_beam_select)
     uint64_t head = 0;
+    if (exact) {
     for (int w = warp; w < W; w += SEL_NT / 32) {
       if (s_row[w] < 0) continue;
       const float* cw = cand + (size_t)w * V;
@@ -657,6 +782,7 @@ __global__ void __launch_bounds__(SEL_NT) k_tsd_select(const __grid_constant__ B
       }
     }
     __syncthreads();
+    }   // exact
     {
       const int ln = min(list_n, cap);
       for (int i = tid; i < ln; i += SEL_NT) {
