@@ -421,6 +421,174 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
   if (warp == 5) tmem_dealloc(tmem, GEMM_BN);
 }
 
+// ------------------------------------------------------------------ persistent GEMM, int32 out
+// The encoder input projection is one large GEMM per layer and direction (thousands of tiles)
+// whose int32 result (128 KB per tile) costs more time to write than its MMAs take.  One CTA per
+// SM walks the tiles t = blockIdx.x, blockIdx.x + gridDim.x, ... (column tile fastest, so the
+// CTAs working at the same time share activation rows and all weights in L2), with two
+// accumulators in tensor memory: the epilogue warps drain one while the MMAs of the next tile
+// fill the other, and the operand ring keeps streaming across tile boundaries.
+constexpr int PG_STAGES = 4;
+
+__global__ void __launch_bounds__(192, 1)
+k_mma_gemm_persistent(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b,
+                      const MmaGemmArgs a, const int tiles_m, const int tiles_n) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr int A_BYTES = BM * BK, B_BYTES = GEMM_BN * BK, STAGE = A_BYTES + B_BYTES;
+  __shared__ uint64_t full[PG_STAGES], empty[PG_STAGES], acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_base_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nk = (a.K + BK - 1) / BK;
+  const int n_tiles = tiles_m * tiles_n;
+
+  if (tid == 0) {
+    for (int s = 0; s < PG_STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 4);   // one arrival per epilogue warp
+    }
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 5) tmem_alloc(&tmem_base_s, 2 * GEMM_BN);
+  if (warp == 4 && lane == 0) {
+    prefetch_tmap(&tma_a);
+    prefetch_tmap(&tma_b);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_s;
+  pdl_wait();
+
+  if (warp == 4 && lane == 0) {
+    // ---- TMA producer: the ring position runs on across tiles
+    bool ok = true;
+    int s = 0, g = 0;
+    uint32_t ph = 0;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      const int m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * GEMM_BN;
+      for (int i = 0; i < nk; ++i, ++g) {
+        if (g >= PG_STAGES) ok = mbar_wait(&empty[s], ph ^ 1);
+        if (!ok) break;
+        mbar_expect_tx(&full[s], STAGE);
+        tma_load_2d(smem + s * STAGE, &tma_a, i * BK, m0, &full[s]);
+        tma_load_2d(smem + s * STAGE + A_BYTES, &tma_b, i * BK, n0, &full[s]);
+        if (++s == PG_STAGES) {
+          s = 0;
+          ph ^= 1;
+        }
+      }
+    }
+    pdl_trigger();
+    if (!ok) flag_timeout(a.status);
+  } else if (warp == 5 && lane == 0) {
+    // ---- MMA issuer: tile `it` of this CTA accumulates into buffer it & 1
+    const uint32_t idesc = umma_idesc_i8(BM, GEMM_BN);
+    bool ok = true;
+    int s = 0, it = 0;
+    uint32_t ph = 0;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+      const int buf = it & 1, use = it >> 1;
+      if (use >= 1) {   // the epilogue must have read the previous contents of this buffer
+        ok = mbar_wait(&acc_empty[buf], (use - 1) & 1);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      const uint32_t d = tmem + (uint32_t)(buf * GEMM_BN);
+      for (int i = 0; i < nk; ++i) {
+        ok = mbar_wait(&full[s], ph);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t da = umma_desc_sw128(smem_u32(smem + s * STAGE));
+        const uint64_t db = umma_desc_sw128(smem_u32(smem + s * STAGE + A_BYTES));
+#pragma unroll
+        for (int kk = 0; kk < BK / 32; ++kk) umma_i8(d, da + 2 * kk, db + 2 * kk, idesc, (i | kk) != 0);
+        umma_commit(&empty[s]);
+        if (++s == PG_STAGES) {
+          s = 0;
+          ph ^= 1;
+        }
+      }
+      if (ok) umma_commit(&acc_full[buf]);
+    }
+    pdl_trigger();
+    if (!ok) flag_timeout(a.status);
+  } else if (warp < 4) {
+    // ---- epilogue: warp w drains TMEM lanes [32 w, 32 w + 32) of the finished accumulator
+    bool ok = true;
+    int it = 0;
+    const bool wide = (reinterpret_cast<uintptr_t>(a.out) & 31) == 0 && ((a.ldo * 4) & 31) == 0;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+      const int buf = it & 1, use = it >> 1;
+      const int m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * GEMM_BN;
+      ok = mbar_wait(&acc_full[buf], use & 1);
+      if (!ok) break;
+      tc_fence_after();
+      const int m = m0 + warp * 32 + lane;
+      const uint32_t taddr = tmem + (uint32_t)(buf * GEMM_BN) + ((uint32_t)(warp * 32) << 16);
+      // two register sets: the TMEM load of the next 32 columns is in flight while these are stored
+      auto store32 = [&](const int (&r)[32], int c0) {
+        const int j0 = n0 + c0;
+        if (m >= a.M || j0 >= a.J) return;
+        int32_t* o = reinterpret_cast<int32_t*>(a.out) + (long long)m * a.ldo + j0;
+        if (j0 + 32 <= a.J && wide) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8)
+            st_global_v8_b32(o + i, r[i], r[i + 1], r[i + 2], r[i + 3], r[i + 4], r[i + 5], r[i + 6], r[i + 7]);
+        } else if (j0 + 32 <= a.J) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) *reinterpret_cast<int4*>(o + i) = make_int4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (j0 + i < a.J) o[i] = r[i];
+        }
+      };
+      int r0[32], r1[32];
+      tmem_ld32(taddr, r0);
+#pragma unroll 1
+      for (int c0 = 0; c0 < GEMM_BN; c0 += 64) {
+        tmem_ld_wait();
+        tmem_ld32(taddr + c0 + 32, r1);
+        store32(r0, c0);
+        tmem_ld_wait();
+        if (c0 + 64 < GEMM_BN) {
+          tmem_ld32(taddr + c0 + 64, r0);
+        } else {
+          // the accumulator has been read completely: hand it back before the last stores
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+        store32(r1, c0 + 32);
+      }
+    }
+    pdl_trigger();
+    if (!ok && lane == 0) flag_timeout(a.status);
+  } else {
+    pdl_trigger();   // idle lanes of the producer and issuer warps
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, 2 * GEMM_BN);
+}
+
+static int g_sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
 // x8: int8 activations [M, K] (pitch x_pitch), w8: int8 weights [J, K] (pitch w_pitch).
 cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const int8_t* w8,
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
@@ -447,13 +615,25 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
   a.status = status;
   a.n_active = n_active;
   const size_t smem = (size_t)GEMM_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
+  const size_t smem_p = (size_t)PG_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(k_mma_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_mma_gemm_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_p);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   dim3 grid((J + GEMM_BN - 1) / GEMM_BN, (M + BM - 1) / BM);
+  if (epi == EPI_I32 && !out_idx && !n_active && (long long)grid.x * grid.y > 2 * g_sm_count()) {
+    // more than two tiles per SM: one persistent CTA per SM with overlapped epilogue
+    timing_begin(s);
+    cudaError_t le = launch_ex(k_mma_gemm_persistent, dim3(g_sm_count()), dim3(192), smem_p, s, dependent, 1, ta, tb,
+                               a, (int)grid.y, (int)grid.x);
+    timing_end(s);
+    ++g_launches;
+    return le != cudaSuccess ? le : cudaGetLastError();
+  }
   timing_begin(s);
   cudaError_t le = launch_ex(k_mma_gemm, grid, dim3(192), smem, s, dependent, 1, ta, tb, a);
   timing_end(s);

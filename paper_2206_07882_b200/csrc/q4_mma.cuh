@@ -147,4 +147,11 @@ __device__ __forceinline__ void st_global_v8(float* p, const float4& lo, const f
                : "memory");
 }
 
+__device__ __forceinline__ void st_global_v8_b32(int32_t* p, int a0, int a1, int a2, int a3, int a4, int a5, int a6,
+                                                 int a7) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a0), "r"(a1), "r"(a2),
+               "r"(a3), "r"(a4), "r"(a5), "r"(a6), "r"(a7)
+               : "memory");
+}
+
 }  // namespace q4

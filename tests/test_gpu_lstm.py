@@ -135,7 +135,10 @@ def test_config0_layer_forward(Bd):
                                                    (12, 33, 128, 96, 1, 4, 4, 8), (7, 1, 1280, 160, 2, 4, 4, 4),
                                                    # 64 and 60 sequences x 2 directions of 640 cells: groups of 16
                                                    # sequences per cluster, full and ragged
-                                                   (6, 64, 64, 640, 2, 4, 4, 4), (5, 60, 32, 640, 2, 8, 8, 4)])
+                                                   (6, 64, 64, 640, 2, 4, 4, 4), (5, 60, 32, 640, 2, 8, 8, 4),
+                                                   # 7620 rows x 1280 gate rows: 298 tiles of the input projection with a
+                                                   # ragged last row tile, more than two per SM (the persistent GEMM)
+                                                   (60, 127, 32, 320, 1, 4, 4, 4)])
 def test_layer_shapes_directions_precisions(Bd, T, B, K, H, dirs, xb, hb, ob):
     layer_case(Bd, T, B, K, H, dirs, xb, hb, ob, seed=11)
 
