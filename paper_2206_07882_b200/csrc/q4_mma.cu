@@ -964,6 +964,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
   constexpr int TCOLS = 2 * LSTM_BN;
   __shared__ uint64_t full[LSTM_STAGES], empty[LSTM_STAGES], acc_full;
   __shared__ uint32_t tmem_base_s;
+  __shared__ float4 s_cst[3][LSTM_BN / 4];   // input scales, recurrent scales, bias of this tile's cells (4 gates each)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * LSTM_BN;   // row tiles slowest: tiles with work are dispatched first
   const int nkx = a.acc_pre ? 0 : (a.Kx_pad + BK - 1) / BK;
@@ -1065,6 +1066,15 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
           cprev_all[ch] = *reinterpret_cast<const float4*>(a.c_in + (long long)src * a.H + cell0);
       }
     }
+    // de-quantization constants of the tile's 32 cells: weights only (nothing of an earlier kernel),
+    // fetched while the main loop runs so that the cell loop reads them from shared memory
+    if (tid < 3 * (LSTM_BN / 4)) {
+      const int which = tid / (LSTM_BN / 4), cell = (n0 >> 2) + tid % (LSTM_BN / 4);
+      const float* src = which == 0 ? a.sc_ih : which == 1 ? a.sc_hh : a.bias;
+      s_cst[which][tid % (LSTM_BN / 4)] =
+          cell < a.H ? __ldg(reinterpret_cast<const float4*>(src) + cell) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(32 * LSTM_EPI_WARPS) : "memory");
     const bool ok = mbar_wait(&acc_full, 0);
     tc_fence_after();
     if (h_first) pdl_wait();   // before the first global write of this thread
@@ -1116,9 +1126,7 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const int cell = cell0 + c;
-        const float4 s_ih = __ldg(reinterpret_cast<const float4*>(a.sc_ih) + cell);
-        const float4 s_hh = __ldg(reinterpret_cast<const float4*>(a.sc_hh) + cell);
-        const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias) + cell);
+        const float4 s_ih = s_cst[0][ct + c], s_hh = s_cst[1][ct + c], bb = s_cst[2][ct + c];
         const float pi = __fmaf_rn((float)hh[4 * c + 0], (PREMUL ? s_hh.x : __fmul_rn(sh, s_hh.x)), __fmaf_rn((float)ih[4 * c + 0], (PREMUL ? s_ih.x : __fmul_rn(sx, s_ih.x)), bb.x));
         const float pf = __fmaf_rn((float)hh[4 * c + 1], (PREMUL ? s_hh.y : __fmul_rn(sh, s_hh.y)), __fmaf_rn((float)ih[4 * c + 1], (PREMUL ? s_ih.y : __fmul_rn(sx, s_ih.y)), bb.y));
         const float pg = __fmaf_rn((float)hh[4 * c + 2], (PREMUL ? s_hh.z : __fmul_rn(sh, s_hh.z)), __fmaf_rn((float)ih[4 * c + 2], (PREMUL ? s_ih.z : __fmul_rn(sx, s_ih.z)), bb.z));
