@@ -200,6 +200,18 @@ def test_config3_full_size_sampled_utterances(Bd):
     compare_search(dd, tokens, lens, scores, ref, utts, T, 8, 16, min_same=1.0)
 
 
+def test_full_size_batch_of_64_sampled_utterance(Bd):
+    # 64 utterances x 16 slots = 1024 hypothesis rows at the full layer widths (the batch of the
+    # end-to-end workload): 512 tiles per target-LM layer, several per SM.  The oracle decodes
+    # one utterance (12 frames, label budget 6).
+    dw = synth.decoder(seed=3, U_max=6)
+    T, B = 12, 64
+    e = config3_inputs(Bd, 12, B).contiguous().cpu().numpy()
+    utts = [37]
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e, utts=utts)
+    compare_search(dd, tokens, lens, scores, ref, utts, T, 6, 16, min_same=1.0)
+
+
 def test_tensor_core_and_dp4a_search_paths_agree(Bd):
     # 8 utterances x 16 slots = 128 rows: enough for the tensor-core path; both paths must give
     # identical beams (same integer accumulators, same fp32 operation sequence).
