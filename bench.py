@@ -47,6 +47,9 @@ WORKLOADS = {
     # everything at 4 bits, beam width from --beam (1..16): 16 hypothesis rows at most, so every
     # step streams all weights for a handful of rows
     "fig2_single_utterance": dict(B=1, T=152, U_max=76, l1_bits=4, out_bits=4, enc=True, dec=True, seed=6),
+    # the same utterance with the precision assignment of the end-to-end workload (first encoder layer
+    # and joint output layer at 8 bits, the rest at 4): the "mixed" point of that figure
+    "fig2_single_utterance_mixed": dict(B=1, T=152, U_max=76, l1_bits=8, out_bits=8, enc=True, dec=True, seed=6),
 }
 
 
@@ -494,7 +497,7 @@ def main():
 # profiles/ (k_mma_lstm_prof_end_to_end.md, k_enc_recurrent_prof_encoder.md); to be reset to None
 # when those kernels change.
 NCU_TRAFFIC = {
-    "k_mma_lstm_tgt_l2": {"bytes": 41248256 + 495616, "rows": 1024, "weights": 2 * 8192 * 2048},
+    "k_mma_lstm_tgt_l2": {"bytes": 41250048 + 625664, "rows": 1024, "weights": 2 * 8192 * 2048},
     "k_enc_recurrent": {"bytes": 167275520 + 6195968},
 }
 

@@ -199,6 +199,16 @@ class DeviceMat:
         a = Act(1.0, 1.0, 0, bits, 1)
         return DeviceMat(quantize_pack_int4(x, a, mode=2, per_row_scale=s), s, rows, k, pad32(k), bits)
 
+    @staticmethod
+    def from_float_max(w: np.ndarray, bits: int, device="cuda") -> "DeviceMat":
+        """Symmetric per-row quantization of real-valued weights with the MAX boundary of
+        Section 3.1 taken per output row (boundary = the row's largest magnitude, an all-zero row
+        gets 1): mode 1 with one group per row; the row scales come back from the device."""
+        rows, k = w.shape
+        x = torch.from_numpy(np.ascontiguousarray(w, dtype=np.float32)).to(device)
+        q, s = quantize_pack_int4(x, Act(1.0, 1.0, 0, bits, 1), mode=1, n_groups=rows)
+        return DeviceMat(q, s, rows, k, pad32(k), bits)
+
     def c(self) -> Mat:
         return Mat(self.q.data_ptr(), self.scale.data_ptr(), self.rows, self.k, self.k_pad, self.bits)
 

@@ -75,6 +75,39 @@ def test_weight_mode_per_row_scale(Bd, bits):
     np.testing.assert_array_equal(gpu_codes(m2.q, k, a), q)
 
 
+@pytest.mark.parametrize("bits", [4, 8])
+def test_weight_mode_max_boundary_per_row(Bd, bits):
+    # real-valued weights -> codes with the MAX boundary (Section 3.1) of every output row: the
+    # row's largest magnitude maps to the largest code, an all-zero row gets boundary 1
+    from _parity import pack_codes
+    st = synth.Stream(6)
+    rows, k = 77, 150
+    w = (st.normal("w", (rows, k), 0.0, 0.2) * st.uniform("g", (rows, 1), 0.1, 3.0)).astype(np.float32)
+    w[5, :] = 0
+    m = Bd.DeviceMat.from_float_max(w, bits)
+    scales = m.scale.cpu().numpy()
+    qmax = (1 << (bits - 1)) - 1
+    got = gpu_codes(m.q, k, O.act_symmetric(1.0, bits))
+    for r in range(rows):
+        a = O.act_symmetric(O.absmax(w[r:r + 1]), bits)
+        assert scales[r] == a.scale
+        np.testing.assert_array_equal(got[r], O.quantize(w[r:r + 1], a)[0])
+        if r != 5:
+            assert np.abs(got[r]).max() == qmax          # the boundary itself reaches the last code
+    # de-quantized weights lie within half a step of the originals (Section 3.1)
+    deq = got.astype(np.float64) * scales[:, None]
+    assert (np.abs(deq - w) <= 0.5 * scales[:, None] * (1 + 1e-6)).all()
+    # the matrix serves a quantized linear layer as it stands
+    xa = O.act_symmetric(1.0, 4)
+    xq = O.quantize(st.normal("x", (9, k)).astype(np.float32), xa)
+    lin = Bd.DeviceLinear.__new__(Bd.DeviceLinear)
+    lin.w, lin.bias = m, None
+    out = Bd.q4_linear_forward(pack_codes(xq, xa), to_act(xa), lin).cpu().numpy()
+    want = (xq.astype(np.int64) @ got.astype(np.int64).T).astype(np.float64) * \
+        (np.float64(xa.scale) * scales.astype(np.float64))[None, :]
+    np.testing.assert_allclose(out, want, rtol=1e-6, atol=1e-6)
+
+
 @pytest.mark.parametrize("B,T100,M", [(1, 4, 1), (3, 20, 40), (2, 1000, 40), (2, 7, 5)])
 def test_feature_prologue(Bd, B, T100, M):
     mel = synth.logmel(9, B, T100, M)
