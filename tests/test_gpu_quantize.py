@@ -98,7 +98,7 @@ def test_weight_mode_max_boundary_per_row(Bd, bits):
     deq = got.astype(np.float64) * scales[:, None]
     assert (np.abs(deq - w) <= 0.5 * scales[:, None] * (1 + 1e-6)).all()
     # the matrix serves a quantized linear layer as it stands
-    xa = O.act_symmetric(1.0, 4)
+    xa = O.act_symmetric(1.0, bits)     # the linear entry point takes codes of the weights' width
     xq = O.quantize(st.normal("x", (9, k)).astype(np.float32), xa)
     lin = Bd.DeviceLinear.__new__(Bd.DeviceLinear)
     lin.w, lin.bias = m, None
