@@ -514,12 +514,20 @@ def roofline(job, tag, ms, n, pk):
         tok = job.dec.tensors["bp_token"][:(wl["T"] * (wl["tsd"] + 1) if "tsd" in wl else wl["T"] + wl["U_max"])]
         N = max(1.0, float((tok > 0).sum().item() + wl["B"]) / float(tok.shape[0]))
         out_rows = N
+        # the mean hides two kinds of launches: iterations that extended some slot by a label (their
+        # successor runs the networks on that many rows) and iterations that extended none
+        per_iter = (tok > 0).reshape(tok.shape[0], -1).sum(1)
+        busy = per_iter > 0
+        rows_split = {"launches_with_rows": int(busy.sum().item()) + 1, "launches_without_rows": int((~busy).sum().item()) - 1,
+                      "mean_rows_when_any": float(per_iter[busy].float().mean().item()) if bool(busy.any()) else 0.0}
     else:
         out_rows = None
+        rows_split = None
     int8_peak = 2.0 * pk["bf16_tflops_sustained"]          # dense int8 : bf16 = 2 : 1
     out = {"kernel": name, "launches_timed": n, "avg_ms": ms, "traffic": None}
     if out_rows is not None:
         out["rows_per_launch"] = out_rows
+        out.update(rows_split)
 
     def lstm_work(l, rows, kx):
         # weights as stored (packed codes + row scales + bias), per row: input codes, previous
