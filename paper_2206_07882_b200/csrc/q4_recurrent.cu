@@ -49,6 +49,9 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& a0, uint32_
                : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3)
                : "r"(addr));
 }
+__device__ __forceinline__ void ldmatrix_x2(uint32_t addr, uint32_t& a0, uint32_t& a1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(a0), "=r"(a1) : "r"(addr));
+}
 // c[16 x 8] += A[16 x 32] * B[32 x 8], signed 8-bit operands, int32 accumulate.
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                        uint32_t b0, uint32_t b1) {
@@ -145,17 +148,20 @@ k_enc_recurrent(const EncRecArgs a) {
 #pragma unroll
       for (int r = 0; r < 4; ++r) acc[j][r] = 0;
     if (warp_valid) {
-      const int8_t* hcur = hb + (size_t)cur * BG * pitch + (size_t)g * pitch + 4 * t4;
+      // B fragments by ldmatrix as well: lane i supplies the row address of matrix i/8 = (sequence tile
+      // i/16, k half (i/8)&1); thread (g, t4) receives bytes 4 t4 .. 4 t4 + 3 of sequence row g of each
+      const uint32_t b_addr = hb_addr + (uint32_t)((cur * BG + (lane & 7) + 8 * (lane >> 4)) * pitch + 16 * ((lane >> 3) & 1));
 #pragma unroll 4
       for (int k0 = 0; k0 < H; k0 += 32) {
         uint32_t a0, a1, a2, a3;
         ldmatrix_x4(a_addr + k0, a0, a1, a2, a3);
+        uint32_t b[4];
+        if (NT == 2)
+          ldmatrix_x4(b_addr + k0, b[0], b[1], b[2], b[3]);
+        else
+          ldmatrix_x2(b_addr + k0, b[0], b[1]);
 #pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(hcur + (size_t)(8 * j) * pitch + k0);
-          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(hcur + (size_t)(8 * j) * pitch + k0 + 16);
-          mma_s8(acc[j], a0, a1, a2, a3, b0, b1);
-        }
+        for (int j = 0; j < NT; ++j) mma_s8(acc[j], a0, a1, a2, a3, b[2 * j], b[2 * j + 1]);
       }
     }
     // cell update for my items
