@@ -714,12 +714,12 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
-  pdl_wait();   // everything above overlaps the tail of the previous kernel of the stream
+  cl_barrier();   // every CTA of the cluster is running before anyone stores into a peer's shared memory
+  pdl_wait();   // everything above (this barrier included) overlaps the tail of the previous kernel of the stream
   if (a.n_active && m0 >= *a.n_active) {   // whole row tile without work: the whole cluster leaves
     if (warp == HEAD_EPI_WARPS + 1) tmem_dealloc(tmem, 512);
     return;
   }
-  cl_barrier();   // every CTA of the cluster is running before anyone stores into a peer's shared memory
 
   if (warp == HEAD_EPI_WARPS && lane == 0) {
     // ---- TMA producer: bottleneck operands, then my block of output-layer weights
@@ -906,7 +906,8 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   if (warp == HEAD_EPI_WARPS + 1) tmem_dealloc(tmem, 512);
-  cl_barrier();   // nobody leaves while a peer may still store into its shared memory
+  // no barrier at the exit: every store into a peer's shared memory precedes the exchange barrier above
+  // (release on arrival, acquire on the wait), after which only local memory is touched
 }
 
 cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h_pitch, const int8_t* wb8,
