@@ -138,11 +138,19 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
           for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
           lse = m + logf(sum);
         }
-        // label proposals of this slot that the merge below folds into another slot's blank
-        for (int w1 = 0; w1 < W; ++w1)
-          if (s_row[w1] >= 0 && s_u[w1] == s_u[w] + 1 && s_prev[w1] == s_hash[w] && labels &&
-              (s_last[w1] & 31) == lane)
-            skip |= 1u << (s_last[w1] >> 5);
+        // label proposals of this slot that the merge below folds into another slot's blank: lane w1
+        // tests slot w1 (all W tests at once), the few hits are then handed round the warp
+        {
+          const bool hit = lane < W && labels && s_row[lane] >= 0 && s_u[lane] == s_u[w] + 1 && s_prev[lane] == s_hash[w];
+          const int tok = hit ? s_last[lane] : 0;
+          unsigned hits = __ballot_sync(0xffffffffu, hit);
+          while (hits) {
+            const int src = __ffs(hits) - 1;
+            hits &= hits - 1;
+            const int t = __shfl_sync(0xffffffffu, tok, src);
+            if ((t & 31) == lane) skip |= 1u << (t >> 5);
+          }
+        }
         float best = NEG;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
