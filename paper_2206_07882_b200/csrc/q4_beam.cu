@@ -152,28 +152,37 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
           }
         }
         float best = NEG;
+        const float blank = (float)(S + (double)(v[0] - lse));   // element 0 of lane 0 is the blank proposal
+        if (labels) {   // uniform per warp: a slot at its label budget skips the double-precision adds
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int k = lane + 32 * i;
-          const float lp = v[i] - lse;
-          float sc;
-          if (k >= V) {
-            sc = NEG;
-            skip |= 1u << i;
-          } else if (k == 0) {
-            sc = (float)(S + (double)lp);
-            skip |= 1u << i;          // the blank proposal is read back after merge and finished list
-          } else if (labels) {
-            // label increment in fp32 (magnitude of tens), one double add onto the running score
-            const float inc = __fmaf_rn(a.lambda_t, ltv[i], __fmaf_rn(-a.lambda_s, lsv[i], lp));
-            sc = (float)(S_rho + (double)inc);
-          } else {
-            sc = NEG;
-            skip |= 1u << i;
+          for (int i = 0; i < 32; ++i) {
+            const int k = lane + 32 * i;
+            const float lp = v[i] - lse;
+            float sc;
+            if (k >= V) {
+              sc = NEG;
+              skip |= 1u << i;
+            } else if (k == 0) {
+              sc = blank;
+              skip |= 1u << i;          // the blank proposal is read back after merge and finished list
+            } else {
+              // label increment in fp32 (magnitude of tens), one double add onto the running score
+              const float inc = __fmaf_rn(a.lambda_t, ltv[i], __fmaf_rn(-a.lambda_s, lsv[i], lp));
+              sc = (float)(S_rho + (double)inc);
+            }
+            v[i] = sc;
+            if (k < V) cw[k] = sc;
+            if (!((skip >> i) & 1u)) best = fmaxf(best, sc);
           }
-          v[i] = sc;
-          if (k < V) cw[k] = sc;
-          if (!((skip >> i) & 1u)) best = fmaxf(best, sc);
+        } else {
+          skip = 0xFFFFFFFFu;       // no label proposals: only the blank, read back from shared memory
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int k = lane + 32 * i;
+            const float sc = k == 0 ? blank : NEG;
+            v[i] = sc;
+            if (k < V) cw[k] = sc;
+          }
         }
         best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, 16));
         if (lane < 16) s_gmax[w][lane] = best;
