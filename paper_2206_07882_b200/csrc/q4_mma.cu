@@ -878,7 +878,29 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
     for (int r = 0; r < nblk; ++r)
       if (part_s[r][rt] > 0.0f) ssum += part_s[r][rt] * __expf(part_m[r][rt] - m);
     const float lse = m + logf(ssum);
-    if (dst >= 0 && ok) {
+    // A thread's 32 log-probabilities belong to one row and the rows of a warp's lanes are V floats
+    // apart, so storing them directly touches 32 lines per instruction.  A full 128-column block goes
+    // through shared memory instead (the operand stages are free: both GEMMs are complete) and leaves
+    // as whole rows, one 512-byte row per warp-wide store.
+    const bool staged = NB == 128 && nb * NB + NB <= a.V && (a.V & 3) == 0 &&
+                        (reinterpret_cast<uintptr_t>(a.lp) & 15) == 0;   // uniform per CTA
+    if (staged) {
+      constexpr int TP = NB + 4;   // row pitch in floats: rows 16-byte aligned, 32 rows spread over the banks
+      float* tile = reinterpret_cast<float*>(smem);
+      int* tdst = reinterpret_cast<int*>(smem + (size_t)BM * TP * sizeof(float));
+      float* trow = tile + rt * TP + CPT * cs;
+#pragma unroll
+      for (int i = 0; i < CPT; i += 4)
+        *reinterpret_cast<float4*>(trow + i) = make_float4(v[i] - lse, v[i + 1] - lse, v[i + 2] - lse, v[i + 3] - lse);
+      if (cs == 0) tdst[rt] = ok ? dst : -1;
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * HEAD_EPI_WARPS) : "memory");
+      for (int r = warp; r < BM; r += HEAD_EPI_WARPS) {
+        const int d = tdst[r];
+        if (d >= 0)
+          *reinterpret_cast<float4*>(a.lp + (long long)d * a.V + nb * NB + 4 * lane) =
+              *reinterpret_cast<const float4*>(tile + r * TP + 4 * lane);
+      }
+    } else if (dst >= 0 && ok) {
       float* out = a.lp + (long long)dst * a.V + col0;
       const int left = a.V - col0;
       if (left >= CPT && (reinterpret_cast<uintptr_t>(out) & 31) == 0) {
