@@ -872,11 +872,20 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
       }
     }
     cl_barrier();
+    // all partials are fetched at once (at most HEAD_MAX_BLOCKS of them), then combined in block order
+    float pm[HEAD_MAX_BLOCKS], ps[HEAD_MAX_BLOCKS];
+#pragma unroll
+    for (int r = 0; r < HEAD_MAX_BLOCKS; ++r) {
+      pm[r] = r < nblk ? part_m[r][rt] : -INFINITY;
+      ps[r] = r < nblk ? part_s[r][rt] : 0.0f;
+    }
     float m = -INFINITY;
-    for (int r = 0; r < nblk; ++r) m = fmaxf(m, part_m[r][rt]);
+#pragma unroll
+    for (int r = 0; r < HEAD_MAX_BLOCKS; ++r) m = fmaxf(m, pm[r]);
     float ssum = 0.0f;
-    for (int r = 0; r < nblk; ++r)
-      if (part_s[r][rt] > 0.0f) ssum += part_s[r][rt] * __expf(part_m[r][rt] - m);
+#pragma unroll
+    for (int r = 0; r < HEAD_MAX_BLOCKS; ++r)
+      if (ps[r] > 0.0f) ssum += ps[r] * __expf(pm[r] - m);
     const float lse = m + logf(ssum);
     // A thread's 32 log-probabilities belong to one row and the rows of a warp's lanes are V floats
     // apart, so storing them directly touches 32 lines per instruction.  A full 128-column block goes
@@ -894,12 +903,17 @@ k_mma_lmhead(const __grid_constant__ CUtensorMap tma_h, const __grid_constant__ 
         *reinterpret_cast<float4*>(trow + i) = make_float4(v[i] - lse, v[i + 1] - lse, v[i + 2] - lse, v[i + 3] - lse);
       if (cs == 0) tdst[rt] = ok ? dst : -1;
       asm volatile("bar.sync 1, %0;" ::"n"(32 * HEAD_EPI_WARPS) : "memory");
-      for (int r = warp; r < BM; r += HEAD_EPI_WARPS) {
-        const int d = tdst[r];
-        if (d >= 0)
-          *reinterpret_cast<float4*>(a.lp + (long long)d * a.V + nb * NB + 4 * lane) =
-              *reinterpret_cast<const float4*>(tile + r * TP + 4 * lane);
+      int d[BM / HEAD_EPI_WARPS];
+      float4 t4[BM / HEAD_EPI_WARPS];
+#pragma unroll
+      for (int j = 0; j < BM / HEAD_EPI_WARPS; ++j) {   // this warp's 8 rows: fetch first, then store
+        const int r = warp + j * HEAD_EPI_WARPS;
+        d[j] = tdst[r];
+        t4[j] = *reinterpret_cast<const float4*>(tile + r * TP + 4 * lane);
       }
+#pragma unroll
+      for (int j = 0; j < BM / HEAD_EPI_WARPS; ++j)
+        if (d[j] >= 0) *reinterpret_cast<float4*>(a.lp + (long long)d[j] * a.V + nb * NB + 4 * lane) = t4[j];
     } else if (dst >= 0 && ok) {
       float* out = a.lp + (long long)dst * a.V + col0;
       const int left = a.V - col0;
