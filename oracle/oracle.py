@@ -79,6 +79,7 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.orc_absmax.restype = C.c_float
+        _lib.orc_quant_calls.restype = C.c_int64
     return _lib
 
 
@@ -113,6 +114,24 @@ def quantize(x: np.ndarray, act: Act) -> np.ndarray:
     q = np.empty(x.shape, dtype=np.int16)
     lib().orc_quantize(_p(x), C.c_int64(x.size), C.byref(act), _p(q))
     return q
+
+
+def quantize_frames(x: np.ndarray, act: Act) -> np.ndarray:
+    """Eq. 2 on [..., F], one quantizer call per frame (leading dimensions)."""
+    x = _c(x, np.float32)
+    q = np.empty(x.shape, dtype=np.int16)
+    F = x.shape[-1]
+    lib().orc_quantize_frames(_p(x), C.c_int64(x.size // F), C.c_int64(F), C.byref(act), _p(q))
+    return q
+
+
+def quant_calls_reset() -> None:
+    lib().orc_quant_calls_reset()
+
+
+def quant_calls() -> int:
+    """Activation-quantizer calls made by the oracle since the last reset (Section 3.4)."""
+    return int(lib().orc_quant_calls())
 
 
 def dequantize(q: np.ndarray, act: Act) -> np.ndarray:
@@ -246,10 +265,56 @@ def lstm_step(L: Lstm, xq, x_act: Act, hq_in, c_in, hid_act: Act, x_scale_row=No
     return r
 
 
+def lstm_step_plain(L: Lstm, xq, x_act: Act, hq_in, c_in, hid_act: Act, x_scale_row=None, d: int = 0):
+    """The textbook step in double (libm gates); returns dict(hq, c, h, tie) where tie is the
+    distance of h / s from the nearest rounding boundary in code units."""
+    xq = _c(xq, np.int16)
+    hq_in = _c(hq_in, np.int16)
+    c_in = _c(c_in, np.float32)
+    N, H = hq_in.shape
+    r = dict(hq=np.empty((N, H), np.int16), c=np.empty((N, H), np.float32),
+             h=np.empty((N, H), np.float32), tie=np.empty((N, H), np.float32))
+    xs = None if x_scale_row is None else _c(x_scale_row, np.float32)
+    lib().orc_lstm_step_plain(C.byref(L.c[d]), _p(xq), C.byref(x_act), _p(xs), _p(hq_in), _p(c_in),
+                              C.byref(hid_act), C.c_int32(N), _p(r["hq"]), _p(r["c"]), _p(r["h"]),
+                              _p(r["tie"]))
+    return r
+
+
+def lstm_layer_inner(L: Lstm, x, x_act: Act, hid_act: Act) -> np.ndarray:
+    """Layer under Inner quantizer placement: real-valued x [T,B,K] in, real-valued h out."""
+    x = _c(x, np.float32)
+    T, B, K = x.shape
+    assert K == L.K
+    h = np.empty((T, B, L.n * L.H), dtype=np.float32)
+    lib().orc_lstm_layer_inner(L.c, C.c_int32(L.n), _p(x), C.byref(x_act), C.c_int32(T), C.c_int32(B),
+                               C.byref(hid_act), _p(h))
+    return h
+
+
+def joint_z_plain(e, p, z_act: Act):
+    """tanh(e * p) in double -> fp32 -> codes; returns (zq, tie)."""
+    e = _c(e, np.float32)
+    p = _c(p, np.float32)
+    zq = np.empty(e.shape, np.int16)
+    tie = np.empty(e.shape, np.float32)
+    lib().orc_joint_z_plain(_p(e), _p(p), C.c_int64(e.size), C.byref(z_act), _p(zq), _p(tie))
+    return zq, tie
+
+
+def linear_plain(L: Linear, xq: np.ndarray, act: Act) -> np.ndarray:
+    """W x + b on de-quantized operands, in double."""
+    xq = _c(xq, np.int16)
+    M = xq.shape[0]
+    out = np.empty((M, L.J), dtype=np.float64)
+    lib().orc_linear_plain(C.byref(L.c), _p(xq), C.byref(act), C.c_int32(M), _p(out))
+    return out
+
+
 def lstm_layer(L: Lstm, xq, x_act: Act, hid_act: Act, out_act: Optional[Act] = None,
                x_scale_b=None, want=("h",), n_threads: int = 8):
     """Whole layer over xq [T,B,K]; returns dict with yq and the requested extras
-    among h, hq_hid, c_n, acc_ih, acc_hh, quant_calls."""
+    among h, hq_hid, c_n, acc_ih, acc_hh."""
     xq = _c(xq, np.int16)
     T, B, K = xq.shape
     assert K == L.K
@@ -266,13 +331,11 @@ def lstm_layer(L: Lstm, xq, x_act: Act, hid_act: Act, out_act: Optional[Act] = N
         r["acc_ih"] = np.empty((T, B, dirs, 4 * H), np.int32)
     if "acc_hh" in want:
         r["acc_hh"] = np.empty((T, B, dirs, 4 * H), np.int32)
-    qc = np.zeros(2, dtype=np.int64)
     xs = None if x_scale_b is None else _c(x_scale_b, np.float32)
     lib().orc_lstm_layer(L.c, C.c_int32(dirs), _p(xq), C.byref(x_act), _p(xs), C.c_int32(T),
                          C.c_int32(B), C.byref(hid_act), C.byref(out_act), _p(r["yq"]),
                          _p(r.get("hq_hid")), _p(r.get("h")), _p(r.get("c_n")),
-                         _p(r.get("acc_ih")), _p(r.get("acc_hh")), _p(qc), C.c_int32(n_threads))
-    r["quant_calls"] = qc
+                         _p(r.get("acc_ih")), _p(r.get("acc_hh")), C.c_int32(n_threads))
     return r
 
 
@@ -293,6 +356,20 @@ def log_softmax(logits: np.ndarray) -> np.ndarray:
 
 
 # ------------------------------------------------------------ encoder pass
+def encoder_forward_inner(enc, features: np.ndarray):
+    """The encoder's LSTM stack under Inner quantizer placement (Section 3.4): real-valued
+    tensors travel between cells and every cell quantizes its two inputs on entry.  FIX
+    boundaries only.  Returns the real-valued output of the last layer [T,B,2H]."""
+    x = np.asarray(features, dtype=np.float32)
+    assert not enc.in_max
+    x_act = act_symmetric(enc.in_clip, enc.in_bits)
+    for dirs in enc.layers:
+        hid_act = act_symmetric(dirs[0].hid_alpha, dirs[0].hid_bits)
+        x = lstm_layer_inner(Lstm(dirs), x, x_act, hid_act)
+        x_act = hid_act
+    return x
+
+
 def encoder_forward(enc, features: np.ndarray, n_threads: int = 8, want_layers: bool = False):
     """Features [T,B,F] (fp16/fp32) -> quantize -> L bidirectional layers ->
     projection.  The first layer's input boundary is FIX (enc.in_clip) or, with
@@ -308,14 +385,12 @@ def encoder_forward(enc, features: np.ndarray, n_threads: int = 8, want_layers: 
         x_scale_b = np.empty(B, dtype=np.float32)
         for b in range(B):
             a = act_symmetric(absmax(x[:, b, :]), enc.in_bits)
-            xq[:, b, :] = quantize(x[:, b, :], a)
+            xq[:, b, :] = quantize_frames(x[:, b, :], a)
             x_scale_b[b] = a.scale
     else:
         x_act = act_symmetric(enc.in_clip, enc.in_bits)
-        xq = quantize(x, x_act)
+        xq = quantize_frames(x, x_act)          # the network input: one call per frame
     outs = []
-    calls = np.zeros(2, dtype=np.int64)
-    calls[0] += T            # the network input is quantized once per frame
     for l, dirs in enumerate(enc.layers):
         lw = dirs[0]
         hid_act = act_symmetric(lw.hid_alpha, lw.hid_bits)
@@ -325,11 +400,10 @@ def encoder_forward(enc, features: np.ndarray, n_threads: int = 8, want_layers: 
         L = Lstm(dirs)
         r = lstm_layer(L, xq, x_act, hid_act, out_act, x_scale_b=x_scale_b,
                        want=("h",) if want_layers else (), n_threads=n_threads)
-        calls += r["quant_calls"]
         xq, x_act, x_scale_b = r["yq"], out_act, None
         if want_layers:
             outs.append(r)
-    res = {"yq": xq, "y_act": x_act, "quant_calls": calls, "layers": outs}
+    res = {"yq": xq, "y_act": x_act, "layers": outs}
     if enc.proj is not None:
         P = Linear(enc.proj)
         res["e"] = linear(P, xq.reshape(T * B, -1), x_act).reshape(T, B, -1)

@@ -17,13 +17,24 @@
 //   * the quantizer itself is fp32 by definition (one multiply by a stored
 //     reciprocal, round-half-even, clamp);
 //   * reductions whose order is free (log-softmax) and the hypothesis scores
-//     of Eq. 1 are evaluated in double and rounded to float where stored.
+//     of Eq. 1 are evaluated in double and rounded to float where stored;
+//   * beside the fixed fp32 sequences stands a PLAIN path written from the
+//     definitions alone (orc_lstm_step_plain, orc_joint_z_plain,
+//     orc_linear_plain: the C library's exp and tanh in double, a value rounded
+//     to fp32 only where the method stores or quantizes it).  It is what the
+//     fixed sequences and the kernels are checked against under teacher
+//     forcing: real values within 1e-5, codes equal except within 1e-3 code
+//     units of a rounding boundary of Eq. 2, where they may differ by one.  A
+//     change of the fixed sequences never touches the plain path;
+//   * Section 3.4's quantizer-call counts are counted (g_quant_calls), under
+//     both placements: Outer (orc_lstm_layer) and Inner (orc_lstm_layer_inner).
 //
 // Parity status: every function below is pinned by tests/test_oracle_*.py
 // (hand tables, closed forms, brute force).  What no test can pin, because it
 // needs trained weights and the NIST test sets, is recognition accuracy
 // (Table 1): parity unpinned for WER, which nothing here computes.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -85,9 +96,22 @@ static inline int32_t quantize_one(float x, const OrcAct& a) {
   return std::min(std::max(q, lo), hi);                 // clamp
 }
 
-// Eq. 2 on n values.
+// Number of activation-quantizer calls made so far: one call = the quantizer applied to one
+// tensor handed to it (orc_quantize).  Section 3.4 counts these per time step and layer.
+static std::atomic<int64_t> g_quant_calls{0};
+void orc_quant_calls_reset() { g_quant_calls.store(0); }
+int64_t orc_quant_calls() { return g_quant_calls.load(); }
+
+// Eq. 2 on n values (one quantizer call).
 void orc_quantize(const float* x, int64_t n, const OrcAct* a, int16_t* q) {
+  g_quant_calls.fetch_add(1);
   for (int64_t i = 0; i < n; ++i) q[i] = (int16_t)quantize_one(x[i], *a);
+}
+
+// The network input [T, B, F] quantized frame by frame: one quantizer call per frame and
+// sequence (the "T" of the T + T L calls of Section 3.4).
+void orc_quantize_frames(const float* x, int64_t frames, int64_t F, const OrcAct* a, int16_t* q) {
+  for (int64_t f = 0; f < frames; ++f) orc_quantize(x + f * F, F, a, q + f * F);
 }
 
 // Eq. 3: x_q = s (x_int - z).
@@ -259,6 +283,8 @@ void orc_activations(const float* x, int64_t n, float* ex, float* sg, float* th)
 }
 
 // ---------------------------------------------------------------- LSTM cell
+static inline double sigmoid(double v) { return 1.0 / (1.0 + std::exp(-v)); }  // plain paths only
+
 struct OrcLstm {
   const int8_t* w_ih;    // [4H, K], gate blocks in the order i, f, g, o
   const float* s_wih;    // [4H]
@@ -268,7 +294,22 @@ struct OrcLstm {
   int32_t K, H;
 };
 
-static inline double sigmoid(double v) { return 1.0 / (1.0 + std::exp(-v)); }  // fp reference only
+// De-quantized pre-activations and cell update of ONE row, without the output quantizer.
+static void lstm_row(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act, float s_x,
+                     const int16_t* hq_in, const float* c_in, const OrcAct* hid_act, float* c_out,
+                     float* h_out, int32_t* a_ih, int32_t* a_hh, float* pre) {
+  const int32_t H = L->H, K = L->K, G = 4 * H;
+  orc_int_matmul(L->w_ih, G, K, xq, x_act->zero_point, 1, a_ih);
+  orc_int_matmul(L->w_hh, G, H, hq_in, hid_act->zero_point, 1, a_hh);
+  const float s_h = hid_act->scale;
+  for (int32_t j = 0; j < G; ++j) {
+    // de-quantize: each accumulator times (activation scale * row scale), plus bias
+    float v = std::fmaf((float)a_ih[j], s_x * L->s_wih[j], L->bias ? L->bias[j] : 0.0f);
+    pre[j] = std::fmaf((float)a_hh[j], s_h * L->s_whh[j], v);
+  }
+  for (int32_t u = 0; u < H; ++u)
+    orc_cell(pre[u], pre[H + u], pre[2 * H + u], pre[3 * H + u], c_in[u], c_out + u, h_out + u);
+}
 
 // One time step for N independent rows.  Cell state is kept in floating point
 // and never quantized; the cell output o * tanh(c) lies in [-1,1] and is
@@ -282,24 +323,13 @@ void orc_lstm_step(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act,
                    int32_t* acc_ih_out, int32_t* acc_hh_out, float* gates_out) {
   const int32_t H = L->H, K = L->K, G = 4 * H;
   std::vector<int32_t> a_ih(G), a_hh(G);
-  std::vector<float> pre(G);
+  std::vector<float> pre(G), h(H);
   for (int32_t n = 0; n < N; ++n) {
-    orc_int_matmul(L->w_ih, G, K, xq + (int64_t)n * K, x_act->zero_point, 1, a_ih.data());
-    orc_int_matmul(L->w_hh, G, H, hq_in + (int64_t)n * H, hid_act->zero_point, 1, a_hh.data());
-    const float s_x = x_scale_row ? x_scale_row[n] : x_act->scale;
-    const float s_h = hid_act->scale;
-    for (int32_t j = 0; j < G; ++j) {
-      // de-quantize: each accumulator times (activation scale * row scale), plus bias
-      float v = std::fmaf((float)a_ih[j], s_x * L->s_wih[j], L->bias ? L->bias[j] : 0.0f);
-      pre[j] = std::fmaf((float)a_hh[j], s_h * L->s_whh[j], v);
-    }
-    for (int32_t u = 0; u < H; ++u) {
-      float c, h;
-      orc_cell(pre[u], pre[H + u], pre[2 * H + u], pre[3 * H + u], c_in[(int64_t)n * H + u], &c, &h);
-      c_out[(int64_t)n * H + u] = c;
-      if (h_out) h_out[(int64_t)n * H + u] = h;
-      hq_out[(int64_t)n * H + u] = (int16_t)quantize_one(h, *hid_act);
-    }
+    lstm_row(L, xq + (int64_t)n * K, x_act, x_scale_row ? x_scale_row[n] : x_act->scale,
+             hq_in + (int64_t)n * H, c_in + (int64_t)n * H, hid_act, c_out + (int64_t)n * H, h.data(),
+             a_ih.data(), a_hh.data(), pre.data());
+    orc_quantize(h.data(), H, hid_act, hq_out + (int64_t)n * H);   // the one call at the cell output
+    if (h_out) std::memcpy(h_out + (int64_t)n * H, h.data(), H * sizeof(float));
     if (acc_ih_out) std::memcpy(acc_ih_out + (int64_t)n * G, a_ih.data(), G * sizeof(int32_t));
     if (acc_hh_out) std::memcpy(acc_hh_out + (int64_t)n * G, a_hh.data(), G * sizeof(int32_t));
     if (gates_out)   // diagnostic: the four gate activations by themselves
@@ -308,15 +338,59 @@ void orc_lstm_step(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act,
   }
 }
 
+// ------------------------------------------------ the plain (textbook) LSTM step
+// The same step written from the definitions alone, independent of the fixed fp32 sequences
+// above: de-quantization (Eq. 3), the gates from the C library's exp and tanh, the cell
+// update c = f c' + i g and the output h = o tanh(c), all in double; a value is rounded to
+// fp32 only where the method stores it (the cell state, Section 3.2) or hands it to the
+// quantizer (the cell output, Section 3.4; the quantizer is an fp32 operation by definition).
+// tie_out [N,H] (nullable) receives how far h / s lies from the nearest rounding boundary of
+// Eq. 2, in code units (0 = exactly between two codes, 0.5 = on a code): a code computed with
+// other floating-point arithmetic may differ by one only where this is tiny.
+void orc_lstm_step_plain(const OrcLstm* L, const int16_t* xq, const OrcAct* x_act,
+                         const float* x_scale_row, const int16_t* hq_in, const float* c_in,
+                         const OrcAct* hid_act, int32_t N, int16_t* hq_out, float* c_out,
+                         float* h_out, float* tie_out) {
+  const int32_t H = L->H, K = L->K, G = 4 * H;
+  std::vector<double> pre(G);
+  std::vector<float> h(H);
+  for (int32_t n = 0; n < N; ++n) {
+    const double s_x = x_scale_row ? (double)x_scale_row[n] : (double)x_act->scale;
+    const double s_h = (double)hid_act->scale;
+    for (int32_t j = 0; j < G; ++j) {
+      double v = L->bias ? (double)L->bias[j] : 0.0;
+      for (int32_t k = 0; k < K; ++k)     // W x with W = s_w Wq and x = s_x (xq - z)   (Eq. 3)
+        v += (double)L->s_wih[j] * (double)L->w_ih[(int64_t)j * K + k] *
+             (s_x * (double)((int32_t)xq[(int64_t)n * K + k] - x_act->zero_point));
+      for (int32_t k = 0; k < H; ++k)
+        v += (double)L->s_whh[j] * (double)L->w_hh[(int64_t)j * H + k] *
+             (s_h * (double)((int32_t)hq_in[(int64_t)n * H + k] - hid_act->zero_point));
+      pre[j] = v;
+    }
+    for (int32_t u = 0; u < H; ++u) {
+      const double i = sigmoid(pre[u]), f = sigmoid(pre[H + u]);
+      const double g = std::tanh(pre[2 * H + u]), o = sigmoid(pre[3 * H + u]);
+      const float c = (float)(f * (double)c_in[(int64_t)n * H + u] + i * g);   // stored: fp32
+      const double hd = o * std::tanh((double)c);
+      h[u] = (float)hd;
+      c_out[(int64_t)n * H + u] = c;
+      if (tie_out) {
+        const double t = hd * (double)hid_act->inv_scale;
+        tie_out[(int64_t)n * H + u] = (float)std::fabs((t - std::floor(t)) - 0.5);
+      }
+    }
+    orc_quantize(h.data(), H, hid_act, hq_out + (int64_t)n * H);
+    if (h_out) std::memcpy(h_out + (int64_t)n * H, h.data(), H * sizeof(float));
+  }
+}
+
 // A uni- or bidirectional layer over time-major input xq [T, B, K].
 // Direction 1 runs t = T-1 .. 0 with its own weights; the output at t is the
 // concatenation [fwd(t) | bwd(t)].  yq [T,B,dirs*H] holds the codes handed to
 // the next layer (out_act); when out_act differs from hid_act (a precision
-// change between layers) both codes are made from the same float h.
-// Optional: h_f [T,B,dirs*H]; hq_hid [T,B,dirs*H] (recurrent codes); c_n
-// [dirs,B,H]; acc_ih/acc_hh [T,B,dirs,4H]; quant_calls[2] receives the number
-// of activation-quantizer calls under Outer placement (one per cell output,
-// per time step and direction) and under Inner placement (two per cell).
+// change between layers) both codes are made from the same float h (a second
+// quantizer call).  Optional: h_f [T,B,dirs*H]; hq_hid [T,B,dirs*H] (recurrent
+// codes); c_n [dirs,B,H]; acc_ih/acc_hh [T,B,dirs,4H].
 static void layer_one_sequence(const OrcLstm* L, int32_t dirs, const int16_t* xq,
                                const OrcAct* x_act, const float* x_scale_b, int32_t T, int32_t B,
                                int32_t b, const OrcAct* hid_act, const OrcAct* out_act,
@@ -324,7 +398,7 @@ static void layer_one_sequence(const OrcLstm* L, int32_t dirs, const int16_t* xq
                                int32_t* acc_ih, int32_t* acc_hh) {
   for (int32_t d = 0; d < dirs; ++d) {
     const int32_t H = L[d].H, K = L[d].K, G = 4 * H, OH = dirs * H;
-    std::vector<int16_t> hq(H, 0), hq2(H);
+    std::vector<int16_t> hq(H, 0), hq2(H), yo(H);
     std::vector<float> c(H, 0.0f), c2(H), h(H);
     const bool same = out_act->bits == hid_act->bits && out_act->scale == hid_act->scale;
     for (int32_t s = 0; s < T; ++s) {
@@ -336,9 +410,10 @@ static void layer_one_sequence(const OrcLstm* L, int32_t dirs, const int16_t* xq
                     acc_hh ? acc_hh + (row * dirs + d) * G : nullptr, nullptr);
       hq.swap(hq2);
       c.swap(c2);
+      if (!same) orc_quantize(h.data(), H, out_act, yo.data());
       for (int32_t u = 0; u < H; ++u) {
         const int64_t o = row * OH + (int64_t)d * H + u;
-        yq[o] = same ? hq[u] : (int16_t)quantize_one(h[u], *out_act);
+        yq[o] = same ? hq[u] : yo[u];
         if (hq_hid) hq_hid[o] = hq[u];
         if (h_f) h_f[o] = h[u];
       }
@@ -350,7 +425,7 @@ static void layer_one_sequence(const OrcLstm* L, int32_t dirs, const int16_t* xq
 void orc_lstm_layer(const OrcLstm* L, int32_t dirs, const int16_t* xq, const OrcAct* x_act,
                     const float* x_scale_b, int32_t T, int32_t B, const OrcAct* hid_act,
                     const OrcAct* out_act, int16_t* yq, int16_t* hq_hid, float* h_f, float* c_n,
-                    int32_t* acc_ih, int32_t* acc_hh, int64_t* quant_calls, int32_t n_threads) {
+                    int32_t* acc_ih, int32_t* acc_hh, int32_t n_threads) {
   n_threads = std::max(1, std::min(n_threads, B));
   std::vector<std::thread> pool;
   for (int32_t w = 0; w < n_threads; ++w)
@@ -360,10 +435,35 @@ void orc_lstm_layer(const OrcLstm* L, int32_t dirs, const int16_t* xq, const Orc
                            h_f, c_n, acc_ih, acc_hh);
     });
   for (auto& th : pool) th.join();
-  if (quant_calls) {
-    quant_calls[0] = (int64_t)T * dirs;      // Outer: one call per cell output
-    quant_calls[1] = 2 * (int64_t)T * dirs;  // Inner: x_t and s_{t-1} on entry
-  }
+}
+
+// The same layer under "Inner" placement of the activation quantizers (Section 3.4, the
+// placement the paper rejects): nothing is quantized at a cell's output; instead every cell
+// quantizes both of its inputs on entry, x_t with x_act and s_{t-1} with hid_act: two calls
+// per cell and time step, 2 T L in a network of L cells.  Input x [T,B,K] and output h
+// [T,B,dirs*H] are real-valued.  When x_act is the quantizer the producing layer would have
+// applied at its output, the result equals that of the Outer placement (same codes reach the
+// same integer MACs); only the number of quantizer calls differs.
+void orc_lstm_layer_inner(const OrcLstm* L, int32_t dirs, const float* x, const OrcAct* x_act,
+                          int32_t T, int32_t B, const OrcAct* hid_act, float* h_out) {
+  for (int32_t b = 0; b < B; ++b)
+    for (int32_t d = 0; d < dirs; ++d) {
+      const int32_t H = L[d].H, K = L[d].K, G = 4 * H, OH = dirs * H;
+      std::vector<int16_t> xq(K), hq(H);
+      std::vector<float> c(H, 0.0f), c2(H), h(H, 0.0f), h2(H), pre(G);
+      std::vector<int32_t> a_ih(G), a_hh(G);
+      for (int32_t s = 0; s < T; ++s) {
+        const int32_t t = d == 0 ? s : T - 1 - s;
+        const int64_t row = (int64_t)t * B + b;
+        orc_quantize(x + row * K, K, x_act, xq.data());       // x_t on entry
+        orc_quantize(h.data(), H, hid_act, hq.data());         // s_{t-1} on entry
+        lstm_row(&L[d], xq.data(), x_act, x_act->scale, hq.data(), c.data(), hid_act, c2.data(),
+                 h2.data(), a_ih.data(), a_hh.data(), pre.data());
+        c.swap(c2);
+        h.swap(h2);
+        std::memcpy(h_out + row * OH + (int64_t)d * H, h.data(), H * sizeof(float));
+      }
+    }
 }
 
 // Full-precision counterpart of the same layer: W = s_w * Wq as real numbers,
@@ -427,6 +527,35 @@ void orc_joint(const OrcJoint* Jn, const float* e, const float* p, int32_t N, fl
   orc_linear(&Jn->out, zq.data(), &Jn->z_act, N, logits.data(), acc_out);
   orc_log_softmax(logits.data(), N, V, logp);
   if (zq_out) std::memcpy(zq_out, zq.data(), zq.size() * sizeof(int16_t));
+}
+
+// Plain counterparts for the joint network's real-valued stages (definitions only, double):
+// z = tanh(e p) rounded to fp32 for the quantizer, with the distance of z / s from the nearest
+// rounding boundary (see orc_lstm_step_plain), and a linear layer W x + b with W = s_w Wq,
+// x = s (xq - z) (Eq. 3).
+void orc_joint_z_plain(const float* e, const float* p, int64_t n, const OrcAct* z_act, int16_t* zq,
+                       float* tie_out) {
+  std::vector<float> z(n);
+  for (int64_t i = 0; i < n; ++i) {
+    const double zd = std::tanh((double)e[i] * (double)p[i]);
+    z[i] = (float)zd;
+    if (tie_out) {
+      const double t = zd * (double)z_act->inv_scale;
+      tie_out[i] = (float)std::fabs((t - std::floor(t)) - 0.5);
+    }
+  }
+  orc_quantize(z.data(), n, z_act, zq);
+}
+void orc_linear_plain(const OrcLinear* L, const int16_t* xq, const OrcAct* x_act, int32_t M,
+                      double* out) {
+  for (int32_t m = 0; m < M; ++m)
+    for (int32_t j = 0; j < L->J; ++j) {
+      double v = L->bias ? (double)L->bias[j] : 0.0;
+      for (int32_t k = 0; k < L->K; ++k)
+        v += (double)L->s_w[j] * (double)L->w[(int64_t)j * L->K + k] *
+             ((double)x_act->scale * (double)((int32_t)xq[(int64_t)m * L->K + k] - x_act->zero_point));
+      out[(int64_t)m * L->J + j] = v;
+    }
 }
 
 // ------------------------------------------------ prediction network and LMs

@@ -328,3 +328,51 @@ def test_time_synchronous_pruned_trace_invariants():
             assert (par[it, :n] >= 0).all()
     # the best final is the first slot of the last frame close
     assert abs(r["score"][0] - sc[-1, 0]) == 0.0 and r["len"][0] == u[-1, 0]
+
+
+# ---------------------------------------------------------------- prediction network by parts
+def test_prediction_network_chain_by_parts():
+    # prediction network = embedding row -> symmetric quantizer with the FIX boundary 1.25
+    # (Section 3.2) -> LSTM step -> linear to D fed with the hidden-state codes under the hidden
+    # quantizer; rebuilt here from the separately pinned parts and compared with the forced routine.
+    dw, dec = tiny_decoder(seed=130, V=9)
+    P = dw.pred
+    assert P.emb_alpha == 1.25
+    toks = np.array([[0, 5, 3, 8]], dtype=np.int32)
+    e = synth.Stream(9).normal("e", (4, 8)).astype(np.float32)
+    fi = np.array([[2, 0, 3, 1]], dtype=np.int32)
+    lp, hq_g, c_g, p_g = O.pred_joint_forced(dec, e, fi, toks, want_state=True)
+    ea = O.act_symmetric(P.emb_alpha, 4)
+    ha = O.act_symmetric(P.lstm.hid_alpha, P.lstm.hid_bits)
+    assert ea.is_signed == 1 and ea.zero_point == 0 and abs(ea.scale - 1.25 / 7) < 1e-7
+    hq, c = np.zeros((1, 8), np.int16), np.zeros((1, 8), np.float32)
+    L, proj = O.Lstm([P.lstm]), O.Linear(P.proj)
+    for s in range(4):
+        xq = O.quantize(P.emb[toks[0, s]][None, :], ea)
+        r = O.lstm_step(L, xq, ea, hq, c, ha)
+        hq, c = r["hq"], r["c"]
+        p = O.linear(proj, hq, ha)                       # hidden codes with the HIDDEN quantizer's scale
+        np.testing.assert_array_equal(hq_g[0, s], hq[0])
+        np.testing.assert_array_equal(c_g[0, s], c[0])
+        np.testing.assert_array_equal(p_g[0, s], p[0])
+        np.testing.assert_array_equal(lp[0, s], O.joint(dec, e[fi[0, s]][None, :], p)[0])
+    # the two quantizers differ, so feeding the projection with the wrong one would show
+    assert not np.array_equal(O.linear(proj, hq, ea), p)
+
+
+def test_joint_and_linear_fixed_sequences_against_plain_definitions():
+    # tanh(e p) by the fixed fp32 sequence vs libm in double: codes equal away from rounding
+    # boundaries; the fp32 linear layer vs W x + b in double
+    dw, dec = tiny_decoder(seed=140, V=11)
+    st = synth.Stream(12)
+    e = st.normal("e", (400, 8)).astype(np.float32)
+    p = (st.normal("p", (400, 8)) * 1.5).astype(np.float32)
+    a = O.act_symmetric(1.0, 4)
+    _, zq, _ = O.joint(dec, e, p, want_zq=True)
+    zq_p, tie = O.joint_z_plain(e, p, a)
+    d = zq.astype(np.int32) - zq_p
+    assert np.abs(d).max() <= 1 and not ((d != 0) & (tie >= 1e-3)).any()
+    out = O.Linear(dw.joint.out)
+    got = O.linear(out, zq, a)
+    want = O.linear_plain(out, zq, a)
+    np.testing.assert_allclose(got, want, rtol=1e-6, atol=1e-6)

@@ -174,15 +174,28 @@ def test_int4_tracks_fp32_and_int8_tracks_closer():
 
 def test_outer_vs_inner_quantizer_calls():
     # Section 3.4: Inner 2*T*L, Outer T + T*L, ratio (L+1)/(2L); 45 % fewer in the encoder.
+    # Both numbers are COUNTED: every call of the oracle's activation quantizer increments a
+    # counter, and the two placements are two code paths that must give the same network output.
     g = gold()
-    enc = synth.encoder(seed=1, T=5, B=2, F=16, H=8, L=6, D=8)
-    r = O.encoder_forward(enc["enc"], enc["features"])
-    outer, inner = int(r["quant_calls"][0]), int(r["quant_calls"][1])
-    T, Lc = 5, int(g["outer_inner_L"])
+    T, Lc = 5, int(g["outer_inner_L"])           # L = 12 cells: 6 layers x 2 directions
+    enc = synth.encoder(seed=1, T=T, B=1, F=16, H=8, L=6, D=8, with_proj=False)
+    O.quant_calls_reset()
+    r = O.encoder_forward(enc["enc"], enc["features"], want_layers=True)
+    outer = O.quant_calls()
+    O.quant_calls_reset()
+    h_inner = O.encoder_forward_inner(enc["enc"], enc["features"])
+    inner = O.quant_calls()
     assert inner == 2 * T * Lc and outer == T + T * Lc
     assert abs(outer / inner - g["outer_inner_ratio"]) < 1e-9
     assert round(100 * (1 - outer / inner)) in (45, 46)
     assert abs(100 * (1 - outer / inner) - g["outer_inner_saving_percent"]) < 1.0
+    # the placement changes the number of calls, not the result
+    np.testing.assert_array_equal(h_inner, r["layers"][-1]["h"])
+    # a batch of B sequences makes B times the calls (the count is per sequence)
+    enc3 = synth.encoder(seed=1, T=T, B=3, F=16, H=8, L=6, D=8, with_proj=False)
+    O.quant_calls_reset()
+    O.encoder_forward(enc3["enc"], enc3["features"])
+    assert O.quant_calls() == 3 * (T + T * Lc)
 
 
 def test_encoder_layers_chain_and_projection():
@@ -283,3 +296,77 @@ def test_fp32_activation_functions_against_libm():
     _, s2, t2 = O.activations(-g)
     np.testing.assert_array_equal(t1, -t2)
     assert np.max(np.abs(s1 + s2 - 1)) < 2e-7
+
+
+# ------------------------------------------------------------------ plain (textbook) step
+def _forced_fixed_vs_plain(layers, xq, x_act, hid, eps=1e-3):
+    """Walks the fixed-sequence step along time (both directions) and, on the very same inputs
+    (teacher forcing), evaluates the plain step: libm gates in double.  Returns counts."""
+    T, B, K = xq.shape
+    L = O.Lstm(layers)
+    H = L.H
+    n = near = moved_at_tie = outside = 0
+    for d in range(L.n):
+        hq = np.zeros((B, H), np.int16)
+        c = np.zeros((B, H), np.float32)
+        for s in range(T):
+            t = s if d == 0 else T - 1 - s
+            f = O.lstm_step(L, xq[t], x_act, hq, c, hid, d=d)
+            p = O.lstm_step_plain(L, xq[t], x_act, hq, c, hid, d=d)
+            np.testing.assert_allclose(f["c"], p["c"], rtol=1e-5, atol=1e-6)
+            np.testing.assert_allclose(f["h"], p["h"], rtol=1e-5, atol=1e-6)
+            tie = p["tie"] < eps
+            diff = f["hq"].astype(np.int32) - p["hq"].astype(np.int32)
+            assert np.abs(diff).max() <= 1
+            n += diff.size
+            near += int(tie.sum())
+            moved_at_tie += int(((diff != 0) & tie).sum())
+            outside += int(((diff != 0) & ~tie).sum())
+            hq, c = f["hq"], f["c"]
+    return n, near, moved_at_tie, outside
+
+
+def test_fixed_sequence_step_against_plain_step_config0():
+    # config 0: one layer, K=64, H=128, B=4, T=50, clip 3.0
+    w = synth.single_layer(seed=0)
+    x_act, hid = O.act_symmetric(w["x_clip"], 4), O.act_symmetric(1.0, 4)
+    n, near, moved, outside = _forced_fixed_vs_plain(w["layers"], O.quantize(w["x"], x_act), x_act, hid)
+    print(f"config 0: {n} codes, {near} within 1e-3 of a rounding boundary, {moved} of those differ by one, "
+          f"{outside} differ elsewhere")
+    assert outside == 0
+    assert near < 0.01 * n
+
+
+def test_fixed_sequence_step_against_plain_step_encoder_layer():
+    # one bidirectional 640-cell layer with the encoder's inner-layer shape (K = 1280), 4 and 8 bit
+    for bits in (4, 8):
+        st = synth.Stream(41 + bits)
+        layers = [synth._lstm(st, f"d{d}", 1280, 640, bits, 0.1, 0.95, bits) for d in range(2)]
+        x_act, hid = O.act_symmetric(0.97, bits), O.act_symmetric(0.95, bits)
+        lo, hi = x_act.lo() + 1, x_act.hi()
+        xq = st.integers("xq", (6, 2, 1280), lo, hi).astype(np.int16)
+        n, near, moved, outside = _forced_fixed_vs_plain(layers, xq, x_act, hid)
+        print(f"{bits} bit: {n} codes, {near} near a boundary, {moved} of those differ, {outside} elsewhere")
+        assert outside == 0
+
+
+def test_plain_step_is_the_library_cell():
+    # the plain step itself against torch's LSTMCell in float64 (gate order, transposes, Eq. 3)
+    st = synth.Stream(5)
+    K, H, N = 24, 16, 5
+    lw = synth._lstm(st, "cell", K, H, 4, bias_std=0.3)
+    rng = np.random.default_rng(1)
+    x_act, hid = O.act_asymmetric(-2.5, 3.5, 4), O.act_symmetric(1.0, 4)
+    xq = rng.integers(0, 16, (N, K)).astype(np.int16)
+    hq = rng.integers(-7, 8, (N, H)).astype(np.int16)
+    c = rng.normal(0, 1, (N, H)).astype(np.float32)
+    p = O.lstm_step_plain(O.Lstm([lw]), xq, x_act, hq, c, hid)
+    with torch.no_grad():
+        h1, c1 = torch_cell(lw)(torch.from_numpy(O.dequantize(xq, x_act)).double(),
+                                (torch.from_numpy(O.dequantize(hq, hid)).double(), torch.from_numpy(c).double()))
+    # de-quantized operands are fp32 products s * q here and exact reals inside the plain step
+    np.testing.assert_allclose(p["c"], c1.numpy(), rtol=2e-6, atol=2e-6)
+    np.testing.assert_allclose(p["h"], h1.numpy(), rtol=2e-6, atol=2e-6)
+    np.testing.assert_array_equal(p["hq"], O.quantize(p["h"], hid))
+    t = p["h"].astype(np.float64) * hid.inv_scale
+    np.testing.assert_allclose(p["tie"], np.abs(t - np.floor(t) - 0.5), atol=1e-5)
