@@ -156,7 +156,8 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
  *   Limit: N * D <= 65536 (D = w_pred->rows), about 320 KB of device memory that every GPU
  *   loading the library keeps until the process exits; larger problems get Q4_ERR_WORKSPACE.
  *   The first call on each device looks up the array's device address (with that device
- *   current); make that first call before starting any stream capture.
+ *   current); make that first call before starting any stream capture.  The address is
+ *   kept for the life of the process: after a cudaDeviceReset reload the library.
  *   All calls on a device share the one array: calls that overlap on the GPU (different
  *   streams) race with each other; calls on one stream are ordered and safe.  Nothing in the
  *   array needs clearing, each call overwrites what it reads.

@@ -7,6 +7,8 @@
 // thread of the process is capturing a stream (an allocation would invalidate that capture).
 // For them the scratch of the joint network lives in a fixed-size array in device memory that
 // is part of the library image.
+#include <mutex>
+
 #include "q4_internal.h"
 
 using namespace q4;
@@ -21,19 +23,21 @@ static __device__ __align__(256) unsigned char g_joint_scratch[Q4_JOINT_STATIC_B
 namespace {
 constexpr int kMaxDevices = 64;
 void* g_scratch_ptr[kMaxDevices];   // device address of g_joint_scratch, per device
-bool g_scratch_ready[kMaxDevices];
+std::once_flag g_scratch_once[kMaxDevices];
 
 // The array's name is only a host-side handle; the device address has to be asked for, once
-// per device, with that device current.
+// per device, with that device current.  Host threads that make their first call at the same
+// time are serialised by the once-flag, and a thread that finds the flag set also sees the
+// stored address.  The address stays valid until the device is reset (cudaDeviceReset): after
+// a reset the library must be reloaded before this entry point is used again.
 int scratch_for_current_device(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return Q4_ERR_CUDA;
-  if (!g_scratch_ready[dev]) {
+  std::call_once(g_scratch_once[dev], [dev]() {
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_joint_scratch) != cudaSuccess || p == nullptr) return Q4_ERR_CUDA;
-    g_scratch_ptr[dev] = p;
-    g_scratch_ready[dev] = true;
-  }
+    if (cudaGetSymbolAddress(&p, g_joint_scratch) == cudaSuccess) g_scratch_ptr[dev] = p;
+  });
+  if (g_scratch_ptr[dev] == nullptr) return Q4_ERR_CUDA;
   *out = g_scratch_ptr[dev];
   return Q4_OK;
 }

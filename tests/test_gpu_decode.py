@@ -385,3 +385,105 @@ def test_time_synchronous_mode_checks(Bd):
         dd.dr_fusion_beam_step(e, 3, 0, 4, mode=2)
     with pytest.raises(RuntimeError):            # beyond the last frame
         dd.dr_fusion_beam_step(e, 3, 9, 4, mode=1)
+
+
+# ------------------------------------------------------------------ gaps closed after review
+def beam_strings(dd, n_iters, B):
+    """Label string of every slot of the beam after n_iters iterations, from the history."""
+    par = dd.tensors["bp_parent"].cpu().numpy()[:n_iters]
+    tok = dd.tensors["bp_token"].cpu().numpy()[:n_iters]
+    out = []
+    for b in range(B):
+        strings = [()]
+        for it in range(n_iters):
+            n = int((par[it, b] >= 0).sum())
+            strings = [strings[p] + ((int(k),) if k > 0 else ()) for p, k in zip(par[it, b, :n], tok[it, b, :n])]
+        out.append(strings)
+    return out
+
+
+@pytest.mark.parametrize("V", [1024, 992])
+def test_lm_logprobs_elementwise_through_the_search(Bd, V):
+    # The LM rows the search caches (LSTM layers -> bottleneck -> re-quantize -> output -> log-softmax,
+    # the fused head kernel) against the oracle's forced LM on each live hypothesis' label string,
+    # element by element; also the joint's projected prediction vectors.  9 utterances x 16 slots.
+    dw = synth.decoder(seed=91, V=V, E=32, Hp=128, D=256, Hs=128, Ht=256, tgt_layers=2, U_max=6, W=16)
+    B, T, n_it = 9, 8, 7
+    e = synth.Stream(14).normal("e", (T, B, 256)).astype(np.float32)
+    dd = Bd.Decoder(dw)
+    dd.alloc_state(B, 16, T + 6)
+    dd.q4_beam_init()
+    e_dev = torch.from_numpy(e).cuda()
+    for it in range(n_it):
+        dd.dr_fusion_beam_step(e_dev, T, it, 6)
+    torch.cuda.synchronize()
+    strings = beam_strings(dd, n_it, B)
+    dec = O.Decoder(dw)
+    # a slot without a pending advance stands on a state row whose networks have been run
+    rows = dd.tensors["row"].cpu().numpy().reshape(B, 16)
+    adv_dst = dd.tensors["adv_dst"].cpu().numpy().reshape(B, 16)
+    tgt_lp = dd.tensors["tgt_lp"].cpu().numpy()
+    src_lp = dd.tensors["src_lp"].cpu().numpy()
+    pred_p = dd.tensors["pred_p"].cpu().numpy()
+    n_rows = worst = 0
+    for b in range(B):
+        for s, y in enumerate(strings[b]):
+            r = rows[b, s]
+            if r < 0 or adv_dst[b, s] >= 0:
+                continue
+            toks = np.array([[0] + list(y)], dtype=np.int32)
+            for which, lp in (("tgt", tgt_lp), ("src", src_lp)):
+                want = O.lm_forced(dec, which, toks)[0, -1]
+                err = np.abs(lp[r] - want).max()
+                worst = max(worst, err)
+                assert err <= LP_ATOL, (b, s, which, err)
+            fi = np.zeros((1, toks.shape[1]), np.int32)
+            _, _, _, p_w = O.pred_joint_forced(dec, e[:, b], fi, toks, want_state=True)
+            np.testing.assert_array_equal(pred_p[r], p_w[0, -1])
+            n_rows += 1
+    print(f"V={V}: {n_rows} cached LM rows compared element-wise, worst |d log P| = {worst:.2e}")
+    assert n_rows >= 100
+
+
+@pytest.mark.parametrize("W", [1, 16])
+def test_single_utterance_full_widths(Bd, W):
+    # ONE utterance at the full layer widths (the regime of the paper's run-time figure, Section 4.1):
+    # at most 16 hypothesis rows in one padded row tile, all three chains on the small-call stream plan
+    dw = synth.decoder(seed=3, U_max=6, W=W)
+    T = 12
+    e = config3_inputs(Bd, T, 1).contiguous().cpu().numpy()
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e)
+    frac, tr = compare_search(dd, tokens, lens, scores, ref, [0], T, 6, W, min_same=1.0)
+    assert tr == 1.0
+
+
+def test_config4_composed_full_widths_sampled_utterances(Bd):
+    # The end-to-end workload as composed, at full widths and with its batch of 64: log-mel ->
+    # prologue -> per-utterance MAX boundary, 8-bit first encoder layer -> 4-bit layers 2-6 ->
+    # projection -> beam-16 fused search with the 8-bit joint output layer.  24 log-mel frames
+    # (12 encoder frames), label budget 6; the oracle runs two of the 64 utterances.
+    B, T100, U = 64, 24, 6
+    T = T100 // 2
+    enc_w = synth.encoder(4, T=T, B=B, first_layer_bits=8, in_max=True, features=False)
+    dw = synth.decoder(3, out_bits=8, U_max=U)
+    mel = synth.logmel(4, B, T100, 40)
+    feats_dev = Bd.q4_feature_prologue(torch.from_numpy(mel).cuda())
+    enc = Bd.Encoder(enc_w["enc"])
+    got = enc.forward(feats_dev, want_layers=True)
+    utts = [5, 58]
+    feats_ref = np.stack([O.features(mel[b]) for b in utts], axis=1).astype(np.float16)
+    np.testing.assert_array_equal(feats_dev.cpu().numpy()[:, utts], feats_ref)
+    ref_enc = O.encoder_forward(enc_w["enc"], feats_ref, want_layers=True)
+    for l, yq in enumerate(got["layers"]):
+        g = gpu_codes(yq, 1280, enc.out_acts[l]).reshape(T, B, 1280)[:, utts]
+        np.testing.assert_array_equal(g, ref_enc["layers"][l]["yq"], err_msg=f"encoder layer {l}")
+    e_gpu = got["e"].cpu().numpy()
+    np.testing.assert_array_equal(e_gpu[:, utts], ref_enc["e"])
+    dd = Bd.Decoder(dw)
+    tokens, lens, scores = dd.decode(got["e"])
+    torch.cuda.synchronize()
+    assert dd.tensors["status"].item() == 0
+    ref = O.alsd(O.Decoder(dw), ref_enc["e"])
+    frac, tr = compare_search(dd, tokens.cpu().numpy(), lens.cpu().numpy(), scores.cpu().numpy(), ref,
+                              utts, T, U, 16, min_same=1.0)
+    assert tr == 1.0

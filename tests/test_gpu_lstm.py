@@ -195,3 +195,50 @@ def test_config1_full_size_sampled_utterances(Bd):
     # oracle recomputes two of the 32 utterances (they are independent).
     enc = synth.encoder(seed=1)
     encoder_case(Bd, enc, enc["features"], utts=[3, 28])
+
+
+# ------------------------------------------------------------------ against the PLAIN oracle path
+def plain_step_case(Bd, lw, x_act, hid, xq, hq, c):
+    """qlstm_step against the textbook step (libm gates in double): real values within the
+    tolerance, codes equal except within 1e-3 code units of a rounding boundary (+-1 there)."""
+    want = O.lstm_step_plain(O.Lstm([lw]), xq, x_act, hq, c, hid)
+    got = Bd.qlstm_step(pack_codes(xq, x_act), to_act(x_act), pack_codes(hq, hid),
+                        torch.from_numpy(c).cuda(), Bd.DeviceLstm(lw))
+    H = c.shape[1]
+    assert_close(got["c"].cpu().numpy(), want["c"], "cell state")
+    assert_close(got["h"].cpu().numpy(), want["h"], "cell output")
+    g = gpu_codes(got["hq"], H, hid)
+    diff = g.astype(np.int32) - want["hq"]
+    tie = want["tie"] < 1e-3
+    assert np.abs(diff).max() <= 1
+    assert not ((diff != 0) & ~tie).any(), "code mismatch away from a rounding boundary"
+    return diff.size, int(tie.sum()), int((diff != 0).sum())
+
+
+def test_config0_teacher_forced_against_plain_step(Bd):
+    w = synth.single_layer(seed=0)
+    lw = w["layers"][0]
+    x_act, hid = O.act_symmetric(w["x_clip"], 4), O.act_symmetric(1.0, 4)
+    xq = O.quantize(w["x"], x_act)
+    hq, c = np.zeros((4, 128), np.int16), np.zeros((4, 128), np.float32)
+    L = O.Lstm([lw])
+    tot = np.zeros(3, np.int64)
+    for t in range(50):
+        tot += plain_step_case(Bd, lw, x_act, hid, xq[t], hq, c)
+        s = O.lstm_step_plain(L, xq[t], x_act, hq, c, hid)      # the plain path's own state feeds the next step
+        hq, c = s["hq"], s["c"]
+    print(f"config 0 vs plain step: {tot[0]} codes, {tot[1]} near a rounding boundary, {tot[2]} differ by one")
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_encoder_shaped_step_against_plain_step(Bd, bits):
+    # 130 rows of the encoder's inner-layer shape (K = 1280, H = 640)
+    st = synth.Stream(51 + bits)
+    lw = synth._lstm(st, "l", 1280, 640, bits, 0.1, 0.95, bits)
+    x_act, hid = O.act_symmetric(0.97, bits), O.act_symmetric(0.95, bits)
+    N = 130
+    xq = st.integers("xq", (N, 1280), x_act.lo() + 1, x_act.hi()).astype(np.int16)
+    hq = st.integers("hq", (N, 640), hid.lo() + 1, hid.hi()).astype(np.int16)
+    c = st.normal("c", (N, 640)).astype(np.float32)
+    n, near, moved = plain_step_case(Bd, lw, x_act, hid, xq, hq, c)
+    print(f"{bits} bit: {n} codes, {near} near a rounding boundary, {moved} differ by one")

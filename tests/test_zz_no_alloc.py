@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as O
 from paper_2206_07882_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -26,9 +27,12 @@ def test_static_scratch_joint_matches_workspace_joint_twice():
     st = synth.Stream(12)
     hid = dd.pred_lstm.hid_act
     R = 64
-    e = torch.from_numpy(st.normal("e", (R, 256)).astype(np.float32)).cuda()
+    e_host = st.normal("e", (R, 256)).astype(np.float32)
+    e = torch.from_numpy(e_host).cuda()
+    dec, o_hid = O.Decoder(dw), O.act_symmetric(dw.pred.lstm.hid_alpha, 4)
     for call, N in enumerate((200, 37)):          # second call is smaller: stale scratch behind it
-        fi = torch.from_numpy(st.integers(f"fi{call}", (N,), 0, R - 1).astype(np.int32)).cuda()
+        fi_host = st.integers(f"fi{call}", (N,), 0, R - 1).astype(np.int32)
+        fi = torch.from_numpy(fi_host).cuda()
         codes = st.integers(f"pq{call}", (N, 1024), -7, 7).astype(np.float32)
         pq = Bd.quantize_pack_int4(torch.from_numpy(codes).cuda(), Bd.Act(1.0, 1.0, 0, 4, 1))
         want = Bd.qjoint_logprobs(e, fi, pq, hid, dd.pred_proj, dd.z_act, dd.joint_out)
@@ -39,6 +43,9 @@ def test_static_scratch_joint_matches_workspace_joint_twice():
         torch.cuda.synchronize()
         assert torch.isfinite(got).all()
         assert (got - want).abs().max().item() <= LP_ATOL
+        # and against the CPU oracle's joint network on the same inputs
+        p_ref = O.linear(O.Linear(dw.pred.proj), codes.astype(np.int16), o_hid)
+        assert np.abs(got.cpu().numpy() - O.joint(dec, e_host[fi_host], p_ref)).max() <= LP_ATOL
     # beyond the built-in limit: a clear error instead of an allocation (N * D > 65536)
     N = 300
     pq = torch.zeros((N, 512), dtype=torch.uint8, device="cuda")
