@@ -36,6 +36,10 @@ WORKLOADS = {
     "cfg4_end_to_end": dict(B=64, T=500, U_max=250, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
     "cfg1_encoder": dict(B=32, T=500, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
     "cfg3_beam": dict(B=16, T=300, U_max=150, l1_bits=4, out_bits=4, enc=False, dec=True, seed=3),
+    # single unidirectional layer (K=64, H=128, B=4, T=50) and the prediction + joint networks driven
+    # with drawn label sequences (256 hypothesis rows x 300 steps)
+    "cfg0_single_layer": dict(B=4, T=50, U_max=0, l1_bits=4, out_bits=4, enc=False, dec=False, seed=0, kind="layer"),
+    "cfg2_pred_joint": dict(B=16, T=300, U_max=0, l1_bits=4, out_bits=4, enc=False, dec=False, seed=2, kind="predjoint"),
     # the same beam workload driven time-synchronously (its wording): at most 2 labels per frame,
     # 3 calls per frame, 900 calls
     "cfg3_beam_time_synchronous": dict(B=16, T=300, U_max=150, l1_bits=4, out_bits=4, enc=False, dec=True,
@@ -126,6 +130,29 @@ def oracle_sample(wl_name: str, cores: int, frames: int = 8):
     seed = wl["seed"]
     t0 = time.perf_counter()
     e = None
+    kind = wl.get("kind", "rnnt")
+    if kind == "layer":      # the whole workload: the oracle finishes it in well under a second
+        w = synth.single_layer(seed=seed, T=wl["T"], B=wl["B"])
+        xa, ha = O.act_symmetric(w["x_clip"], 4), O.act_symmetric(1.0, 4)
+        t0 = time.perf_counter()
+        O.lstm_layer(O.Lstm(w["layers"]), O.quantize(w["x"], xa), xa, ha, n_threads=n)
+        dt = time.perf_counter() - t0
+        return dt, wl["B"] * wl["T"] * 0.02, f"the whole workload ({wl['B']} sequences x {wl['T']} steps)"
+    if kind == "predjoint":  # `cores` of the 256 rows over the first 4 * frames steps
+        steps = 4 * frames
+        dw = synth.decoder(seed)
+        act = O.act_symmetric(1.0, 4)
+        fr = synth.enc_frames(seed, steps, 1, 1280).astype(np.float32)
+        proj = synth._linear(synth.Stream(seed), "enc.proj", 256, 1280)
+        toks = np.concatenate([np.zeros((n, 1), np.int32), synth.labels(seed, n, steps - 1, 1024)], axis=1)
+        fi = np.tile(np.arange(steps, dtype=np.int32)[None, :], (n, 1))
+        dec = O.Decoder(dw)
+        t0 = time.perf_counter()
+        e = O.linear(O.Linear(proj), O.quantize(fr.reshape(steps, 1280), act), act)
+        O.pred_joint_forced(dec, e, fi, toks, n_threads=n)
+        dt = time.perf_counter() - t0
+        # scaled to the unit of the line: seconds per second of "audio" at 16 rows per utterance
+        return dt, n * steps * 0.02 / 16.0, f"{n} of the 256 rows x first {steps} of 300 steps, full layer widths, one row per thread"
     if wl["enc"]:
         enc_w = synth.encoder(seed, T=frames, B=n, first_layer_bits=wl["l1_bits"], in_max=wl["l1_bits"] == 8,
                               features=False)
@@ -193,6 +220,29 @@ class Job:
         seed = sharding.rank_seed(wl["seed"], rank)    # every rank gets its own utterances
         self.enc = self.dec = None
         self.host_in = None
+        self.kind = wl.get("kind", "rnnt")
+        if self.kind == "layer":
+            w = synth.single_layer(seed=wl["seed"], T=T, B=B)
+            self.layer = [Bd.DeviceLstm(l) for l in w["layers"]]
+            self.layer_act = Bd.q4_act_symmetric(w["x_clip"], 4)
+            self.host_in = torch.from_numpy(synth.single_layer(seed=seed, T=T, B=B)["x"].reshape(T * B, -1)).pin_memory()
+            self.layer_ws = None
+        if self.kind == "predjoint":
+            dw = synth.decoder(wl["seed"])
+            self.pj = Bd.Decoder(dw)
+            N = B * 16
+            self.pj_tok = torch.from_numpy(np.ascontiguousarray(np.concatenate(
+                [np.zeros((N, 1), np.int32), synth.labels(seed, N, T - 1, 1024)], axis=1).T)).cuda()   # [T, N]
+            self.pj_fi = torch.from_numpy((np.arange(T, dtype=np.int32)[:, None] * B +
+                                           (np.arange(N, dtype=np.int32)[None, :] // 16)).astype(np.int32)).cuda()
+            self.host_in = torch.from_numpy(synth.enc_frames(seed, T, B, 1280)).pin_memory()
+            self.frame_act = Bd.q4_act_symmetric(1.0, 4)
+            self.frame_proj = Bd.DeviceLinear(synth._linear(synth.Stream(wl["seed"]), "enc.proj", 256, 1280))
+            Hp = self.pj.pred_lstm.H
+            self.pj_buf = dict(hq=[torch.zeros((N, Hp // 2), dtype=torch.uint8, device="cuda") for _ in range(2)],
+                               c=torch.zeros((N, Hp), dtype=torch.float32, device="cuda"),
+                               logp=torch.empty((N, 1024), dtype=torch.float32, device="cuda"),
+                               ws=torch.empty(Bd.workspace_bytes(Bd.WS_JOINT, [N, 256]), dtype=torch.uint8, device="cuda"))
         if wl["enc"]:
             enc_w = synth.encoder(wl["seed"], T=T, B=B, first_layer_bits=wl["l1_bits"],
                                   in_max=wl["l1_bits"] == 8, features=False)
@@ -246,6 +296,11 @@ class Job:
         """Encoder side of a pass: returns (projected frames e [T,B,D], last result so far)."""
         Bd, wl = self.Bd, self.wl
         B, T = wl["B"], wl["T"]
+        if self.kind == "layer":
+            xq = Bd.quantize_pack_int4(x, self.layer_act)
+            r = Bd.qlstm_layer_forward(xq, self.layer_act, T, B, self.layer, workspace=self.layer_ws)
+            self.layer_ws = r["workspace"]
+            return None, r["yq"]
         if self.enc is not None:
             feats = Bd.q4_feature_prologue(x) if self.name.startswith("cfg4") else x
             r = self.enc.forward(feats)
@@ -255,6 +310,19 @@ class Job:
 
     def search(self, enc_out):
         e, res = enc_out if isinstance(enc_out, tuple) else (enc_out, None)
+        if self.kind == "predjoint":
+            # teacher-forced prediction network + joint: every step feeds the drawn label of each of the
+            # 256 rows (embedding lookup inside qlstm_step), then scores the row against its frame
+            Bd, d, b = self.Bd, self.pj, self.pj_buf
+            b["hq"][0].zero_()
+            b["c"].zero_()
+            e2 = e.reshape(-1, 256)
+            for s in range(self.wl["T"]):
+                Bd.qlstm_step(d.pred_emb_q, d.pred_emb_act, b["hq"][s & 1], b["c"], d.pred_lstm,
+                              x_row_idx=self.pj_tok[s], out=dict(hq=b["hq"][(s + 1) & 1], c=b["c"]))
+                Bd.qjoint_logprobs(e2, self.pj_fi[s], b["hq"][(s + 1) & 1], d.pred_lstm.hid_act, d.pred_proj,
+                                   d.z_act, d.joint_out, logp=b["logp"], workspace=b["ws"])
+            return (b["logp"],)
         if self.dec is not None:
             if "tsd" in self.wl:
                 res = self.dec.decode_time_synchronous(e, self.wl["tsd"], u_max=self.wl["U_max"], W=self.W)
@@ -293,6 +361,8 @@ def main():
     ap.add_argument("--ref-frames", type=int, default=8)
     ap.add_argument("--beam", type=int, default=16, help="beam width W (1..16)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the single-utterance beam sweep appended to the end-to-end line")
     ap.add_argument("--no-dependent-launch", action="store_true",
                     help="launch the beam step's kernels in plain stream order")
     ap.add_argument("--eager", action="store_true",
@@ -321,6 +391,7 @@ def main():
         from paper_2206_07882_b200 import binding as _Bd
         _Bd.dependent_launch_set(False)
     job = Job(args.workload, rank, args.beam)
+    job.passes = args.steps
     wl = job.wl
     B, T, U = wl["B"], wl["T"], wl["U_max"]
     iters = (T * (wl["tsd"] + 1) if "tsd" in wl else T + U) if wl["dec"] else 0
@@ -393,7 +464,7 @@ def main():
     # ---- instrumented eager passes (rank 0): every launch of the pass bracketed by CUDA
     # events on its own stream -> per-kernel shares, the dominant kernel's launch duration,
     # the encoder / search split, and the number of launches per pass
-    shares, dom_tag, dom_ms, dom_n, n_launch_step, rec_extra = {}, None, None, 0, 0, None
+    shares, dom_tag, dom_ms, dom_n, n_launch_step, rec_extra, series = {}, None, None, 0, 0, None, {}
     if rank == 0:
         cap = 40000
         evs, start, stop, tags = events(cap)
@@ -412,7 +483,7 @@ def main():
             st = job.dec.state
             saved_aux = (st.aux_stream[0], st.aux_stream[1])
             st.aux_stream[0], st.aux_stream[1] = None, None
-        tot, cnt = {}, {}
+        tot, cnt, series = {}, {}, {}
         for _ in range(K):
             lib.q4_timing_set(C.c_uint32(0xFFFFFFFF), start, stop, tags, C.c_int32(cap))
             la = Bd.launch_count()
@@ -421,10 +492,14 @@ def main():
             n_launch_step = Bd.launch_count() - la
             n = lib.q4_timing_count()
             lib.q4_timing_set(C.c_uint32(0), None, None, None, C.c_int32(0))
+            per_pass = {}
             for i in range(n):
                 ms = evs[i].elapsed_time(evs[cap + i])
                 tot[tags[i]] = tot.get(tags[i], 0.0) + ms
                 cnt[tags[i]] = cnt.get(tags[i], 0) + 1
+                per_pass.setdefault(tags[i], []).append(ms)
+            for t_, v_ in per_pass.items():          # launch-ordered durations, one list per pass
+                series.setdefault(t_, []).append(v_)
         if saved_aux is not None:
             job.dec.state.aux_stream[0], job.dec.state.aux_stream[1] = saved_aux
         allms = sum(tot.values()) or 1.0
@@ -435,7 +510,7 @@ def main():
         # function they launch: the fused LSTM step serves tags 5, 7, 9 and 10), and of that
         # kernel the launch site with the largest time; the encoder recurrence is reported beside
         # it when it is not the dominant one.
-        families = {"k_mma_lstm": (5, 7, 9, 10), "k_enc_recurrent": (3,), "k_mma_gemm": (2,)}
+        families = {"k_mma_lstm": (5, 7, 9, 10), "k_enc_recurrent": (3,), "k_mma_gemm": (2,), "joint": (12,)}
         fam_ms = {f: sum(tot.get(t, 0.0) for t in ts) for f, ts in families.items()}
         dom_tag = None
         if any(v > 0 for v in fam_ms.values()):
@@ -467,16 +542,23 @@ def main():
                                  "state through the 126 MB L2 between two uses of any input"},
                 "parts": {"encoder_ms": enc_ms, "decode_ms": dec_ms,
                           "encoder_frames_per_s": (B * T / (enc_ms / 1e3)) if wl["enc"] and enc_ms else None,
-                          "beam_hyps_per_s": (B * job.W * iters / (dec_ms / 1e3)) if wl["dec"] and dec_ms else None},
+                          "beam_hyps_per_s": (B * job.W * iters / (dec_ms / 1e3)) if wl["dec"] and dec_ms else None,
+                          "layer_frames_per_s": (B * T / (enc_ms / 1e3)) if job.kind == "layer" and enc_ms else None,
+                          "pred_joint_hyps_per_s": (B * 16 * T / (dec_ms / 1e3)) if job.kind == "predjoint" and dec_ms else None},
                 "e2e": {"value": rtf_e2e, "unit": "s/s", "h2d_bytes_per_step": job.h2d_bytes(),
                         "d2h_bytes_per_step": d2h},
                 "gpu_launches": n_launch_step * K, "launches_per_step": n_launch_step, "kernels": shares,
                 "clocks": clocks, "peaks": pk,
                 "paper_context": {"rtf_int4_simulated": 0.065, "speedup_fp16_to_int4_simulated": 3.4,
                                   "note": "simulated accelerator, 1 utterance of 152 frames, beam 16"}}
-        line["roofline"] = roofline(job, dom_tag, dom_ms, dom_n, pk) if dom_tag is not None else None
+        pk["int8_tops_yardstick"] = int8_yardstick(torch)
+        line["roofline"] = roofline(job, dom_tag, dom_ms, dom_n, pk, series.get(dom_tag)) if dom_tag is not None else None
         if rec_extra is not None:
             line["roofline_encoder_recurrence"] = roofline(job, 3, rec_extra[0], rec_extra[1], pk)
+        if wl["dec"] and "tsd" not in wl:
+            line["parts"].update(search_regimes(job, dec_ms, torch))
+        if args.workload == "cfg4_end_to_end" and world == 1 and not args.no_sweep:
+            line["fig2_beam_sweep"] = fig2_sweep(torch)
         if line["roofline"] is not None:
             line["roofline"]["timing"] = ("CUDA events around every launch of this kernel in eager, single-stream "
                                           "passes of the same step; the headline region replays CUDA graphs, "
@@ -493,41 +575,121 @@ def main():
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the captures summarised under
-# profiles/ (k_mma_lstm_prof_end_to_end.md, k_enc_recurrent_prof_encoder.md); to be reset to None
-# when those kernels change.
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch, copied by hand from an ncu capture of
+# the kernel revision named in "captured"; None once the kernel has changed since.  The capture runs
+# with cold caches; inside the timed loop the weights of an iteration stay in the L2, so the real
+# DRAM traffic of a launch is lower.
 NCU_TRAFFIC = {
-    "k_mma_lstm_tgt_l2": {"bytes": 41252864 + 545536, "rows": 1024, "weights": 2 * 8192 * 2048},
-    "k_enc_recurrent": {"bytes": 167211520 + 6564096},
+    "k_mma_lstm_tgt_l2": None,
+    "k_enc_recurrent": None,
 }
 
 
-def roofline(job, tag, ms, n, pk):
-    """Roofline entry of the dominant kernel.  Algorithmic work per launch: the weight bytes
-    the kernel must read once plus per-row state traffic, and 2*rows*J*K integer ops."""
+def int8_yardstick(torch):
+    """Dense int8 GEMM rate of the library routine torch._int_mm at 8192^3, measured in this run as a
+    yardstick for the int8 tensor peak (never on the timed path).  TOP/s, or None if unavailable."""
+    try:
+        a = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda")
+        b = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda")
+        for _ in range(3):
+            torch._int_mm(a, b)
+        best = None
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._int_mm(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+        return 2.0 * 8192 ** 3 / (best / 1e3) / 1e12
+    except Exception:
+        return None
+
+
+def search_regimes(job, dec_ms, torch):
+    """Splits the search time into its two kinds of iterations.  With the synthetic weights an
+    iteration either extends (nearly) every slot by a label, so that the next one runs all three
+    networks on those rows, or extends none (label budgets spent: only the joint network and the
+    selection run).  The label-free kind is timed by itself: the same search with a label budget of
+    zero, replayed as a CUDA graph; the other kind follows from the measured search time."""
+    wl, d = job.wl, job.dec
+    T, B, W = wl["T"], wl["B"], job.W
+    iters = T + wl["U_max"]
+    tok = d.tensors["bp_token"][:iters]
+    per_iter = (tok > 0).reshape(iters, -1).sum(1)
+    n_busy = int((per_iter > 0).sum().item()) + 1          # launch 0 advances the start symbols
+    n_free = iters - n_busy
+    e = job.graph[0].result[0] if job.graph is not None else job.encode(job.dev_in)[0]
+    g = job.Bd.GraphedStep(lambda: d.decode(e, u_max=0, W=W))
+    g()
+    g()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(3):
+        g()
+    e1.record()
+    torch.cuda.synchronize()
+    free_us = e0.elapsed_time(e1) / 3 * 1e3 / T
+    busy_us = (dec_ms * 1e3 - n_free * free_us) / max(n_busy, 1)
+    return {"iterations_with_network_rows": n_busy, "iterations_label_free": n_free,
+            "us_per_iteration_with_network_rows": busy_us, "us_per_iteration_label_free": free_us,
+            "hyps_per_s_with_network_rows": B * W / (busy_us * 1e-6) if busy_us > 0 else None,
+            "hyps_per_s_label_free": B * W / (free_us * 1e-6)}
+
+
+def fig2_sweep(torch):
+    """The regime of the paper's run-time figure (Section 4.1): ONE utterance of 152 encoder frames,
+    beam width 1..16, everything at 4 bits; ms per utterance (graph replay, inputs resident)."""
+    out = {}
+    job = Job("fig2_single_utterance", 0, 16)
+    for W in (1, 2, 4, 8, 16):
+        job.W = W
+        job.dec.alloc_state(job.wl["B"], W, job.wl["T"] + job.wl["U_max"])
+        job.graph = None
+        job.step(job.dev_in)
+        for _ in range(3):
+            job.step_graphed()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(5):
+            job.step_graphed()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 5
+        out[str(W)] = {"ms_per_utterance": ms, "rtf": ms / 1e3 / (job.wl["T"] * 0.02)}
+    return out
+
+
+def roofline(job, tag, ms, n, pk, series=None):
+    """Roofline entry of one kernel.  Algorithmic work per launch: the weight bytes the kernel must
+    read once plus per-row state traffic, and 2*rows*J*K integer ops.  `series`: the launch-ordered
+    event durations (ms) of this launch site, one list per instrumented pass."""
     name = TAG_NAMES[tag]
     wl = job.wl
-    N = wl["B"] * job.W
-    if job.dec is not None and tag in (5, 7, 9, 10):
-        # rows a launch really advances: label extensions of the previous selection (blank
-        # extensions keep their parent's state), counted from the search history of the last pass
-        tok = job.dec.tensors["bp_token"][:(wl["T"] * (wl["tsd"] + 1) if "tsd" in wl else wl["T"] + wl["U_max"])]
-        N = max(1.0, float((tok > 0).sum().item() + wl["B"]) / float(tok.shape[0]))
-        out_rows = N
-        # the mean hides two kinds of launches: iterations that extended some slot by a label (their
-        # successor runs the networks on that many rows) and iterations that extended none
-        per_iter = (tok > 0).reshape(tok.shape[0], -1).sum(1)
-        busy = per_iter > 0
-        rows_split = {"launches_with_rows": int(busy.sum().item()) + 1, "launches_without_rows": int((~busy).sum().item()) - 1,
-                      "mean_rows_when_any": float(per_iter[busy].float().mean().item()) if bool(busy.any()) else 0.0}
-    else:
-        out_rows = None
-        rows_split = None
-    int8_peak = 2.0 * pk["bf16_tflops_sustained"]          # dense int8 : bf16 = 2 : 1
-    out = {"kernel": name, "launches_timed": n, "avg_ms": ms, "traffic": None}
-    if out_rows is not None:
-        out["rows_per_launch"] = out_rows
-        out.update(rows_split)
+    int8_peak = 2.0 * pk["bf16_tflops_sustained"]          # dense int8 : bf16 = 2 : 1 (nominal ratio)
+    tensor_unit = "TOP/s (int8; peak = 2 x measured sustained bf16)"
+    out = {"kernel": name, "launches_timed": n, "avg_ms": ms, "traffic": None,
+           "traffic_note": "no ncu capture of the current kernel revision", "peak_source": pk["source"]}
+
+    def entry(bytes_, ops, sec):
+        t_hbm = bytes_ / (pk["hbm_gbs"] * 1e9)
+        t_tensor = ops / (int8_peak * 1e12)
+        r = {"algorithmic_bytes": bytes_, "algorithmic_ops": ops,
+             "hbm": {"achieved": bytes_ / sec / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": bytes_ / sec / 1e9 / pk["hbm_gbs"]},
+             "tensor": {"achieved": ops / sec / 1e12, "peak": int8_peak, "unit": tensor_unit,
+                        "frac": ops / sec / 1e12 / int8_peak,
+                        "peak_measured_int8_yardstick": pk.get("int8_tops_yardstick")}}
+        if t_tensor > t_hbm:
+            r.update(bound="tensor", achieved=ops / sec / 1e12, peak=int8_peak, unit="TFLOP/s",
+                     frac=ops / sec / 1e12 / int8_peak)
+        else:
+            r.update(bound="hbm", achieved=bytes_ / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s",
+                     frac=bytes_ / sec / 1e9 / pk["hbm_gbs"])
+        return r
 
     def lstm_work(l, rows, kx):
         # weights as stored (packed codes + row scales + bias), per row: input codes, previous
@@ -538,59 +700,92 @@ def roofline(job, tag, ms, n, pk):
         ops = 2.0 * rows * 4 * H * (l.w_ih.k_pad + H)
         return wbytes + rows * per_row, ops
 
-    if tag in (5, 7, 9, 10):
+    if job.dec is not None and tag in (5, 7, 9, 10):
         d = job.dec
         l, kx = {5: (d.pred_lstm, 256), 7: (d.src.lstm[0], 256), 9: (d.tgt.lstm[0], 256),
                  10: (d.tgt.lstm[-1], d.tgt.lstm[0].H)}[tag]
-        bytes_, ops = lstm_work(l, N, kx)
-        if tag == 10 and l.H == 2048:
-            # DRAM bytes of one launch from the ncu capture (cold caches, 1024 rows): the weights do
-            # not depend on the rows, the rest scales with them
-            t = NCU_TRAFFIC["k_mma_lstm_tgt_l2"]
-            out["traffic"] = t["weights"] + (t["bytes"] - t["weights"]) * N / t["rows"]
-    elif tag == 3:
+        # rows a launch really advances: the label extensions of the previous selection (blank
+        # extensions keep their parent's state), counted from the search history of the last pass;
+        # launch 0 advances the start symbol of every utterance
+        iters = wl["T"] * (wl["tsd"] + 1) if "tsd" in wl else wl["T"] + wl["U_max"]
+        tok = job.dec.tensors["bp_token"][:iters]
+        per_iter = (tok > 0).reshape(iters, -1).sum(1).cpu().numpy().astype(np.float64)
+        rows = np.concatenate([[float(wl["B"])], per_iter[:-1]])
+        busy = rows > 0
+        mean_rows = float(rows.mean())
+        out.update(rows_per_launch_mean=mean_rows, launches_with_rows=int(busy.sum()),
+                   launches_without_rows=int((~busy).sum()), mean_rows_when_any=float(rows[busy].mean()))
+        times = None
+        if series and all(len(v) == iters for v in series):
+            times = np.asarray(series, dtype=np.float64)            # [passes, launches]
+        if times is not None and busy.any():
+            # the headline fraction describes the launches that HAVE rows (ops at their mean row count
+            # over their mean duration); the all-launch mean, which mixes them with launches that find
+            # no pending row and exit at once, is kept beside it
+            ms_busy = float(times[:, busy].mean())
+            b_, o_ = lstm_work(l, float(rows[busy].mean()), kx)
+            out.update(entry(b_, o_, ms_busy / 1e3))
+            out["avg_ms_with_rows"] = ms_busy
+            out["avg_ms_without_rows"] = float(times[:, ~busy].mean()) if (~busy).any() else None
+            b2, o2 = lstm_work(l, mean_rows, kx)
+            out["frac_mean"] = entry(b2, o2, ms / 1e3)["frac"]
+            out["regime"] = "launches with pending rows"
+        else:
+            b_, o_ = lstm_work(l, mean_rows, kx)
+            out.update(entry(b_, o_, ms / 1e3))
+        t = NCU_TRAFFIC["k_mma_lstm_tgt_l2"]
+        if tag == 10 and l.H == 2048 and t is not None:
+            # the weights do not depend on the rows, the rest scales with them
+            out["traffic"] = t["weights"] + (t["bytes"] - t["weights"]) * out["mean_rows_when_any"] / t["rows"]
+            out["traffic_note"] = t["captured"]
+        return out
+    if tag == 3:
         # persistent recurrence: one launch = all T steps of a layer, both directions.  It must
         # read the int32 input accumulators once, the recurrent weights once, and write the codes.
         # By bytes it is an HBM kernel; in practice the T dependent steps (MMA, cell update,
         # exchange of the new codes, cluster barrier) bind it, so the fraction is small by nature.
         l = job.enc.layers[1][0]
         Bn, Tn, H = wl["B"], wl["T"], l.H
-        bytes_ = 2 * (4 * H * H + Tn * Bn * 4 * H * 4 + Tn * Bn * H // 2)
+        bytes_ = 2 * (4 * H * H // 2 + Tn * Bn * 4 * H * 4 + Tn * Bn * H // 2)
         ops = 2 * 2.0 * Tn * Bn * 4 * H * H
         sec = ms / 1e3
         out.update(bound="hbm", achieved=bytes_ / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s",
                    frac=bytes_ / sec / 1e9 / pk["hbm_gbs"], algorithmic_bytes=bytes_, algorithmic_ops=ops,
-                   tensor={"achieved": ops / sec / 1e12, "peak": int8_peak, "unit": "TOP/s (int8, 2x measured bf16)",
+                   tensor={"achieved": ops / sec / 1e12, "peak": int8_peak, "unit": tensor_unit,
                            "frac": ops / sec / 1e12 / int8_peak},
-                   us_per_step=ms * 1e3 / Tn, peak_source=pk["source"],
+                   us_per_step=ms * 1e3 / Tn,
                    note="latency-bound: T dependent steps per launch, each ending in a cluster barrier")
-        # captured at 250 steps x 32 sequences; the traffic (input accumulators read once, codes
-        # written once) grows in proportion to steps x sequences
-        out["traffic"] = NCU_TRAFFIC["k_enc_recurrent"]["bytes"] * (Tn * Bn) / (250.0 * 32.0)
+        t = NCU_TRAFFIC["k_enc_recurrent"]
+        if t is not None:
+            # the traffic (input accumulators read once, codes written once) grows in proportion to
+            # steps x sequences
+            out["traffic"] = t["bytes"] * (Tn * Bn) / float(t["steps"] * t["sequences"])
+            out["traffic_note"] = t["captured"]
         return out
-    elif tag == 2:
+    if tag == 2:
         l = job.enc.layers[1][0]
         M = wl["B"] * wl["T"]
         bytes_ = M * l.w_ih.k_pad // 2 + l.w_ih.q.numel() + M * 4 * l.H * 4
         ops = 2.0 * M * 4 * l.H * l.w_ih.k_pad
-    else:
-        out.update(bound="hbm", achieved=None, peak=pk["hbm_gbs"], unit="GB/s", frac=None)
+        out.update(entry(bytes_, ops, ms / 1e3))
         return out
-    t_hbm = bytes_ / (pk["hbm_gbs"] * 1e9)
-    t_tensor = ops / (int8_peak * 1e12)
-    sec = ms / 1e3
-    out.update(algorithmic_bytes=bytes_, algorithmic_ops=ops,
-               hbm={"achieved": bytes_ / sec / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                    "frac": bytes_ / sec / 1e9 / pk["hbm_gbs"]},
-               tensor={"achieved": ops / sec / 1e12, "peak": int8_peak, "unit": "TOP/s (int8, 2x measured bf16)",
-                       "frac": ops / sec / 1e12 / int8_peak})
-    if t_tensor > t_hbm:
-        out.update(bound="tensor", achieved=ops / sec / 1e12, peak=int8_peak, unit="TFLOP/s",
-                   frac=ops / sec / 1e12 / int8_peak)
-    else:
-        out.update(bound="hbm", achieved=bytes_ / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s",
-                   frac=bytes_ / sec / 1e9 / pk["hbm_gbs"])
-    out["peak_source"] = pk["source"]
+    if tag == 12 and job.kind == "predjoint":
+        # joint of the teacher-forced workload: projection Hp -> D and output layer D -> V for N rows
+        d, N = job.pj, wl["B"] * 16
+        Hp, D, V = d.pred_lstm.H, d.D, d.V
+        bytes_ = d.pred_proj.nbytes() + d.joint_out.nbytes() + N * (Hp // 2 + D * 4 + V * 4)
+        ops = 2.0 * N * (D * Hp + V * D)
+        per_call_ms = ms * n / max(job.passes, 1) / wl["T"]      # all launches of one qjoint_logprobs call
+        out.update(entry(bytes_, ops, per_call_ms / 1e3))
+        out["ms_per_call"] = per_call_ms
+        out["launches_per_call"] = n / max(job.passes, 1) / wl["T"]
+        return out
+    if tag == 5 and job.kind == "predjoint":
+        d, N = job.pj, wl["B"] * 16
+        b_, o_ = lstm_work(d.pred_lstm, N, 256)
+        out.update(entry(b_, o_, ms / 1e3))
+        return out
+    out.update(bound="hbm", achieved=None, peak=pk["hbm_gbs"], unit="GB/s", frac=None)
     return out
 
 

@@ -281,20 +281,25 @@ def qlstm_layer_forward(xq: torch.Tensor, x_act: Act, T: int, B: int, layers: Se
 
 
 def qlstm_step(xq: torch.Tensor, x_act: Act, hq_in: torch.Tensor, c_in: torch.Tensor,
-               layer: DeviceLstm, x_row_idx: Optional[torch.Tensor] = None, want_dbg: bool = False):
-    """One step for N rows.  Returns dict(hq, c, h [, acc_ih, acc_hh])."""
+               layer: DeviceLstm, x_row_idx: Optional[torch.Tensor] = None, want_dbg: bool = False,
+               out: Optional[dict] = None):
+    """One step for N rows.  Returns dict(hq, c, h [, acc_ih, acc_hh]).  `out` may hold
+    preallocated tensors hq, c (c may be c_in itself) and optionally h; then nothing is allocated."""
     _need_cuda()
     N, H = c_in.shape
     dev = c_in.device
-    r = {"hq": torch.empty_like(hq_in), "c": torch.empty_like(c_in),
-         "h": torch.empty((N, H), dtype=torch.float32, device=dev)}
+    if out is not None:
+        r = dict(out)
+    else:
+        r = {"hq": torch.empty_like(hq_in), "c": torch.empty_like(c_in),
+             "h": torch.empty((N, H), dtype=torch.float32, device=dev)}
     if want_dbg:
         r["acc_ih"] = torch.empty((N, 4 * H), dtype=torch.int32, device=dev)
         r["acc_hh"] = torch.empty((N, 4 * H), dtype=torch.int32, device=dev)
     wih, whh = layer.w_ih.c(), layer.w_hh.c()
     _chk(lib().qlstm_step(_p(xq), C.byref(x_act), _p(x_row_idx), _p(hq_in), _p(c_in), C.c_int32(N),
                           C.byref(wih), C.byref(whh), _p(layer.bias), C.byref(layer.hid_act),
-                          _p(r["hq"]), _p(r["c"]), _p(r["h"]), _p(r.get("acc_ih")),
+                          _p(r["hq"]), _p(r["c"]), _p(r.get("h")), _p(r.get("acc_ih")),
                           _p(r.get("acc_hh")), _stream()), "qlstm_step")
     return r
 
