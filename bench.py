@@ -744,10 +744,16 @@ def roofline(job, tag, ms, n, pk, series=None):
         # read the int32 input accumulators once, the recurrent weights once, and write the codes.
         # By bytes it is an HBM kernel; in practice the T dependent steps (MMA, cell update,
         # exchange of the new codes, cluster barrier) bind it, so the fraction is small by nature.
-        l = job.enc.layers[1][0]
+        l = job.layer[0] if job.kind == "layer" else job.enc.layers[1][0]
+        nd = 1 if job.kind == "layer" else 2
         Bn, Tn, H = wl["B"], wl["T"], l.H
-        bytes_ = 2 * (4 * H * H // 2 + Tn * Bn * 4 * H * 4 + Tn * Bn * H // 2)
-        ops = 2 * 2.0 * Tn * Bn * 4 * H * H
+        bytes_ = nd * (4 * H * H // 2 + Tn * Bn * 4 * H * 4 + Tn * Bn * H // 2)
+        ops = nd * 2.0 * Tn * Bn * 4 * H * H
+        if job.kind == "layer":
+            # 50 launches of the one-step kernel (200 rows: below the persistent kernel's threshold)
+            ms = ms * n / max(job.passes, 1)
+            out["note_launches"] = "one launch per time step; avg_ms is the sum over the T launches of a pass"
+            out["avg_ms"] = ms
         sec = ms / 1e3
         out.update(bound="hbm", achieved=bytes_ / sec / 1e9, peak=pk["hbm_gbs"], unit="GB/s",
                    frac=bytes_ / sec / 1e9 / pk["hbm_gbs"], algorithmic_bytes=bytes_, algorithmic_ops=ops,
@@ -763,7 +769,7 @@ def roofline(job, tag, ms, n, pk, series=None):
             out["traffic_note"] = t["captured"]
         return out
     if tag == 2:
-        l = job.enc.layers[1][0]
+        l = job.layer[0] if job.kind == "layer" else job.enc.layers[1][0]
         M = wl["B"] * wl["T"]
         bytes_ = M * l.w_ih.k_pad // 2 + l.w_ih.q.numel() + M * 4 * l.H * 4
         ops = 2.0 * M * 4 * l.H * l.w_ih.k_pad

@@ -371,6 +371,8 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
     ra.B = B;
     ra.H = H;
     ra.dirs = dirs;
+    ra.w_bits = w_hh[0].bits;
+    ra.status = status;
     ra.x_scale = x_act->scale;
     ra.x_scale_b = x_scale_b;
     ra.hid_act = *hid_act;

@@ -148,6 +148,8 @@ struct EncRecDir {
 struct EncRecArgs {
   EncRecDir d[2];
   int32_t T, B, H, dirs, n_groups;
+  int32_t w_bits;           // storage width of the recurrent weights the int8 copies were made from
+  int32_t* status;          // device status word: receives Q4_ERR_TIMEOUT when a bounded wait expires
   float x_scale;
   const float* x_scale_b;
   q4_act hid_act, out_act;

@@ -15,6 +15,7 @@
 #include <string.h>
 
 #include "q4_internal.h"
+#include "q4_mma.cuh"
 
 namespace q4 {
 
@@ -254,6 +255,342 @@ k_enc_recurrent(const EncRecArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same recurrence for 4-bit recurrent weights and 4-bit hidden codes (five of the six encoder
+// layers, Section 3.2) with the weights held in REGISTERS for the whole sequence.
+//
+// A warp's 16 weight rows x H columns are 20 A fragments of the m16n8k32 MMA at H = 640; as 4-bit
+// codes they fill 2 registers per fragment instead of 4, 40 registers per thread for the whole
+// slice (102 KB per CTA).  Register 2s of thread (g, t4) holds, nibble 2i = W[row r(g)][32s + 4 t4 + i]
+// and nibble 2i+1 = W[row r(g+8)][32s + 4 t4 + i] (register 2s+1 the same for columns + 16), so that
+// two masks and one shift turn it into the fragment registers (a0, a1) with every code in the HIGH
+// nibble of its byte: the int8 operand is 16 x code, exact, and the accumulator 16 x the true sum
+// (|16 w h| <= 1024 per product, far from overflow); an arithmetic shift by 4 restores it.  The
+// main loop therefore reads only the hidden codes from shared memory, not the weight slice (205 KB
+// per step in the int8 kernel above: that kernel's limit).
+//
+// Tile row g holds gate (g & 1) of the warp's cell g >> 1 and tile row g + 8 gate 2 + (g & 1) of
+// the same cell, so after the MMA the lanes g and g ^ 1 hold the four gates of one cell for two
+// sequences: one exchange of two values with lane ^ 4 gives every lane the four gates of its item
+// (cell g >> 1, sequence 2 t4 + (g & 1)).
+//
+// A cluster serves NU independent units of 8 sequences of one direction, one after the other within
+// a step.  The hidden codes of a unit are laid out [source CTA][sequence][cells of that CTA], so a
+// CTA's new codes are one contiguous block of 8 x H/8 bytes in every receiver: they travel as ONE
+// bulk copy per destination through distributed shared memory (8 per unit and step instead of 320
+// 16-byte stores), counted on an mbarrier of the receiving CTA; a CTA waits on its own mbarrier
+// before the unit's next step.  (Rows of 80 bytes put the eight sequences of an ldmatrix on
+// distinct banks.)  There is no cluster-wide barrier in the loop: while the
+// codes of one unit are in flight the CTA computes the other unit.  Buffers are double buffered by
+// step parity; a sender can only be a step ahead of a receiver after that receiver's own codes of
+// the previous step have arrived, which it sends after its last read of the buffer in question.
+// Every wait is bounded; when one expires the CTA records Q4_ERR_TIMEOUT, leaves the loop, and all
+// CTAs still meet at the closing cluster barrier (the others' waits expire in turn).
+// The input accumulators of the next step are fetched into shared memory by cp.async one step
+// ahead.  The layer output codes leave through a staging buffer as 8-byte stores.
+// `bytes` (a multiple of 16) from this CTA's shared memory into the shared memory of a CTA of the
+// cluster by the bulk-copy engine; their arrival is counted on the mbarrier at `mbar_addr`, an
+// address in the receiving CTA's window.  No multicast: one destination per copy.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_addr, uint32_t src_addr, uint32_t bytes,
+                                                     uint32_t mbar_addr) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_addr), "r"(src_addr), "r"(bytes), "r"(mbar_addr)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr int REC_BG = 8;   // sequences per unit of the register-resident kernel
+constexpr int REC4_THREADS = REC_THREADS;
+
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(int id, int count) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+template <int NU, int KS>
+__global__ void __cluster_dims__(REC_CLUSTER, 1, 1) __launch_bounds__(REC4_THREADS, 1)
+k_enc_recurrent_w4(const EncRecArgs a) {
+  extern __shared__ __align__(16) uint8_t rec_smem[];
+  constexpr int BG = REC_BG;
+  constexpr int H = 32 * KS;
+  constexpr int cpc = H / REC_CLUSTER;      // cells per CTA
+  constexpr int rows = 4 * cpc;
+  constexpr int chunks = cpc >> 4;          // 16-byte chunks of a sequence's new codes per CTA
+  constexpr int UB = BG * H;                // bytes of one unit's hidden codes
+  constexpr int CW = REC_THREADS / 32;      // warps
+  constexpr int KR = KS - 4;                // k-steps whose weight fragments stay in registers; the last
+                                            // four come from shared memory (8 bytes per thread and k-step),
+                                            // which leaves the cell update enough registers
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_rank();
+  const int cid = blockIdx.x / REC_CLUSTER;
+  const int cpd = a.n_groups;               // clusters per direction
+  const int d = cid / cpd;
+  const int grp0 = (cid % cpd) * NU;        // first 8-sequence group of this cluster
+  const EncRecDir& D = a.d[d];
+  const int T = a.T, B = a.B;
+  int8_t* hb = reinterpret_cast<int8_t*>(rec_smem);                       // [NU][2][source CTA][BG][cpc] h_{t-1}
+  int4* pre_s = reinterpret_cast<int4*>(hb + (size_t)NU * 2 * UB);        // [2][NU][threads] input accumulators
+  float4* cst = reinterpret_cast<float4*>(pre_s + (size_t)2 * NU * REC_THREADS);   // [3][cpc] per-cell constants
+  int8_t* stage = reinterpret_cast<int8_t*>(cst + 3 * cpc);                // [2][NU][BG][cpc] new recurrent codes
+  int8_t* stage_y = stage + (size_t)2 * NU * BG * cpc;                     // [2][NU][BG][cpc] new output codes
+  uint64_t* full = reinterpret_cast<uint64_t*>(stage_y + (size_t)2 * NU * BG * cpc);   // [NU][2]
+  volatile int* dead = reinterpret_cast<volatile int*>(full + NU * 2);     // a bounded wait has expired
+  uint2* wsm = reinterpret_cast<uint2*>(full + NU * 2 + 2);                // [KS - KR][threads] packed weights
+
+  const int g = lane >> 2, t4 = lane & 3;   // MMA fragment coordinates
+  const int e = g & 1, ci = g >> 1;         // this lane's item: cell ci of the warp's 4 ...
+  const int n = 2 * t4 + e;                 // ... and sequence n of the unit's 8
+  const int cl = warp * 4 + ci;             // cell within the CTA
+  const int cell = (int)rank * cpc + cl;    // cell within the layer
+  const float sh = a.hid_act.scale;
+  const uint32_t hb_addr = smem_u32(hb), pre_addr = smem_u32(pre_s), full_addr = smem_u32(full);
+
+  // resident weights: this warp's 16 rows (stored in 4*cell+gate order), packed two codes per byte;
+  // tile row g = gate e of cell ci, tile row g + 8 = gate 2 + e of cell ci
+  uint32_t wreg[2 * KR];
+  {
+    const int8_t* W = D.w_hh + ((size_t)rank * rows + (size_t)(16 * warp)) * H;
+    const int8_t* r0 = W + (size_t)(4 * ci + e) * H + 4 * t4;
+    const int8_t* r1 = r0 + (size_t)2 * H;
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      const uint32_t q0 = *reinterpret_cast<const uint32_t*>(r0 + 32 * s);
+      const uint32_t p0 = *reinterpret_cast<const uint32_t*>(r1 + 32 * s);
+      const uint32_t q1 = *reinterpret_cast<const uint32_t*>(r0 + 32 * s + 16);
+      const uint32_t p1 = *reinterpret_cast<const uint32_t*>(r1 + 32 * s + 16);
+      const uint32_t w0 = (q0 & 0x0F0F0F0Fu) | ((p0 << 4) & 0xF0F0F0F0u);
+      const uint32_t w1 = (q1 & 0x0F0F0F0Fu) | ((p1 << 4) & 0xF0F0F0F0u);
+      if (s < KR) {
+        wreg[2 * s] = w0;
+        wreg[2 * s + 1] = w1;
+      } else {
+        wsm[(s - KR) * REC_THREADS + tid] = make_uint2(w0, w1);
+      }
+    }
+  }
+  for (int i = tid; i < NU * 2 * UB / 16; i += REC4_THREADS)
+    reinterpret_cast<uint4*>(hb)[i] = make_uint4(0, 0, 0, 0);   // h_0 = 0
+  for (int i = tid; i < cpc; i += REC4_THREADS) {
+    // de-quantization products per gate row: input scale * row scale, hidden scale * row scale; bias
+    const int c = (int)rank * cpc + i;
+    const float4 w = reinterpret_cast<const float4*>(D.sc_hh)[c], v = reinterpret_cast<const float4*>(D.sc_ih)[c];
+    const float sxs = a.x_scale;
+    cst[i] = make_float4(__fmul_rn(sxs, v.x), __fmul_rn(sxs, v.y), __fmul_rn(sxs, v.z), __fmul_rn(sxs, v.w));
+    cst[cpc + i] = make_float4(__fmul_rn(sh, w.x), __fmul_rn(sh, w.y), __fmul_rn(sh, w.z), __fmul_rn(sh, w.w));
+    cst[2 * cpc + i] = reinterpret_cast<const float4*>(D.bias)[c];
+  }
+  if (tid == 0) {
+    *dead = 0;
+    for (int i = 0; i < NU * 2; ++i) mbar_init(&full[i], 1);
+    fence_barrier_init();
+    // the first fill of either buffer of every unit: BG x H bytes from the eight CTAs
+    for (int i = 0; i < NU * 2; ++i) mbar_expect_tx(&full[i], (uint32_t)UB);
+  }
+  fence_proxy_async();   // the zeroed buffers are later written by the bulk-copy engine
+  __syncthreads();
+  cluster_barrier();   // every CTA's buffers and barriers are initialised before anyone stores into them
+
+  float c_state[NU];
+  bool live[NU];
+#pragma unroll
+  for (int u = 0; u < NU; ++u) {
+    c_state[u] = 0.0f;
+    live[u] = (grp0 + u) * BG + n < B;
+  }
+  constexpr int G = 4 * H;
+
+  {
+    const int hlo = act_lo(a.hid_act), hhi = act_hi(a.hid_act);
+    const int ylo = act_lo(a.out_act), yhi = act_hi(a.out_act);
+    const bool y4 = a.out_act.bits == 4;
+#pragma unroll
+    for (int u = 0; u < NU; ++u) {
+      const int b = (grp0 + u) * BG + n;
+      // input accumulators of the first step
+      if (live[u]) {
+        const int t = d == 0 ? 0 : T - 1;
+        cp_async16(pre_addr + (uint32_t)((u * REC_THREADS + tid) * 16), D.acc_pre + ((size_t)t * B + b) * G + 4 * cell);
+      }
+      cp_async_commit();
+    }
+    bool ok = true;
+    for (int step = 0; step < T; ++step) {
+      const int t = d == 0 ? step : T - 1 - step;
+      const int cur = step & 1, nxt = cur ^ 1;
+#pragma unroll
+      for (int u = 0; u < NU; ++u) {
+        const int b = (grp0 + u) * BG + n;
+        // the next step's input accumulators for this unit, one step ahead
+        if (step + 1 < T && live[u]) {
+          const int tn = d == 0 ? step + 1 : T - 2 - step;
+          cp_async16(pre_addr + (uint32_t)(((nxt * NU + u) * REC_THREADS + tid) * 16),
+                     D.acc_pre + ((size_t)tn * B + b) * G + 4 * cell);
+        }
+        cp_async_commit();
+        // h_{t-1} of this unit is complete in this CTA once all eight CTAs' copies have landed.  Every
+        // thread looks for itself (no block barrier: with several units the codes are long there).
+        // After a wait has expired anywhere in the CTA nobody waits any more; the loop is walked to its
+        // end all the same, so that every named barrier still gets its arrivals
+        if (step > 0 && ok) {
+          uint64_t* bar = &full[u * 2 + cur];
+          const uint32_t parity = (uint32_t)(((step - 1) >> 1) & 1);
+          bool got = false;
+          for (uint32_t i = 0; i < (1u << 22); ++i) {
+            if (mbar_try_wait(bar, parity)) {
+              got = true;
+              break;
+            }
+            if ((i & 255u) == 255u && *dead) break;
+          }
+          if (!got) {
+            ok = false;
+            *dead = 1;
+            if (a.status) atomicExch(a.status, Q4_ERR_TIMEOUT);
+          }
+          // arm the barrier for the next fill of this buffer; nobody can send that fill before this
+          // CTA's codes of the present step have arrived, which are sent after every thread got here
+          if (tid == 0 && got) mbar_expect_tx(bar, (uint32_t)UB);
+        }
+        // recurrent MACs: weights from registers, hidden codes by ldmatrix
+        int acc[2][4];
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+          for (int r = 0; r < 4; ++r) acc[c][r] = 0;
+        {
+          // lanes 0-15 supply the row addresses: matrix i/8 = k half, row i%8 = sequence; the 16-byte
+          // chunk j = 2s + half of a sequence's codes lies in source block j / chunks at chunk j % chunks
+          // (the second half's chunk is 16 bytes on, or in the next source block when j % chunks wraps)
+          const uint32_t half = (uint32_t)((lane >> 3) & 1);
+          const uint32_t b_addr = hb_addr + (uint32_t)((u * 2 + cur) * UB + (lane & 7) * cpc);
+          const uint32_t b_in = b_addr + half * 16u, b_wrap = b_addr + half * (uint32_t)(BG * cpc - (chunks - 1) * 16);
+#pragma unroll
+          for (int s = 0; s < KS; ++s) {
+            uint32_t w0, w1;
+            if (s < KR) {
+              w0 = wreg[2 * s];
+              w1 = wreg[2 * s + 1];
+            } else {
+              const uint2 w = wsm[(s - KR) * REC_THREADS + tid];
+              w0 = w.x;
+              w1 = w.y;
+            }
+            const uint32_t a0 = (w0 << 4) & 0xF0F0F0F0u, a1 = w0 & 0xF0F0F0F0u;
+            const uint32_t a2 = (w1 << 4) & 0xF0F0F0F0u, a3 = w1 & 0xF0F0F0F0u;
+            const uint32_t o0 = (uint32_t)(((2 * s) / chunks) * BG * cpc + ((2 * s) % chunks) * 16);
+            uint32_t b0, b1;
+            ldmatrix_x2(((2 * s) % chunks == chunks - 1 ? b_wrap : b_in) + o0, b0, b1);
+            mma_s8(acc[s & 1], a0, a1, a2, a3, b0, b1);
+          }
+        }
+        // the four gates of my item: mine are rows g (gate e) and g + 8 (gate 2 + e) at column e of the
+        // pair; the other two come from lane ^ 4, which needs my values at the other column
+        int hh[4];
+        {
+          const int v0 = acc[0][0] + acc[1][0], v1 = acc[0][1] + acc[1][1];
+          const int v2 = acc[0][2] + acc[1][2], v3 = acc[0][3] + acc[1][3];
+          const int r0 = __shfl_xor_sync(0xffffffffu, e ? v0 : v1, 4);
+          const int r1 = __shfl_xor_sync(0xffffffffu, e ? v2 : v3, 4);
+          const int m0 = e ? v1 : v0, m1 = e ? v3 : v2;
+          hh[0] = (e ? r0 : m0) >> 4;     // the operand was 16 x code
+          hh[1] = (e ? m0 : r0) >> 4;
+          hh[2] = (e ? r1 : m1) >> 4;
+          hh[3] = (e ? m1 : r1) >> 4;
+        }
+        cp_async_wait<NU>();              // this thread's accumulators of the present step have landed
+        int q = 0, q2 = 0;
+        if (live[u]) {
+          const int4 pre = pre_s[(cur * NU + u) * REC_THREADS + tid];
+          const float4 s_ih = cst[cl], s_hh = cst[cpc + cl], bb = cst[2 * cpc + cl];
+          const float pi = __fmaf_rn((float)hh[0], s_hh.x, __fmaf_rn((float)pre.x, s_ih.x, bb.x));
+          const float pf = __fmaf_rn((float)hh[1], s_hh.y, __fmaf_rn((float)pre.y, s_ih.y, bb.y));
+          const float pg = __fmaf_rn((float)hh[2], s_hh.z, __fmaf_rn((float)pre.z, s_ih.z, bb.z));
+          const float po = __fmaf_rn((float)hh[3], s_hh.w, __fmaf_rn((float)pre.w, s_ih.w, bb.w));
+          float hval;
+          cell_fixed(pi, pf, pg, po, c_state[u], c_state[u], hval);
+          q = quantize1(hval, a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
+          q2 = quantize1(hval, a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
+        }
+        // staged by step parity: the engine may still be reading the other buffer (the previous step's
+        // block), but not this one (its block of two steps ago has been received by every CTA)
+        stage[((cur * NU + u) * BG + n) * cpc + cl] = (int8_t)q;
+        stage_y[((cur * NU + u) * BG + n) * cpc + cl] = (int8_t)q2;
+        if (step == T - 1 && D.hq_n) {   // final recurrent codes, two cells per byte: the even cell's lane writes
+          const int qn = __shfl_down_sync(0xffffffffu, q, 8);
+          if (live[u] && (cl & 1) == 0)
+            D.hq_n[(size_t)b * (H >> 1) + (cell >> 1)] = (uint8_t)((q & 0xF) | ((qn & 0xF) << 4));
+        }
+        fence_proxy_async();   // the staged codes are read by the bulk-copy engine
+        // One warp, a different one every time, waits until all threads have staged their codes (the
+        // others only arrive at the named barrier and go on with the next unit), sends the staged
+        // block [BG][cpc] to [source = this CTA] of every CTA's buffer for the next step (one bulk copy
+        // per destination, counted on the receiver's mbarrier), and writes the CTA's share of the
+        // layer output: 16 cells per lane and pass, packed when 4 bit
+        if (warp != (step * NU + u) % CW) {
+          named_bar_arrive(1 + u * 2 + cur, REC4_THREADS);
+        } else {
+          named_bar_sync(1 + u * 2 + cur, REC4_THREADS);
+          if (lane < REC_CLUSTER) {
+            const uint32_t r = (uint32_t)lane;
+            bulk_copy_to_cluster(map_to_rank(hb_addr + (uint32_t)((u * 2 + nxt) * UB + (int)rank * BG * cpc), r),
+                                 smem_u32(stage + (size_t)(cur * NU + u) * BG * cpc), (uint32_t)(BG * cpc),
+                                 map_to_rank(full_addr + (uint32_t)((u * 2 + nxt) * 8), r));
+          }
+          for (int i = lane; i < BG * chunks; i += 32) {
+            const int ch = i % chunks, bl = i / chunks;
+            const int by = (grp0 + u) * BG + bl;
+            if (by >= B) continue;
+            const uint4 v = *reinterpret_cast<const uint4*>(stage_y + ((cur * NU + u) * BG + bl) * cpc + ch * 16);
+            uint8_t* y = D.yq + ((size_t)t * B + by) * a.yq_ld;
+            const int c0 = (int)rank * cpc + ch * 16;
+            if (y4) {
+              // bytes (c, c+1) -> one byte: low nibble c, high nibble c+1
+              auto pk = [](uint32_t w) -> uint32_t {
+                const uint32_t m = (w & 0x000F000Fu) | ((w >> 4) & 0x00F000F0u);   // bytes 0 and 2 hold the pairs
+                return (m & 0xFFu) | ((m >> 8) & 0xFF00u);
+              };
+              *reinterpret_cast<uint2*>(y + (c0 >> 1)) = make_uint2(pk(v.x) | (pk(v.y) << 16), pk(v.z) | (pk(v.w) << 16));
+            } else {
+              *reinterpret_cast<uint4*>(y + c0) = v;
+            }
+          }
+        }
+      }
+    }
+  }
+  cp_async_wait<0>();
+  // the codes sent in the last step are still on their way into this CTA: wait for them (bounded), so
+  // that nobody leaves while copies into its shared memory are in flight
+  if (T > 0) {
+#pragma unroll
+    for (int u = 0; u < NU; ++u) {
+      const uint32_t parity = (uint32_t)(((T - 1) >> 1) & 1);
+      for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(&full[u * 2 + (T & 1)], parity)) break;
+        if ((i & 255u) == 255u && *dead) break;
+      }
+    }
+  }
+  __syncthreads();
+  cluster_barrier();
+  // final states
+#pragma unroll
+  for (int u = 0; u < NU; ++u) {
+    const int b = (grp0 + u) * BG + n;
+    if (live[u] && D.c_n) D.c_n[(size_t)b * H + cell] = c_state[u];
+  }
+}
+
 constexpr size_t REC_SMEM_MAX = 232448 - 128;   // 227 KB per CTA on sm_100, minus a margin
 
 size_t enc_recurrent_smem(int H, int BG) {
@@ -325,7 +662,44 @@ bool enc_recurrent_supported(int H, int B, int dirs) {
   return enc_recurrent_smem(H, 8) <= REC_SMEM_MAX;
 }
 
+static size_t enc_recurrent_w4_smem(int H, int NU) {
+  const int cpc = H / REC_CLUSTER;
+  return (size_t)NU * 2 * REC_BG * H + (size_t)2 * NU * REC_THREADS * sizeof(int4) +
+         (size_t)3 * cpc * sizeof(float4) + (size_t)4 * NU * REC_BG * cpc + (size_t)NU * 2 * sizeof(uint64_t) + 32 + (size_t)4 * REC_THREADS * sizeof(uint2);
+}
+
+template <int NU, int KS>
+static cudaError_t rec_w4_launch(const EncRecArgs& a, cudaStream_t s) {
+  const size_t smem = enc_recurrent_w4_smem(32 * KS, NU);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_enc_recurrent_w4<NU, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  k_enc_recurrent_w4<NU, KS><<<(unsigned)(a.dirs * a.n_groups * REC_CLUSTER), REC4_THREADS, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s) {
+  // 4-bit recurrent weights and hidden codes at 640 cells: the register-resident kernel, with as few
+  // units of 8 sequences per cluster as keeps all clusters resident at once
+  // (no per-sequence input scale and no accumulator dump: those take the general kernel)
+  if (a.w_bits == 4 && a.hid_act.bits == 4 && a.hid_act.is_signed && a.H == 640 && !a.x_scale_b &&
+      !a.d[0].dbg_ih) {
+    const int groups = (a.B + REC_BG - 1) / REC_BG, maxc = rec_max_clusters(a.H);
+    int nu = 1;
+    while (nu <= 4 && a.dirs * ((groups + nu - 1) / nu) > maxc) ++nu;
+    if (nu <= 4) {
+      a.n_groups = (groups + nu - 1) / nu;   // clusters per direction
+      timing_begin(s);
+      cudaError_t e = nu == 1 ? rec_w4_launch<1, 20>(a, s) : nu == 2 ? rec_w4_launch<2, 20>(a, s)
+                      : nu == 3 ? rec_w4_launch<3, 20>(a, s) : rec_w4_launch<4, 20>(a, s);
+      timing_end(s);
+      ++g_launches;
+      return e;
+    }
+  }
   const int BG = enc_recurrent_group(a.B, a.dirs, a.H);
   a.n_groups = (a.B + BG - 1) / BG;
   const size_t smem = enc_recurrent_smem(a.H, BG);

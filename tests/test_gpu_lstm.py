@@ -115,6 +115,13 @@ def layer_case(Bd, T, B, K, H, dirs, xb=4, hb=4, ob=None, seed=0, x_clip=3.0, ma
         alt = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), x_act), to_act(x_act), T, B, layers,
                                      to_act(out), want_dbg=True, tensor_cores=False)
         assert torch.equal(alt["acc_ih"], got["acc_ih"]) and torch.equal(alt["yq"], got["yq"])
+    # the same call without the accumulator dumps (at 640 cells and 4 bits this takes the kernel that
+    # keeps the recurrent weights in registers)
+    lean = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), x_act), to_act(x_act), T, B, layers,
+                                  to_act(out), want_state=True)
+    assert Bd.q4_poll_status(lean["workspace"]) == 0
+    for k in ("yq", "hq_n", "c_n"):
+        assert torch.equal(lean[k], got[k]), k
     yq = gpu_codes(got["yq"], dirs * H, out).reshape(T, B, dirs * H)
     # free-running over the whole sequence and still bit-exact: codes, accumulators, states
     np.testing.assert_array_equal(yq, ref["yq"])
