@@ -316,6 +316,8 @@ __device__ __forceinline__ void named_bar_arrive(int id, int count) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
+__host__ __device__ constexpr int rec_w4_ksmem(int nu) { return nu <= 2 ? 6 : 8; }
+
 template <int NU, int KS>
 __global__ void __cluster_dims__(REC_CLUSTER, 1, 1) __launch_bounds__(REC4_THREADS, 1)
 k_enc_recurrent_w4(const EncRecArgs a) {
@@ -327,9 +329,9 @@ k_enc_recurrent_w4(const EncRecArgs a) {
   constexpr int chunks = cpc >> 4;          // 16-byte chunks of a sequence's new codes per CTA
   constexpr int UB = BG * H;                // bytes of one unit's hidden codes
   constexpr int CW = REC_THREADS / 32;      // warps
-  constexpr int KR = KS - 4;                // k-steps whose weight fragments stay in registers; the last
-                                            // four come from shared memory (8 bytes per thread and k-step),
-                                            // which leaves the cell update enough registers
+  constexpr int KR = KS - rec_w4_ksmem(NU);   // k-steps whose weight fragments stay in registers; the last
+                                              // six or eight come from shared memory (8 bytes per thread and
+                                              // k-step), which leaves the cell update enough registers: no spills
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_rank();
   const int cid = blockIdx.x / REC_CLUSTER;
@@ -665,7 +667,7 @@ bool enc_recurrent_supported(int H, int B, int dirs) {
 static size_t enc_recurrent_w4_smem(int H, int NU) {
   const int cpc = H / REC_CLUSTER;
   return (size_t)NU * 2 * REC_BG * H + (size_t)2 * NU * REC_THREADS * sizeof(int4) +
-         (size_t)3 * cpc * sizeof(float4) + (size_t)4 * NU * REC_BG * cpc + (size_t)NU * 2 * sizeof(uint64_t) + 32 + (size_t)4 * REC_THREADS * sizeof(uint2);
+         (size_t)3 * cpc * sizeof(float4) + (size_t)4 * NU * REC_BG * cpc + (size_t)NU * 2 * sizeof(uint64_t) + 32 + (size_t)rec_w4_ksmem(NU) * REC_THREADS * sizeof(uint2);
 }
 
 template <int NU, int KS>
