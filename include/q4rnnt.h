@@ -12,15 +12,19 @@
  *   codes, 4 bit : two per byte, element 2i in bits 0-3, element 2i+1 in bits
  *                  4-7; two's complement when signed, plain when unsigned.
  *   codes, 8 bit : one per byte, two's complement (signed only).
- *   rows         : row-major, k_pad elements per row, k_pad a multiple of 32,
- *                  elements k..k_pad-1 hold the code of the real value 0 (0 for
- *                  signed codes, the zero point for unsigned ones).
+ *   codes, 2 bit : weights only (the 2-bit weight rows of the paper's Table 1): four per
+ *                  byte, element 4i+j in bits 2j, 2j+1, two's complement (-2..1).
+ *   rows         : row-major, k_pad elements per row, k_pad a multiple of 32 (of 64 for
+ *                  2-bit weights: rows are multiples of 16 bytes), elements k..k_pad-1 hold
+ *                  the code of the real value 0 (0 for signed codes, the zero point for
+ *                  unsigned ones).
  *   weights      : symmetric signed codes with one fp32 scale per output row
  *                  (W[j,k] ~ scale[j] * q[j,k]); biases and LSTM cell states
  *                  are fp32 and never quantized (paper Section 3.2).
  *   LSTM gates   : the 4H rows of w_ih / w_hh / bias are ordered i, f, g, o.
- * A matrix product needs its weight and its input activation at the same bit
- * width (both 4 or both 8).
+ * Weights may be stored at 2, 4 or 8 bits and activations at 4 or 8 bits in any combination
+ * (the paper's mixed assignments: 8-bit first layer, 2-bit weights with 4-bit activations);
+ * a weight matrix and the activation rows it multiplies share k_pad.
  */
 #ifndef Q4RNNT_H_
 #define Q4RNNT_H_
@@ -36,7 +40,7 @@ extern "C" {
 #define Q4_ERR_NULL (-1)        /* a required pointer is NULL */
 #define Q4_ERR_DIM (-2)         /* a size is non-positive or inconsistent */
 #define Q4_ERR_ALIGN (-3)       /* a pointer or k_pad breaks the alignment rule */
-#define Q4_ERR_BITS (-4)        /* bit width not 4/8, or operands disagree */
+#define Q4_ERR_BITS (-4)        /* bit width not supported (weights 2/4/8, activations 4/8) */
 #define Q4_ERR_WORKSPACE (-5)   /* workspace smaller than q4_workspace_bytes says */
 #define Q4_ERR_UNSUPPORTED (-6) /* valid request this build does not implement */
 #define Q4_ERR_CUDA (-7)        /* a CUDA runtime call failed (launch error) */
@@ -76,6 +80,7 @@ int q4_act_asymmetric(float lo, float hi, int32_t bits, q4_act* out);
  *          boundary per utterance).  The per-group scale is written to group_scale_out
  *          [n_groups] (device); an all-zero group gets boundary 1.  act->bits selects the width.
  *   mode 2 (weights): symmetric, row r uses scale per_row_scale[r] (device), act->bits wide.
+ *   Modes 1 and 2 also accept act->bits = 2 (weight storage; k_pad a multiple of 64).
  * x_is_fp16: 1 = half precision input, 0 = fp32.  x rows are dense (k values per row).
  */
 int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k, int32_t k_pad,

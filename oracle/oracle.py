@@ -168,6 +168,23 @@ def unpack4(b: np.ndarray, k: int, is_signed: bool) -> np.ndarray:
     return q
 
 
+def pack2(q: np.ndarray, k_pad: int) -> np.ndarray:
+    """2-bit codes (-2..1) -> four per byte."""
+    q = _c(q, np.int16)
+    rows, k = q.shape
+    out = np.empty((rows, k_pad // 4), dtype=np.uint8)
+    lib().orc_pack2(_p(q), C.c_int64(rows), C.c_int64(k), C.c_int64(k_pad), _p(out))
+    return out
+
+
+def unpack2(b: np.ndarray, k: int) -> np.ndarray:
+    b = _c(b, np.uint8)
+    rows, kp4 = b.shape
+    q = np.empty((rows, k), dtype=np.int16)
+    lib().orc_unpack2(_p(b), C.c_int64(rows), C.c_int64(k), C.c_int64(kp4 * 4), _p(q))
+    return q
+
+
 def activations(x: np.ndarray):
     """The oracle's fp32 2^x, sigmoid and tanh on an array."""
     x = _c(x, np.float32)

@@ -158,6 +158,29 @@ void orc_unpack4(const uint8_t* in, int64_t rows, int64_t k, int64_t k_pad, int3
     }
 }
 
+// Storage format for 2-bit weight codes (the 2-bit weight rows of Table 1): four per byte,
+// element 4i+j in bits 2j, 2j+1, two's complement (codes -2..1), rows padded with zeros.
+void orc_pack2(const int16_t* q, int64_t rows, int64_t k, int64_t k_pad, uint8_t* out) {
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t i = 0; i < k_pad; i += 4) {
+      uint32_t b = 0;
+      for (int64_t j = 0; j < 4; ++j) {
+        const int32_t v = i + j < k ? q[r * k + i + j] : 0;
+        b |= (uint32_t)(v & 0x3) << (2 * j);
+      }
+      out[r * (k_pad / 4) + i / 4] = (uint8_t)b;
+    }
+}
+
+void orc_unpack2(const uint8_t* in, int64_t rows, int64_t k, int64_t k_pad, int16_t* q) {
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t i = 0; i < k; ++i) {
+      int32_t v = (in[r * (k_pad / 4) + i / 4] >> ((i & 3) * 2)) & 0x3;
+      if (v >= 2) v -= 4;
+      q[r * k + i] = (int16_t)v;
+    }
+}
+
 // ------------------------------------------------------------ integer MACs
 // acc[m, j] = sum_k W[j,k] * (xq[m,k] - z).  Weights are symmetric (no zero point).
 void orc_int_matmul(const int8_t* w, int32_t J, int32_t K, const int16_t* xq, int32_t zero_point,

@@ -121,6 +121,12 @@ def pad32(k: int) -> int:
     return (k + 31) // 32 * 32
 
 
+def pad_for(k: int, bits: int) -> int:
+    """Row length in elements: rows are multiples of 16 bytes, so 2-bit rows pad to 64."""
+    m = 64 if bits == 2 else 32
+    return (k + m - 1) // m * m
+
+
 def launch_count() -> int:
     return int(lib().q4_launch_count())
 
@@ -186,9 +192,9 @@ class DeviceMat:
         x = torch.from_numpy(np.ascontiguousarray(codes, dtype=np.float32)).to(device)
         ones = torch.ones(rows, dtype=torch.float32, device=device)
         a = Act(1.0, 1.0, 0, bits, 1)
-        q = quantize_pack_int4(x, a, mode=2, per_row_scale=ones)
+        q = quantize_pack_int4(x, a, mode=2, per_row_scale=ones, k_pad=pad_for(k, bits))
         s = torch.from_numpy(np.ascontiguousarray(scale, dtype=np.float32)).to(device)
-        return DeviceMat(q, s, rows, k, pad32(k), bits)
+        return DeviceMat(q, s, rows, k, pad_for(k, bits), bits)
 
     @staticmethod
     def from_float(w: np.ndarray, scale: np.ndarray, bits: int, device="cuda") -> "DeviceMat":
@@ -197,7 +203,8 @@ class DeviceMat:
         x = torch.from_numpy(np.ascontiguousarray(w, dtype=np.float32)).to(device)
         s = torch.from_numpy(np.ascontiguousarray(scale, dtype=np.float32)).to(device)
         a = Act(1.0, 1.0, 0, bits, 1)
-        return DeviceMat(quantize_pack_int4(x, a, mode=2, per_row_scale=s), s, rows, k, pad32(k), bits)
+        return DeviceMat(quantize_pack_int4(x, a, mode=2, per_row_scale=s, k_pad=pad_for(k, bits)), s, rows, k,
+                         pad_for(k, bits), bits)
 
     @staticmethod
     def from_float_max(w: np.ndarray, bits: int, device="cuda") -> "DeviceMat":
@@ -206,8 +213,8 @@ class DeviceMat:
         gets 1): mode 1 with one group per row; the row scales come back from the device."""
         rows, k = w.shape
         x = torch.from_numpy(np.ascontiguousarray(w, dtype=np.float32)).to(device)
-        q, s = quantize_pack_int4(x, Act(1.0, 1.0, 0, bits, 1), mode=1, n_groups=rows)
-        return DeviceMat(q, s, rows, k, pad32(k), bits)
+        q, s = quantize_pack_int4(x, Act(1.0, 1.0, 0, bits, 1), mode=1, n_groups=rows, k_pad=pad_for(k, bits))
+        return DeviceMat(q, s, rows, k, pad_for(k, bits), bits)
 
     def c(self) -> Mat:
         return Mat(self.q.data_ptr(), self.scale.data_ptr(), self.rows, self.k, self.k_pad, self.bits)
@@ -388,10 +395,11 @@ class Encoder:
         T, B, F = features.shape
         x2 = features.reshape(T * B, F)
         x_scale_b = None
+        kp = self.layers[0][0].w_ih.k_pad          # rows padded like the first layer's weight rows
         if self.in_max:
-            xq, x_scale_b = quantize_pack_int4(x2, self.in_act, mode=1, n_groups=B)
+            xq, x_scale_b = quantize_pack_int4(x2, self.in_act, mode=1, n_groups=B, k_pad=kp)
         else:
-            xq = quantize_pack_int4(x2, self.in_act)
+            xq = quantize_pack_int4(x2, self.in_act, k_pad=kp)
         x_act = self.in_act
         H = self.layers[0][0].H
         kmax = max(dirs[0].w_ih.k_pad for dirs in self.layers)
@@ -415,8 +423,8 @@ class DeviceLm:
     def __init__(self, m, device="cuda"):
         self.emb_act = q4_act_asymmetric(m.emb_lo, m.emb_hi, 4)
         emb = torch.from_numpy(np.ascontiguousarray(m.emb, dtype=np.float32)).to(device)
-        self.emb_q = quantize_pack_int4(emb, self.emb_act)           # table quantized once
         self.lstm = [DeviceLstm(l, device) for l in m.lstm]
+        self.emb_q = quantize_pack_int4(emb, self.emb_act, k_pad=self.lstm[0].w_ih.k_pad)   # table quantized once
         self.bott = DeviceLinear(m.bott, device)
         self.bott_act = q4_act_asymmetric(m.bott_lo, m.bott_hi, 4)
         self.out = DeviceLinear(m.out, device)
@@ -445,8 +453,8 @@ class Decoder:
         self.V, self.E = dw.pred.emb.shape
         self.pred_emb_act = q4_act_symmetric(dw.pred.emb_alpha, 4)
         emb = torch.from_numpy(np.ascontiguousarray(dw.pred.emb, dtype=np.float32)).to(device)
-        self.pred_emb_q = quantize_pack_int4(emb, self.pred_emb_act)
         self.pred_lstm = DeviceLstm(dw.pred.lstm, device)
+        self.pred_emb_q = quantize_pack_int4(emb, self.pred_emb_act, k_pad=self.pred_lstm.w_ih.k_pad)
         self.pred_proj = DeviceLinear(dw.pred.proj, device)
         self.D = self.pred_proj.w.rows
         self.z_act = q4_act_symmetric(1.0, dw.joint.z_bits)

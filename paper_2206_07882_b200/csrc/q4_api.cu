@@ -35,9 +35,9 @@ int check_act(const q4_act* a) {
 
 int check_mat(const q4_mat* m, int rows, int k_pad_expected) {
   if (!m || !m->q || !m->scale) return Q4_ERR_NULL;
-  if (m->bits != 4 && m->bits != 8) return Q4_ERR_BITS;
+  if (m->bits != 2 && m->bits != 4 && m->bits != 8) return Q4_ERR_BITS;
   if (m->rows <= 0 || m->k <= 0 || m->k_pad < m->k) return Q4_ERR_DIM;
-  if (m->k_pad % 32 != 0) return Q4_ERR_ALIGN;
+  if (m->k_pad % (m->bits == 2 ? 64 : 32) != 0) return Q4_ERR_ALIGN;   // rows are 16-byte multiples
   if (rows > 0 && m->rows != rows) return Q4_ERR_DIM;
   if (k_pad_expected > 0 && m->k_pad != k_pad_expected) return Q4_ERR_DIM;
   if (!aligned16(m->q) || (reinterpret_cast<uintptr_t>(m->scale) & 3u)) return Q4_ERR_ALIGN;
@@ -56,6 +56,8 @@ GemmArgs gemm_args(const void* x, long long x_stride, const int32_t* x_idx, cons
   g.x.idx = x_idx;
   g.x_signed = xa.is_signed;
   g.x_zp = xa.zero_point;
+  g.x_bits = xa.bits;
+  g.w_bits = w.bits;
   g.M = M;
   g.w = static_cast<const uint8_t*>(w.q);
   g.w_scale = w.scale;
@@ -185,8 +187,9 @@ int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k
   if (rows < 0 || k <= 0 || k_pad < k) return Q4_ERR_DIM;
   if (rows > 0 && (!x || !q_out)) return Q4_ERR_NULL;
   if (k_pad % 32 != 0 || !aligned16(q_out)) return Q4_ERR_ALIGN;
-  if (act->bits != 4 && act->bits != 8) return Q4_ERR_BITS;
   if (mode < 0 || mode > 2) return Q4_ERR_UNSUPPORTED;
+  if (act->bits != 4 && act->bits != 8 && !(act->bits == 2 && mode != 0)) return Q4_ERR_BITS;   // 2 bit: weights
+  if (act->bits == 2 && k_pad % 64 != 0) return Q4_ERR_ALIGN;
   q4_act a = *act;
   if (mode == 0) {
     Q4_CHECK(check_act(act));
@@ -210,13 +213,12 @@ int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_m
   Q4_CHECK(check_act(x_act));
   Q4_CHECK(check_mat(w, 0, 0));
   if (M < 0) return Q4_ERR_DIM;
-  if (w->bits != x_act->bits) return Q4_ERR_BITS;
   if (!aligned16(xq) || !aligned16(out)) return Q4_ERR_ALIGN;
-  GemmArgs g = gemm_args(xq, row_bytes(w->k_pad, w->bits), nullptr, *x_act, M, *w, bias, out,
+  GemmArgs g = gemm_args(xq, row_bytes(w->k_pad, x_act->bits), nullptr, *x_act, M, *w, bias, out,
                          w->rows, nullptr);
   g.dbg_acc = dbg_acc;
   TagScope tag(TAG_LINEAR);
-  Q4_TRY(launch_gemm(g, w->bits, EPI_F32, S(stream)));
+  Q4_TRY(launch_gemm(g, EPI_F32, S(stream)));
   return Q4_OK;
 }
 
@@ -231,7 +233,6 @@ static int check_lstm(const q4_mat* w_ih, const q4_mat* w_hh, const q4_act* x_ac
   const int H = w_ih->rows / 4;
   if (w_hh->k != H || w_hh->k_pad != H) return Q4_ERR_DIM;
   if (H % 32 != 0) return Q4_ERR_ALIGN;
-  if (w_ih->bits != x_act->bits || w_hh->bits != hid_act->bits) return Q4_ERR_BITS;
   *H_out = H;
   return Q4_OK;
 }
@@ -240,6 +241,9 @@ static void fill_lstm_weights(LstmArgs& a, const q4_mat& w_ih, const q4_mat& w_h
                               const q4_act& x_act, const q4_act& hid_act) {
   a.x_signed = x_act.is_signed;
   a.x_zp = x_act.zero_point;
+  a.x_bits = x_act.bits;
+  a.wih_bits = w_ih.bits;
+  a.whh_bits = w_hh.bits;
   a.kx_pad = w_ih.k_pad;
   a.x_scale = x_act.scale;
   a.w_ih = static_cast<const uint8_t*>(w_ih.q);
@@ -269,7 +273,7 @@ int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, co
   LstmArgs& a = args.d[0];
   fill_lstm_weights(a, *w_ih, *w_hh, bias, *x_act, *hid_act);
   a.x.base = static_cast<const uint8_t*>(xq);
-  a.x.stride = row_bytes(w_ih->k_pad, w_ih->bits);
+  a.x.stride = row_bytes(w_ih->k_pad, x_act->bits);
   a.x.idx = x_row_idx;
   a.hin.base = static_cast<const uint8_t*>(hq_in);
   a.hin.stride = row_bytes(H, hid_act->bits);
@@ -283,7 +287,7 @@ int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, co
   a.dbg_hh = dbg_acc_hh;
   a.dbg_stride = 4LL * H;
   TagScope tag(TAG_PRED_LSTM);
-  Q4_TRY(launch_lstm(args, 1, w_ih->bits, w_hh->bits, S(stream)));
+  Q4_TRY(launch_lstm(args, 1, S(stream)));
   return Q4_OK;
 }
 
@@ -335,7 +339,7 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
   const bool persistent = use_mma && enc_recurrent_supported(H, B, dirs);
   const long long hb = row_bytes(H, hid_act->bits);
   const long long yb = row_bytes(dirs * H, out_act->bits);
-  const long long xb = row_bytes(w_ih[0].k_pad, w_ih[0].bits);
+  const long long xb = row_bytes(w_ih[0].k_pad, x_act->bits);
 
   // time-parallel input projections for all frames
   if (use_mma) {
@@ -361,7 +365,7 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
     } else {
       GemmArgs g = gemm_args(xq, xb, nullptr, *x_act, (int)TB, w_ih[d], nullptr,
                              acc_ih + (size_t)d * TB * G, G, nullptr);
-      Q4_TRY(launch_gemm(g, w_ih[d].bits, EPI_I32, s));
+      Q4_TRY(launch_gemm(g, EPI_I32, s));
     }
   }
   if (persistent) {
@@ -426,7 +430,7 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
       a.dbg_stride = (long long)dirs * G;
     }
     TagScope tag(TAG_ENC_STEP);
-    Q4_TRY(launch_lstm(args, dirs, w_ih[0].bits, w_hh[0].bits, s));
+    Q4_TRY(launch_lstm(args, dirs, s));
   }
   for (int d = 0; d < dirs; ++d) {
     if (hq_n)
@@ -452,7 +456,6 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
   if (N < 0) return Q4_ERR_DIM;
   const int D = w_pred->rows, V = w_out->rows;
   if (w_out->k != D || w_out->k_pad != D || D % 32 != 0) return Q4_ERR_DIM;
-  if (w_pred->bits != p_act->bits || w_out->bits != z_act->bits) return Q4_ERR_BITS;
   if (!aligned16(pq) || !aligned16(workspace) || !aligned16(e)) return Q4_ERR_ALIGN;
   const int32_t dims[2] = {N, D};
   if (workspace_bytes < q4_workspace_bytes(Q4_WS_JOINT, dims, 2)) return Q4_ERR_WORKSPACE;
@@ -461,13 +464,13 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
   TagScope tag(TAG_JOINT);
   float* p = static_cast<float*>(workspace);
   uint8_t* zq = static_cast<uint8_t*>(workspace) + align_up((size_t)N * D * sizeof(float));
-  GemmArgs g1 = gemm_args(pq, row_bytes(w_pred->k_pad, w_pred->bits), nullptr, *p_act, N, *w_pred,
+  GemmArgs g1 = gemm_args(pq, row_bytes(w_pred->k_pad, p_act->bits), nullptr, *p_act, N, *w_pred,
                           b_pred, p, D, nullptr);
-  Q4_TRY(launch_gemm(g1, w_pred->bits, EPI_F32, s));
+  Q4_TRY(launch_gemm(g1, EPI_F32, s));
   Q4_TRY(launch_joint_z(e, frame_idx, nullptr, 1, 1, p, nullptr, N, D, *z_act, zq, nullptr, nullptr, s));
   GemmArgs g2 = gemm_args(zq, row_bytes(D, z_act->bits), nullptr, *z_act, N, *w_out, b_out, logp, V,
                           nullptr);
-  Q4_TRY(launch_gemm(g2, w_out->bits, EPI_F32, s));
+  Q4_TRY(launch_gemm(g2, EPI_F32, s));
   Q4_TRY(launch_logsoftmax(logp, logp, N, V, V, nullptr, s));
   return Q4_OK;
 }
@@ -623,7 +626,7 @@ static int advance_lstm(int tag_id, const q4_lstm& L, const void* x, long long x
   a.c_out = c;
   a.dbg_stride = 4LL * H;
   a.n_active = n_active;
-  Q4_TRY(launch_lstm(args, 1, L.w_ih.bits, L.w_hh.bits, s));
+  Q4_TRY(launch_lstm(args, 1, s));
   return Q4_OK;
 }
 
@@ -662,8 +665,6 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   Q4_CHECK(check_mat(&m.pred_proj.w, D, m.pred_lstm.w_hh.k_pad));
   Q4_CHECK(check_act(&m.z_act));
   Q4_CHECK(check_mat(&m.joint_out.w, V, D));
-  if (m.joint_out.w.bits != m.z_act.bits || m.pred_proj.w.bits != m.pred_lstm.hid_act.bits)
-    return Q4_ERR_BITS;
   const q4_lm* lms[2] = {&m.src, &m.tgt};
   for (const q4_lm* lm : lms) {
     Q4_CHECK(check_model_lstm(lm->lstm[0], lm->emb_act));
@@ -672,7 +673,6 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     Q4_CHECK(check_mat(&lm->bott.w, D, last.w_hh.k_pad));
     Q4_CHECK(check_act(&lm->bott_act));
     Q4_CHECK(check_mat(&lm->out.w, V, D));
-    if (lm->bott.w.bits != last.hid_act.bits || lm->out.w.bits != lm->bott_act.bits) return Q4_ERR_BITS;
   }
   if ((size_t)W * V * sizeof(float) > 200 * 1024) return Q4_ERR_UNSUPPORTED;
   const int32_t dims[4] = {B, W, V, D};
@@ -768,9 +768,9 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
         j.dst = dst;
         j.dst_stride = k_pad;
       };
-      add(m.pred_emb_q, row_bytes(Ep, m.pred_lstm.w_ih.bits), cst.adv_tok, m.pred_emb_act, Ep, xa8[0]);
-      add(m.src.emb_q, row_bytes(Ep, m.src.lstm[0].w_ih.bits), cst.adv_tok, m.src.emb_act, Ep, xa8[1]);
-      add(m.tgt.emb_q, row_bytes(Ep, m.tgt.lstm[0].w_ih.bits), cst.adv_tok, m.tgt.emb_act, Ep, xa8[2]);
+      add(m.pred_emb_q, row_bytes(Ep, m.pred_emb_act.bits), cst.adv_tok, m.pred_emb_act, Ep, xa8[0]);
+      add(m.src.emb_q, row_bytes(Ep, m.src.emb_act.bits), cst.adv_tok, m.src.emb_act, Ep, xa8[1]);
+      add(m.tgt.emb_q, row_bytes(Ep, m.tgt.emb_act.bits), cst.adv_tok, m.tgt.emb_act, Ep, xa8[2]);
       add(st.pred_hq, row_bytes(Hp, m.pred_lstm.hid_act.bits), cst.adv_src, m.pred_lstm.hid_act, Hp, ha8[0]);
       add(st.src_hq, row_bytes(Hs, m.src.lstm[0].hid_act.bits), cst.adv_src, m.src.lstm[0].hid_act, Hs, ha8[1]);
       add(st.tgt_hq[0], row_bytes(Ht, m.tgt.lstm[0].hid_act.bits), cst.adv_src, m.tgt.lstm[0].hid_act, Ht, ha8[2]);
@@ -947,13 +947,13 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     // 1. pending advances -------------------------------------------------------------
     if (nets) {  // prediction network: embedding row -> LSTM -> projection to D
       const q4_lstm& L = m.pred_lstm;
-      Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, L.w_ih.bits), cst.adv_tok,
+      Q4_CHECK(advance_lstm(TAG_PRED_LSTM, L, m.pred_emb_q, row_bytes(L.w_ih.k_pad, m.pred_emb_act.bits), cst.adv_tok,
                             m.pred_emb_act, st.pred_hq, st.pred_c, cst, N, n_active, s));
       GemmArgs g = gemm_args(st.pred_hq, row_bytes(L.w_hh.k_pad, L.hid_act.bits), cst.adv_dst,
                              L.hid_act, N, m.pred_proj.w, m.pred_proj.bias, st.pred_p, D, cst.adv_dst);
       g.n_active = n_active;
       TagScope tag(TAG_PRED_PROJ);
-      Q4_TRY(launch_gemm(g, m.pred_proj.w.bits, EPI_F32, s));
+      Q4_TRY(launch_gemm(g, EPI_F32, s));
     }
     for (int which = 0; which < 2 && nets; ++which) {
       const q4_lm& lm = *lms[which];
@@ -962,7 +962,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       float* lp = which == 0 ? st.src_lp : st.tgt_lp;
       uint8_t* bq = which == 0 ? bq_src : bq_tgt;
       const q4_lstm& L0 = lm.lstm[0];
-      Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, L0.w_ih.bits), cst.adv_tok,
+      Q4_CHECK(advance_lstm(which == 0 ? TAG_SRC_LSTM : TAG_TGT_L1, L0, lm.emb_q, row_bytes(L0.w_ih.k_pad, lm.emb_act.bits), cst.adv_tok,
                             lm.emb_act, hq0, c0, cst, N, n_active, s));
       const void* top = hq0;
       const q4_lstm* last = &L0;
@@ -980,11 +980,11 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
       gb.out_act = lm.bott_act;
       gb.n_active = n_active;
       TagScope tag(which == 0 ? TAG_SRC_HEAD : TAG_TGT_HEAD);
-      Q4_TRY(launch_gemm(gb, lm.bott.w.bits, EPI_QUANT, s));
+      Q4_TRY(launch_gemm(gb, EPI_QUANT, s));
       GemmArgs go = gemm_args(bq, row_bytes(D, lm.bott_act.bits), nullptr, lm.bott_act, N, lm.out.w,
                               lm.out.bias, lp, V, cst.adv_dst);
       go.n_active = n_active;
-      Q4_TRY(launch_gemm(go, lm.out.w.bits, EPI_F32, s));
+      Q4_TRY(launch_gemm(go, EPI_F32, s));
       Q4_TRY(launch_logsoftmax(lp, lp, N, V, V, cst.adv_dst, s, nullptr, n_active));
     }
 
@@ -993,7 +993,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, zq, nullptr, live, s));
     GemmArgs gj = gemm_args(zq, row_bytes(D, m.z_act.bits), live, m.z_act, N, m.joint_out.w,
                             m.joint_out.bias, logits, V, nullptr);
-    Q4_TRY(launch_gemm(gj, m.joint_out.w.bits, EPI_F32, s));
+    Q4_TRY(launch_gemm(gj, EPI_F32, s));
   }
 
   // 3. Eq. 1 proposals, merge, finished list, next beam --------------------------------

@@ -51,23 +51,54 @@ __device__ __forceinline__ void unpack8(uint32_t w, bool is_signed, uint32_t zp4
   }
 }
 
-// Stage one K chunk [k0, k0+KC) of a 64-row operand tile into shared memory as int8.
+// 16 packed 2-bit codes (two's complement, element i in bits 2i, 2i+1) -> four words of 4 int8,
+// natural element order.
+__device__ __forceinline__ void unpack16x2(uint32_t w, uint32_t (&o)[4]) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint32_t v = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int c = (int)((w >> (2 * (4 * j + e))) & 3u);
+      v |= (uint32_t)(((c ^ 2) - 2) & 0xFF) << (8 * e);
+    }
+    o[j] = v;
+  }
+}
+// 8 packed nibbles -> two words of 4 int8 in natural element order (elements 0..3, 4..7).
+__device__ __forceinline__ void unpack8_natural(uint32_t w, bool is_signed, uint32_t zp4, uint32_t& lo,
+                                                uint32_t& hi) {
+  uint32_t even, odd;
+  unpack8(w, is_signed, zp4, even, odd);
+  lo = __byte_perm(even, odd, 0x5140);   // e0 o0 e1 o1
+  hi = __byte_perm(even, odd, 0x7362);   // e2 o2 e3 o3
+}
+
+// Stage one K chunk [k0, k0+KC) of a 64-row operand tile into shared memory as int8, natural
+// element order whatever the storage width, so that operands of different widths can meet (2-bit
+// or 4-bit weights with 4- or 8-bit activations).
 // rowp[s] = first byte of the global row that belongs in shared row s (nullptr = zeros).
-// Thread t handles 32 elements of row t/4.  BITS = storage width of the codes.
-template <int BITS>
+// Thread t handles 32 elements of row t/4.  bits = storage width of the codes (2: signed only).
 __device__ __forceinline__ void stage_chunk(int8_t* smem, const uint8_t* const* rowp, int k0,
-                                            int k_pad, bool is_signed, uint32_t zp4, int tid) {
+                                            int k_pad, int bits, bool is_signed, uint32_t zp4, int tid) {
   const int s = tid >> 2, seg = tid & 3;
   const int k = k0 + 32 * seg;
   uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
   const uint8_t* p = rowp[s];
   if (p != nullptr && k < k_pad) {
-    if (BITS == 4) {
+    if (bits == 4) {
       const uint4 v = *reinterpret_cast<const uint4*>(p + (k >> 1));
-      unpack8(v.x, is_signed, zp4, o0.x, o0.y);
-      unpack8(v.y, is_signed, zp4, o0.z, o0.w);
-      unpack8(v.z, is_signed, zp4, o1.x, o1.y);
-      unpack8(v.w, is_signed, zp4, o1.z, o1.w);
+      unpack8_natural(v.x, is_signed, zp4, o0.x, o0.y);
+      unpack8_natural(v.y, is_signed, zp4, o0.z, o0.w);
+      unpack8_natural(v.z, is_signed, zp4, o1.x, o1.y);
+      unpack8_natural(v.w, is_signed, zp4, o1.z, o1.w);
+    } else if (bits == 2) {
+      const uint2 v = *reinterpret_cast<const uint2*>(p + (k >> 2));
+      uint32_t a[4], b[4];
+      unpack16x2(v.x, a);
+      unpack16x2(v.y, b);
+      o0 = make_uint4(a[0], a[1], a[2], a[3]);
+      o1 = make_uint4(b[0], b[1], b[2], b[3]);
     } else {
       o0 = *reinterpret_cast<const uint4*>(p + k);
       o1 = *reinterpret_cast<const uint4*>(p + k + 16);
@@ -164,6 +195,7 @@ enum { EPI_I32 = 0, EPI_F32 = 1, EPI_QUANT = 2 };
 struct GemmArgs {
   RowSrc x;                 // activation codes
   int32_t x_signed, x_zp, M;
+  int32_t x_bits, w_bits;   // storage widths of the activation and weight codes
   const uint8_t* w;         // weight codes [J, k_pad]
   const float* w_scale;
   const float* bias;
@@ -180,6 +212,7 @@ struct GemmArgs {
 struct LstmArgs {
   RowSrc x;                 // input codes (ignored when acc_pre is set)
   int32_t x_signed, x_zp, kx_pad;
+  int32_t x_bits, wih_bits, whh_bits;   // storage widths: input codes, input weights, recurrent weights
   float x_scale;
   const float* x_scale_vec; // optional per-row input scale, indexed n % x_scale_mod
   int32_t x_scale_mod;

@@ -4,8 +4,8 @@
 
 namespace q4 {
 
-cudaError_t launch_gemm(const GemmArgs& a, int bits, int epi, cudaStream_t s);
-cudaError_t launch_lstm(const LstmArgs2& a, int dirs, int x_bits, int h_bits, cudaStream_t s);
+cudaError_t launch_gemm(const GemmArgs& a, int epi, cudaStream_t s);
+cudaError_t launch_lstm(const LstmArgs2& a, int dirs, cudaStream_t s);
 cudaError_t launch_logsoftmax(const float* in, float* out, int rows, int V, long long stride,
                               const int32_t* idx, cudaStream_t s, float* second = nullptr,
                               const int32_t* n_active = nullptr);

@@ -53,7 +53,7 @@ int timing_count() { return g_timing.n; }
 // Thread (ty, tx) owns rows 4ty..4ty+3 and columns 4tx..4tx+3; column c is staged in
 // shared row c/4 + 16*(c%4) so that the 16-byte reads of a quarter warp hit distinct banks.
 // =====================================================================================
-template <int BITS, int EPI>
+template <int EPI>
 __global__ void __launch_bounds__(NT) k_gemm(const __grid_constant__ GemmArgs a) {
   __shared__ __align__(16) int8_t Xs[TILE * PITCH];
   __shared__ __align__(16) int8_t Ws[TILE * PITCH];
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(NT) k_gemm(const __grid_constant__ GemmArgs a)
     const int s = tid - TILE;
     const int c = ((s & 15) << 2) | (s >> 4);
     const int j = j0 + c;
-    wrow[s] = j < a.J ? a.w + (long long)j * (a.k_pad * BITS / 8) : nullptr;
+    wrow[s] = j < a.J ? a.w + (long long)j * (a.k_pad * a.w_bits / 8) : nullptr;
   }
   if (!__syncthreads_or(active)) return;
 
@@ -93,8 +93,8 @@ __global__ void __launch_bounds__(NT) k_gemm(const __grid_constant__ GemmArgs a)
     for (int j = 0; j < 4; ++j) acc[i][j] = 0;
 
   for (int k0 = 0; k0 < a.k_pad; k0 += KC) {
-    stage_chunk<BITS>(Xs, xrow, k0, a.k_pad, a.x_signed != 0, zp4, tid);
-    stage_chunk<BITS>(Ws, wrow, k0, a.k_pad, true, 0u, tid);
+    stage_chunk(Xs, xrow, k0, a.k_pad, a.x_bits, a.x_signed != 0, zp4, tid);
+    stage_chunk(Ws, wrow, k0, a.k_pad, a.w_bits, true, 0u, tid);
     __syncthreads();
 #pragma unroll
     for (int kk = 0; kk < KC; kk += 16) {
@@ -174,23 +174,20 @@ __global__ void __launch_bounds__(NT) k_gemm(const __grid_constant__ GemmArgs a)
   }
 }
 
-cudaError_t launch_gemm(const GemmArgs& a, int bits, int epi, cudaStream_t s) {
+cudaError_t launch_gemm(const GemmArgs& a, int epi, cudaStream_t s) {
   if (a.M <= 0 || a.J <= 0) return cudaSuccess;
   dim3 grid((a.M + TILE - 1) / TILE, (a.J + TILE - 1) / TILE);
-#define Q4_GEMM_CASE(B_, E_)                           \
-  if (bits == B_ && epi == E_) {                       \
+#define Q4_GEMM_CASE(E_)                               \
+  if (epi == E_) {                                     \
     timing_begin(s);                                   \
-    k_gemm<B_, E_><<<grid, NT, 0, s>>>(a);             \
+    k_gemm<E_><<<grid, NT, 0, s>>>(a);                 \
     timing_end(s);                                     \
     ++g_launches;                                      \
     return cudaGetLastError();                         \
   }
-  Q4_GEMM_CASE(4, EPI_I32)
-  Q4_GEMM_CASE(4, EPI_F32)
-  Q4_GEMM_CASE(4, EPI_QUANT)
-  Q4_GEMM_CASE(8, EPI_I32)
-  Q4_GEMM_CASE(8, EPI_F32)
-  Q4_GEMM_CASE(8, EPI_QUANT)
+  Q4_GEMM_CASE(EPI_I32)
+  Q4_GEMM_CASE(EPI_F32)
+  Q4_GEMM_CASE(EPI_QUANT)
 #undef Q4_GEMM_CASE
   return cudaErrorInvalidValue;
 }
@@ -201,7 +198,6 @@ cudaError_t launch_gemm(const GemmArgs& a, int bits, int epi, cudaStream_t s) {
 // update and the packing of two 4-bit codes into a byte stay in registers.
 // Cell c of the tile is staged in shared row gate*16 + (c%2)*8 + c/2.
 // =====================================================================================
-template <int BITS>
 __device__ __forceinline__ void lstm_mac(int (&acc)[2][2][4], const int8_t* Xs, const int8_t* Ws,
                                          int rp, int cp) {
 #pragma unroll
@@ -230,7 +226,6 @@ __device__ __forceinline__ void lstm_mac(int (&acc)[2][2][4], const int8_t* Xs, 
   }
 }
 
-template <int XB, int HB>
 __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 args) {
   const LstmArgs& a = args.d[blockIdx.z];
   __shared__ __align__(16) int8_t Xs[TILE * PITCH];
@@ -264,7 +259,7 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
   } else if (tid < 2 * TILE) {
     const int s = tid - TILE, g = s >> 4, q = s & 15;
     const int cell = c0 + (((q & 7) << 1) | (q >> 3));
-    wrow[s] = cell < H ? a.w_ih + (long long)(g * H + cell) * (a.kx_pad * XB / 8) : nullptr;
+    wrow[s] = cell < H ? a.w_ih + (long long)(g * H + cell) * (a.kx_pad * a.wih_bits / 8) : nullptr;
   }
   if (!__syncthreads_or(active)) return;
 
@@ -297,10 +292,10 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
   } else {
     const uint32_t zp4 = (uint32_t)a.x_zp * 0x01010101u;
     for (int k0 = 0; k0 < a.kx_pad; k0 += KC) {
-      stage_chunk<XB>(Xs, xrow, k0, a.kx_pad, a.x_signed != 0, zp4, tid);
-      stage_chunk<XB>(Ws, wrow, k0, a.kx_pad, true, 0u, tid);
+      stage_chunk(Xs, xrow, k0, a.kx_pad, a.x_bits, a.x_signed != 0, zp4, tid);
+      stage_chunk(Ws, wrow, k0, a.kx_pad, a.wih_bits, true, 0u, tid);
       __syncthreads();
-      lstm_mac<XB>(acc, Xs, Ws, rp, cp);
+      lstm_mac(acc, Xs, Ws, rp, cp);
       __syncthreads();
     }
   }
@@ -328,14 +323,14 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
   } else if (tid < 2 * TILE) {
     const int s = tid - TILE, g = s >> 4, q = s & 15;
     const int cell = c0 + (((q & 7) << 1) | (q >> 3));
-    wrow[s] = cell < H ? a.w_hh + (long long)(g * H + cell) * (a.kh_pad * HB / 8) : nullptr;
+    wrow[s] = cell < H ? a.w_hh + (long long)(g * H + cell) * (a.kh_pad * a.whh_bits / 8) : nullptr;
   }
   __syncthreads();
   for (int k0 = 0; k0 < a.kh_pad; k0 += KC) {
-    stage_chunk<HB>(Xs, xrow, k0, a.kh_pad, true, 0u, tid);
-    stage_chunk<HB>(Ws, wrow, k0, a.kh_pad, true, 0u, tid);
+    stage_chunk(Xs, xrow, k0, a.kh_pad, a.hid_act.bits, true, 0u, tid);
+    stage_chunk(Ws, wrow, k0, a.kh_pad, a.whh_bits, true, 0u, tid);
     __syncthreads();
-    lstm_mac<HB>(acc, Xs, Ws, rp, cp);
+    lstm_mac(acc, Xs, Ws, rp, cp);
     __syncthreads();
   }
 
@@ -385,24 +380,15 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
   }
 }
 
-cudaError_t launch_lstm(const LstmArgs2& a, int dirs, int x_bits, int h_bits, cudaStream_t s) {
+cudaError_t launch_lstm(const LstmArgs2& a, int dirs, cudaStream_t s) {
   const LstmArgs& a0 = a.d[0];
   if (a0.N <= 0) return cudaSuccess;
   dim3 grid((a0.N + TILE - 1) / TILE, (a0.H + 15) / 16, dirs);
-#define Q4_LSTM_CASE(X_, H_)                    \
-  if (x_bits == X_ && h_bits == H_) {           \
-    timing_begin(s);                            \
-    k_lstm<X_, H_><<<grid, NT, 0, s>>>(a);      \
-    timing_end(s);                              \
-    ++g_launches;                               \
-    return cudaGetLastError();                  \
-  }
-  Q4_LSTM_CASE(4, 4)
-  Q4_LSTM_CASE(4, 8)
-  Q4_LSTM_CASE(8, 4)
-  Q4_LSTM_CASE(8, 8)
-#undef Q4_LSTM_CASE
-  return cudaErrorInvalidValue;
+  timing_begin(s);
+  k_lstm<<<grid, NT, 0, s>>>(a);
+  timing_end(s);
+  ++g_launches;
+  return cudaGetLastError();
 }
 
 // =====================================================================================
@@ -545,6 +531,11 @@ __global__ void __launch_bounds__(256) k_quantize(const void* x, long long rows,
 #pragma unroll
     for (int j = 0; j < 8; ++j) w |= (uint32_t)(q[j] & 0xF) << (4 * j);
     *reinterpret_cast<uint32_t*>(out + r * (k_pad >> 1) + (kb >> 1)) = w;
+  } else if (a.bits == 2) {   // weights only: four codes per byte, element i in bits 2i, 2i+1
+    uint32_t w = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w |= (uint32_t)(q[j] & 0x3) << (2 * j);
+    *reinterpret_cast<uint16_t*>(out + r * (k_pad >> 2) + (kb >> 2)) = (uint16_t)w;
   } else {
     uint2 w = make_uint2(0, 0);
 #pragma unroll

@@ -187,6 +187,16 @@ __global__ void __launch_bounds__(256) k_prepare_w(const uint8_t* src, int bits,
       hi |= (uint32_t)(c & 0xFF) << (8 * e);
     }
     o = make_uint2(lo, hi);
+  } else if (bits == 2) {   // four codes per byte, element i in bits 2i, 2i+1 of the 16-bit group
+    const uint32_t w = *reinterpret_cast<const uint16_t*>(src + (long long)r * (k_pad >> 2) + (k >> 2));
+    uint32_t lo = 0, hi = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int a = (int)(((w >> (2 * e)) & 3u) ^ 2u) - 2, c = (int)(((w >> (2 * (e + 4))) & 3u) ^ 2u) - 2;
+      lo |= (uint32_t)(a & 0xFF) << (8 * e);
+      hi |= (uint32_t)(c & 0xFF) << (8 * e);
+    }
+    o = make_uint2(lo, hi);
   } else {
     o = *reinterpret_cast<const uint2*>(src + (long long)r * k_pad + k);
   }

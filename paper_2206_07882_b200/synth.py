@@ -160,6 +160,9 @@ def _qmat(st: Stream, name: str, rows: int, k: int, bits: int = 4) -> QMat:
     if bits == 8:
         # keep the dequantized weight range of the 4-bit layers (same alpha)
         scale = (scale * np.float32(7.0 / 127.0)).astype(np.float32)
+    if bits == 2:
+        # codes -2..1 with the same boundary: one step is the whole boundary
+        scale = (scale * np.float32(7.0)).astype(np.float32)
     return QMat(codes, scale, bits)
 
 
@@ -201,7 +204,7 @@ def single_layer(seed: int = 0, T: int = 50, B: int = 4, K: int = 64, H: int = 1
 
 def encoder(seed: int = 1, T: int = 500, B: int = 32, F: int = 240, H: int = 640, L: int = 6,
             D: int = 256, first_layer_bits: int = 4, in_max: bool = False,
-            with_proj: bool = True, features: bool = True):
+            with_proj: bool = True, features: bool = True, w_bits: int = 4, proj_bits: int = 4):
     """Bidirectional LSTM encoder.  Features fp16 ~ N(0,1); input clip U(2.5,3.5);
     per-layer hidden boundary U(.9,1.0) (the paper observes MAX boundaries of LSTM
     outputs in [0.9,1], Section 3.2); biases N(0,.1)."""
@@ -215,9 +218,11 @@ def encoder(seed: int = 1, T: int = 500, B: int = 32, F: int = 240, H: int = 640
     for l in range(L):
         k = F if l == 0 else 2 * H
         bits = first_layer_bits if l == 0 else 4
-        layers.append([_lstm(st, f"enc.l{l}.d{d}", k, H, bits, 0.1, float(alphas[l]), bits)
+        # w_bits < 4: weight codes stored narrower than the activation codes (Table 1's 2/4 rows)
+        wb = bits if bits == 8 else w_bits
+        layers.append([_lstm(st, f"enc.l{l}.d{d}", k, H, wb, 0.1, float(alphas[l]), bits)
                        for d in range(2)])
-    proj = _linear(st, "enc.proj", D, 2 * H) if with_proj else None
+    proj = _linear(st, "enc.proj", D, 2 * H, proj_bits) if with_proj else None
     out["enc"] = EncoderW(layers, in_clip, first_layer_bits, in_max, proj)
     out.update(T=T, B=B, F=F, H=H, L=L, D=D)
     return out
@@ -240,14 +245,15 @@ def _lm(st: Stream, name: str, V: int, E: int, H: int, n_layers: int, D: int) ->
 def decoder(seed: int = 3, V: int = 1024, E: int = 256, Hp: int = 1024, D: int = 256,
             Hs: int = 1024, Ht: int = 2048, tgt_layers: int = 2, out_bits: int = 4,
             W: int = 16, U_max: int = 150, lambda_t: float = 0.5, lambda_s: float = 0.3,
-            rho: float = 0.2) -> DecoderW:
+            rho: float = 0.2, rnnt_w_bits: int = 4, proj_bits: int = 4) -> DecoderW:
     """Prediction network, joint network and the two fusion LMs.  Embeddings
     N(0,.5); prediction-input boundary 1.25 and hidden boundary 1 (Section 3.2);
     learned LM input boundaries stand-ins alpha- ~ -U(1,2), alpha+ ~ U(1,2)."""
     st = Stream(seed)
     pred = PredW(st.normal("pred.emb", (V, E), 0.0, 0.5).astype(np.float32), 1.25,
-                 _lstm(st, "pred.lstm", E, Hp, 4, 0.1, 1.0), _linear(st, "pred.proj", D, Hp))
-    joint = JointW(_linear(st, "joint.out", V, D, out_bits), out_bits)
+                 _lstm(st, "pred.lstm", E, Hp, rnnt_w_bits, 0.1, 1.0, 4),
+                 _linear(st, "pred.proj", D, Hp, proj_bits if proj_bits != 4 else rnnt_w_bits))
+    joint = JointW(_linear(st, "joint.out", V, D, out_bits if out_bits != 4 else rnnt_w_bits), out_bits)
     src = _lm(st, "src", V, E, Hs, 1, D)
     tgt = _lm(st, "tgt", V, E, Ht, tgt_layers, D)
     return DecoderW(pred, joint, src, tgt, lambda_t, lambda_s, rho, W, U_max)

@@ -487,3 +487,16 @@ def test_config4_composed_full_widths_sampled_utterances(Bd):
     frac, tr = compare_search(dd, tokens.cpu().numpy(), lens.cpu().numpy(), scores.cpu().numpy(), ref,
                               utts, T, U, 16, min_same=1.0)
     assert tr == 1.0
+
+
+@pytest.mark.parametrize("tensor_cores", [True, False])
+def test_search_two_bit_rnnt_weights(Bd, tensor_cores):
+    # Table 1's 2/4 rows: prediction and joint network weights stored at 2 bits under 4-bit
+    # activations, LMs at 4 bits; 8 utterances x 16 slots, every beam of every iteration
+    dw = synth.decoder(seed=95, V=64, E=64, Hp=128, D=64, Hs=128, Ht=128, tgt_layers=2, U_max=6, W=16,
+                       rnnt_w_bits=2)
+    assert dw.pred.lstm.w_ih.bits == 2 and dw.joint.out.w.bits == 2 and dw.tgt.lstm[0].w_ih.bits == 4
+    e = synth.Stream(15).normal("e", (10, 8, 64)).astype(np.float32)
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e, tensor_cores=tensor_cores)
+    frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(8)), 10, 6, 16, min_same=1.0)
+    assert tr == 1.0

@@ -23,7 +23,7 @@ def step_case(Bd, lw, x_act, hid, xq, hq, c):
     want = O.lstm_step(L, xq, x_act, hq, c, hid)
     dl = Bd.DeviceLstm(lw)
     assert dl.hid_act.scale == hid.scale
-    got = Bd.qlstm_step(pack_codes(xq, x_act), to_act(x_act), pack_codes(hq, hid),
+    got = Bd.qlstm_step(pack_codes(xq, x_act, dl.w_ih.k_pad), to_act(x_act), pack_codes(hq, hid),
                         torch.from_numpy(c).cuda(), dl, want_dbg=True)
     H = c.shape[1]
     np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), want["acc_ih"])     # bit-exact
@@ -249,3 +249,39 @@ def test_encoder_shaped_step_against_plain_step(Bd, bits):
     c = st.normal("c", (N, 640)).astype(np.float32)
     n, near, moved = plain_step_case(Bd, lw, x_act, hid, xq, hq, c)
     print(f"{bits} bit: {n} codes, {near} near a rounding boundary, {moved} differ by one")
+
+
+# ------------------------------------------------------------------ 2-bit weights, mixed widths
+@pytest.mark.parametrize("N,K,H,wb,xb,hb", [(70, 200, 64, 2, 4, 4), (130, 256, 128, 2, 8, 4), (9, 64, 64, 4, 8, 8),
+                                             (33, 96, 64, 8, 4, 4), (5, 1280, 640, 2, 4, 4)])
+def test_step_weight_and_activation_widths_mix(Bd, N, K, H, wb, xb, hb):
+    # weights stored at 2, 4 or 8 bits under activations of 4 or 8 bits (Table 1's 2/4 rows; the
+    # 8-bit first layer): integer accumulators, cell state and codes exact
+    st = synth.Stream(300 + N)
+    lw = synth._lstm(st, "l", K, H, wb, bias_std=0.2, hid_alpha=0.95, hid_bits=hb)
+    x_act, hid = O.act_symmetric(3.0, xb), O.act_symmetric(0.95, hb)
+    xq = st.integers("xq", (N, K), x_act.lo(), x_act.hi()).astype(np.int16)
+    hq = st.integers("hq", (N, H), hid.lo() + 1, hid.hi()).astype(np.int16)
+    c = st.normal("c", (N, H)).astype(np.float32)
+    assert lw.w_ih.codes.min() == -(1 << (wb - 1)) and lw.w_ih.codes.max() == (1 << (wb - 1)) - 1
+    step_case(Bd, lw, x_act, hid, xq, hq, c)
+
+
+def test_layer_two_bit_weights(Bd):
+    # bidirectional layer with 2-bit weights under 4-bit activations, 160 rows: tensor-core input
+    # projection and persistent recurrence from int8 operand copies of the 2-bit codes
+    T, B, K, H = 20, 8, 128, 64
+    w = synth.single_layer(seed=21, T=T, B=B, K=K, H=H, bits=2, dirs=2)
+    for lw in w["layers"]:
+        lw.hid_bits = 4
+    x_act, hid = O.act_symmetric(3.0, 4), O.act_symmetric(1.0, 4)
+    xq = O.quantize(w["x"], x_act)
+    ref = O.lstm_layer(O.Lstm(w["layers"]), xq, x_act, hid, want=("c_n", "acc_ih"))
+    layers = [Bd.DeviceLstm(lw) for lw in w["layers"]]
+    assert layers[0].w_ih.bits == 2 and layers[0].w_ih.q.shape[1] == K // 4
+    for tc in (True, False):
+        got = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), x_act), to_act(x_act), T, B, layers,
+                                     want_state=True, want_dbg=True, tensor_cores=tc)
+        np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), ref["acc_ih"])
+        np.testing.assert_array_equal(gpu_codes(got["yq"], 2 * H, hid).reshape(T, B, 2 * H), ref["yq"])
+        np.testing.assert_array_equal(got["c_n"].cpu().numpy(), ref["c_n"])

@@ -116,3 +116,21 @@ def test_feature_prologue(Bd, B, T100, M):
     for b in range(B):
         want = O.features(mel[b]).astype(np.float16)
         np.testing.assert_array_equal(got[:, b, :], want)
+
+
+def test_weight_mode_two_bit_storage(Bd):
+    # symmetric per-row quantization to 2-bit codes, four per byte: byte-identical to the oracle's packing
+    st = synth.Stream(31)
+    rows, k = 37, 200
+    w = st.normal("w", (rows, k), 0, 1.0).astype(np.float32)
+    sc = st.uniform("s", (rows,), 0.5, 1.5).astype(np.float32)
+    dm = Bd.DeviceMat.from_float(w, sc, 2)
+    assert dm.k_pad == 256 and dm.q.shape == (rows, 64)
+    want = O.pack2(O.quantize_weights(w, sc, 2).astype(np.int16), 256)
+    np.testing.assert_array_equal(dm.q.cpu().numpy(), want)
+    # MAX boundary per row at 2 bits: the row's largest magnitude maps to code 1 (or -1 / -2 by sign)
+    dm2 = Bd.DeviceMat.from_float_max(w, 2)
+    amax = np.abs(w).max(1)
+    np.testing.assert_array_equal(dm2.scale.cpu().numpy(), amax.astype(np.float32))
+    want2 = O.pack2(O.quantize_weights(w, amax.astype(np.float32), 2).astype(np.int16), 256)
+    np.testing.assert_array_equal(dm2.q.cpu().numpy(), want2)

@@ -71,14 +71,14 @@ def test_argument_errors_are_reported_on_the_host(Bd):
     assert lib.quantize_pack_int4(fake, 0, C.c_int64(4), 32, 32, C.byref(ok), 2, 1, None, fake, None, None) == -1
     bad_bits = Bd.Act(1.0, 1.0, 0, 3, 1)
     assert lib.quantize_pack_int4(fake, 0, C.c_int64(4), 32, 32, C.byref(bad_bits), 0, 1, None, fake, None, None) == -4
-    # LSTM: mismatched bit widths, misaligned k_pad, aliasing
+    # LSTM: unsupported weight width, misaligned k_pad (2-bit rows need multiples of 64), aliasing
     w_ih = Bd.Mat(4096, 4096, 128, 64, 64, 4)
     w_hh = Bd.Mat(4096, 4096, 128, 32, 32, 4)
-    act8 = Bd.q4_act_symmetric(1.0, 8)
     args = lambda x_act, wi=w_ih, wh=w_hh, hin=fake, hout=C.c_void_p(8192): lib.qlstm_step(
         fake, C.byref(x_act), None, hin, fake, 4, C.byref(wi), C.byref(wh), None, C.byref(ok), hout,
         fake, None, None, None, None)
-    assert args(act8) == -4
+    assert args(ok, wi=Bd.Mat(4096, 4096, 128, 64, 64, 3)) == -4
+    assert args(ok, wi=Bd.Mat(4096, 4096, 128, 32, 32, 2)) == -3
     assert args(ok, wi=Bd.Mat(4096, 4096, 128, 60, 60, 4)) == -3
     assert args(ok, wh=Bd.Mat(4096, 4096, 128, 64, 64, 4)) == -2
     assert args(ok, hout=fake) == -6

@@ -190,3 +190,21 @@ def test_size_accounting_matches_paper():
     # packed bytes of a matrix = rows * k_pad * bits / 8 in the oracle's storage format
     q = np.zeros((10, 64), dtype=np.int16)
     assert O.pack4(q, 64).nbytes == 10 * 64 * 4 // 8
+
+
+def test_two_bit_weight_storage_by_hand_and_round_trip():
+    # four codes per byte, element 4i+j in bits 2j, 2j+1, two's complement: -2..1 -> 10, 11, 00, 01
+    q = np.array([[1, -1, 0, -2, -2, 1, 1, 0, 0, 0, -1]], dtype=np.int16)
+    b = O.pack2(q, 12)
+    #   byte 0: 1 | (-1&3)<<2 | 0<<4 | (-2&3)<<6 = 1 + 12 + 0 + 128 = 141
+    #   byte 1: (-2&3) | 1<<2 | 1<<4 | 0<<6 = 2 + 4 + 16 = 22
+    #   byte 2: 0 | 0 | (-1&3)<<4 | padding 0 = 48
+    assert b.tolist() == [[141, 22, 48]]
+    np.testing.assert_array_equal(O.unpack2(b, 11), q)
+    rng = np.random.default_rng(3)
+    q = rng.integers(-2, 2, (7, 130)).astype(np.int16)
+    np.testing.assert_array_equal(O.unpack2(O.pack2(q, 192), 130), q)
+    # the symmetric weight quantizer at 2 bits: step = boundary, codes clamp to -2..1
+    w = np.array([[0.0, 0.49, 0.51, 1.0, 1.6, -0.6, -1.4, -1.6, -9.0]], dtype=np.float32)
+    codes = O.quantize_weights(w, np.array([1.0], np.float32), 2)
+    assert codes.tolist() == [[0, 0, 1, 1, 1, -1, -1, -2, -2]]
