@@ -126,6 +126,9 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
  *   alias hq_in (every output cell reads the whole previous row).
  *   h_f32_out [N, H] (nullable) receives the fp32 cell output before quantization;
  *   dbg_acc_ih / dbg_acc_hh [N, 4H] int32 (nullable).
+ *   hq_out == NULL (then h_f32_out is required) leaves the cell output unquantized: the "Inner"
+ *   placement of Section 3.4, where every cell quantizes its two inputs on entry instead
+ *   (quantize_pack_int4 on x_t and on the previous real-valued cell output, then this call).
  */
 int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, const void* hq_in,
                const float* c_in, int32_t N, const q4_mat* w_ih, const q4_mat* w_hh,
@@ -344,6 +347,13 @@ int q4_poll_status(const int32_t* device_status, q4_stream stream);
  * benchmark reads to report its launch count). */
 int q4_version(void);
 int64_t q4_launch_count(void);
+/* Number of activation-quantizer applications enqueued so far (Section 3.4 counts them: T + T L
+ * per sequence with the quantizer at the cell outputs, 2 T L with quantizers at the cell inputs):
+ * +1 per quantize_pack_int4 call on activations (modes 0 and 1), +1 per qlstm_step with hq_out,
+ * +T*dirs per qlstm_layer_forward (twice that when out_act differs from hid_act), +1 per joint
+ * call, and the corresponding sum per beam step.  A call covers all rows it is given (a batch of
+ * sequences counts once).  reset != 0 sets the counter back to zero after reading it. */
+int64_t q4_quantizer_calls(int32_t reset);
 
 /* dr_fusion_beam_step launches consecutive kernels of one stream as programmatic dependents
  * (each kernel sets itself up while its predecessor drains and waits for the predecessor's

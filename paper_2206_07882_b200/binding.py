@@ -80,7 +80,7 @@ class BeamStateS(C.Structure):
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
-           "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_beam_select_exact_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static"]
+           "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_beam_select_exact_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static", "q4_quantizer_calls"]
 
 _lib = None
 
@@ -96,6 +96,7 @@ def lib() -> C.CDLL:
         _lib.q4_workspace_bytes.restype = C.c_size_t
         _lib.q4_launch_count.restype = C.c_int64
         _lib.q4_prepared_bytes.restype = C.c_size_t
+        _lib.q4_quantizer_calls.restype = C.c_int64
     return _lib
 
 
@@ -129,6 +130,11 @@ def pad_for(k: int, bits: int) -> int:
 
 def launch_count() -> int:
     return int(lib().q4_launch_count())
+
+
+def quantizer_calls(reset: bool = False) -> int:
+    """Activation-quantizer applications enqueued so far by the library (Section 3.4)."""
+    return int(lib().q4_quantizer_calls(C.c_int32(1 if reset else 0)))
 
 
 def dependent_launch_set(enabled: bool) -> bool:
@@ -306,9 +312,32 @@ def qlstm_step(xq: torch.Tensor, x_act: Act, hq_in: torch.Tensor, c_in: torch.Te
     wih, whh = layer.w_ih.c(), layer.w_hh.c()
     _chk(lib().qlstm_step(_p(xq), C.byref(x_act), _p(x_row_idx), _p(hq_in), _p(c_in), C.c_int32(N),
                           C.byref(wih), C.byref(whh), _p(layer.bias), C.byref(layer.hid_act),
-                          _p(r["hq"]), _p(r["c"]), _p(r.get("h")), _p(r.get("acc_ih")),
+                          _p(r.get("hq")), _p(r["c"]), _p(r.get("h")), _p(r.get("acc_ih")),
                           _p(r.get("acc_hh")), _stream()), "qlstm_step")
     return r
+
+
+def lstm_layer_inner(x: torch.Tensor, x_act: Act, layers: Sequence[DeviceLstm]) -> torch.Tensor:
+    """One layer under the Inner placement of the activation quantizers (Section 3.4): real-valued
+    x [T, B, K] in, real-valued cell outputs [T, B, dirs*H] out; every step of every direction
+    quantizes its two inputs on entry (two quantize_pack_int4 calls) and runs qlstm_step without
+    the output quantizer.  Marshalling only: a loop over library calls."""
+    _need_cuda()
+    T, B, K = x.shape
+    dirs, H = len(layers), layers[0].H
+    hid = layers[0].hid_act
+    out = torch.empty((T, B, dirs * H), dtype=torch.float32, device=x.device)
+    for d, L in enumerate(layers):
+        h = torch.zeros((B, H), dtype=torch.float32, device=x.device)
+        c = torch.zeros((B, H), dtype=torch.float32, device=x.device)
+        for s in range(T):
+            t = s if d == 0 else T - 1 - s
+            xq = quantize_pack_int4(x[t].contiguous(), x_act, k_pad=L.w_ih.k_pad)     # x_t on entry
+            hq = quantize_pack_int4(h, hid)                                            # s_{t-1} on entry
+            r = qlstm_step(xq, x_act, hq, c, L, out=dict(c=c, h=torch.empty_like(h)))
+            h = r["h"]
+            out[t, :, d * H:(d + 1) * H] = h
+    return out
 
 
 def q4_poll_status(status: torch.Tensor) -> int:

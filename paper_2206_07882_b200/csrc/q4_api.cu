@@ -86,6 +86,11 @@ int q4_timing_set(uint32_t tag_mask, void** start_events, void** stop_events, in
 }
 int q4_timing_count(void) { return timing_count(); }
 int64_t q4_launch_count(void) { return g_launches; }
+int64_t q4_quantizer_calls(int32_t reset) {
+  const int64_t n = g_quant_calls;
+  if (reset) g_quant_calls = 0;
+  return n;
+}
 static int g_select_exact = 0;
 static int select_exact_only() { return g_select_exact; }
 int q4_beam_select_exact_set(int32_t enabled) {
@@ -202,6 +207,7 @@ int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k
   }
   if (rows == 0) return Q4_OK;
   TagScope tag(TAG_QUANT);
+  if (mode != 2) ++g_quant_calls;   // an activation tensor (weights are quantized once, off line)
   Q4_TRY(launch_quantize(x, x_is_fp16 != 0, rows, k, k_pad, a, mode, n_groups, per_row_scale,
                          static_cast<uint8_t*>(q_out), group_scale_out, S(stream)));
   return Q4_OK;
@@ -261,13 +267,15 @@ int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, co
                const float* c_in, int32_t N, const q4_mat* w_ih, const q4_mat* w_hh,
                const float* bias, const q4_act* hid_act, void* hq_out, float* c_out,
                float* h_f32_out, int32_t* dbg_acc_ih, int32_t* dbg_acc_hh, q4_stream stream) {
-  if (!xq || !hq_in || !c_in || !hq_out || !c_out) return Q4_ERR_NULL;
+  if (!xq || !hq_in || !c_in || !c_out) return Q4_ERR_NULL;
+  if (!hq_out && !h_f32_out) return Q4_ERR_NULL;   // Inner placement needs the real-valued output
   int H = 0;
   Q4_CHECK(check_lstm(w_ih, w_hh, x_act, hid_act, &H));
   if (N < 0) return Q4_ERR_DIM;
   if (hq_in == hq_out) return Q4_ERR_UNSUPPORTED;
   if (!aligned16(xq) || !aligned16(hq_in) || !aligned16(hq_out)) return Q4_ERR_ALIGN;
   if (N == 0) return Q4_OK;
+  if (hq_out) ++g_quant_calls;   // the one quantizer call at the cell output (Outer placement)
   LstmArgs2 args;
   memset(&args, 0, sizeof(args));
   LstmArgs& a = args.d[0];
@@ -368,6 +376,10 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
       Q4_TRY(launch_gemm(g, EPI_I32, s));
     }
   }
+  // per step and direction one quantizer call at the cell output; a second one where the next
+  // layer wants the same real value at another precision
+  g_quant_calls += (int64_t)T * dirs *
+                   ((out_act->bits == hid_act->bits && out_act->scale == hid_act->scale) ? 1 : 2);
   if (persistent) {
     EncRecArgs ra;
     memset(&ra, 0, sizeof(ra));
@@ -462,6 +474,7 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
   if (N == 0) return Q4_OK;
   cudaStream_t s = S(stream);
   TagScope tag(TAG_JOINT);
+  ++g_quant_calls;   // tanh(e * p)
   float* p = static_cast<float*>(workspace);
   uint8_t* zq = static_cast<uint8_t*>(workspace) + align_up((size_t)N * D * sizeof(float));
   GemmArgs g1 = gemm_args(pq, row_bytes(w_pred->k_pad, p_act->bits), nullptr, *p_act, N, *w_pred,
@@ -682,6 +695,9 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   cudaStream_t s = S(stream);
   const q4_beam_state& st = *state;
   const int N = B * W;
+  // quantizer applications of one iteration: the cell outputs of the advanced networks, the two
+  // bottleneck outputs, tanh(e * p)
+  g_quant_calls += 1 + 1 + m.tgt.n_layers + 2 + 1;
   int joint_normalized = 0;   // the tensor-core joint kernel leaves log-probabilities, not logits
   // the first call of a frame of the time-synchronous search follows a frame close, which creates
   // no label extension: no network has anything to advance, only the joint runs

@@ -24,6 +24,7 @@ constexpr int PITCH = KC + 16;  // shared-memory row pitch in bytes (16 B aligne
 constexpr int NT = 256;         // threads per CTA of the tile kernels
 
 extern int64_t g_launches;      // kernels launched by this process
+extern int64_t g_quant_calls;   // activation-quantizer applications enqueued by this process
 
 // Where the rows of an operand live: row n is at base + (idx ? idx[n] : n) * stride bytes;
 // a negative index means "no row" (reads as zeros / is not written).

@@ -7,6 +7,7 @@
 namespace q4 {
 
 int64_t g_launches = 0;
+int64_t g_quant_calls = 0;   // activation-quantizer applications (Section 3.4), see q4_quantizer_calls
 int g_tag = TAG_NONE;
 int g_dependent_launch = 1;
 
@@ -363,7 +364,9 @@ __global__ void __launch_bounds__(NT) k_lstm(const __grid_constant__ LstmArgs2 a
       q[cc] = quantize1(h, a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
       q2[cc] = quantize1(h, a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
     }
-    if (a.hid_act.bits == 4) {
+    if (a.hq_out == nullptr) {
+      // Inner placement (Section 3.4): nothing is quantized at the cell output
+    } else if (a.hid_act.bits == 4) {
       a.hq_out[(long long)oi * a.hq_stride + (cell0 >> 1)] = (uint8_t)((q[0] & 0xF) | ((q[1] & 0xF) << 4));
     } else {
       *reinterpret_cast<uint16_t*>(a.hq_out + (long long)oi * a.hq_stride + cell0) =

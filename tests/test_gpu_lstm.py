@@ -285,3 +285,37 @@ def test_layer_two_bit_weights(Bd):
         np.testing.assert_array_equal(got["acc_ih"].cpu().numpy(), ref["acc_ih"])
         np.testing.assert_array_equal(gpu_codes(got["yq"], 2 * H, hid).reshape(T, B, 2 * H), ref["yq"])
         np.testing.assert_array_equal(got["c_n"].cpu().numpy(), ref["c_n"])
+
+
+def test_outer_and_inner_quantizer_placement_counted_on_the_device(Bd):
+    # Section 3.4 on the device: the library counts its activation-quantizer applications.  Outer
+    # placement (quantize once at each cell output; the input once per frame): T + T L.  Inner
+    # placement (every cell quantizes its two inputs on entry): 2 T L.  L = 12 cells (6 layers x 2
+    # directions).  Both placements give the same network output; the oracle's two paths agree
+    # with both, value for value.
+    T, B, Lc = 5, 3, 12
+    enc = synth.encoder(seed=1, T=T, B=B, F=32, H=32, L=6, D=32, with_proj=False)
+    E = enc["enc"]
+    feats = torch.from_numpy(enc["features"].astype(np.float32)).cuda()
+    dev = Bd.Encoder(E)
+    # Outer, input quantized frame by frame
+    Bd.quantizer_calls(reset=True)
+    frames = [Bd.quantize_pack_int4(feats[t].contiguous(), dev.in_act) for t in range(T)]
+    xq, x_act = torch.cat(frames, 0), dev.in_act
+    for l, dirs in enumerate(dev.layers):
+        r = Bd.qlstm_layer_forward(xq, x_act, T, B, dirs, dev.out_acts[l])
+        xq, x_act = r["yq"], dev.out_acts[l]
+    outer = Bd.quantizer_calls(reset=True)
+    # Inner
+    x = feats
+    x_act = dev.in_act
+    for l, dirs in enumerate(dev.layers):
+        x = Bd.lstm_layer_inner(x, x_act, dirs)
+        x_act = dirs[0].hid_act
+    inner = Bd.quantizer_calls(reset=True)
+    assert outer == T + T * Lc and inner == 2 * T * Lc
+    assert round(100 * (1 - outer / inner)) in (45, 46)
+    ref = O.encoder_forward(E, enc["features"], want_layers=True)
+    np.testing.assert_array_equal(gpu_codes(xq, 64, dev.out_acts[-1]).reshape(T, B, 64), ref["yq"])
+    np.testing.assert_array_equal(x.cpu().numpy(), ref["layers"][-1]["h"])
+    np.testing.assert_array_equal(x.cpu().numpy(), O.encoder_forward_inner(E, enc["features"]))
