@@ -54,6 +54,9 @@ WORKLOADS = {
     # the same utterance with the precision assignment of the end-to-end workload (first encoder layer
     # and joint output layer at 8 bits, the rest at 4): the "mixed" point of that figure
     "fig2_single_utterance_mixed": dict(B=1, T=152, U_max=76, l1_bits=8, out_bits=8, enc=True, dec=True, seed=6),
+    # and with every weight and every activation quantizer at 8 bits: the "INT8" bar of that figure
+    "fig2_single_utterance_int8": dict(B=1, T=152, U_max=76, l1_bits=8, out_bits=8, enc=True, dec=True, seed=6,
+                                       all8=True),
 }
 
 
@@ -244,8 +247,9 @@ class Job:
                                logp=torch.empty((N, 1024), dtype=torch.float32, device="cuda"),
                                ws=torch.empty(Bd.workspace_bytes(Bd.WS_JOINT, [N, 256]), dtype=torch.uint8, device="cuda"))
         if wl["enc"]:
+            a8 = 8 if wl.get("all8") else 4
             enc_w = synth.encoder(wl["seed"], T=T, B=B, first_layer_bits=wl["l1_bits"],
-                                  in_max=wl["l1_bits"] == 8, features=False)
+                                  in_max=wl["l1_bits"] == 8, features=False, layer_bits=a8, proj_bits=a8)
             self.enc = Bd.Encoder(enc_w["enc"])
             if wl_name.startswith("cfg4"):
                 self.host_in = torch.from_numpy(synth.logmel(seed, B, 2 * T, 40)).pin_memory()
@@ -253,7 +257,7 @@ class Job:
                 self.host_in = torch.from_numpy(
                     synth.Stream(seed).normal("features", (T, B, 240)).astype(np.float16)).pin_memory()
         if wl["dec"]:
-            dw = synth.decoder(3, out_bits=wl["out_bits"], U_max=wl["U_max"])
+            dw = synth.decoder(3, out_bits=wl["out_bits"], U_max=wl["U_max"], all_bits=8 if wl.get("all8") else 4)
             self.dec = Bd.Decoder(dw)
             if "tsd" in wl:
                 self.dec.alloc_state(B, self.W, T * (wl["tsd"] + 1), wl["tsd"])
@@ -660,6 +664,24 @@ def fig2_sweep(torch):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / 5
         out[str(W)] = {"ms_per_utterance": ms, "rtf": ms / 1e3 / (job.wl["T"] * 0.02)}
+    # the precision axis of the same figure at beam 16 (the paper's simulated accelerator: RTF 0.116 all
+    # 8 bit, 0.065 all 4 bit)
+    for name, key in (("fig2_single_utterance_int8", "all_int8_beam16"), ("fig2_single_utterance_mixed", "mixed_beam16")):
+        del job
+        torch.cuda.empty_cache()
+        job = Job(name, 0, 16)
+        job.step(job.dev_in)
+        for _ in range(3):
+            job.step_graphed()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(5):
+            job.step_graphed()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 5
+        out[key] = {"ms_per_utterance": ms, "rtf": ms / 1e3 / (job.wl["T"] * 0.02)}
     return out
 
 

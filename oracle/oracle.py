@@ -434,7 +434,8 @@ class Decoder:
         d = self.c = _Decoder()
         self.dw = dw
         V, E = dw.pred.emb.shape
-        d.pred = _Pred(k.arr(dw.pred.emb, np.float32), V, E, act_symmetric(dw.pred.emb_alpha, 4),
+        d.pred = _Pred(k.arr(dw.pred.emb, np.float32), V, E,
+                       act_symmetric(dw.pred.emb_alpha, getattr(dw, "emb_bits", 4)),
                        _mk_lstm(k, dw.pred.lstm),
                        act_symmetric(dw.pred.lstm.hid_alpha, dw.pred.lstm.hid_bits),
                        _mk_linear(k, dw.pred.proj))
@@ -450,13 +451,16 @@ class Decoder:
         V, E = m.emb.shape
         lm = _Lm()
         lm.emb, lm.V, lm.E = k.arr(m.emb, np.float32), V, E
-        lm.emb_act = act_asymmetric(m.emb_lo, m.emb_hi, 4)
+        # learned-boundary input quantizers: asymmetric at 4 bits (Eq. 2); at 8 bits symmetric with
+        # the wider of the two boundaries (no clipping is added, codes stay signed)
+        wide = getattr(m, "act_bits", 4) == 8
+        lm.emb_act = act_symmetric(max(-m.emb_lo, m.emb_hi), 8) if wide else act_asymmetric(m.emb_lo, m.emb_hi, 4)
         lm.n_layers = len(m.lstm)
         for i, l in enumerate(m.lstm):
             lm.lstm[i] = _mk_lstm(k, l)
             lm.hid_act[i] = act_symmetric(l.hid_alpha, l.hid_bits)
         lm.bott = _mk_linear(k, m.bott)
-        lm.bott_act = act_asymmetric(m.bott_lo, m.bott_hi, 4)
+        lm.bott_act = act_symmetric(max(-m.bott_lo, m.bott_hi), 8) if wide else act_asymmetric(m.bott_lo, m.bott_hi, 4)
         lm.out = _mk_linear(k, m.out)
         return lm
 

@@ -450,12 +450,13 @@ class Encoder:
 
 class DeviceLm:
     def __init__(self, m, device="cuda"):
-        self.emb_act = q4_act_asymmetric(m.emb_lo, m.emb_hi, 4)
+        wide = getattr(m, "act_bits", 4) == 8     # 8 bits: symmetric with the wider boundary (signed codes)
+        self.emb_act = q4_act_symmetric(max(-m.emb_lo, m.emb_hi), 8) if wide else q4_act_asymmetric(m.emb_lo, m.emb_hi, 4)
         emb = torch.from_numpy(np.ascontiguousarray(m.emb, dtype=np.float32)).to(device)
         self.lstm = [DeviceLstm(l, device) for l in m.lstm]
         self.emb_q = quantize_pack_int4(emb, self.emb_act, k_pad=self.lstm[0].w_ih.k_pad)   # table quantized once
         self.bott = DeviceLinear(m.bott, device)
-        self.bott_act = q4_act_asymmetric(m.bott_lo, m.bott_hi, 4)
+        self.bott_act = q4_act_symmetric(max(-m.bott_lo, m.bott_hi), 8) if wide else q4_act_asymmetric(m.bott_lo, m.bott_hi, 4)
         self.out = DeviceLinear(m.out, device)
 
     def c(self) -> LmS:
@@ -480,7 +481,7 @@ class Decoder:
         self.tensor_cores = tensor_cores
         self.concurrent = concurrent and tensor_cores
         self.V, self.E = dw.pred.emb.shape
-        self.pred_emb_act = q4_act_symmetric(dw.pred.emb_alpha, 4)
+        self.pred_emb_act = q4_act_symmetric(dw.pred.emb_alpha, getattr(dw, "emb_bits", 4))
         emb = torch.from_numpy(np.ascontiguousarray(dw.pred.emb, dtype=np.float32)).to(device)
         self.pred_lstm = DeviceLstm(dw.pred.lstm, device)
         self.pred_emb_q = quantize_pack_int4(emb, self.pred_emb_act, k_pad=self.pred_lstm.w_ih.k_pad)
@@ -521,13 +522,14 @@ class Decoder:
         R, N = B * RW, B * W
         Hp, Hs, Ht = self.pred_lstm.H, self.src.lstm[0].H, self.tgt.lstm[0].H
         z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
+        bp, bs, bt = (self.pred_lstm.hid_act.bits, self.src.lstm[0].hid_act.bits, self.tgt.lstm[0].hid_act.bits)
         t = self.tensors = dict(
-            pred_hq=z((R, Hp // 2), torch.uint8), pred_c=z((R, Hp), torch.float32),
+            pred_hq=z((R, Hp * bp // 8), torch.uint8), pred_c=z((R, Hp), torch.float32),
             pred_p=z((R, self.D), torch.float32),
-            src_hq=z((R, Hs // 2), torch.uint8), src_c=z((R, Hs), torch.float32),
+            src_hq=z((R, Hs * bs // 8), torch.uint8), src_c=z((R, Hs), torch.float32),
             src_lp=z((R, self.V), torch.float32),
-            tgt_hq0=z((R, Ht // 2), torch.uint8), tgt_c0=z((R, Ht), torch.float32),
-            tgt_hq1=z((R, Ht // 2), torch.uint8), tgt_c1=z((R, Ht), torch.float32),
+            tgt_hq0=z((R, Ht * bt // 8), torch.uint8), tgt_c0=z((R, Ht), torch.float32),
+            tgt_hq1=z((R, Ht * bt // 8), torch.uint8), tgt_c1=z((R, Ht), torch.float32),
             tgt_lp=z((R, self.V), torch.float32),
             score=z(N, torch.float32), t=z(N, torch.int32), u=z(N, torch.int32),
             hash=z(N, torch.int64), prev_hash=z(N, torch.int64), last_tok=z(N, torch.int32),

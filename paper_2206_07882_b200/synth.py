@@ -138,6 +138,8 @@ class LmW:
     bott_lo: float
     bott_hi: float
     out: LinearW               # D -> V
+    act_bits: int = 4          # width of the two input quantizers; at 8 bits they are symmetric with
+                               # the boundary max(|lo|, hi) (signed codes), at 4 bits asymmetric
 
 
 @dataclass
@@ -151,6 +153,7 @@ class DecoderW:
     rho: float = 0.2
     W: int = 16
     U_max: int = 0
+    emb_bits: int = 4          # width of the prediction network's input quantizer
 
 
 def _qmat(st: Stream, name: str, rows: int, k: int, bits: int = 4) -> QMat:
@@ -204,7 +207,8 @@ def single_layer(seed: int = 0, T: int = 50, B: int = 4, K: int = 64, H: int = 1
 
 def encoder(seed: int = 1, T: int = 500, B: int = 32, F: int = 240, H: int = 640, L: int = 6,
             D: int = 256, first_layer_bits: int = 4, in_max: bool = False,
-            with_proj: bool = True, features: bool = True, w_bits: int = 4, proj_bits: int = 4):
+            with_proj: bool = True, features: bool = True, w_bits: int = 4, proj_bits: int = 4,
+            layer_bits: int = 4):
     """Bidirectional LSTM encoder.  Features fp16 ~ N(0,1); input clip U(2.5,3.5);
     per-layer hidden boundary U(.9,1.0) (the paper observes MAX boundaries of LSTM
     outputs in [0.9,1], Section 3.2); biases N(0,.1)."""
@@ -217,7 +221,7 @@ def encoder(seed: int = 1, T: int = 500, B: int = 32, F: int = 240, H: int = 640
     layers = []
     for l in range(L):
         k = F if l == 0 else 2 * H
-        bits = first_layer_bits if l == 0 else 4
+        bits = first_layer_bits if l == 0 else layer_bits
         # w_bits < 4: weight codes stored narrower than the activation codes (Table 1's 2/4 rows)
         wb = bits if bits == 8 else w_bits
         layers.append([_lstm(st, f"enc.l{l}.d{d}", k, H, wb, 0.1, float(alphas[l]), bits)
@@ -228,35 +232,37 @@ def encoder(seed: int = 1, T: int = 500, B: int = 32, F: int = 240, H: int = 640
     return out
 
 
-def _lm(st: Stream, name: str, V: int, E: int, H: int, n_layers: int, D: int) -> LmW:
+def _lm(st: Stream, name: str, V: int, E: int, H: int, n_layers: int, D: int, bits: int = 4) -> LmW:
     emb = st.normal(name + ".emb", (V, E), 0.0, 0.5).astype(np.float32)
     lo = -float(st.uniform(name + ".emb_lo", (1,), 1.0, 2.0)[0])
     hi = float(st.uniform(name + ".emb_hi", (1,), 1.0, 2.0)[0])
     alphas = st.uniform(name + ".hid_alpha", (n_layers,), 0.9, 1.0)
-    lstm = [_lstm(st, f"{name}.l{l}", E if l == 0 else H, H, 4, 0.1, float(alphas[l]))
+    lstm = [_lstm(st, f"{name}.l{l}", E if l == 0 else H, H, bits, 0.1, float(alphas[l]))
             for l in range(n_layers)]
-    bott = _linear(st, name + ".bott", D, H)
+    bott = _linear(st, name + ".bott", D, H, bits)
     blo = -float(st.uniform(name + ".bott_lo", (1,), 1.0, 2.0)[0])
     bhi = float(st.uniform(name + ".bott_hi", (1,), 1.0, 2.0)[0])
-    out = _linear(st, name + ".out", V, D)
-    return LmW(emb, lo, hi, lstm, bott, blo, bhi, out)
+    out = _linear(st, name + ".out", V, D, bits)
+    return LmW(emb, lo, hi, lstm, bott, blo, bhi, out, bits)
 
 
 def decoder(seed: int = 3, V: int = 1024, E: int = 256, Hp: int = 1024, D: int = 256,
             Hs: int = 1024, Ht: int = 2048, tgt_layers: int = 2, out_bits: int = 4,
             W: int = 16, U_max: int = 150, lambda_t: float = 0.5, lambda_s: float = 0.3,
-            rho: float = 0.2, rnnt_w_bits: int = 4, proj_bits: int = 4) -> DecoderW:
+            rho: float = 0.2, rnnt_w_bits: int = 4, proj_bits: int = 4, all_bits: int = 4) -> DecoderW:
     """Prediction network, joint network and the two fusion LMs.  Embeddings
     N(0,.5); prediction-input boundary 1.25 and hidden boundary 1 (Section 3.2);
     learned LM input boundaries stand-ins alpha- ~ -U(1,2), alpha+ ~ U(1,2)."""
     st = Stream(seed)
+    if all_bits == 8:      # the all-8-bit point of the paper's run-time figure: every weight and quantizer at 8
+        rnnt_w_bits = out_bits = proj_bits = 8
     pred = PredW(st.normal("pred.emb", (V, E), 0.0, 0.5).astype(np.float32), 1.25,
-                 _lstm(st, "pred.lstm", E, Hp, rnnt_w_bits, 0.1, 1.0, 4),
+                 _lstm(st, "pred.lstm", E, Hp, rnnt_w_bits, 0.1, 1.0, all_bits),
                  _linear(st, "pred.proj", D, Hp, proj_bits if proj_bits != 4 else rnnt_w_bits))
     joint = JointW(_linear(st, "joint.out", V, D, out_bits if out_bits != 4 else rnnt_w_bits), out_bits)
-    src = _lm(st, "src", V, E, Hs, 1, D)
-    tgt = _lm(st, "tgt", V, E, Ht, tgt_layers, D)
-    return DecoderW(pred, joint, src, tgt, lambda_t, lambda_s, rho, W, U_max)
+    src = _lm(st, "src", V, E, Hs, 1, D, all_bits)
+    tgt = _lm(st, "tgt", V, E, Ht, tgt_layers, D, all_bits)
+    return DecoderW(pred, joint, src, tgt, lambda_t, lambda_s, rho, W, U_max, all_bits)
 
 
 def enc_frames(seed: int, T: int, B: int, dim: int = 1280) -> np.ndarray:
@@ -274,16 +280,36 @@ def logmel(seed: int, B: int, T100: int = 1000, n_mel: int = 40) -> np.ndarray:
     return Stream(seed).normal("logmel", (B, T100, n_mel)).astype(np.float32)
 
 
-def paper_dimensions(seed: int = 5, T: int = 12, B: int = 2, U_max: int = 6):
+def paper_dimensions(seed: int = 5, T: int = 12, B: int = 2, U_max: int = 6, section_3_2: bool = False):
     """The model sizes the paper states in Section 2: 340-d encoder input, 6 bidirectional layers of
     640 cells, 256-d encoder/prediction outputs, prediction LSTM of 768 cells behind a small
     embedding (10-d reproduces the 2.6 M parameters quoted), 46 output characters, external LM of
     two 2048-cell layers with a 256 bottleneck, source LM shaped like the prediction network;
-    fusion weights 0.7 / 0.5 / 0.2 as after Eq. 1."""
-    enc = encoder(seed, T=T, B=B, F=340, H=640, L=6, D=256)
+    fusion weights 0.7 / 0.5 / 0.2 as after Eq. 1.  section_3_2 = the precision assignment of
+    Section 3.2: first encoder layer at 8 bits with the per-utterance MAX boundary on its input, the
+    linear layers of the RNN-T (encoder and prediction projections, joint output) at 8 bits,
+    everything else, both LMs included, at 4 bits."""
+    kw_e = dict(first_layer_bits=8, in_max=True, proj_bits=8) if section_3_2 else {}
+    kw_d = dict(out_bits=8, proj_bits=8) if section_3_2 else {}
+    enc = encoder(seed, T=T, B=B, F=340, H=640, L=6, D=256, **kw_e)
     dec = decoder(seed + 1000, V=46, E=10, Hp=768, D=256, Hs=768, Ht=2048, tgt_layers=2, U_max=U_max,
-                  lambda_t=0.7, lambda_s=0.5, rho=0.2)
+                  lambda_t=0.7, lambda_s=0.5, rho=0.2, **kw_d)
     return enc, dec
+
+
+def weight_storage(enc: EncoderW, dec: DecoderW, with_src_lm: bool = False) -> dict:
+    """Weight-matrix parameters by storage width (biases and embeddings aside): count, the share
+    held at 4 bits, bytes as stored and the ratio to fp32 storage."""
+    mats = [m for layer in enc.layers for l in layer for m in (l.w_ih, l.w_hh)]
+    if enc.proj is not None:
+        mats.append(enc.proj.w)
+    mats += [dec.pred.lstm.w_ih, dec.pred.lstm.w_hh, dec.pred.proj.w, dec.joint.out.w]
+    for m in [dec.tgt] + ([dec.src] if with_src_lm else []):
+        mats += [w for l in m.lstm for w in (l.w_ih, l.w_hh)] + [m.bott.w, m.out.w]
+    n = sum(m.codes.size for m in mats)
+    by = sum(m.codes.size * m.bits / 8 for m in mats)
+    return {"params": n, "frac_4bit": sum(m.codes.size for m in mats if m.bits == 4) / n, "bytes": by,
+            "compression": 4.0 * n / by}
 
 
 def parameter_counts(enc: EncoderW, dec: DecoderW) -> dict:

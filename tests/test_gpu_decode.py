@@ -500,3 +500,16 @@ def test_search_two_bit_rnnt_weights(Bd, tensor_cores):
     dd, tokens, lens, scores, ref = run_search(Bd, dw, e, tensor_cores=tensor_cores)
     frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(8)), 10, 6, 16, min_same=1.0)
     assert tr == 1.0
+
+
+@pytest.mark.parametrize("dims", [dict(V=64, E=32, Hp=64, D=32, Hs=32, Ht=64), dict(V=128, E=32, Hp=128, D=256, Hs=128, Ht=256)])
+def test_search_all_eight_bit(Bd, dims):
+    # every weight and every activation quantizer of the decoder at 8 bits (the all-8-bit point of the
+    # paper's run-time figure): 8-bit search state, DP4A kernels (small) and tensor-core kernels
+    dw = synth.decoder(seed=97, tgt_layers=2, U_max=6, W=16, all_bits=8, **dims)
+    assert dw.pred.lstm.w_hh.bits == 8 and dw.tgt.out.w.bits == 8 and dw.pred.lstm.hid_bits == 8
+    e = synth.Stream(16).normal("e", (10, 8, dims["D"])).astype(np.float32)
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e)
+    assert dd.tensors["pred_hq"].shape[1] == dims["Hp"]           # one byte per hidden code
+    frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(8)), 10, 6, 16, min_same=1.0)
+    assert tr == 1.0
