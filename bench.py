@@ -233,6 +233,10 @@ class Job:
         if self.kind == "predjoint":
             dw = synth.decoder(wl["seed"])
             self.pj = Bd.Decoder(dw)
+            # one-time int8 operands: from 128 rows on the library runs these calls on the tensor cores
+            self.pj.pred_lstm.prepare()
+            self.pj.pred_proj.prepare()
+            self.pj.joint_out.prepare()
             N = B * 16
             self.pj_tok = torch.from_numpy(np.ascontiguousarray(np.concatenate(
                 [np.zeros((N, 1), np.int32), synth.labels(seed, N, T - 1, 1024)], axis=1).T)).cuda()   # [T, N]
@@ -240,12 +244,12 @@ class Job:
                                            (np.arange(N, dtype=np.int32)[None, :] // 16)).astype(np.int32)).cuda()
             self.host_in = torch.from_numpy(synth.enc_frames(seed, T, B, 1280)).pin_memory()
             self.frame_act = Bd.q4_act_symmetric(1.0, 4)
-            self.frame_proj = Bd.DeviceLinear(synth._linear(synth.Stream(wl["seed"]), "enc.proj", 256, 1280))
+            self.frame_proj = Bd.DeviceLinear(synth._linear(synth.Stream(wl["seed"]), "enc.proj", 256, 1280)).prepare()
             Hp = self.pj.pred_lstm.H
             self.pj_buf = dict(hq=[torch.zeros((N, Hp // 2), dtype=torch.uint8, device="cuda") for _ in range(2)],
                                c=torch.zeros((N, Hp), dtype=torch.float32, device="cuda"),
                                logp=torch.empty((N, 1024), dtype=torch.float32, device="cuda"),
-                               ws=torch.empty(Bd.workspace_bytes(Bd.WS_JOINT, [N, 256]), dtype=torch.uint8, device="cuda"))
+                               ws=torch.empty(Bd.workspace_bytes(Bd.WS_JOINT, [N, 256, Hp]), dtype=torch.uint8, device="cuda"))
         if wl["enc"]:
             a8 = 8 if wl.get("all8") else 4
             enc_w = synth.encoder(wl["seed"], T=T, B=B, first_layer_bits=wl["l1_bits"],
@@ -266,7 +270,7 @@ class Job:
             if not wl["enc"]:
                 self.host_in = torch.from_numpy(synth.enc_frames(seed, T, B, 1280)).pin_memory()
                 self.frame_act = Bd.q4_act_symmetric(1.0, 4)
-                self.frame_proj = Bd.DeviceLinear(synth._linear(synth.Stream(wl["seed"]), "enc.proj", 256, 1280))
+                self.frame_proj = Bd.DeviceLinear(synth._linear(synth.Stream(wl["seed"]), "enc.proj", 256, 1280)).prepare()
         self.dev_in = self.host_in.cuda()
         self.graph = None
 

@@ -129,19 +129,37 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
  *   hq_out == NULL (then h_f32_out is required) leaves the cell output unquantized: the "Inner"
  *   placement of Section 3.4, where every cell quantizes its two inputs on entry instead
  *   (quantize_pack_int4 on x_t and on the previous real-valued cell output, then this call).
+ *   prepared / workspace (all nullable): with the buffer filled by q4_prepare_lstm for these weights
+ *   and a workspace of q4_workspace_bytes(Q4_WS_LSTM_STEP, {N, kx_pad, H}) bytes, calls with N >= 128
+ *   and H a multiple of 128 run on the tensor cores (same results, bit for bit); otherwise, and
+ *   always without them, the DP4A kernel reads the packed weights directly.
  */
 int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, const void* hq_in,
                const float* c_in, int32_t N, const q4_mat* w_ih, const q4_mat* w_hh,
                const float* bias, const q4_act* hid_act, void* hq_out, float* c_out,
-               float* h_f32_out, int32_t* dbg_acc_ih, int32_t* dbg_acc_hh, q4_stream stream);
+               float* h_f32_out, int32_t* dbg_acc_ih, int32_t* dbg_acc_hh, const void* prepared,
+               void* workspace, size_t workspace_bytes, q4_stream stream);
+
+/* One-time int8 operands of an LSTM's weights for the tensor-core path of qlstm_step (weights are
+ * quantized once, activations at every step: Section 3.2): rows reordered to 4*cell+gate, row
+ * scales and bias in the same order.  buffer: device, q4_prepared_lstm_bytes bytes, caller-owned.
+ * q4_prepare_linear: the same for a linear layer (q4_linear_forward, qjoint_logprobs). */
+size_t q4_prepared_lstm_bytes(const q4_mat* w_ih, const q4_mat* w_hh);
+int q4_prepare_lstm(const q4_mat* w_ih, const q4_mat* w_hh, const float* bias, void* buffer, size_t bytes,
+                    q4_stream stream);
+size_t q4_prepared_linear_bytes(const q4_mat* w);
+int q4_prepare_linear(const q4_mat* w, void* buffer, size_t bytes, q4_stream stream);
 
 /*
  * q4_linear_forward — quantized linear layer (Section 3.2): out[m, j] = acc[m, j] *
  * (x_act.scale * w.scale[j]) + bias[j], fp32, out [M, w.rows].  Used for the encoder ->
- * joint projection.  dbg_acc [M, w.rows] int32 nullable.
+ * joint projection.  dbg_acc [M, w.rows] int32 nullable.  prepared / workspace (nullable): with
+ * the buffer of q4_prepare_linear and q4_workspace_bytes(Q4_WS_LINEAR, {M, k_pad}) bytes, calls
+ * with M >= 128 and no dbg_acc run on the tensor cores.
  */
 int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_mat* w,
-                      const float* bias, float* out, int32_t* dbg_acc, q4_stream stream);
+                      const float* bias, float* out, int32_t* dbg_acc, const void* prepared,
+                      void* workspace, size_t workspace_bytes, q4_stream stream);
 
 /*
  * qjoint_logprobs — joint network (Section 2): the prediction-network cell output codes pq
@@ -149,11 +167,15 @@ int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_m
  * the projected encoder frame e[frame_idx[n]] ([*, D] fp32), z = tanh(e * p), z is quantized
  * with z_act, passed through the output layer (w_out [V, D], b_out) and a log-softmax.
  * logp [N, V] fp32.  workspace: q4_workspace_bytes(Q4_WS_JOINT, {N, D}).
+ * prepared_pred / prepared_out (nullable): buffers of q4_prepare_linear for w_pred and w_out; with
+ * both, a workspace of q4_workspace_bytes(Q4_WS_JOINT, {N, D, Hp_pad}) bytes, N >= 128 and V a
+ * multiple of 32 the call runs on the tensor cores in three launches (the projection's epilogue forms
+ * tanh(e * p) and quantizes it; the output layer's epilogue takes the log-softmax).
  */
 int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, const q4_act* p_act,
                     int32_t N, const q4_mat* w_pred, const float* b_pred, const q4_act* z_act,
-                    const q4_mat* w_out, const float* b_out, float* logp, void* workspace,
-                    size_t workspace_bytes, q4_stream stream);
+                    const q4_mat* w_out, const float* b_out, float* logp, const void* prepared_pred,
+                    const void* prepared_out, void* workspace, size_t workspace_bytes, q4_stream stream);
 
 /*
  * qjoint_logprobs_static — qjoint_logprobs for callers that cannot allocate device memory when
@@ -336,8 +358,10 @@ int q4_feature_prologue(const float* mel, int32_t B, int32_t T100, int32_t M, vo
                         q4_stream stream);
 
 #define Q4_WS_LSTM_LAYER 1 /* dims = {T, B, dirs, H} or {T, B, dirs, H, kx_pad} */
-#define Q4_WS_JOINT 2      /* dims = {N, D} */
+#define Q4_WS_JOINT 2      /* dims = {N, D} or {N, D, Hp_pad} (tensor-core path) */
 #define Q4_WS_BEAM 3       /* dims = {B, W, V, D} or {B, W, V, D, E_pad, Hp, Hs, Ht} */
+#define Q4_WS_LSTM_STEP 4  /* dims = {N, kx_pad, H} (tensor-core path of qlstm_step) */
+#define Q4_WS_LINEAR 5     /* dims = {M, k_pad} (tensor-core path of q4_linear_forward) */
 size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims);
 
 /* Synchronise `stream`, read the device status word and return 0 or the error it holds. */

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libq4rnnt.so")
 
 ERRORS = {-1: "Q4_ERR_NULL", -2: "Q4_ERR_DIM", -3: "Q4_ERR_ALIGN", -4: "Q4_ERR_BITS",
           -5: "Q4_ERR_WORKSPACE", -6: "Q4_ERR_UNSUPPORTED", -7: "Q4_ERR_CUDA", -8: "Q4_ERR_TIMEOUT"}
-WS_LSTM_LAYER, WS_JOINT, WS_BEAM = 1, 2, 3
+WS_LSTM_LAYER, WS_JOINT, WS_BEAM, WS_LSTM_STEP, WS_LINEAR = 1, 2, 3, 4, 5
 
 
 class Q4Error(RuntimeError):
@@ -80,7 +80,8 @@ class BeamStateS(C.Structure):
 EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm_layer_forward",
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
-           "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_beam_select_exact_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static", "q4_quantizer_calls"]
+           "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_beam_select_exact_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static", "q4_quantizer_calls", "q4_prepared_lstm_bytes", "q4_prepare_lstm",
+           "q4_prepared_linear_bytes", "q4_prepare_linear"]
 
 _lib = None
 
@@ -97,6 +98,8 @@ def lib() -> C.CDLL:
         _lib.q4_launch_count.restype = C.c_int64
         _lib.q4_prepared_bytes.restype = C.c_size_t
         _lib.q4_quantizer_calls.restype = C.c_int64
+        _lib.q4_prepared_lstm_bytes.restype = C.c_size_t
+        _lib.q4_prepared_linear_bytes.restype = C.c_size_t
     return _lib
 
 
@@ -240,6 +243,17 @@ class DeviceLstm:
         self.bias = _dev_f32(lw.bias, device)
         self.hid_act = q4_act_symmetric(lw.hid_alpha, lw.hid_bits)
         self.H = self.w_hh.k
+        self.prepared = None
+        self.ws = None
+
+    def prepare(self):
+        """One-time int8 operands for the tensor-core path of qlstm_step (q4_prepare_lstm)."""
+        wi, wh = self.w_ih.c(), self.w_hh.c()
+        n = int(lib().q4_prepared_lstm_bytes(C.byref(wi), C.byref(wh)))
+        self.prepared = torch.empty(n, dtype=torch.uint8, device=self.w_ih.q.device)
+        _chk(lib().q4_prepare_lstm(C.byref(wi), C.byref(wh), _p(self.bias), _p(self.prepared), C.c_size_t(n),
+                                   _stream()), "q4_prepare_lstm")
+        return self
 
     def c(self) -> LstmS:
         return LstmS(self.w_ih.c(), self.w_hh.c(), self.bias.data_ptr() if self.bias is not None else None,
@@ -253,6 +267,16 @@ class DeviceLinear:
     def __init__(self, lw, device="cuda"):
         self.w = DeviceMat.from_codes(lw.w.codes, lw.w.scale, lw.w.bits, device)
         self.bias = _dev_f32(lw.bias, device)
+        self.prepared = None
+        self.ws = None
+
+    def prepare(self):
+        """One-time int8 operand for the tensor-core paths (q4_prepare_linear)."""
+        w = self.w.c()
+        n = int(lib().q4_prepared_linear_bytes(C.byref(w)))
+        self.prepared = torch.empty(n, dtype=torch.uint8, device=self.w.q.device)
+        _chk(lib().q4_prepare_linear(C.byref(w), _p(self.prepared), C.c_size_t(n), _stream()), "q4_prepare_linear")
+        return self
 
     def c(self) -> LinearS:
         return LinearS(self.w.c(), self.bias.data_ptr() if self.bias is not None else None)
@@ -310,10 +334,17 @@ def qlstm_step(xq: torch.Tensor, x_act: Act, hq_in: torch.Tensor, c_in: torch.Te
         r["acc_ih"] = torch.empty((N, 4 * H), dtype=torch.int32, device=dev)
         r["acc_hh"] = torch.empty((N, 4 * H), dtype=torch.int32, device=dev)
     wih, whh = layer.w_ih.c(), layer.w_hh.c()
+    ws = None
+    if layer.prepared is not None:      # tensor-core path (taken by the library from 128 rows on)
+        need = workspace_bytes(WS_LSTM_STEP, [N, layer.w_ih.k_pad, H])
+        if layer.ws is None or layer.ws.numel() < need:
+            layer.ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        ws = layer.ws
     _chk(lib().qlstm_step(_p(xq), C.byref(x_act), _p(x_row_idx), _p(hq_in), _p(c_in), C.c_int32(N),
                           C.byref(wih), C.byref(whh), _p(layer.bias), C.byref(layer.hid_act),
                           _p(r.get("hq")), _p(r["c"]), _p(r.get("h")), _p(r.get("acc_ih")),
-                          _p(r.get("acc_hh")), _stream()), "qlstm_step")
+                          _p(r.get("acc_hh")), _p(layer.prepared), _p(ws),
+                          C.c_size_t(ws.numel() if ws is not None else 0), _stream()), "qlstm_step")
     return r
 
 
@@ -351,8 +382,15 @@ def q4_linear_forward(xq: torch.Tensor, x_act: Act, lin: DeviceLinear, want_acc:
     out = torch.empty((M, lin.w.rows), dtype=torch.float32, device=xq.device)
     acc = torch.empty((M, lin.w.rows), dtype=torch.int32, device=xq.device) if want_acc else None
     w = lin.w.c()
+    ws = None
+    if getattr(lin, "prepared", None) is not None and not want_acc:
+        need = workspace_bytes(WS_LINEAR, [M, lin.w.k_pad])
+        if lin.ws is None or lin.ws.numel() < need:
+            lin.ws = torch.empty(need, dtype=torch.uint8, device=xq.device)
+        ws = lin.ws
     _chk(lib().q4_linear_forward(_p(xq), C.byref(x_act), C.c_int32(M), C.byref(w), _p(lin.bias),
-                                 _p(out), _p(acc), _stream()), "q4_linear_forward")
+                                 _p(out), _p(acc), _p(getattr(lin, "prepared", None)), _p(ws),
+                                 C.c_size_t(ws.numel() if ws is not None else 0), _stream()), "q4_linear_forward")
     return (out, acc) if want_acc else out
 
 
@@ -364,13 +402,15 @@ def qjoint_logprobs(e: torch.Tensor, frame_idx: torch.Tensor, pq: torch.Tensor, 
     D, V = proj.w.rows, out.w.rows
     if logp is None:
         logp = torch.empty((N, V), dtype=torch.float32, device=pq.device)
-    need = workspace_bytes(WS_JOINT, [N, D])
+    tc = proj.prepared is not None and out.prepared is not None
+    need = workspace_bytes(WS_JOINT, [N, D] + ([proj.w.k_pad] if tc else []))
     if workspace is None or workspace.numel() < need:
         workspace = torch.empty(need, dtype=torch.uint8, device=pq.device)
     wp, wo = proj.w.c(), out.w.c()
     _chk(lib().qjoint_logprobs(_p(e), _p(frame_idx), _p(pq), C.byref(p_act), C.c_int32(N),
                                C.byref(wp), _p(proj.bias), C.byref(z_act), C.byref(wo), _p(out.bias),
-                               _p(logp), _p(workspace), C.c_size_t(workspace.numel()), _stream()),
+                               _p(logp), _p(proj.prepared if tc else None), _p(out.prepared if tc else None),
+                               _p(workspace), C.c_size_t(workspace.numel()), _stream()),
          "qjoint_logprobs")
     return logp
 
@@ -405,7 +445,7 @@ class Encoder:
 
     def __init__(self, enc, device="cuda"):
         self.layers = [[DeviceLstm(d, device) for d in dirs] for dirs in enc.layers]
-        self.proj = DeviceLinear(enc.proj, device) if enc.proj is not None else None
+        self.proj = DeviceLinear(enc.proj, device).prepare() if enc.proj is not None else None
         self.in_bits, self.in_max, self.in_clip = enc.in_bits, enc.in_max, enc.in_clip
         self.in_act = q4_act_symmetric(1.0 if enc.in_max else enc.in_clip, enc.in_bits)
         self.out_acts = []

@@ -156,7 +156,20 @@ size_t q4_workspace_bytes(int32_t call_id, const int32_t* dims, int32_t ndims) {
   }
   if (call_id == Q4_WS_JOINT && ndims >= 2) {
     const size_t N = dims[0], D = dims[1];
-    return align_up(N * D * sizeof(float)) + align_up(N * D);
+    size_t n = align_up(N * D * sizeof(float)) + align_up(N * D);
+    if (ndims >= 3) {   // tensor-core path: status word, int8 copies of the hidden codes and of z
+      const size_t Np = (N + 127) / 128 * 128, Hp = dims[2];
+      n += 256 + align_up(Np * Hp) + align_up(Np * D);
+    }
+    return n;
+  }
+  if (call_id == Q4_WS_LSTM_STEP && ndims >= 3) {   // status word, int8 copies of x and h rows
+    const size_t Np = ((size_t)dims[0] + 127) / 128 * 128;
+    return 256 + align_up(Np * (size_t)dims[1]) + align_up(Np * (size_t)dims[2]);
+  }
+  if (call_id == Q4_WS_LINEAR && ndims >= 2) {      // status word, int8 copy of the input rows
+    const size_t Np = ((size_t)dims[0] + 127) / 128 * 128;
+    return 256 + align_up(Np * (size_t)dims[1]);
   }
   if (call_id == Q4_WS_BEAM && ndims >= 4) {
     const size_t N = (size_t)dims[0] * dims[1], V = dims[2], D = dims[3];
@@ -214,12 +227,33 @@ int quantize_pack_int4(const void* x, int32_t x_is_fp16, int64_t rows, int32_t k
 }
 
 int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_mat* w,
-                      const float* bias, float* out, int32_t* dbg_acc, q4_stream stream) {
+                      const float* bias, float* out, int32_t* dbg_acc, const void* prepared,
+                      void* workspace, size_t workspace_bytes, q4_stream stream) {
   if (!xq || !out) return Q4_ERR_NULL;
   Q4_CHECK(check_act(x_act));
   Q4_CHECK(check_mat(w, 0, 0));
   if (M < 0) return Q4_ERR_DIM;
   if (!aligned16(xq) || !aligned16(out)) return Q4_ERR_ALIGN;
+  {
+    const int32_t wd[2] = {M, w->k_pad};
+    if (prepared && workspace && !dbg_acc && M >= 128 && aligned16(workspace) && aligned16(prepared) &&
+        workspace_bytes >= q4_workspace_bytes(Q4_WS_LINEAR, wd, 2)) {
+      // tensor cores: int8 copy of the input rows, then the tiled GEMM on the prepared int8 weights
+      cudaStream_t s = S(stream);
+      uint8_t* ws = static_cast<uint8_t*>(workspace);
+      int32_t* status = reinterpret_cast<int32_t*>(ws);
+      int8_t* x8 = reinterpret_cast<int8_t*>(ws + 256);
+      const int Mp = (M + 127) / 128 * 128;
+      TagScope tag(TAG_LINEAR);
+      Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
+      Q4_TRY(launch_unpack_rows(xq, row_bytes(w->k_pad, x_act->bits), nullptr, *x_act, w->k_pad, M, x8, w->k_pad, 0,
+                                Mp, s));
+      Q4_TRY(launch_mma_gemm(x8, w->k_pad, M, static_cast<const int8_t*>(prepared), w->k_pad, w->rows, w->k_pad,
+                             EPI_F32, out, w->rows, nullptr, w->scale, bias, x_act->scale, nullptr, status, nullptr,
+                             s));
+      return Q4_OK;
+    }
+  }
   GemmArgs g = gemm_args(xq, row_bytes(w->k_pad, x_act->bits), nullptr, *x_act, M, *w, bias, out,
                          w->rows, nullptr);
   g.dbg_acc = dbg_acc;
@@ -266,7 +300,8 @@ static void fill_lstm_weights(LstmArgs& a, const q4_mat& w_ih, const q4_mat& w_h
 int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, const void* hq_in,
                const float* c_in, int32_t N, const q4_mat* w_ih, const q4_mat* w_hh,
                const float* bias, const q4_act* hid_act, void* hq_out, float* c_out,
-               float* h_f32_out, int32_t* dbg_acc_ih, int32_t* dbg_acc_hh, q4_stream stream) {
+               float* h_f32_out, int32_t* dbg_acc_ih, int32_t* dbg_acc_hh, const void* prepared,
+               void* workspace, size_t workspace_bytes, q4_stream stream) {
   if (!xq || !hq_in || !c_in || !c_out) return Q4_ERR_NULL;
   if (!hq_out && !h_f32_out) return Q4_ERR_NULL;   // Inner placement needs the real-valued output
   int H = 0;
@@ -276,6 +311,55 @@ int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, co
   if (!aligned16(xq) || !aligned16(hq_in) || !aligned16(hq_out)) return Q4_ERR_ALIGN;
   if (N == 0) return Q4_OK;
   if (hq_out) ++g_quant_calls;   // the one quantizer call at the cell output (Outer placement)
+  {
+    const int32_t wd[3] = {N, w_ih->k_pad, H};
+    if (prepared && workspace && hq_out && N >= 128 && H % 128 == 0 && aligned16(workspace) && aligned16(prepared) &&
+        (dbg_acc_ih == nullptr) == (dbg_acc_hh == nullptr) && c_out != nullptr &&
+        workspace_bytes >= q4_workspace_bytes(Q4_WS_LSTM_STEP, wd, 3)) {
+      // tensor cores: int8 copies of the x rows (gathered) and h rows, then the fused LSTM kernel on the
+      // prepared int8 weights (rows 4*cell+gate, scales and bias in the same order)
+      cudaStream_t s = S(stream);
+      const size_t G = 4 * (size_t)H, Kx = w_ih->k_pad;
+      const uint8_t* pb = static_cast<const uint8_t*>(prepared);
+      const int8_t* xw8 = reinterpret_cast<const int8_t*>(pb);
+      const int8_t* hw8 = xw8 + align_up(G * Kx);
+      const float* sc_ih = reinterpret_cast<const float*>(hw8 + align_up(G * H));
+      const float* sc_hh = sc_ih + align_up(G * sizeof(float)) / sizeof(float);
+      const float* bi = sc_hh + align_up(G * sizeof(float)) / sizeof(float);
+      uint8_t* ws = static_cast<uint8_t*>(workspace);
+      int32_t* status = reinterpret_cast<int32_t*>(ws);
+      const int Np = (N + 127) / 128 * 128;
+      int8_t* x8 = reinterpret_cast<int8_t*>(ws + 256);
+      int8_t* h8 = x8 + align_up((size_t)Np * Kx);
+      TagScope tag(TAG_PRED_LSTM);
+      Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
+      Q4_TRY(launch_unpack_rows(xq, row_bytes(w_ih->k_pad, x_act->bits), x_row_idx, *x_act, (int)Kx, N, x8, (long long)Kx,
+                                0, Np, s));
+      Q4_TRY(launch_unpack_rows(hq_in, row_bytes(H, hid_act->bits), nullptr, *hid_act, H, N, h8, H, 0, Np, s));
+      MmaLstmArgs a;
+      memset(&a, 0, sizeof(a));
+      a.N = N;
+      a.H = H;
+      a.Kx_pad = (int)Kx;
+      a.sc_ih = sc_ih;
+      a.sc_hh = sc_hh;
+      a.bias = bi;
+      a.x_scale = x_act->scale;
+      a.hid_act = *hid_act;
+      a.out_act = *hid_act;
+      a.c_in = c_in;
+      a.c_out = c_out;
+      a.hq_out = static_cast<uint8_t*>(hq_out);
+      a.hq_ld = row_bytes(H, hid_act->bits);
+      a.h_f32 = h_f32_out;
+      a.dbg_ih = dbg_acc_ih;
+      a.dbg_hh = dbg_acc_hh;
+      a.dbg_ld = 4LL * H;
+      a.status = status;
+      Q4_TRY(launch_mma_lstm(a, x8, (long long)Kx, xw8, (long long)Kx, h8, H, hw8, H, s));
+      return Q4_OK;
+    }
+  }
   LstmArgs2 args;
   memset(&args, 0, sizeof(args));
   LstmArgs& a = args.d[0];
@@ -458,8 +542,8 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
 
 int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, const q4_act* p_act,
                     int32_t N, const q4_mat* w_pred, const float* b_pred, const q4_act* z_act,
-                    const q4_mat* w_out, const float* b_out, float* logp, void* workspace,
-                    size_t workspace_bytes, q4_stream stream) {
+                    const q4_mat* w_out, const float* b_out, float* logp, const void* prepared_pred,
+                    const void* prepared_out, void* workspace, size_t workspace_bytes, q4_stream stream) {
   if (!e || !frame_idx || !pq || !logp || !workspace) return Q4_ERR_NULL;
   Q4_CHECK(check_act(p_act));
   Q4_CHECK(check_act(z_act));
@@ -475,6 +559,41 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
   cudaStream_t s = S(stream);
   TagScope tag(TAG_JOINT);
   ++g_quant_calls;   // tanh(e * p)
+  const int32_t dims3[3] = {N, D, w_pred->k_pad};
+  if (prepared_pred && prepared_out && N >= 128 && V % 32 == 0 && z_act->is_signed && aligned16(prepared_pred) &&
+      aligned16(prepared_out) && workspace_bytes >= q4_workspace_bytes(Q4_WS_JOINT, dims3, 3)) {
+    // tensor cores, three launches: int8 copy of the hidden codes; projection GEMM whose epilogue forms
+    // tanh(e * p) and quantizes it; output layer with the log-softmax in its epilogue (fused head kernel
+    // when D = 256, else GEMM + row log-softmax)
+    const int Hp = w_pred->k_pad, Np = (N + 127) / 128 * 128;
+    uint8_t* ws = static_cast<uint8_t*>(workspace) + align_up((size_t)N * D * sizeof(float)) + align_up((size_t)N * D);
+    int32_t* status = reinterpret_cast<int32_t*>(ws);
+    int8_t* p8 = reinterpret_cast<int8_t*>(ws + 256);
+    int8_t* z8 = p8 + align_up((size_t)Np * Hp);
+    Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
+    Q4_TRY(launch_unpack_rows(pq, row_bytes(Hp, p_act->bits), nullptr, *p_act, Hp, N, p8, Hp, 0, Np, s));
+    Q4_TRY(launch_mma_gemm(p8, Hp, N, static_cast<const int8_t*>(prepared_pred), Hp, D, Hp, EPI_JOINTZ, z8, D,
+                           nullptr, w_pred->scale, b_pred, p_act->scale, z_act, status, nullptr, s, false, e,
+                           frame_idx));
+    if (D == 256 && V <= 2048) {
+      LmHeadArgs ja;
+      memset(&ja, 0, sizeof(ja));
+      ja.N = N;
+      ja.H = 0;
+      ja.V = V;
+      ja.q_scale = z_act->scale;
+      ja.sc_out = w_out->scale;
+      ja.b_out = b_out;
+      ja.lp = logp;
+      ja.status = status;
+      Q4_TRY(launch_mma_lmhead(ja, z8, D, nullptr, static_cast<const int8_t*>(prepared_out), s, false));
+    } else {
+      Q4_TRY(launch_mma_gemm(z8, D, N, static_cast<const int8_t*>(prepared_out), D, V, D, EPI_F32, logp, V, nullptr,
+                             w_out->scale, b_out, z_act->scale, nullptr, status, nullptr, s));
+      Q4_TRY(launch_logsoftmax(logp, logp, N, V, V, nullptr, s));
+    }
+    return Q4_OK;
+  }
   float* p = static_cast<float*>(workspace);
   uint8_t* zq = static_cast<uint8_t*>(workspace) + align_up((size_t)N * D * sizeof(float));
   GemmArgs g1 = gemm_args(pq, row_bytes(w_pred->k_pad, p_act->bits), nullptr, *p_act, N, *w_pred,
@@ -589,6 +708,47 @@ int q4_prepare_model(q4_model* model, void* buffer, size_t bytes, q4_stream stre
     Q4_TRY(launch_prepare_w(L->w, 0, reinterpret_cast<int8_t*>(b + p.lin[i]), L->w.k_pad, 0, s));
   }
   model->prepared = buffer;
+  return Q4_OK;
+}
+
+// One-time int8 operands for the tensor-core variants of the step calls.
+size_t q4_prepared_lstm_bytes(const q4_mat* w_ih, const q4_mat* w_hh) {
+  if (!w_ih || !w_hh) return 0;
+  const size_t G = w_ih->rows;
+  return align_up(G * w_ih->k_pad) + align_up(G * w_hh->k_pad) + 3 * align_up(G * sizeof(float));
+}
+int q4_prepare_lstm(const q4_mat* w_ih, const q4_mat* w_hh, const float* bias, void* buffer, size_t bytes,
+                    q4_stream stream) {
+  if (!buffer) return Q4_ERR_NULL;
+  Q4_CHECK(check_mat(w_ih, 0, 0));
+  Q4_CHECK(check_mat(w_hh, 0, 0));
+  if (w_ih->rows != w_hh->rows || w_ih->rows % 4 != 0) return Q4_ERR_DIM;
+  if (!aligned16(buffer)) return Q4_ERR_ALIGN;
+  if (bytes < q4_prepared_lstm_bytes(w_ih, w_hh)) return Q4_ERR_WORKSPACE;
+  cudaStream_t s = S(stream);
+  const size_t G = w_ih->rows;
+  uint8_t* b = static_cast<uint8_t*>(buffer);
+  int8_t* xw8 = reinterpret_cast<int8_t*>(b);
+  int8_t* hw8 = xw8 + align_up(G * w_ih->k_pad);
+  float* sc_ih = reinterpret_cast<float*>(hw8 + align_up(G * w_hh->k_pad));
+  float* sc_hh = sc_ih + align_up(G * sizeof(float)) / sizeof(float);
+  float* bi = sc_hh + align_up(G * sizeof(float)) / sizeof(float);
+  TagScope tag(TAG_MISC);
+  Q4_TRY(launch_prepare_w(*w_ih, 1, xw8, w_ih->k_pad, 0, s));
+  Q4_TRY(launch_prepare_w(*w_hh, 1, hw8, w_hh->k_pad, 0, s));
+  Q4_TRY(launch_prepare_vec(w_ih->scale, (int)G, 1, sc_ih, s));
+  Q4_TRY(launch_prepare_vec(w_hh->scale, (int)G, 1, sc_hh, s));
+  Q4_TRY(launch_prepare_vec(bias, (int)G, 1, bi, s));
+  return Q4_OK;
+}
+size_t q4_prepared_linear_bytes(const q4_mat* w) { return w ? align_up((size_t)w->rows * w->k_pad) : 0; }
+int q4_prepare_linear(const q4_mat* w, void* buffer, size_t bytes, q4_stream stream) {
+  if (!buffer) return Q4_ERR_NULL;
+  Q4_CHECK(check_mat(w, 0, 0));
+  if (!aligned16(buffer)) return Q4_ERR_ALIGN;
+  if (bytes < q4_prepared_linear_bytes(w)) return Q4_ERR_WORKSPACE;
+  TagScope tag(TAG_MISC);
+  Q4_TRY(launch_prepare_w(*w, 0, static_cast<int8_t*>(buffer), w->k_pad, 0, S(stream)));
   return Q4_OK;
 }
 

@@ -101,7 +101,8 @@ struct LmHeadArgs {
 };
 cudaError_t launch_mma_lmhead(const LmHeadArgs& a, const int8_t* h8, long long h_pitch, const int8_t* wb8,
                               const int8_t* wo8, cudaStream_t s, bool dependent = false);
-enum { EPI_QUANT8 = 3 };    // re-quantize and store (code - zero_point) as int8, one per byte
+enum { EPI_QUANT8 = 3,      // re-quantize and store (code - zero_point) as int8, one per byte
+       EPI_JOINTZ = 4 };    // tanh(other factor * value), quantized, stored like EPI_QUANT8
 cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
                                const q4_act& act, int k_pad, int n_rows, int8_t* dst,
                                long long dst_stride, int col0, int n_rows_pad, cudaStream_t s);
@@ -127,7 +128,8 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
                             const int32_t* out_idx, const float* w_scale, const float* bias,
                             float x_scale, const q4_act* out_act, int32_t* status,
-                            const int32_t* n_active, cudaStream_t s, bool dependent = false);
+                            const int32_t* n_active, cudaStream_t s, bool dependent = false,
+                            const float* mul_e = nullptr, const int32_t* mul_idx = nullptr);
 cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa_pitch,
                             const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
                             const int8_t* hw, long long hw_pitch, cudaStream_t s, bool dependent = false);

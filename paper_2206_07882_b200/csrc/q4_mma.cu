@@ -280,6 +280,8 @@ struct MmaGemmArgs {
   q4_act out_act;
   int32_t* status;
   const int32_t* n_active;
+  const float* mul_e;       // EPI_JOINTZ: the other factor, row mul_idx[m] of [*, J] fp32
+  const int32_t* mul_idx;
 };
 
 __global__ void __launch_bounds__(192, 1)
@@ -382,6 +384,18 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = __fmaf_rn((float)r[i], s_sc[c0 + i], s_bi[c0 + i]);
+        if (a.epi == EPI_JOINTZ) {
+          // joint network: z = tanh(e * p) with p the projected value just formed; quantized below
+          const float* er = a.mul_e + (long long)a.mul_idx[mi] * a.J + j0;
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            const float4 ev = *reinterpret_cast<const float4*>(er + i);
+            v[i] = tanh_fixed(__fmul_rn(ev.x, v[i]));
+            v[i + 1] = tanh_fixed(__fmul_rn(ev.y, v[i + 1]));
+            v[i + 2] = tanh_fixed(__fmul_rn(ev.z, v[i + 2]));
+            v[i + 3] = tanh_fixed(__fmul_rn(ev.w, v[i + 3]));
+          }
+        }
         if (a.epi == EPI_F32) {
           float* o = reinterpret_cast<float*>(a.out) + (long long)m * a.ldo + j0;
           if (j0 + 32 <= a.J && (reinterpret_cast<uintptr_t>(o) & 31) == 0) {
@@ -398,7 +412,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
         } else {  // EPI_QUANT / EPI_QUANT8 (J a multiple of 32)
           const int lo = act_lo(a.out_act), hi = act_hi(a.out_act);
           uint8_t* o = reinterpret_cast<uint8_t*>(a.out) + (long long)m * a.ldo;
-          if (a.epi == EPI_QUANT8) {
+          if (a.epi == EPI_QUANT8 || a.epi == EPI_JOINTZ) {
             uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
             for (int i = 0; i < 32; ++i)
@@ -604,8 +618,10 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
                             long long w_pitch, int J, int K, int epi, void* out, long long ldo,
                             const int32_t* out_idx, const float* w_scale, const float* bias,
                             float x_scale, const q4_act* out_act, int32_t* status,
-                            const int32_t* n_active, cudaStream_t s, bool dependent) {
+                            const int32_t* n_active, cudaStream_t s, bool dependent, const float* mul_e,
+                            const int32_t* mul_idx) {
   if (M <= 0 || J <= 0) return cudaSuccess;
+  if (epi == EPI_JOINTZ && (!mul_e || !mul_idx || J % 32 != 0)) return cudaErrorInvalidValue;
   CUtensorMap ta, tb;
   if (!make_tmap_i8(&ta, x8, K, M, x_pitch, BM) || !make_tmap_i8(&tb, w8, K, J, w_pitch, GEMM_BN))
     return cudaErrorInvalidValue;
@@ -624,6 +640,8 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
   if (out_act) a.out_act = *out_act;
   a.status = status;
   a.n_active = n_active;
+  a.mul_e = mul_e;
+  a.mul_idx = mul_idx;
   const size_t smem = (size_t)GEMM_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
   const size_t smem_p = (size_t)PG_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
   static bool configured = false;

@@ -55,6 +55,6 @@ extern "C" int qjoint_logprobs_static(const float* e, const int32_t* frame_idx, 
   if (r != Q4_OK) return r;
   // Same kernels as qjoint_logprobs; every scratch element that is read is written first by
   // the call itself, so nothing has to be cleared between calls.
-  return qjoint_logprobs(e, frame_idx, pq, p_act, N, w_pred, b_pred, z_act, w_out, b_out, logp, scratch,
-                         Q4_JOINT_STATIC_BYTES, stream);
+  return qjoint_logprobs(e, frame_idx, pq, p_act, N, w_pred, b_pred, z_act, w_out, b_out, logp, nullptr, nullptr,
+                         scratch, Q4_JOINT_STATIC_BYTES, stream);
 }

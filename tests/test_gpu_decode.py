@@ -20,8 +20,13 @@ def Bd():
     return binding
 
 
-@pytest.mark.parametrize("N,V,D,Hp,zb", [(5, 64, 32, 64, 4), (70, 1024, 256, 1024, 4), (33, 200, 64, 96, 8)])
-def test_joint_logprobs(Bd, N, V, D, Hp, zb):
+@pytest.mark.parametrize("N,V,D,Hp,zb,prep", [(5, 64, 32, 64, 4, False), (70, 1024, 256, 1024, 4, False),
+                                                  (33, 200, 64, 96, 8, False),
+                                                  # tensor-core path: fused head (D = 256), ragged last row tile;
+                                                  # GEMM + row log-softmax (D = 64); 8-bit output layer
+                                                  (200, 1024, 256, 1024, 4, True), (130, 96, 64, 128, 4, True),
+                                                  (257, 992, 256, 256, 8, True)])
+def test_joint_logprobs(Bd, N, V, D, Hp, zb, prep):
     dw = synth.decoder(seed=5, V=V, E=32, Hp=Hp, D=D, Hs=32, Ht=32, out_bits=zb)
     dec = O.Decoder(dw)
     st = synth.Stream(9)
@@ -33,8 +38,13 @@ def test_joint_logprobs(Bd, N, V, D, Hp, zb):
     p = O.linear(O.Linear(dw.pred.proj), pq, hid)
     want = O.joint(dec, e[fi], p)
     dd = Bd.Decoder(dw)
+    if prep:
+        dd.pred_proj.prepare()
+        dd.joint_out.prepare()
+    n0 = Bd.launch_count()
     got = Bd.qjoint_logprobs(torch.from_numpy(e).cuda(), torch.from_numpy(fi).cuda(), pack_codes(pq, hid),
                              to_act(hid), dd.pred_proj, dd.z_act, dd.joint_out).cpu().numpy()
+    assert Bd.launch_count() - n0 == ((3 if D == 256 else 4) if prep else 4)
     assert np.abs(got - want).max() <= LP_ATOL
     np.testing.assert_allclose(np.exp(got.astype(np.float64)).sum(1), 1.0, atol=1e-5)
 
@@ -43,6 +53,10 @@ def pred_joint_gpu(Bd, dd, e_dev, frame_idx, tokens):
     """Teacher-forced prediction network + joint on the GPU: logp [N,S,V], hq codes [N,S,Hp]."""
     N, S = tokens.shape
     Hp, V = dd.pred_lstm.H, dd.V
+    # one-time int8 operands: from 128 rows on these calls run on the tensor-core kernels
+    dd.pred_lstm.prepare()
+    dd.pred_proj.prepare()
+    dd.joint_out.prepare()
     hq = torch.zeros((N, Hp // 2), dtype=torch.uint8, device="cuda")
     c = torch.zeros((N, Hp), dtype=torch.float32, device="cuda")
     tok = torch.from_numpy(tokens).cuda()

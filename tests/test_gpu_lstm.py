@@ -18,10 +18,12 @@ def Bd():
     return binding
 
 
-def step_case(Bd, lw, x_act, hid, xq, hq, c):
+def step_case(Bd, lw, x_act, hid, xq, hq, c, prepare=False):
     L = O.Lstm([lw])
     want = O.lstm_step(L, xq, x_act, hq, c, hid)
     dl = Bd.DeviceLstm(lw)
+    if prepare:
+        dl.prepare()
     assert dl.hid_act.scale == hid.scale
     got = Bd.qlstm_step(pack_codes(xq, x_act, dl.w_ih.k_pad), to_act(x_act), pack_codes(hq, hid),
                         torch.from_numpy(c).cuda(), dl, want_dbg=True)
@@ -319,3 +321,24 @@ def test_outer_and_inner_quantizer_placement_counted_on_the_device(Bd):
     np.testing.assert_array_equal(gpu_codes(xq, 64, dev.out_acts[-1]).reshape(T, B, 64), ref["yq"])
     np.testing.assert_array_equal(x.cpu().numpy(), ref["layers"][-1]["h"])
     np.testing.assert_array_equal(x.cpu().numpy(), O.encoder_forward_inner(E, enc["features"]))
+
+
+@pytest.mark.parametrize("N,K,H,xb,hb,signed", [(130, 256, 128, 4, 4, True), (300, 96, 256, 4, 4, False),
+                                                 (128, 240, 128, 8, 8, True), (257, 64, 384, 4, 8, True)])
+def test_step_on_the_tensor_cores_with_prepared_weights(Bd, N, K, H, xb, hb, signed):
+    # qlstm_step with the one-time int8 operands: tcgen05 kernel, same integers and floats as the oracle
+    st = synth.Stream(400 + N)
+    lw = synth._lstm(st, "l", K, H, 4, bias_std=0.2, hid_alpha=0.95, hid_bits=hb)
+    if xb == 8:
+        lw.w_ih = synth._qmat(st, "w8", 4 * H, K, 8)
+    if hb == 8:
+        lw.w_hh = synth._qmat(st, "h8", 4 * H, H, 8)
+    x_act = O.act_symmetric(3.0, xb) if signed else O.act_asymmetric(-1.7, 1.4, 4)
+    hid = O.act_symmetric(0.95, hb)
+    xq = st.integers("xq", (N, K), x_act.lo(), x_act.hi()).astype(np.int16)
+    hq = st.integers("hq", (N, H), hid.lo() + 1, hid.hi()).astype(np.int16)
+    c = st.normal("c", (N, H)).astype(np.float32)
+    n0 = Bd.launch_count()
+    step_case(Bd, lw, x_act, hid, xq, hq, c, prepare=True)
+    # packing of the test operands aside: two gathers and one fused kernel (not the DP4A kernel alone)
+    assert Bd.launch_count() - n0 >= 3

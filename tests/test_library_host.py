@@ -76,7 +76,7 @@ def test_argument_errors_are_reported_on_the_host(Bd):
     w_hh = Bd.Mat(4096, 4096, 128, 32, 32, 4)
     args = lambda x_act, wi=w_ih, wh=w_hh, hin=fake, hout=C.c_void_p(8192): lib.qlstm_step(
         fake, C.byref(x_act), None, hin, fake, 4, C.byref(wi), C.byref(wh), None, C.byref(ok), hout,
-        fake, None, None, None, None)
+        fake, None, None, None, None, None, C.c_size_t(0), None)
     assert args(ok, wi=Bd.Mat(4096, 4096, 128, 64, 64, 3)) == -4
     assert args(ok, wi=Bd.Mat(4096, 4096, 128, 32, 32, 2)) == -3
     assert args(ok, wi=Bd.Mat(4096, 4096, 128, 60, 60, 4)) == -3
