@@ -392,6 +392,18 @@ int q4_dependent_launch_set(int32_t enabled);
  * take the exact search (for tests; both give the same beam).  Returns the previous setting. */
 int q4_beam_select_exact_set(int32_t enabled);
 
+/* Test hook for the bounded device-side waits (not an operation of the paper): while skip_producer
+ * is non-zero the tiled tensor-core GEMM (the tensor-core paths of q4_linear_forward and of the
+ * projections) launches with a producer that issues no copy at all, so that the consumer's wait
+ * runs out after wait_limit polls (0 = the normal limit); nothing asynchronous is in flight, every
+ * thread of the kernel still reaches its final barrier, tensor memory is freed, nothing is stored
+ * and the status word reads Q4_ERR_TIMEOUT.  (0, 0) restores normal operation.  Process-wide. */
+int q4_test_wait_expiry_set(int32_t skip_producer, uint32_t wait_limit);
+
+/* Threads: the library keeps a few process-wide host variables (launch and quantizer counters, the
+ * timing hook, the switches above); calls from several host threads must be serialised by the
+ * caller. */
+
 /* Optional timing of the library's own launches with CUDA events lent by the caller (host
  * arrays of cudaEvent_t, `capacity` entries each).  Every launch whose tag bit is set in
  * tag_mask records start_events[i] before and stop_events[i] after itself on the stream it

@@ -98,6 +98,10 @@ int q4_beam_select_exact_set(int32_t enabled) {
   g_select_exact = enabled ? 1 : 0;
   return prev;
 }
+int q4_test_wait_expiry_set(int32_t skip_producer, uint32_t wait_limit) {
+  test_wait_expiry_set(skip_producer ? 1 : 0, wait_limit);
+  return Q4_OK;
+}
 int q4_dependent_launch_set(int32_t enabled) {
   const int prev = g_dependent_launch;
   g_dependent_launch = enabled ? 1 : 0;

@@ -130,6 +130,7 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
                             float x_scale, const q4_act* out_act, int32_t* status,
                             const int32_t* n_active, cudaStream_t s, bool dependent = false,
                             const float* mul_e = nullptr, const int32_t* mul_idx = nullptr);
+void test_wait_expiry_set(int skip_producer, uint32_t wait_limit);
 cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa_pitch,
                             const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
                             const int8_t* hw, long long hw_pitch, cudaStream_t s, bool dependent = false);

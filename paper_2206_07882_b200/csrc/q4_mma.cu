@@ -282,7 +282,17 @@ struct MmaGemmArgs {
   const int32_t* n_active;
   const float* mul_e;       // EPI_JOINTZ: the other factor, row mul_idx[m] of [*, J] fp32
   const int32_t* mul_idx;
+  uint32_t wait_limit;      // polls before a wait gives up
+  int32_t skip_producer;    // test hook: the producer issues no copy, so the consumer's wait runs out
 };
+
+// Test hook (q4_test_wait_expiry_set): the next launches of k_mma_gemm get this limit and flag.
+static uint32_t g_wait_limit = 1u << 22;
+static int g_skip_producer = 0;
+void test_wait_expiry_set(int skip_producer, uint32_t wait_limit) {
+  g_skip_producer = skip_producer;
+  g_wait_limit = wait_limit ? wait_limit : (1u << 22);
+}
 
 __global__ void __launch_bounds__(192, 1)
 k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b,
@@ -322,9 +332,9 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
     // whole tile without work
   } else if (warp == 4 && lane == 0) {
     bool ok = true;
-    for (int i = 0; i < nk && ok; ++i) {
+    for (int i = 0; i < nk && ok && !a.skip_producer; ++i) {
       const int s = i % GEMM_STAGES;
-      if (i >= GEMM_STAGES) ok = mbar_wait(&empty[s], ((i / GEMM_STAGES) - 1) & 1);
+      if (i >= GEMM_STAGES) ok = mbar_wait(&empty[s], ((i / GEMM_STAGES) - 1) & 1, a.wait_limit);
       if (!ok) break;
       mbar_expect_tx(&full[s], STAGE);
       tma_load_2d(smem + s * STAGE, &tma_a, i * BK, m0, &full[s]);
@@ -337,7 +347,7 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
     bool ok = true;
     for (int i = 0; i < nk && ok; ++i) {
       const int s = i % GEMM_STAGES;
-      ok = mbar_wait(&full[s], (i / GEMM_STAGES) & 1);
+      ok = mbar_wait(&full[s], (i / GEMM_STAGES) & 1, a.wait_limit);
       if (!ok) break;
       tc_fence_after();
       const uint64_t da = umma_desc_sw128(smem_u32(smem + s * STAGE));
@@ -346,9 +356,12 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
       for (int kk = 0; kk < BK / 32; ++kk) umma_i8(tmem, da + 2 * kk, db + 2 * kk, idesc, (i | kk) != 0);
       umma_commit(&empty[s]);
     }
+    if (!ok) {   // recorded before the epilogue is released, so that it stores nothing
+      flag_timeout(a.status);
+      __threadfence();
+    }
     umma_commit(&acc_full);
     pdl_trigger();
-    if (!ok) flag_timeout(a.status);
   } else if (warp < 4) {
     if (a.epi != EPI_I32) {   // stage scale * row scale and bias while the MMAs run
       for (int c = tid; c < GEMM_BN; c += 128) {
@@ -358,7 +371,8 @@ k_mma_gemm(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CU
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
     }
-    const bool ok = mbar_wait(&acc_full, 0);
+    bool ok = mbar_wait(&acc_full, 0, a.wait_limit);
+    if (ok && a.status && *reinterpret_cast<volatile int32_t*>(a.status) != 0) ok = false;   // a wait gave up somewhere
     tc_fence_after();
     pdl_trigger();   // the main loop is over: the next kernel may set itself up
     if (!ok && lane == 0) flag_timeout(a.status);
@@ -642,6 +656,8 @@ cudaError_t launch_mma_gemm(const int8_t* x8, long long x_pitch, int M, const in
   a.n_active = n_active;
   a.mul_e = mul_e;
   a.mul_idx = mul_idx;
+  a.wait_limit = g_wait_limit;
+  a.skip_producer = g_skip_producer;
   const size_t smem = (size_t)GEMM_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
   const size_t smem_p = (size_t)PG_STAGES * (BM * BK + GEMM_BN * BK) + 1024;
   static bool configured = false;

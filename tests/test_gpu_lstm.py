@@ -342,3 +342,30 @@ def test_step_on_the_tensor_cores_with_prepared_weights(Bd, N, K, H, xb, hb, sig
     step_case(Bd, lw, x_act, hid, xq, hq, c, prepare=True)
     # packing of the test operands aside: two gathers and one fused kernel (not the DP4A kernel alone)
     assert Bd.launch_count() - n0 >= 3
+
+
+def test_bounded_wait_runs_out_and_the_stream_stays_usable(Bd):
+    # The consumer of the tiled tensor-core GEMM waits for operand tiles a bounded number of polls.  With
+    # the test hook the producer issues nothing (so nothing asynchronous is in flight): the wait runs
+    # out, every role of the kernel returns, the status word reads Q4_ERR_TIMEOUT, nothing was stored,
+    # and the next call on the same stream is correct.
+    import ctypes as C
+    st = synth.Stream(77)
+    M, K, J = 200, 256, 256
+    lw = synth._linear(st, "lin", J, K)
+    a = O.act_symmetric(1.0, 4)
+    xq = st.integers("xq", (M, K), -7, 7).astype(np.int16)
+    want = O.linear(O.Linear(lw), xq, a)
+    lin = Bd.DeviceLinear(lw).prepare()
+    x_dev = pack_codes(xq, a)
+    lib = Bd.lib()
+    assert lib.q4_test_wait_expiry_set(C.c_int32(1), C.c_uint32(1 << 12)) == 0
+    try:
+        out = Bd.q4_linear_forward(x_dev, to_act(a), lin)
+        assert Bd.q4_poll_status(lin.ws) == -8                      # Q4_ERR_TIMEOUT
+    finally:
+        lib.q4_test_wait_expiry_set(C.c_int32(0), C.c_uint32(0))
+    torch.cuda.synchronize()
+    out = Bd.q4_linear_forward(x_dev, to_act(a), lin)               # same stream, same buffers
+    assert Bd.q4_poll_status(lin.ws) == 0
+    np.testing.assert_array_equal(out.cpu().numpy(), want)
