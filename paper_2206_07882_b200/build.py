@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libq4rnnt.so")
-SOURCES = ["q4_kernels.cu", "q4_beam.cu", "q4_mma.cu", "q4_recurrent.cu", "q4_api.cu", "q4_noalloc.cu"]
+SOURCES = ["q4_kernels.cu", "q4_beam.cu", "q4_mma.cu", "q4_recurrent.cu", "q4_skinny.cu", "q4_api.cu", "q4_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -930,9 +930,18 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     const PrepPlan pp = plan_prepared(m);
     const uint8_t* pb = static_cast<const uint8_t*>(m.prepared);
 
+    // at most 32 hypothesis rows (one utterance): the LSTM steps are bound by reading the weights once,
+    // and a weight-streaming kernel reads them as stored (packed 4-bit), the state rows and embedding
+    // rows too, so the gathers below are not needed
+    const bool skinny =
+        skinny_lstm_supported(N, Hp, Ep, m.pred_lstm.w_ih.bits, m.pred_lstm.w_hh.bits, m.pred_emb_act, m.pred_lstm.hid_act) &&
+        skinny_lstm_supported(N, Hs, Ep, m.src.lstm[0].w_ih.bits, m.src.lstm[0].w_hh.bits, m.src.emb_act, m.src.lstm[0].hid_act) &&
+        skinny_lstm_supported(N, Ht, Ep, m.tgt.lstm[0].w_ih.bits, m.tgt.lstm[0].w_hh.bits, m.tgt.emb_act, m.tgt.lstm[0].hid_act) &&
+        (m.tgt.n_layers == 1 || skinny_lstm_supported(N, Ht, Ht, m.tgt.lstm[1].w_ih.bits, m.tgt.lstm[1].w_hh.bits,
+                                                      m.tgt.lstm[0].hid_act, m.tgt.lstm[1].hid_act));
     // all gathers of the iteration in one launch: embedding rows by pending symbol, previous
     // cell-output codes by parent state row, unpacked to int8 operand rows
-    if (nets) {
+    if (nets && !skinny) {
       UnpackJobs uj;
       memset(&uj, 0, sizeof(uj));
       auto add = [&](const void* src, long long stride, const int32_t* idx, const q4_act& act, int k_pad,
@@ -990,6 +999,38 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
                         int trigger_early = 0) -> int {
       TagScope tag(tag_id);
       const int H = L.w_hh.k_pad, Kx = L.w_ih.k_pad;
+      if (skinny) {
+        // x rows: the embedding table by pending symbol, or (second layer) the first layer's fresh state rows
+        const bool second = li == 3;
+        SkinnyLstmArgs k;
+        memset(&k, 0, sizeof(k));
+        k.N = N;
+        k.H = H;
+        k.Kx = Kx;
+        k.w_ih = static_cast<const uint8_t*>(L.w_ih.q);
+        k.w_hh = static_cast<const uint8_t*>(L.w_hh.q);
+        k.s_wih = L.w_ih.scale;
+        k.s_whh = L.w_hh.scale;
+        k.bias = L.bias;
+        k.x = static_cast<const uint8_t*>(second ? st.tgt_hq[0] : li == 0 ? m.pred_emb_q : li == 1 ? m.src.emb_q : m.tgt.emb_q);
+        k.x_stride = row_bytes(Kx, 4);
+        k.x_idx = second ? cst.adv_dst : cst.adv_tok;
+        k.x_signed = x_act.is_signed;
+        k.x_zp = x_act.zero_point;
+        k.x_scale = x_act.scale;
+        k.hid_act = L.hid_act;
+        k.hq_in = static_cast<const uint8_t*>(hq);
+        k.c_in = c;
+        k.src_row = cst.adv_src;
+        k.dst_row = cst.adv_dst;
+        k.hq_out = static_cast<uint8_t*>(hq);
+        k.c_out = c;
+        k.h8_out = h8;
+        k.h8_ld = H;
+        k.n_active = n_active;
+        Q4_TRY(launch_skinny_lstm(k, s, dep));
+        return Q4_OK;
+      }
       MmaLstmArgs a;
       memset(&a, 0, sizeof(a));
       a.N = N;

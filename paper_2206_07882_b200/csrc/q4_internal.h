@@ -135,6 +135,34 @@ cudaError_t launch_mma_lstm(const MmaLstmArgs& a, const int8_t* xa, long long xa
                             const int8_t* xw, long long xw_pitch, const int8_t* ha, long long ha_pitch,
                             const int8_t* hw, long long hw_pitch, cudaStream_t s, bool dependent = false);
 
+// ---- weight-streaming LSTM step for at most 32 rows (q4_skinny.cu)
+struct SkinnyLstmArgs {
+  int32_t N, H, Kx;         // launch rows (<= 32), cells, input width (both multiples of 128)
+  const uint8_t* w_ih;      // packed 4-bit [4H, Kx], gate blocks i, f, g, o
+  const uint8_t* w_hh;      // packed 4-bit [4H, H]
+  const float* s_wih;       // [4H] row scales
+  const float* s_whh;
+  const float* bias;        // [4H] or null
+  const uint8_t* x;         // packed 4-bit input code rows, row n at x + x_idx[n] * x_stride
+  long long x_stride;
+  const int32_t* x_idx;     // null = n, negative = zero row
+  int32_t x_signed, x_zp;
+  float x_scale;
+  q4_act hid_act;
+  const uint8_t* hq_in;     // packed state rows [*, H/2], row src_row[n] (negative = zero state)
+  const float* c_in;        // [*, H], same rows
+  const int32_t* src_row;   // null = n
+  const int32_t* dst_row;   // null = n, negative = row inactive
+  uint8_t* hq_out;          // packed codes at dst row
+  float* c_out;
+  int8_t* h8_out;           // int8 codes at launch row n (nullable)
+  long long h8_ld;
+  const int32_t* n_active;  // optional device count: rows >= *n_active carry no work
+};
+bool skinny_lstm_supported(int N, int H, int Kx, int w_bits_ih, int w_bits_hh, const q4_act& x_act,
+                           const q4_act& hid_act);
+cudaError_t launch_skinny_lstm(const SkinnyLstmArgs& a, cudaStream_t s, bool dependent = false);
+
 // ---- persistent encoder recurrence (q4_recurrent.cu)
 struct EncRecDir {
   const int8_t* w_hh;       // int8 [4H, H], rows in 4*cell+gate order

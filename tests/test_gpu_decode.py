@@ -527,3 +527,16 @@ def test_search_all_eight_bit(Bd, dims):
     assert dd.tensors["pred_hq"].shape[1] == dims["Hp"]           # one byte per hidden code
     frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(8)), 10, 6, 16, min_same=1.0)
     assert tr == 1.0
+
+
+@pytest.mark.parametrize("B,W", [(1, 5), (1, 16), (2, 16), (3, 7)])
+def test_search_few_rows_weight_streaming_kernels(Bd, B, W):
+    # at most 32 hypothesis rows and widths that are multiples of 128: the LSTM steps run on the
+    # weight-streaming kernel that reads packed 4-bit weights, state rows and embedding rows as stored
+    # (signed prediction-network input, unsigned LM input with its zero point); every beam of every
+    # iteration as the oracle's
+    dw = synth.decoder(seed=99, V=128, E=128, Hp=128, D=256, Hs=128, Ht=256, tgt_layers=2, U_max=6, W=W)
+    e = synth.Stream(17).normal("e", (9, B, 256)).astype(np.float32)
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e)
+    frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(B)), 9, 6, W, min_same=1.0)
+    assert tr == 1.0
