@@ -3,8 +3,10 @@
 // reading the weights once, so they are read as stored: packed 4-bit codes, 128-bit loads, no int8
 // copies, no staging through shared memory.
 //
-// One CTA owns the 16 weight rows of 4 cells (their i, f, g, o rows); its 8 warps split K in chunks
-// of 128 codes (the input part, then the recurrent part).  A lane loads 16 bytes (32 codes) of two
+// One CTA owns the 16 weight rows of 4 cells (their i, f, g, o rows); its 16 warps split K in chunks
+// of 128 codes (the input part, then the recurrent part); a warp fetches its next chunk while it
+// multiplies the present one.  Four CTAs fit an SM, so all CTAs of a layer (at most 512) are resident
+// together and the whole weight matrix is requested within the first microsecond.  A lane loads 16 bytes (32 codes) of two
 // weight rows and of one activation row per 8-row tile and chunk and turns every 32-bit word (8 codes)
 // into two operand registers of the warp-level int8 MMA m16n8k32 by two masks and a shift: the
 // even-numbered codes of the word, each in the high nibble of a byte (16 x code), and the odd-numbered
@@ -24,6 +26,7 @@ namespace q4 {
 
 constexpr int SK_WARPS = 8;
 constexpr int SK_THREADS = 32 * SK_WARPS;
+constexpr int SK_CTAS_PER_SM = 4;   // registers are capped so that every CTA of a layer is resident at once
 
 __device__ __forceinline__ void mma_s8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -42,11 +45,17 @@ __device__ __forceinline__ void mma_s8u8(int (&c)[4], uint32_t a0, uint32_t a1, 
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void cp_async4(float* dst_smem, const float* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src)
+               : "memory");
+}
+
 template <int NT>
-__global__ void __launch_bounds__(SK_THREADS) k_skinny_lstm(const SkinnyLstmArgs a) {
+__global__ void __launch_bounds__(SK_THREADS, NT == 4 ? 2 : SK_CTAS_PER_SM) k_skinny_lstm(const SkinnyLstmArgs a) {
   // partial sums: [warp][part: input, recurrent][16 tile rows][8 NT rows], and the weight row sums
-  __shared__ int part[SK_WARPS][2][16][8 * NT];
-  __shared__ int wsum[SK_WARPS][16];
+  extern __shared__ __align__(16) int sk_smem[];
+  int (*part)[2][16][8 * NT] = reinterpret_cast<int (*)[2][16][8 * NT]>(sk_smem);
+  int (*wsum)[16] = reinterpret_cast<int (*)[16]>(sk_smem + SK_WARPS * 2 * 16 * 8 * NT);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t4 = lane & 3;
   const int e = g & 1, ci = g >> 1;
@@ -55,26 +64,53 @@ __global__ void __launch_bounds__(SK_THREADS) k_skinny_lstm(const SkinnyLstmArgs
   // tile row g = gate e of cell ci, tile row g + 8 = gate 2 + e of the same cell
   const long long r0 = (long long)e * H + cell0 + ci, r1 = (long long)(2 + e) * H + cell0 + ci;
   const int nxc = a.Kx >> 7, nhc = H >> 7;
+  const uint32_t M = 0xF0F0F0F0u;
+  const bool x_unsigned = a.x_signed == 0;
 
+  // the de-quantization constants of the thread's item of the closing stage (cell ec of the CTA's 4,
+  // row en) do not depend on the previous kernel of the stream: they are sent on their way to shared
+  // memory first (row scales and bias of the item's four gate rows; no registers are held for them)
+  const int ec = tid & 3, en = tid >> 2;
+  float* ecst = reinterpret_cast<float*>(sk_smem + SK_WARPS * 2 * 16 * 8 * NT + SK_WARPS * 16);   // [12][32 NT]
+  if (tid < 32 * NT) {
+#pragma unroll
+    for (int gate = 0; gate < 4; ++gate) {
+      const long long row = (long long)gate * H + cell0 + ec;
+      cp_async4(ecst + (gate * 3 + 0) * 32 * NT + tid, a.s_wih + row);
+      cp_async4(ecst + (gate * 3 + 1) * 32 * NT + tid, a.s_whh + row);
+      if (a.bias) cp_async4(ecst + (gate * 3 + 2) * 32 * NT + tid, a.bias + row);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
   pdl_wait();   // nothing produced by an earlier kernel is read before this
+  // row bookkeeping: every index is requested at once (the arrays hold an entry for each of the N launch
+  // rows), the count of rows with work only masks them afterwards
   int n_act = a.N;
-  if (a.n_active) n_act = min(n_act, *a.n_active);
-  if (n_act <= 0) return;
-
-  // activation row pointers of this lane: row 8 j + g of every tile (nullptr: no such row / zero state)
-  const uint8_t* xrow[NT];
-  const uint8_t* hrow[NT];
+  int xrow[NT], hrow[NT], drow[NT];   // row indices of this lane's rows 8 j + g, negative = none
 #pragma unroll
   for (int j = 0; j < NT; ++j) {
     const int n = 8 * j + g;
-    xrow[j] = hrow[j] = nullptr;
-    if (n < n_act && (a.dst_row ? a.dst_row[n] : n) >= 0) {
-      const int xi = a.x_idx ? a.x_idx[n] : n;
-      if (xi >= 0) xrow[j] = a.x + (long long)xi * a.x_stride;
-      const int hi = a.src_row ? a.src_row[n] : n;
-      if (hi >= 0) hrow[j] = a.hq_in + (long long)hi * (H >> 1);
-    }
+    const bool in = n < a.N;
+    drow[j] = in ? (a.dst_row ? a.dst_row[n] : n) : -1;
+    xrow[j] = in ? (a.x_idx ? a.x_idx[n] : n) : -1;
+    hrow[j] = in ? (a.src_row ? a.src_row[n] : n) : -1;
   }
+  int e_dst = -1, e_src = -1;
+  if (tid < 32 * NT && en < a.N) {
+    e_dst = a.dst_row ? a.dst_row[en] : en;
+    e_src = a.src_row ? a.src_row[en] : en;
+  }
+  if (a.n_active) n_act = min(n_act, *a.n_active);
+  if (n_act <= 0) return;
+#pragma unroll
+  for (int j = 0; j < NT; ++j)
+    if (8 * j + g >= n_act || drow[j] < 0) xrow[j] = hrow[j] = -1;
+  // the item's parent cell state, fetched beside the main loop
+  float e_cprev = 0.0f;
+  if (en >= n_act) e_dst = -1;
+  if (e_dst >= 0 && e_src >= 0) e_cprev = a.c_in[(long long)e_src * H + cell0 + ec];
+
+  // activation row pointers of this lane: row 8 j + g of every tile (nullptr: no such row / zero state)
   int acc[2][NT][4];
   int accs[4] = {0, 0, 0, 0};
 #pragma unroll
@@ -83,42 +119,53 @@ __global__ void __launch_bounds__(SK_THREADS) k_skinny_lstm(const SkinnyLstmArgs
     for (int j = 0; j < NT; ++j)
 #pragma unroll
       for (int r = 0; r < 4; ++r) acc[p][j][r] = 0;
-  const uint32_t M = 0xF0F0F0F0u;
-  const bool x_unsigned = a.x_signed == 0;
 
-  for (int q = warp; q < nxc + nhc; q += SK_WARPS) {
+  // chunk q of this warp: weight pieces of two rows and activation pieces of NT rows, 16 bytes each
+  auto fetch = [&](int q, uint4& wa, uint4& wb, uint4 (&xb)[NT]) {
+    wa = wb = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int j = 0; j < NT; ++j) xb[j] = make_uint4(0, 0, 0, 0);
+    if (q >= nxc + nhc) return;
     const bool is_x = q < nxc;
     const int kb = ((is_x ? q : q - nxc) << 6) + 16 * t4;   // byte offset of this lane's 32 codes in a row
     const uint8_t* wbase = is_x ? a.w_ih : a.w_hh;
     const long long wpitch = is_x ? (a.Kx >> 1) : (H >> 1);
-    const uint4 wa = *reinterpret_cast<const uint4*>(wbase + r0 * wpitch + kb);
-    const uint4 wb = *reinterpret_cast<const uint4*>(wbase + r1 * wpitch + kb);
-    uint4 xb[NT];
+    wa = *reinterpret_cast<const uint4*>(wbase + r0 * wpitch + kb);
+    wb = *reinterpret_cast<const uint4*>(wbase + r1 * wpitch + kb);
 #pragma unroll
     for (int j = 0; j < NT; ++j) {
-      const uint8_t* p = is_x ? xrow[j] : hrow[j];
-      xb[j] = p ? *reinterpret_cast<const uint4*>(p + kb) : make_uint4(0, 0, 0, 0);
+      const int r = is_x ? xrow[j] : hrow[j];
+      if (r >= 0)
+        xb[j] = *reinterpret_cast<const uint4*>((is_x ? a.x + (long long)r * a.x_stride : a.hq_in + (long long)r * (H >> 1)) + kb);
     }
+  };
+  uint4 wa, wb, xb[NT];
+  fetch(warp, wa, wb, xb);
+  for (int q = warp; q < nxc + nhc; q += SK_WARPS) {
+    const bool is_x = q < nxc;
     const uint32_t aw[4] = {wa.x, wa.y, wa.z, wa.w}, bw[4] = {wb.x, wb.y, wb.z, wb.w};
+    uint32_t xw[NT][4];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      xw[j][0] = xb[j].x;
+      xw[j][1] = xb[j].y;
+      xw[j][2] = xb[j].z;
+      xw[j][3] = xb[j].w;
+    }
+    fetch(q + SK_WARPS, wa, wb, xb);   // the next chunk is on its way while this one is multiplied
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint32_t a0 = (aw[i] << 4) & M, a2 = aw[i] & M, a1 = (bw[i] << 4) & M, a3 = bw[i] & M;
       if (is_x && x_unsigned) {
         mma_s8u8(accs, a0, a1, a2, a3, 0x01010101u, 0x01010101u);
 #pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          const uint32_t w = i == 0 ? xb[j].x : i == 1 ? xb[j].y : i == 2 ? xb[j].z : xb[j].w;
-          mma_s8u8(acc[0][j], a0, a1, a2, a3, (w << 4) & M, w & M);
-        }
+        for (int j = 0; j < NT; ++j) mma_s8u8(acc[0][j], a0, a1, a2, a3, (xw[j][i] << 4) & M, xw[j][i] & M);
+      } else if (is_x) {
+#pragma unroll
+        for (int j = 0; j < NT; ++j) mma_s8s8(acc[0][j], a0, a1, a2, a3, (xw[j][i] << 4) & M, xw[j][i] & M);
       } else {
 #pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          const uint32_t w = i == 0 ? xb[j].x : i == 1 ? xb[j].y : i == 2 ? xb[j].z : xb[j].w;
-          if (is_x)
-            mma_s8s8(acc[0][j], a0, a1, a2, a3, (w << 4) & M, w & M);
-          else
-            mma_s8s8(acc[1][j], a0, a1, a2, a3, (w << 4) & M, w & M);
-        }
+        for (int j = 0; j < NT; ++j) mma_s8s8(acc[1][j], a0, a1, a2, a3, (xw[j][i] << 4) & M, xw[j][i] & M);
       }
     }
   }
@@ -139,9 +186,10 @@ __global__ void __launch_bounds__(SK_THREADS) k_skinny_lstm(const SkinnyLstmArgs
   }
   __syncthreads();
   if (tid >= 32 * NT) return;
+  asm volatile("cp.async.wait_all;" ::: "memory");   // this thread's constants have landed
   // item: cell c of the CTA's 4, row n
-  const int c = tid & 3, n = tid >> 2;
-  const int dst = (n < n_act) ? (a.dst_row ? a.dst_row[n] : n) : -1;
+  const int c = ec, n = en;
+  const int dst = e_dst;
   int q = 0;
   if (dst >= 0) {
     const int cell = cell0 + c;
@@ -150,7 +198,7 @@ __global__ void __launch_bounds__(SK_THREADS) k_skinny_lstm(const SkinnyLstmArgs
     for (int gate = 0; gate < 4; ++gate) {
       const int r = gate < 2 ? 2 * c + gate : 8 + 2 * c + (gate - 2);
       int ih = 0, hh = 0, ws = 0;
-#pragma unroll
+#pragma unroll 4
       for (int w = 0; w < SK_WARPS; ++w) {
         ih += part[w][0][r][n];
         hh += part[w][1][r][n];
@@ -159,15 +207,13 @@ __global__ void __launch_bounds__(SK_THREADS) k_skinny_lstm(const SkinnyLstmArgs
       if (x_unsigned) ih -= 16 * a.x_zp * ws;   // 256 sum w (x - z) = 256 sum w x - 16 z (16 sum w)
       ih >>= 8;                                // both operands were 16 x code
       hh >>= 8;
-      const long long row = (long long)gate * H + cell;
-      const float b = a.bias ? a.bias[row] : 0.0f;
-      const float v = __fmaf_rn((float)ih, __fmul_rn(a.x_scale, a.s_wih[row]), b);
-      pre[gate] = __fmaf_rn((float)hh, __fmul_rn(a.hid_act.scale, a.s_whh[row]), v);
+      const float sih = ecst[(gate * 3 + 0) * 32 * NT + tid], shh = ecst[(gate * 3 + 1) * 32 * NT + tid];
+      const float bi = a.bias ? ecst[(gate * 3 + 2) * 32 * NT + tid] : 0.0f;
+      const float v = __fmaf_rn((float)ih, __fmul_rn(a.x_scale, sih), bi);
+      pre[gate] = __fmaf_rn((float)hh, __fmul_rn(a.hid_act.scale, shh), v);
     }
-    const int src = a.src_row ? a.src_row[n] : n;
-    const float cprev = src >= 0 ? a.c_in[(long long)src * H + cell] : 0.0f;
     float cn, hn;
-    cell_fixed(pre[0], pre[1], pre[2], pre[3], cprev, cn, hn);
+    cell_fixed(pre[0], pre[1], pre[2], pre[3], e_cprev, cn, hn);
     a.c_out[(long long)dst * H + cell] = cn;
     q = quantize1(hn, a.hid_act.inv_scale, a.hid_act.zero_point, act_lo(a.hid_act), act_hi(a.hid_act));
     if (a.h8_out) a.h8_out[(long long)n * a.h8_ld + cell] = (int8_t)q;
@@ -187,14 +233,21 @@ bool skinny_lstm_supported(int N, int H, int Kx, int w_bits_ih, int w_bits_hh, c
 cudaError_t launch_skinny_lstm(const SkinnyLstmArgs& a, cudaStream_t s, bool dependent) {
   if (a.N <= 0) return cudaSuccess;
   const dim3 grid(a.H / 4), block(SK_THREADS);
+  auto smem = [](int nt) { return (size_t)(SK_WARPS * 2 * 16 * 8 * nt + SK_WARPS * 16 + 12 * 32 * nt) * sizeof(int); };
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t ce = cudaFuncSetAttribute(k_skinny_lstm<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem(4));
+    if (ce != cudaSuccess) return ce;
+    configured = true;
+  }
   timing_begin(s);
   cudaError_t e;
   if (a.N <= 8)
-    e = launch_ex(k_skinny_lstm<1>, grid, block, 0, s, dependent, 1, a);
+    e = launch_ex(k_skinny_lstm<1>, grid, block, smem(1), s, dependent, 1, a);
   else if (a.N <= 16)
-    e = launch_ex(k_skinny_lstm<2>, grid, block, 0, s, dependent, 1, a);
+    e = launch_ex(k_skinny_lstm<2>, grid, block, smem(2), s, dependent, 1, a);
   else
-    e = launch_ex(k_skinny_lstm<4>, grid, block, 0, s, dependent, 1, a);
+    e = launch_ex(k_skinny_lstm<4>, grid, block, smem(4), s, dependent, 1, a);
   timing_end(s);
   ++g_launches;
   return e != cudaSuccess ? e : cudaGetLastError();
