@@ -96,6 +96,63 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
   if (lane < 16) s_gmax[warp][lane] = NEG;
   __syncthreads();
 
+  // ---- no slot of this utterance may emit a label (all at their label budget, or empty): the only
+  // proposals are the blanks of the live slots, at most W of them, no two of which can describe the
+  // same string.  One warp, lane = slot: the same score arithmetic, the same finished list and the
+  // same order (score descending, then slot) as the general path below, without its passes over V.
+  const int cap = 16 * ((V + 31) / 32);
+  bool any_labels = false;
+  for (int w = 0; w < W; ++w) any_labels |= s_row[w] >= 0 && s_u[w] < a.u_max;
+  const bool blank_only = fast && a.normalized != 0 && !any_labels;
+  if (blank_only) {
+    if (warp == 0) {
+      const int w = lane;
+      const bool alive = w < W && s_row[w] >= 0;
+      float sc = NEG;
+      if (alive) sc = (float)((double)s_score[w] + (double)(a.logits[(size_t)(base + w) * V] - 0.0f));
+      const bool fin = alive && s_t[w] + 1 == a.T;   // consumed the last frame: goes to the finished list
+      if (__any_sync(0xffffffffu, fin)) {
+        if (w < W) win_score[w] = sc;                // staging only; overwritten by the ranking below
+        __syncwarp();
+        if (lane == 0) {
+          float* fs = st.fin_score + base;
+          int* fi = st.fin_iter + base;
+          int* fl = st.fin_slot + base;
+          int n = st.fin_n[b];
+          for (int x = 0; x < W; ++x) {
+            if (s_row[x] < 0 || s_t[x] + 1 != a.T) continue;
+            const float S = win_score[x];
+            int pos = n;
+            while (pos > 0 && fs[pos - 1] < S) --pos;
+            if (pos >= W) continue;
+            const int last = min(n, W - 1);
+            for (int i = last; i > pos; --i) {
+              fs[i] = fs[i - 1];
+              fi[i] = fi[i - 1];
+              fl[i] = fl[i - 1];
+            }
+            fs[pos] = S;
+            fi[pos] = a.iter;
+            fl[pos] = x;
+            n = min(n + 1, W);
+          }
+          st.fin_n[b] = n;
+        }
+        __syncwarp();
+      }
+      const bool cnd = alive && !fin && sc > NEG;
+      const uint64_t key = cnd ? make_key(sc, (uint32_t)w * (uint32_t)V) : 0ull;
+      int rank = 0;
+      for (int x = 0; x < W; ++x) rank += __shfl_sync(0xffffffffu, key, x) > key;
+      if (cnd) {
+        win_idx[rank] = w * V;
+        win_score[rank] = sc;
+      }
+      const int n_c = __popc(__ballot_sync(0xffffffffu, cnd));
+      if (lane == 0) list_n = n_c;
+    }
+    __syncthreads();
+  } else {
   // ---- proposals
   uint32_t skip = 0;   // fast path: bit i = element lane + 32 i is not a label proposal that can win
   if (fast) {
@@ -296,7 +353,6 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
   __syncthreads();
 
   // ---- the W best remaining proposals
-  const int cap = 16 * ((V + 31) / 32);
   bool exact = !fast;
   if (fast) {
     // everything at or above the bound goes to the short list (label proposals from registers,
@@ -387,8 +443,9 @@ __global__ void __launch_bounds__(SEL_NT) k_beam_select(const __grid_constant__ 
     }
     __syncthreads();
   }
+  }
   // each list entry's rank is counted in parallel
-  {
+  if (!blank_only) {
     const int ln = min(list_n, cap);
     for (int i = tid; i < ln; i += SEL_NT) {
       const uint64_t mine = list[i];
