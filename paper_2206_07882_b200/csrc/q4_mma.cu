@@ -100,41 +100,24 @@ __global__ void __launch_bounds__(256) k_unpack_multi(const UnpackJobs jobs) {
     rows = jobs.n_rows;
     if (jobs.n_active) rows = min(rows, *jobs.n_active);
   }
+  const int n_work = jobs.n_active ? min(jobs.n_rows, *jobs.n_active) : jobs.n_rows;
+  const uint32_t zp4 = (uint32_t)j.zp * 0x01010101u;
   const long long total = (long long)rows * per_row;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const int n = (int)(i / per_row), k = (int)(i % per_row) * 32;
     uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
     int r = -1;
-    const bool has_work = n < jobs.n_rows && !(jobs.n_active && n >= *jobs.n_active);
-    if (has_work) r = j.idx ? j.idx[n] : n;
+    if (n < n_work) r = j.idx ? j.idx[n] : n;
     if (r >= 0) {
       const uint8_t* p = j.src + (long long)r * j.src_stride;
       if (j.bits == 4) {
+        // eight codes per word -> two words of four int8 in natural element order
         const uint4 v = *reinterpret_cast<const uint4*>(p + (k >> 1));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t o[8];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint32_t lo = 0, hi = 0;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            int a = (w[q] >> (4 * e)) & 0xF, c = (w[q] >> (4 * (e + 4))) & 0xF;
-            if (j.is_signed) {
-              a = (a ^ 8) - 8;
-              c = (c ^ 8) - 8;
-            } else {
-              a -= j.zp;
-              c -= j.zp;
-            }
-            lo |= (uint32_t)(a & 0xFF) << (8 * e);
-            hi |= (uint32_t)(c & 0xFF) << (8 * e);
-          }
-          o[2 * q] = lo;
-          o[2 * q + 1] = hi;
-        }
-        o0 = make_uint4(o[0], o[1], o[2], o[3]);
-        o1 = make_uint4(o[4], o[5], o[6], o[7]);
+        unpack8_natural(v.x, j.is_signed != 0, zp4, o0.x, o0.y);
+        unpack8_natural(v.y, j.is_signed != 0, zp4, o0.z, o0.w);
+        unpack8_natural(v.z, j.is_signed != 0, zp4, o1.x, o1.y);
+        unpack8_natural(v.w, j.is_signed != 0, zp4, o1.z, o1.w);
       } else {
         o0 = *reinterpret_cast<const uint4*>(p + k);
         o1 = *reinterpret_cast<const uint4*>(p + k + 16);
@@ -152,7 +135,8 @@ cudaError_t launch_unpack_multi(const UnpackJobs& jobs, cudaStream_t s, bool dep
   for (int i = 0; i < jobs.n_jobs; ++i) kmax = jobs.job[i].k_pad > kmax ? jobs.job[i].k_pad : kmax;
   const long long total = (long long)jobs.n_rows_pad * (kmax >> 5);
   long long blocks = (total + 255) / 256;
-  const long long cap = (2 * 148 + jobs.n_jobs - 1) / jobs.n_jobs;   // about two CTAs per SM in all
+  const long long cap = (6 * 148 + jobs.n_jobs - 1) / jobs.n_jobs;   // about six CTAs per SM in all: one or two
+                                                                     // pieces per thread at 1024 rows
   if (blocks > cap) blocks = cap;
   dim3 grid((unsigned)blocks, jobs.n_jobs);
   timing_begin(s);
