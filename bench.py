@@ -210,7 +210,7 @@ def run_reference(args):
 class Job:
     """Holds device weights and buffers of one workload and runs whole steps."""
 
-    def __init__(self, wl_name: str, rank: int, beam: int = 16):
+    def __init__(self, wl_name: str, rank: int, beam: int = 16, groups: int = 1):
         import torch
         from paper_2206_07882_b200 import binding as Bd
         from paper_2206_07882_b200 import synth
@@ -262,7 +262,10 @@ class Job:
                     synth.Stream(seed).normal("features", (T, B, 240)).astype(np.float16)).pin_memory()
         if wl["dec"]:
             dw = synth.decoder(3, out_bits=wl["out_bits"], U_max=wl["U_max"], all_bits=8 if wl.get("all8") else 4)
-            self.dec = Bd.Decoder(dw)
+            # optionally the batch is searched as `groups` sets side by side (same weights, separate states
+            # and streams)
+            self.groups = groups if (groups > 1 and B >= 32 and "tsd" not in wl) else 1
+            self.dec = Bd.GroupedDecoder(dw, self.groups) if self.groups > 1 else Bd.Decoder(dw)
             if "tsd" in wl:
                 self.dec.alloc_state(B, self.W, T * (wl["tsd"] + 1), wl["tsd"])
             else:
@@ -368,6 +371,9 @@ def main():
     ap.add_argument("--workload", default="cfg4_end_to_end", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-frames", type=int, default=8)
     ap.add_argument("--beam", type=int, default=16, help="beam width W (1..16)")
+    ap.add_argument("--groups", type=int, default=1,
+                    help="sets of utterances searched side by side on their own streams (batches of 32 "
+                         "utterances and more); measured: no gain over one set, hence 1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true",
                     help="skip the single-utterance beam sweep appended to the end-to-end line")
@@ -398,7 +404,7 @@ def main():
     if args.no_dependent_launch:
         from paper_2206_07882_b200 import binding as _Bd
         _Bd.dependent_launch_set(False)
-    job = Job(args.workload, rank, args.beam)
+    job = Job(args.workload, rank, args.beam, args.groups)
     job.passes = args.steps
     wl = job.wl
     B, T, U = wl["B"], wl["T"], wl["U_max"]
@@ -487,10 +493,11 @@ def main():
         # (auxiliary streams withdrawn for these passes), so that an event pair brackets one
         # kernel running alone, as in the profiler's launch list
         saved_aux = None
-        if job.dec is not None and job.dec.state is not None:
-            st = job.dec.state
-            saved_aux = (st.aux_stream[0], st.aux_stream[1])
-            st.aux_stream[0], st.aux_stream[1] = None, None
+        parts = list(getattr(job.dec, "parts", [job.dec])) if job.dec is not None else []
+        if parts and parts[0].state is not None:
+            saved_aux = [(p.state.aux_stream[0], p.state.aux_stream[1]) for p in parts]
+            for p in parts:
+                p.state.aux_stream[0], p.state.aux_stream[1] = None, None
         tot, cnt, series = {}, {}, {}
         for _ in range(K):
             lib.q4_timing_set(C.c_uint32(0xFFFFFFFF), start, stop, tags, C.c_int32(cap))
@@ -509,7 +516,8 @@ def main():
             for t_, v_ in per_pass.items():          # launch-ordered durations, one list per pass
                 series.setdefault(t_, []).append(v_)
         if saved_aux is not None:
-            job.dec.state.aux_stream[0], job.dec.state.aux_stream[1] = saved_aux
+            for p, sv in zip(parts, saved_aux):
+                p.state.aux_stream[0], p.state.aux_stream[1] = sv
         allms = sum(tot.values()) or 1.0
         shares = {TAG_NAMES.get(t, str(t)): {"launches": cnt[t] // K, "ms": round(tot[t] / K, 3),
                                              "avg_us": round(1e3 * tot[t] / cnt[t], 2),
@@ -624,7 +632,7 @@ def search_regimes(job, dec_ms, torch):
     wl, d = job.wl, job.dec
     T, B, W = wl["T"], wl["B"], job.W
     iters = T + wl["U_max"]
-    tok = d.tensors["bp_token"][:iters]
+    tok = (d.history("bp_token") if hasattr(d, "parts") else d.tensors["bp_token"])[:iters]
     per_iter = (tok > 0).reshape(iters, -1).sum(1)
     n_busy = int((per_iter > 0).sum().item()) + 1          # launch 0 advances the start symbols
     n_free = iters - n_busy
@@ -734,9 +742,16 @@ def roofline(job, tag, ms, n, pk, series=None):
         # extensions keep their parent's state), counted from the search history of the last pass;
         # launch 0 advances the start symbol of every utterance
         iters = wl["T"] * (wl["tsd"] + 1) if "tsd" in wl else wl["T"] + wl["U_max"]
-        tok = job.dec.tensors["bp_token"][:iters]
-        per_iter = (tok > 0).reshape(iters, -1).sum(1).cpu().numpy().astype(np.float64)
-        rows = np.concatenate([[float(wl["B"])], per_iter[:-1]])
+        # (with the batch searched as several sets, a launch serves one set: launches come in
+        # iteration-major order, one per set)
+        parts = list(getattr(job.dec, "parts", [job.dec]))
+        cols = []
+        for p_ in parts:
+            tk = p_.tensors["bp_token"][:iters]
+            pi = (tk > 0).reshape(iters, -1).sum(1).cpu().numpy().astype(np.float64)
+            cols.append(np.concatenate([[float(p_.B)], pi[:-1]]))
+        rows = np.stack(cols, axis=1).reshape(-1)
+        iters = iters * len(parts)
         busy = rows > 0
         mean_rows = float(rows.mean())
         out.update(rows_per_launch_mean=mean_rows, launches_with_rows=int(busy.sum()),

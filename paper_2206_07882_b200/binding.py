@@ -515,11 +515,19 @@ class Decoder:
     """Device copy of prediction network, joint network and both fusion LMs, the search
     state, and the iteration loop (one library call per search iteration)."""
 
-    def __init__(self, dw, device="cuda", tensor_cores: bool = True, concurrent: bool = True):
+    def __init__(self, dw, device="cuda", tensor_cores: bool = True, concurrent: bool = True, share_from=None):
         self.dw = dw
         self.device = device
         self.tensor_cores = tensor_cores
         self.concurrent = concurrent and tensor_cores
+        self.state = None
+        self.S_max = None
+        if share_from is not None:
+            # a second search state over the same device weights (read-only, prepared operands included)
+            for name in ("V", "E", "D", "pred_emb_act", "pred_emb_q", "pred_lstm", "pred_proj", "z_act", "joint_out",
+                         "src", "tgt", "model", "prepared"):
+                setattr(self, name, getattr(share_from, name))
+            return
         self.V, self.E = dw.pred.emb.shape
         self.pred_emb_act = q4_act_symmetric(dw.pred.emb_alpha, getattr(dw, "emb_bits", 4))
         emb = torch.from_numpy(np.ascontiguousarray(dw.pred.emb, dtype=np.float32)).to(device)
@@ -670,6 +678,64 @@ class Decoder:
         for it in range(n_iters):
             self.dr_fusion_beam_step(e, T, it, u_max, mode=2 if it % (S_max + 1) == S_max else 1)
         return self.q4_traceback(n_iters, u_max)
+
+
+class GroupedDecoder:
+    """The fused search over a batch split into `groups` sets of utterances, each with its own search
+    state and streams over ONE copy of the device weights.  Utterances are independent (Eq. 1 has no
+    cross-utterance term), so the sets advance side by side: while one set's selection and LM heads (short,
+    latency-bound kernels) run, the other set's LSTM GEMMs have the SMs.  Marshalling only."""
+
+    def __init__(self, dw, groups: int = 2, device="cuda"):
+        first = Decoder(dw, device)
+        self.parts = [first] + [Decoder(dw, device, share_from=first) for _ in range(groups - 1)]
+        self.dw, self.device = dw, device
+        self.streams = [torch.cuda.Stream(device=device) for _ in range(groups)]
+        for name in ("V", "E", "D", "pred_lstm", "pred_proj", "joint_out", "src", "tgt"):
+            setattr(self, name, getattr(first, name))
+
+    def step_weight_bytes(self) -> int:
+        return self.parts[0].step_weight_bytes()
+
+    def _bounds(self, B):
+        G = len(self.parts)
+        return [(g * B // G, (g + 1) * B // G) for g in range(G)]
+
+    def alloc_state(self, B: int, W: int, n_iters: int):
+        for part, (b0, b1) in zip(self.parts, self._bounds(B)):
+            part.alloc_state(b1 - b0, W, n_iters)
+
+    def history(self, name: str) -> torch.Tensor:
+        """A history tensor [iter, B, W] of all sets, utterances in batch order."""
+        return torch.cat([p.tensors[name] for p in self.parts], dim=1)
+
+    def decode(self, e: torch.Tensor, u_max: Optional[int] = None, W: Optional[int] = None):
+        T, B, D = e.shape
+        u_max = self.dw.U_max if u_max is None else u_max
+        W = self.dw.W if W is None else W
+        n_iters = T + u_max
+        bounds = self._bounds(B)
+        main = torch.cuda.current_stream()
+        es = [e[:, b0:b1].contiguous() for b0, b1 in bounds]     # each set's frames as one dense block
+        for part, (b0, b1) in zip(self.parts, bounds):
+            if part.state is None or (part.B, part.W) != (b1 - b0, W) or part.n_iters < n_iters or part.S_max is not None:
+                part.alloc_state(b1 - b0, W, n_iters)
+        for st in self.streams:
+            st.wait_stream(main)
+        for part, st in zip(self.parts, self.streams):
+            with torch.cuda.stream(st):
+                part.q4_beam_init()
+        for it in range(n_iters):
+            for part, st, eg in zip(self.parts, self.streams, es):
+                with torch.cuda.stream(st):
+                    part.dr_fusion_beam_step(eg, T, it, u_max)
+        res = []
+        for part, st in zip(self.parts, self.streams):
+            with torch.cuda.stream(st):
+                res.append(part.q4_traceback(n_iters, u_max))
+        for st in self.streams:
+            main.wait_stream(st)
+        return tuple(torch.cat([r[i] for r in res], dim=0) for i in range(3))
 
 
 class GraphedStep:

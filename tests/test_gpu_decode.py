@@ -540,3 +540,27 @@ def test_search_few_rows_weight_streaming_kernels(Bd, B, W):
     dd, tokens, lens, scores, ref = run_search(Bd, dw, e)
     frac, tr = compare_search(dd, tokens, lens, scores, ref, list(range(B)), 9, 6, W, min_same=1.0)
     assert tr == 1.0
+
+
+def test_grouped_search_equals_single_state_search(Bd):
+    # the batch searched as two and three sets of utterances side by side (own states and streams, one copy
+    # of the weights): token for token, score for score, the result of the one-state search
+    dw = synth.decoder(seed=101, V=64, E=32, Hp=128, D=32, Hs=128, Ht=256, tgt_layers=2, U_max=8, W=16)
+    e = synth.Stream(18).normal("e", (14, 12, 32)).astype(np.float32)
+    e_dev = torch.from_numpy(e).cuda()
+    one = Bd.Decoder(dw)
+    t1, l1, s1 = one.decode(e_dev)
+    torch.cuda.synchronize()
+    for G in (2, 3):
+        gd = Bd.GroupedDecoder(dw, G)
+        t2, l2, s2 = gd.decode(e_dev)
+        torch.cuda.synchronize()
+        assert torch.equal(t1, t2) and torch.equal(l1, l2) and torch.equal(s1, s2)
+        assert torch.equal(gd.history("bp_parent")[:22], one.tensors["bp_parent"][:22])
+        assert torch.equal(gd.history("bp_token")[:22], one.tensors["bp_token"][:22])
+        # and replayed as a CUDA graph
+        g = Bd.GraphedStep(lambda: gd.decode(e_dev))
+        t3, l3, s3 = g()
+        t3, l3, s3 = g()
+        torch.cuda.synchronize()
+        assert torch.equal(t1, t3) and torch.equal(s1, s3)
