@@ -32,7 +32,7 @@ def _worker(rank, world, port, out):
 
 def test_two_ranks_shard_and_reduce():
     world = 2
-    mgr = mp.Manager()
+    mgr = mp.get_context("spawn").Manager()
     out = mgr.dict()
     mp.spawn(_worker, args=(world, _free_port(), out), nprocs=world, join=True)
     (lo0, hi0, s0, rtf0, t0), (lo1, hi1, s1, rtf1, t1) = out[0], out[1]
