@@ -392,6 +392,12 @@ int q4_dependent_launch_set(int32_t enabled);
  * take the exact search (for tests; both give the same beam).  Returns the previous setting. */
 int q4_beam_select_exact_set(int32_t enabled);
 
+/* qlstm_layer_forward, 4-bit layers of 640 cells: when the sequences form one group of 8 more (per
+ * direction) than thread-block clusters can be resident, the clusters of a direction take turns at
+ * that group instead of every cluster serving two groups.  enabled = 0 switches this off (for tests
+ * and measurements; the results are identical).  Returns the previous setting. */
+int q4_encoder_time_slicing_set(int32_t enabled);
+
 /* Test hook for the bounded device-side waits (not an operation of the paper): while skip_producer
  * is non-zero the tiled tensor-core GEMM (the tensor-core paths of q4_linear_forward and of the
  * projections) launches with a producer that issues no copy at all, so that the consumer's wait

@@ -81,7 +81,7 @@ EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
            "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_beam_select_exact_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static", "q4_quantizer_calls", "q4_prepared_lstm_bytes", "q4_prepare_lstm",
-           "q4_prepared_linear_bytes", "q4_prepare_linear", "q4_test_wait_expiry_set"]
+           "q4_prepared_linear_bytes", "q4_prepare_linear", "q4_test_wait_expiry_set", "q4_encoder_time_slicing_set"]
 
 _lib = None
 
@@ -143,6 +143,11 @@ def quantizer_calls(reset: bool = False) -> int:
 def dependent_launch_set(enabled: bool) -> bool:
     """Switch programmatic dependent launches of the beam step on or off; returns the previous setting."""
     return bool(lib().q4_dependent_launch_set(1 if enabled else 0))
+
+
+def encoder_time_slicing_set(enabled: bool) -> bool:
+    """Let the clusters of the encoder recurrence take turns at a surplus group of sequences (default) or not; returns the previous setting."""
+    return bool(lib().q4_encoder_time_slicing_set(1 if enabled else 0))
 
 
 def beam_select_exact_set(enabled: bool) -> bool:

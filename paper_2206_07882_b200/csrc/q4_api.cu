@@ -102,6 +102,7 @@ int q4_test_wait_expiry_set(int32_t skip_producer, uint32_t wait_limit) {
   test_wait_expiry_set(skip_producer ? 1 : 0, wait_limit);
   return Q4_OK;
 }
+int q4_encoder_time_slicing_set(int32_t enabled) { return enc_recurrent_sliced_set(enabled ? 1 : 0); }
 int q4_dependent_launch_set(int32_t enabled) {
   const int prev = g_dependent_launch;
   g_dependent_launch = enabled ? 1 : 0;
@@ -483,6 +484,13 @@ int qlstm_layer_forward(const void* xq, const q4_act* x_act, const float* x_scal
     ra.out_act = *out_act;
     ra.yq_ld = yb;
     ra.dbg_ld = (long long)dirs * G;
+    // scratch of the time-sliced kernel: counters in the status block (zeroed above), the shared
+    // group's state in the buffers the step-by-step path would use
+    ra.flags = status + 16;
+    for (int d = 0; d < dirs && B >= 8; ++d) {
+      ra.hand_h[d] = hbuf + (size_t)d * 2 * B * H;
+      ra.hand_c[d] = cbuf + (size_t)d * B * H;
+    }
     for (int d = 0; d < dirs; ++d) {
       EncRecDir& D = ra.d[d];
       D.w_hh = whh8 + (size_t)d * G * H;

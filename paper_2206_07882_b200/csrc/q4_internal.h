@@ -186,8 +186,17 @@ struct EncRecArgs {
   q4_act hid_act, out_act;
   long long yq_ld;          // bytes per (t, b) output row
   long long dbg_ld;         // elements per (t, b) debug row
+  // One group of 8 sequences more than clusters (time-sliced kernel): set by the launcher from the
+  // scratch below, which the caller provides (nullptr = that kernel is not used)
+  int32_t ncl[2];           // clusters of each direction
+  int32_t sliced[2];        // 1: the direction's clusters take turns at its last group
+  int32_t groups;           // groups of 8 sequences per direction
+  int32_t* flags;           // [2][8] hand-over counters, zero before the launch
+  uint8_t* hand_h[2];       // [8][8][H / 8] hidden codes of the shared group at a hand-over, per direction
+  float* hand_c[2];         // [8][H] its cell states
 };
 bool enc_recurrent_supported(int H, int B, int dirs);
+int enc_recurrent_sliced_set(int enabled);   // returns the previous setting
 cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s);
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }

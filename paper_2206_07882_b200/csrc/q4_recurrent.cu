@@ -593,6 +593,327 @@ k_enc_recurrent_w4(const EncRecArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same step with one group too many for the clusters that can be resident: G groups of 8
+// sequences of a direction on G - 1 clusters.  Cluster j owns group j; group G - 1 is shared: it
+// advances on cluster 0 during its first T / (G - 1) steps, then on cluster 1, and so on; while a
+// cluster advances the shared group its own group rests.  Every cluster therefore walks
+// T + T / (G - 1) steps of ONE group each instead of 2 T (two groups per cluster), and all clusters
+// of the direction end together.  At a hand-over the shared group's cell states and hidden codes go
+// through global memory: every CTA of the giving cluster stores its part, fences, and adds one to a
+// counter; the taking cluster (always the next higher one, so a waiting cluster only ever waits for
+// clusters that were dispatched before it) polls the counter, bounded, and loads the state.
+// A direction with as many clusters as groups runs plain (sliced = 0).
+// Slot 0 = the cluster's own group, slot 1 = the shared group while it is here.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+template <int KS>
+__global__ void __cluster_dims__(REC_CLUSTER, 1, 1) __launch_bounds__(REC4_THREADS, 1)
+k_enc_recurrent_w4s(const EncRecArgs a) {
+  extern __shared__ __align__(16) uint8_t rec_smem[];
+  constexpr int BG = REC_BG;
+  constexpr int NS = 2;                     // slots
+  constexpr int H = 32 * KS;
+  constexpr int cpc = H / REC_CLUSTER;      // cells per CTA
+  constexpr int rows = 4 * cpc;
+  constexpr int chunks = cpc >> 4;          // 16-byte chunks of a sequence's new codes per CTA
+  constexpr int UB = BG * H;                // bytes of one group's hidden codes
+  constexpr int CW = REC_THREADS / 32;      // warps
+  constexpr int KR = KS - rec_w4_ksmem(NS);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_rank();
+  const int cid = blockIdx.x / REC_CLUSTER;
+  const int d = cid < a.ncl[0] ? 0 : 1;     // the clusters of direction 0 come first
+  const int j = d == 0 ? cid : cid - a.ncl[0];
+  const int C = a.ncl[d];
+  const bool host = a.sliced[d] != 0;
+  const EncRecDir& D = a.d[d];
+  const int T = a.T, B = a.B;
+  // the shared group's steps [w0, w1) run here
+  const int w0 = host ? (int)((long long)j * T / C) : 0, w1 = host ? (int)((long long)(j + 1) * T / C) : 0;
+  const int n_it = T + (w1 - w0);
+  int8_t* hb = reinterpret_cast<int8_t*>(rec_smem);                       // [NS][2][source CTA][BG][cpc] h_{t-1}
+  int4* pre_s = reinterpret_cast<int4*>(hb + (size_t)NS * 2 * UB);        // [2][threads] input accumulators
+  float4* cst = reinterpret_cast<float4*>(pre_s + (size_t)2 * REC_THREADS);   // [3][cpc] per-cell constants
+  int8_t* stage = reinterpret_cast<int8_t*>(cst + 3 * cpc);                // [NS][2][BG][cpc] new recurrent codes
+  int8_t* stage_y = stage + (size_t)2 * NS * BG * cpc;                     // [NS][2][BG][cpc] new output codes
+  uint64_t* full = reinterpret_cast<uint64_t*>(stage_y + (size_t)2 * NS * BG * cpc);   // [NS][2]
+  volatile int* dead = reinterpret_cast<volatile int*>(full + NS * 2);     // a bounded wait has expired
+  uint2* wsm = reinterpret_cast<uint2*>(full + NS * 2 + 2);                // [KS - KR][threads] packed weights
+
+  const int g = lane >> 2, t4 = lane & 3;   // MMA fragment coordinates
+  const int e = g & 1, ci = g >> 1;         // this lane's item: cell ci of the warp's 4 ...
+  const int n = 2 * t4 + e;                 // ... and sequence n of the group's 8
+  const int cl = warp * 4 + ci;             // cell within the CTA
+  const int cell = (int)rank * cpc + cl;    // cell within the layer
+  const float sh = a.hid_act.scale;
+  const uint32_t hb_addr = smem_u32(hb), pre_addr = smem_u32(pre_s), full_addr = smem_u32(full);
+
+  uint32_t wreg[2 * KR];
+  {
+    const int8_t* W = D.w_hh + ((size_t)rank * rows + (size_t)(16 * warp)) * H;
+    const int8_t* r0 = W + (size_t)(4 * ci + e) * H + 4 * t4;
+    const int8_t* r1 = r0 + (size_t)2 * H;
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      const uint32_t q0 = *reinterpret_cast<const uint32_t*>(r0 + 32 * s);
+      const uint32_t p0 = *reinterpret_cast<const uint32_t*>(r1 + 32 * s);
+      const uint32_t q1 = *reinterpret_cast<const uint32_t*>(r0 + 32 * s + 16);
+      const uint32_t p1 = *reinterpret_cast<const uint32_t*>(r1 + 32 * s + 16);
+      const uint32_t w0p = (q0 & 0x0F0F0F0Fu) | ((p0 << 4) & 0xF0F0F0F0u);
+      const uint32_t w1p = (q1 & 0x0F0F0F0Fu) | ((p1 << 4) & 0xF0F0F0F0u);
+      if (s < KR) {
+        wreg[2 * s] = w0p;
+        wreg[2 * s + 1] = w1p;
+      } else {
+        wsm[(s - KR) * REC_THREADS + tid] = make_uint2(w0p, w1p);
+      }
+    }
+  }
+  for (int i = tid; i < NS * 2 * UB / 16; i += REC4_THREADS)
+    reinterpret_cast<uint4*>(hb)[i] = make_uint4(0, 0, 0, 0);   // h_0 = 0
+  for (int i = tid; i < cpc; i += REC4_THREADS) {
+    const int c = (int)rank * cpc + i;
+    const float4 w = reinterpret_cast<const float4*>(D.sc_hh)[c], v = reinterpret_cast<const float4*>(D.sc_ih)[c];
+    const float sxs = a.x_scale;
+    cst[i] = make_float4(__fmul_rn(sxs, v.x), __fmul_rn(sxs, v.y), __fmul_rn(sxs, v.z), __fmul_rn(sxs, v.w));
+    cst[cpc + i] = make_float4(__fmul_rn(sh, w.x), __fmul_rn(sh, w.y), __fmul_rn(sh, w.z), __fmul_rn(sh, w.w));
+    cst[2 * cpc + i] = reinterpret_cast<const float4*>(D.bias)[c];
+  }
+  if (tid == 0) {
+    *dead = 0;
+    for (int i = 0; i < NS * 2; ++i) mbar_init(&full[i], 1);
+    fence_barrier_init();
+    for (int i = 0; i < NS * 2; ++i) mbar_expect_tx(&full[i], (uint32_t)UB);
+  }
+  fence_proxy_async();   // the zeroed buffers are later written by the bulk-copy engine
+  __syncthreads();
+  cluster_barrier();   // every CTA's buffers and barriers are initialised before anyone stores into them
+
+  const int b_own = j * BG + n, b_shared = (a.groups - 1) * BG + n;
+  const bool live_own = b_own < B, live_shared = host && b_shared < B;
+  float c_own = 0.0f, c_shared = 0.0f;
+  constexpr int G = 4 * H;
+  const int hlo = act_lo(a.hid_act), hhi = act_hi(a.hid_act);
+  const int ylo = act_lo(a.out_act), yhi = act_hi(a.out_act);
+  const bool y4 = a.out_act.bits == 4;
+  int32_t* const flag_out = a.flags + d * 8 + j;
+
+  // walk: own steps [0, w0), shared steps [w0, w1), own steps [w0, T)
+  auto walk = [&](int i, int& u, int& step) {
+    if (i < w0) {
+      u = 0;
+      step = i;
+    } else if (i < w1) {
+      u = 1;
+      step = i;
+    } else {
+      u = 0;
+      step = i - (w1 - w0);
+    }
+  };
+  auto fetch_pre = [&](int i) {   // input accumulators of walk position i into buffer i & 1
+    int u, step;
+    walk(i, u, step);
+    const int b = u ? b_shared : b_own;
+    if (u ? live_shared : live_own) {
+      const int t = d == 0 ? step : T - 1 - step;
+      cp_async16(pre_addr + (uint32_t)(((i & 1) * REC_THREADS + tid) * 16), D.acc_pre + ((size_t)t * B + b) * G + 4 * cell);
+    }
+    cp_async_commit();
+  };
+  if (n_it > 0) fetch_pre(0);
+  bool ok = true;
+  for (int i = 0; i < n_it; ++i) {
+    int u, step;
+    walk(i, u, step);
+    const int ls = u ? step - w0 : step;          // steps of this slot made here so far
+    const int t = d == 0 ? step : T - 1 - step;
+    const int cur = ls & 1, nxt = cur ^ 1;
+    const int b = u ? b_shared : b_own;
+    const bool live = u ? live_shared : live_own;
+    if (i + 1 < n_it)
+      fetch_pre(i + 1);
+    else
+      cp_async_commit();
+    if (u == 1 && ls == 0 && j > 0) {
+      // take the shared group over from cluster j - 1: all eight of its CTAs have stored their parts
+      if (tid == 0 && ok) {
+        bool got = false;
+        for (uint32_t it = 0; it < (1u << 22); ++it) {
+          if (ld_acquire_gpu(flag_out - 1) >= REC_CLUSTER) {
+            got = true;
+            break;
+          }
+          if (*dead) break;
+          __nanosleep(100);
+        }
+        if (!got) {
+          *dead = 1;
+          if (a.status) atomicExch(a.status, Q4_ERR_TIMEOUT);
+        }
+      }
+      __syncthreads();
+      if (*dead) ok = false;
+      if (ok) {
+        const uint4* src = reinterpret_cast<const uint4*>(a.hand_h[d]);
+        for (int k = tid; k < UB / 16; k += REC4_THREADS)
+          reinterpret_cast<uint4*>(hb + (size_t)(1 * 2 + 0) * UB)[k] = __ldcg(src + k);
+        c_shared = live_shared ? __ldcg(a.hand_c[d] + (size_t)n * H + cell) : 0.0f;
+      }
+      fence_proxy_async();   // this buffer is written by the bulk-copy engine two steps on
+      __syncthreads();
+    }
+    if (ls > 0 && ok) {
+      uint64_t* bar = &full[u * 2 + cur];
+      const uint32_t parity = (uint32_t)(((ls - 1) >> 1) & 1);
+      bool got = false;
+      for (uint32_t it = 0; it < (1u << 22); ++it) {
+        if (mbar_try_wait(bar, parity)) {
+          got = true;
+          break;
+        }
+        if ((it & 255u) == 255u && *dead) break;
+      }
+      if (!got) {
+        ok = false;
+        *dead = 1;
+        if (a.status) atomicExch(a.status, Q4_ERR_TIMEOUT);
+      }
+      if (tid == 0 && got) mbar_expect_tx(bar, (uint32_t)UB);
+    }
+    int acc[2][4];
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) acc[c][r] = 0;
+    {
+      const uint32_t half = (uint32_t)((lane >> 3) & 1);
+      const uint32_t b_addr = hb_addr + (uint32_t)((u * 2 + cur) * UB + (lane & 7) * cpc);
+      const uint32_t b_in = b_addr + half * 16u, b_wrap = b_addr + half * (uint32_t)(BG * cpc - (chunks - 1) * 16);
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        uint32_t w0p, w1p;
+        if (s < KR) {
+          w0p = wreg[2 * s];
+          w1p = wreg[2 * s + 1];
+        } else {
+          const uint2 w = wsm[(s - KR) * REC_THREADS + tid];
+          w0p = w.x;
+          w1p = w.y;
+        }
+        const uint32_t a0 = (w0p << 4) & 0xF0F0F0F0u, a1 = w0p & 0xF0F0F0F0u;
+        const uint32_t a2 = (w1p << 4) & 0xF0F0F0F0u, a3 = w1p & 0xF0F0F0F0u;
+        const uint32_t o0 = (uint32_t)(((2 * s) / chunks) * BG * cpc + ((2 * s) % chunks) * 16);
+        uint32_t b0, b1;
+        ldmatrix_x2(((2 * s) % chunks == chunks - 1 ? b_wrap : b_in) + o0, b0, b1);
+        mma_s8(acc[s & 1], a0, a1, a2, a3, b0, b1);
+      }
+    }
+    int hh[4];
+    {
+      const int v0 = acc[0][0] + acc[1][0], v1 = acc[0][1] + acc[1][1];
+      const int v2 = acc[0][2] + acc[1][2], v3 = acc[0][3] + acc[1][3];
+      const int r0 = __shfl_xor_sync(0xffffffffu, e ? v0 : v1, 4);
+      const int r1 = __shfl_xor_sync(0xffffffffu, e ? v2 : v3, 4);
+      const int m0 = e ? v1 : v0, m1 = e ? v3 : v2;
+      hh[0] = (e ? r0 : m0) >> 4;     // the operand was 16 x code
+      hh[1] = (e ? m0 : r0) >> 4;
+      hh[2] = (e ? r1 : m1) >> 4;
+      hh[3] = (e ? m1 : r1) >> 4;
+    }
+    cp_async_wait<1>();               // this thread's accumulators of the present step have landed
+    int q = 0, q2 = 0;
+    if (live) {
+      const int4 pre = pre_s[(i & 1) * REC_THREADS + tid];
+      const float4 s_ih = cst[cl], s_hh = cst[cpc + cl], bb = cst[2 * cpc + cl];
+      const float pi = __fmaf_rn((float)hh[0], s_hh.x, __fmaf_rn((float)pre.x, s_ih.x, bb.x));
+      const float pf = __fmaf_rn((float)hh[1], s_hh.y, __fmaf_rn((float)pre.y, s_ih.y, bb.y));
+      const float pg = __fmaf_rn((float)hh[2], s_hh.z, __fmaf_rn((float)pre.z, s_ih.z, bb.z));
+      const float po = __fmaf_rn((float)hh[3], s_hh.w, __fmaf_rn((float)pre.w, s_ih.w, bb.w));
+      float cs = u ? c_shared : c_own, hval;
+      cell_fixed(pi, pf, pg, po, cs, cs, hval);
+      if (u)
+        c_shared = cs;
+      else
+        c_own = cs;
+      q = quantize1(hval, a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
+      q2 = quantize1(hval, a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
+    }
+    stage[((u * 2 + cur) * BG + n) * cpc + cl] = (int8_t)q;
+    stage_y[((u * 2 + cur) * BG + n) * cpc + cl] = (int8_t)q2;
+    if (step == T - 1 && D.hq_n) {   // final recurrent codes, two cells per byte: the even cell's lane writes
+      const int qn = __shfl_down_sync(0xffffffffu, q, 8);
+      if (live && (cl & 1) == 0)
+        D.hq_n[(size_t)b * (H >> 1) + (cell >> 1)] = (uint8_t)((q & 0xF) | ((qn & 0xF) << 4));
+    }
+    fence_proxy_async();   // the staged codes are read by the bulk-copy engine
+    const bool window_end = u == 1 && step == w1 - 1;   // the shared group leaves after this step
+    if (warp != i % CW) {
+      named_bar_arrive(1 + u * 2 + cur, REC4_THREADS);
+    } else {
+      named_bar_sync(1 + u * 2 + cur, REC4_THREADS);
+      if (!window_end) {
+        if (lane < REC_CLUSTER) {
+          const uint32_t r = (uint32_t)lane;
+          bulk_copy_to_cluster(map_to_rank(hb_addr + (uint32_t)((u * 2 + nxt) * UB + (int)rank * BG * cpc), r),
+                               smem_u32(stage + (size_t)(u * 2 + cur) * BG * cpc), (uint32_t)(BG * cpc),
+                               map_to_rank(full_addr + (uint32_t)((u * 2 + nxt) * 8), r));
+        }
+      } else if (w1 < T) {
+        // this CTA's block of the shared group's codes, in the layout of a receiver's buffer
+        const uint4* src = reinterpret_cast<const uint4*>(stage + (size_t)(u * 2 + cur) * BG * cpc);
+        uint4* dst = reinterpret_cast<uint4*>(a.hand_h[d] + (size_t)rank * BG * cpc);
+        for (int k = lane; k < BG * cpc / 16; k += 32) dst[k] = src[k];
+      }
+      for (int k = lane; k < BG * chunks; k += 32) {
+        const int ch = k % chunks, bl = k / chunks;
+        const int by = (u ? a.groups - 1 : j) * BG + bl;
+        if (by >= B) continue;
+        const uint4 v = *reinterpret_cast<const uint4*>(stage_y + ((u * 2 + cur) * BG + bl) * cpc + ch * 16);
+        uint8_t* y = D.yq + ((size_t)t * B + by) * a.yq_ld;
+        const int c0 = (int)rank * cpc + ch * 16;
+        if (y4) {
+          auto pk = [](uint32_t w) -> uint32_t {
+            const uint32_t m = (w & 0x000F000Fu) | ((w >> 4) & 0x00F000F0u);   // bytes 0 and 2 hold the pairs
+            return (m & 0xFFu) | ((m >> 8) & 0xFF00u);
+          };
+          *reinterpret_cast<uint2*>(y + (c0 >> 1)) = make_uint2(pk(v.x) | (pk(v.y) << 16), pk(v.z) | (pk(v.w) << 16));
+        } else {
+          *reinterpret_cast<uint4*>(y + c0) = v;
+        }
+      }
+    }
+    if (window_end && w1 < T) {
+      // hand the shared group on: cell states by every thread, codes by the sending warp above
+      a.hand_c[d][(size_t)n * H + cell] = c_shared;
+      __threadfence();
+      __syncthreads();
+      if (tid == 0) atomicAdd(flag_out, 1);
+    }
+  }
+  cp_async_wait<0>();
+  // the own group's codes sent in its last step are still on their way into this CTA: wait for them
+  // (bounded), so that nobody leaves while copies into its shared memory are in flight.  (The shared
+  // group sends nothing in the last step of its stay.)
+  if (T > 0) {
+    const uint32_t parity = (uint32_t)(((T - 1) >> 1) & 1);
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+      if (mbar_try_wait(&full[0 * 2 + (T & 1)], parity)) break;
+      if ((it & 255u) == 255u && *dead) break;
+    }
+  }
+  __syncthreads();
+  cluster_barrier();
+  if (live_own && D.c_n) D.c_n[(size_t)b_own * H + cell] = c_own;
+  if (live_shared && w1 == T && D.c_n) D.c_n[(size_t)b_shared * H + cell] = c_shared;
+}
+
 constexpr size_t REC_SMEM_MAX = 232448 - 128;   // 227 KB per CTA on sm_100, minus a margin
 
 size_t enc_recurrent_smem(int H, int BG) {
@@ -657,6 +978,13 @@ int enc_recurrent_group(int B, int dirs, int H) {
   return best;
 }
 
+static int g_rec_sliced = 1;
+int enc_recurrent_sliced_set(int enabled) {
+  const int prev = g_rec_sliced;
+  g_rec_sliced = enabled ? 1 : 0;
+  return prev;
+}
+
 bool enc_recurrent_supported(int H, int B, int dirs) {
   (void)B;
   (void)dirs;
@@ -668,6 +996,22 @@ static size_t enc_recurrent_w4_smem(int H, int NU) {
   const int cpc = H / REC_CLUSTER;
   return (size_t)NU * 2 * REC_BG * H + (size_t)2 * NU * REC_THREADS * sizeof(int4) +
          (size_t)3 * cpc * sizeof(float4) + (size_t)4 * NU * REC_BG * cpc + (size_t)NU * 2 * sizeof(uint64_t) + 32 + (size_t)rec_w4_ksmem(NU) * REC_THREADS * sizeof(uint2);
+}
+
+template <int KS>
+static cudaError_t rec_w4s_launch(const EncRecArgs& a, cudaStream_t s) {
+  const int H = 32 * KS, cpc = H / REC_CLUSTER;
+  const size_t smem = (size_t)2 * 2 * REC_BG * H + (size_t)2 * REC_THREADS * sizeof(int4) + (size_t)3 * cpc * sizeof(float4) +
+                      (size_t)4 * 2 * REC_BG * cpc + (size_t)2 * 2 * sizeof(uint64_t) + 32 +
+                      (size_t)rec_w4_ksmem(2) * REC_THREADS * sizeof(uint2);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_enc_recurrent_w4s<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  k_enc_recurrent_w4s<KS><<<(unsigned)((a.ncl[0] + a.ncl[1]) * REC_CLUSTER), REC4_THREADS, smem, s>>>(a);
+  return cudaGetLastError();
 }
 
 template <int NU, int KS>
@@ -690,6 +1034,21 @@ cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s) {
   if (a.w_bits == 4 && a.hid_act.bits == 4 && a.hid_act.is_signed && a.H == 640 && !a.x_scale_b &&
       !a.d[0].dbg_ih) {
     const int groups = (a.B + REC_BG - 1) / REC_BG, maxc = rec_max_clusters(a.H);
+    // one or two groups more than clusters: a direction's clusters take turns at its last group
+    const int lack = a.dirs * groups - maxc;
+    if (g_rec_sliced && lack >= 1 && lack <= a.dirs && groups >= 2 && groups <= 8 && a.T >= 8 * groups && a.flags &&
+        a.hand_h[0] && a.hand_c[0]) {
+      a.groups = groups;
+      for (int d = 0; d < 2; ++d) {
+        a.sliced[d] = d < a.dirs && d < lack ? 1 : 0;
+        a.ncl[d] = d < a.dirs ? groups - a.sliced[d] : 0;
+      }
+      timing_begin(s);
+      cudaError_t e = rec_w4s_launch<20>(a, s);
+      timing_end(s);
+      ++g_launches;
+      return e;
+    }
     int nu = 1;
     while (nu <= 4 && a.dirs * ((groups + nu - 1) / nu) > maxc) ++nu;
     if (nu <= 4) {

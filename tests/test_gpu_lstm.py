@@ -152,6 +152,35 @@ def test_layer_shapes_directions_precisions(Bd, T, B, K, H, dirs, xb, hb, ob):
     layer_case(Bd, T, B, K, H, dirs, xb, hb, ob, seed=11)
 
 
+def test_layer_clusters_taking_turns_at_a_surplus_group(Bd):
+    # 57 sequences x 2 directions of 640 cells = 16 groups of 8 for the 15 clusters that fit: the seven
+    # clusters of one direction take turns at its eighth group (9 of 64 steps each, one more on the
+    # last; the group holds one live sequence), the other direction runs one group per cluster
+    diff = layer_case(Bd, T=64, B=57, K=64, H=640, dirs=2, seed=23)
+    assert (diff > 0).sum() == 0
+
+
+def test_layer_time_slicing_equals_two_groups_per_cluster(Bd):
+    # longer windows, full groups: codes and final states of the time-sliced launch against the launch
+    # that gives every cluster two groups
+    T, B, K, H = 150, 64, 64, 640
+    w = synth.single_layer(seed=29, T=T, B=B, K=K, H=H, bits=4, dirs=2)
+    x_act, out = O.act_symmetric(3.0, 4), O.act_symmetric(1.0, 4)
+    xq = pack_codes(O.quantize(w["x"], x_act).reshape(T * B, K), x_act)
+    layers = [Bd.DeviceLstm(lw) for lw in w["layers"]]
+    run = lambda: Bd.qlstm_layer_forward(xq, to_act(x_act), T, B, layers, to_act(out), want_state=True)
+    a = run()
+    assert Bd.q4_poll_status(a["workspace"]) == 0
+    prev = Bd.encoder_time_slicing_set(False)
+    try:
+        b = run()
+    finally:
+        Bd.encoder_time_slicing_set(prev)
+    assert Bd.q4_poll_status(b["workspace"]) == 0
+    for k in ("yq", "hq_n", "c_n"):
+        assert torch.equal(a[k], b[k]), k
+
+
 def test_layer_per_sequence_input_scale(Bd):
     T, B, K, H = 8, 5, 64, 32
     w = synth.single_layer(seed=5, T=T, B=B, K=K, H=H, bits=8, dirs=2)
