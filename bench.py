@@ -790,7 +790,7 @@ def roofline(job, tag, ms, n, pk, series=None):
         # persistent recurrence: one launch = all T steps of a layer, both directions.  It must
         # read the int32 input accumulators once, the recurrent weights once, and write the codes.
         # By bytes it is an HBM kernel; in practice the T dependent steps (MMA, cell update,
-        # exchange of the new codes, cluster barrier) bind it, so the fraction is small by nature.
+        # exchange of the new codes between the CTAs of a cluster) bind it, so the fraction is small by nature.
         l = job.layer[0] if job.kind == "layer" else job.enc.layers[1][0]
         nd = 1 if job.kind == "layer" else 2
         Bn, Tn, H = wl["B"], wl["T"], l.H
@@ -807,7 +807,7 @@ def roofline(job, tag, ms, n, pk, series=None):
                    tensor={"achieved": ops / sec / 1e12, "peak": int8_peak, "unit": tensor_unit,
                            "frac": ops / sec / 1e12 / int8_peak},
                    us_per_step=ms * 1e3 / Tn,
-                   note="latency-bound: T dependent steps per launch, each ending in a cluster barrier")
+                   note="latency-bound: T dependent steps per launch, each waiting for the hidden codes of the other CTAs of its cluster")
         t = NCU_TRAFFIC["k_enc_recurrent"]
         if t is not None:
             # the traffic (input accumulators read once, codes written once) grows in proportion to

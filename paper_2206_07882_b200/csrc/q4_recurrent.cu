@@ -317,6 +317,8 @@ __device__ __forceinline__ void named_bar_arrive(int id, int count) {
 }
 
 __host__ __device__ constexpr int rec_w4_ksmem(int nu) { return nu <= 2 ? 6 : 8; }
+// k-steps of weights in shared memory, kernel whose clusters may take turns: packed 4-bit / int8
+__host__ __device__ constexpr int rec_turns_ksmem(bool w8) { return w8 ? 13 : 6; }
 
 template <int NU, int KS>
 __global__ void __cluster_dims__(REC_CLUSTER, 1, 1) __launch_bounds__(REC4_THREADS, 1)
@@ -612,7 +614,7 @@ __device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
   return v;
 }
 
-template <int KS>
+template <int KS, bool W8>
 __global__ void __cluster_dims__(REC_CLUSTER, 1, 1) __launch_bounds__(REC4_THREADS, 1)
 k_enc_recurrent_w4s(const EncRecArgs a) {
   extern __shared__ __align__(16) uint8_t rec_smem[];
@@ -624,7 +626,8 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
   constexpr int chunks = cpc >> 4;          // 16-byte chunks of a sequence's new codes per CTA
   constexpr int UB = BG * H;                // bytes of one group's hidden codes
   constexpr int CW = REC_THREADS / 32;      // warps
-  constexpr int KR = KS - rec_w4_ksmem(NS);
+  constexpr int KR = KS - rec_turns_ksmem(W8);   // k-steps whose weight fragments stay in registers
+  constexpr int WPK = W8 ? 4 : 2;                // 32-bit words of weights per thread and k-step
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_rank();
   const int cid = blockIdx.x / REC_CLUSTER;
@@ -644,7 +647,7 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
   int8_t* stage_y = stage + (size_t)2 * NS * BG * cpc;                     // [NS][2][BG][cpc] new output codes
   uint64_t* full = reinterpret_cast<uint64_t*>(stage_y + (size_t)2 * NS * BG * cpc);   // [NS][2]
   volatile int* dead = reinterpret_cast<volatile int*>(full + NS * 2);     // a bounded wait has expired
-  uint2* wsm = reinterpret_cast<uint2*>(full + NS * 2 + 2);                // [KS - KR][threads] packed weights
+  uint32_t* wsm = reinterpret_cast<uint32_t*>(full + NS * 2 + 2);          // [KS - KR][threads][WPK] weights
 
   const int g = lane >> 2, t4 = lane & 3;   // MMA fragment coordinates
   const int e = g & 1, ci = g >> 1;         // this lane's item: cell ci of the warp's 4 ...
@@ -654,7 +657,7 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
   const float sh = a.hid_act.scale;
   const uint32_t hb_addr = smem_u32(hb), pre_addr = smem_u32(pre_s), full_addr = smem_u32(full);
 
-  uint32_t wreg[2 * KR];
+  uint32_t wreg[WPK * KR];
   {
     const int8_t* W = D.w_hh + ((size_t)rank * rows + (size_t)(16 * warp)) * H;
     const int8_t* r0 = W + (size_t)(4 * ci + e) * H + 4 * t4;
@@ -665,13 +668,24 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
       const uint32_t p0 = *reinterpret_cast<const uint32_t*>(r1 + 32 * s);
       const uint32_t q1 = *reinterpret_cast<const uint32_t*>(r0 + 32 * s + 16);
       const uint32_t p1 = *reinterpret_cast<const uint32_t*>(r1 + 32 * s + 16);
-      const uint32_t w0p = (q0 & 0x0F0F0F0Fu) | ((p0 << 4) & 0xF0F0F0F0u);
-      const uint32_t w1p = (q1 & 0x0F0F0F0Fu) | ((p1 << 4) & 0xF0F0F0F0u);
-      if (s < KR) {
-        wreg[2 * s] = w0p;
-        wreg[2 * s + 1] = w1p;
-      } else {
-        wsm[(s - KR) * REC_THREADS + tid] = make_uint2(w0p, w1p);
+      if (W8) {   // one code per byte: the MMA fragment as it is
+        if (s < KR) {
+          wreg[WPK * s] = q0;
+          wreg[WPK * s + 1] = p0;
+          wreg[WPK * s + 2] = q1;
+          wreg[WPK * s + 3] = p1;
+        } else {
+          reinterpret_cast<uint4*>(wsm)[(s - KR) * REC_THREADS + tid] = make_uint4(q0, p0, q1, p1);
+        }
+      } else {    // two codes per byte
+        const uint32_t w0p = (q0 & 0x0F0F0F0Fu) | ((p0 << 4) & 0xF0F0F0F0u);
+        const uint32_t w1p = (q1 & 0x0F0F0F0Fu) | ((p1 << 4) & 0xF0F0F0F0u);
+        if (s < KR) {
+          wreg[WPK * s] = w0p;
+          wreg[WPK * s + 1] = w1p;
+        } else {
+          reinterpret_cast<uint2*>(wsm)[(s - KR) * REC_THREADS + tid] = make_uint2(w0p, w1p);
+        }
       }
     }
   }
@@ -680,8 +694,7 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
   for (int i = tid; i < cpc; i += REC4_THREADS) {
     const int c = (int)rank * cpc + i;
     const float4 w = reinterpret_cast<const float4*>(D.sc_hh)[c], v = reinterpret_cast<const float4*>(D.sc_ih)[c];
-    const float sxs = a.x_scale;
-    cst[i] = make_float4(__fmul_rn(sxs, v.x), __fmul_rn(sxs, v.y), __fmul_rn(sxs, v.z), __fmul_rn(sxs, v.w));
+    cst[i] = v;   // multiplied with the sequence's input scale at every use (the same fp32 product)
     cst[cpc + i] = make_float4(__fmul_rn(sh, w.x), __fmul_rn(sh, w.y), __fmul_rn(sh, w.z), __fmul_rn(sh, w.w));
     cst[2 * cpc + i] = reinterpret_cast<const float4*>(D.bias)[c];
   }
@@ -698,6 +711,9 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
   const int b_own = j * BG + n, b_shared = (a.groups - 1) * BG + n;
   const bool live_own = b_own < B, live_shared = host && b_shared < B;
   float c_own = 0.0f, c_shared = 0.0f;
+  const float sx_own = (a.x_scale_b && live_own) ? a.x_scale_b[b_own] : a.x_scale;
+  const float sx_shared = (a.x_scale_b && live_shared) ? a.x_scale_b[b_shared] : a.x_scale;
+  const bool h4 = a.hid_act.bits == 4;
   constexpr int G = 4 * H;
   const int hlo = act_lo(a.hid_act), hhi = act_hi(a.hid_act);
   const int ylo = act_lo(a.out_act), yhi = act_hi(a.out_act);
@@ -798,17 +814,35 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
       const uint32_t b_in = b_addr + half * 16u, b_wrap = b_addr + half * (uint32_t)(BG * cpc - (chunks - 1) * 16);
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        uint32_t w0p, w1p;
-        if (s < KR) {
-          w0p = wreg[2 * s];
-          w1p = wreg[2 * s + 1];
+        uint32_t a0, a1, a2, a3;
+        if (W8) {
+          if (s < KR) {
+            a0 = wreg[WPK * s];
+            a1 = wreg[WPK * s + 1];
+            a2 = wreg[WPK * s + 2];
+            a3 = wreg[WPK * s + 3];
+          } else {
+            const uint4 w = reinterpret_cast<const uint4*>(wsm)[(s - KR) * REC_THREADS + tid];
+            a0 = w.x;
+            a1 = w.y;
+            a2 = w.z;
+            a3 = w.w;
+          }
         } else {
-          const uint2 w = wsm[(s - KR) * REC_THREADS + tid];
-          w0p = w.x;
-          w1p = w.y;
+          uint32_t w0p, w1p;
+          if (s < KR) {
+            w0p = wreg[WPK * s];
+            w1p = wreg[WPK * s + 1];
+          } else {
+            const uint2 w = reinterpret_cast<const uint2*>(wsm)[(s - KR) * REC_THREADS + tid];
+            w0p = w.x;
+            w1p = w.y;
+          }
+          a0 = (w0p << 4) & 0xF0F0F0F0u;   // 16 x code
+          a1 = w0p & 0xF0F0F0F0u;
+          a2 = (w1p << 4) & 0xF0F0F0F0u;
+          a3 = w1p & 0xF0F0F0F0u;
         }
-        const uint32_t a0 = (w0p << 4) & 0xF0F0F0F0u, a1 = w0p & 0xF0F0F0F0u;
-        const uint32_t a2 = (w1p << 4) & 0xF0F0F0F0u, a3 = w1p & 0xF0F0F0F0u;
         const uint32_t o0 = (uint32_t)(((2 * s) / chunks) * BG * cpc + ((2 * s) % chunks) * 16);
         uint32_t b0, b1;
         ldmatrix_x2(((2 * s) % chunks == chunks - 1 ? b_wrap : b_in) + o0, b0, b1);
@@ -822,20 +856,22 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
       const int r0 = __shfl_xor_sync(0xffffffffu, e ? v0 : v1, 4);
       const int r1 = __shfl_xor_sync(0xffffffffu, e ? v2 : v3, 4);
       const int m0 = e ? v1 : v0, m1 = e ? v3 : v2;
-      hh[0] = (e ? r0 : m0) >> 4;     // the operand was 16 x code
-      hh[1] = (e ? m0 : r0) >> 4;
-      hh[2] = (e ? r1 : m1) >> 4;
-      hh[3] = (e ? m1 : r1) >> 4;
+      constexpr int SH = W8 ? 0 : 4;   // the packed operand was 16 x code
+      hh[0] = (e ? r0 : m0) >> SH;
+      hh[1] = (e ? m0 : r0) >> SH;
+      hh[2] = (e ? r1 : m1) >> SH;
+      hh[3] = (e ? m1 : r1) >> SH;
     }
     cp_async_wait<1>();               // this thread's accumulators of the present step have landed
     int q = 0, q2 = 0;
     if (live) {
       const int4 pre = pre_s[(i & 1) * REC_THREADS + tid];
       const float4 s_ih = cst[cl], s_hh = cst[cpc + cl], bb = cst[2 * cpc + cl];
-      const float pi = __fmaf_rn((float)hh[0], s_hh.x, __fmaf_rn((float)pre.x, s_ih.x, bb.x));
-      const float pf = __fmaf_rn((float)hh[1], s_hh.y, __fmaf_rn((float)pre.y, s_ih.y, bb.y));
-      const float pg = __fmaf_rn((float)hh[2], s_hh.z, __fmaf_rn((float)pre.z, s_ih.z, bb.z));
-      const float po = __fmaf_rn((float)hh[3], s_hh.w, __fmaf_rn((float)pre.w, s_ih.w, bb.w));
+      const float sx = u ? sx_shared : sx_own;
+      const float pi = __fmaf_rn((float)hh[0], s_hh.x, __fmaf_rn((float)pre.x, __fmul_rn(sx, s_ih.x), bb.x));
+      const float pf = __fmaf_rn((float)hh[1], s_hh.y, __fmaf_rn((float)pre.y, __fmul_rn(sx, s_ih.y), bb.y));
+      const float pg = __fmaf_rn((float)hh[2], s_hh.z, __fmaf_rn((float)pre.z, __fmul_rn(sx, s_ih.z), bb.z));
+      const float po = __fmaf_rn((float)hh[3], s_hh.w, __fmaf_rn((float)pre.w, __fmul_rn(sx, s_ih.w), bb.w));
       float cs = u ? c_shared : c_own, hval;
       cell_fixed(pi, pf, pg, po, cs, cs, hval);
       if (u)
@@ -847,9 +883,11 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
     }
     stage[((u * 2 + cur) * BG + n) * cpc + cl] = (int8_t)q;
     stage_y[((u * 2 + cur) * BG + n) * cpc + cl] = (int8_t)q2;
-    if (step == T - 1 && D.hq_n) {   // final recurrent codes, two cells per byte: the even cell's lane writes
+    if (step == T - 1 && D.hq_n) {   // final recurrent codes; at 4 bits two cells per byte: the even cell's lane writes
       const int qn = __shfl_down_sync(0xffffffffu, q, 8);
-      if (live && (cl & 1) == 0)
+      if (live && !h4)
+        D.hq_n[(size_t)b * H + cell] = (uint8_t)q;
+      else if (live && (cl & 1) == 0)
         D.hq_n[(size_t)b * (H >> 1) + (cell >> 1)] = (uint8_t)((q & 0xF) | ((qn & 0xF) << 4));
     }
     fence_proxy_async();   // the staged codes are read by the bulk-copy engine
@@ -998,19 +1036,19 @@ static size_t enc_recurrent_w4_smem(int H, int NU) {
          (size_t)3 * cpc * sizeof(float4) + (size_t)4 * NU * REC_BG * cpc + (size_t)NU * 2 * sizeof(uint64_t) + 32 + (size_t)rec_w4_ksmem(NU) * REC_THREADS * sizeof(uint2);
 }
 
-template <int KS>
+template <int KS, bool W8>
 static cudaError_t rec_w4s_launch(const EncRecArgs& a, cudaStream_t s) {
   const int H = 32 * KS, cpc = H / REC_CLUSTER;
   const size_t smem = (size_t)2 * 2 * REC_BG * H + (size_t)2 * REC_THREADS * sizeof(int4) + (size_t)3 * cpc * sizeof(float4) +
                       (size_t)4 * 2 * REC_BG * cpc + (size_t)2 * 2 * sizeof(uint64_t) + 32 +
-                      (size_t)rec_w4_ksmem(2) * REC_THREADS * sizeof(uint2);
+                      (size_t)rec_turns_ksmem(W8) * REC_THREADS * (W8 ? sizeof(uint4) : sizeof(uint2));
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_enc_recurrent_w4s<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_enc_recurrent_w4s<KS, W8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  k_enc_recurrent_w4s<KS><<<(unsigned)((a.ncl[0] + a.ncl[1]) * REC_CLUSTER), REC4_THREADS, smem, s>>>(a);
+  k_enc_recurrent_w4s<KS, W8><<<(unsigned)((a.ncl[0] + a.ncl[1]) * REC_CLUSTER), REC4_THREADS, smem, s>>>(a);
   return cudaGetLastError();
 }
 
@@ -1028,27 +1066,37 @@ static cudaError_t rec_w4_launch(const EncRecArgs& a, cudaStream_t s) {
 }
 
 cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s) {
-  // 4-bit recurrent weights and hidden codes at 640 cells: the register-resident kernel, with as few
-  // units of 8 sequences per cluster as keeps all clusters resident at once
-  // (no per-sequence input scale and no accumulator dump: those take the general kernel)
-  if (a.w_bits == 4 && a.hid_act.bits == 4 && a.hid_act.is_signed && a.H == 640 && !a.x_scale_b &&
-      !a.d[0].dbg_ih) {
-    const int groups = (a.B + REC_BG - 1) / REC_BG, maxc = rec_max_clusters(a.H);
-    // one or two groups more than clusters: a direction's clusters take turns at its last group
+  // 640 cells, no accumulator dump: the kernels that keep (most of) a CTA's recurrent weights in
+  // registers; the general kernel otherwise
+  const int groups = (a.B + REC_BG - 1) / REC_BG;
+  const bool regs_ok = a.hid_act.is_signed && a.H == 640 && !a.d[0].dbg_ih && (a.w_bits == 4 || a.w_bits == 8) &&
+                       (a.hid_act.bits == 4 || a.hid_act.bits == 8);
+  if (regs_ok) {
+    // The kernel whose clusters may take turns: with one group more than clusters per sliced
+    // direction, and (all directions plain) for what the packed kernel below does not take: int8
+    // weights, 8-bit hidden codes, an input scale per sequence.
+    const int maxc = rec_max_clusters(a.H);
     const int lack = a.dirs * groups - maxc;
-    if (g_rec_sliced && lack >= 1 && lack <= a.dirs && groups >= 2 && groups <= 8 && a.T >= 8 * groups && a.flags &&
-        a.hand_h[0] && a.hand_c[0]) {
+    const bool plain_only = a.w_bits == 8 || a.hid_act.bits == 8 || a.x_scale_b;
+    const bool turns = g_rec_sliced && lack >= 1 && lack <= a.dirs && groups >= 2 && groups <= 8 && a.T >= 8 * groups &&
+                       a.flags && a.hand_h[0] && a.hand_c[0];
+    if (turns || (lack <= 0 && plain_only && groups <= 8 && a.flags)) {
       a.groups = groups;
       for (int d = 0; d < 2; ++d) {
-        a.sliced[d] = d < a.dirs && d < lack ? 1 : 0;
+        a.sliced[d] = turns && d < a.dirs && d < lack ? 1 : 0;
         a.ncl[d] = d < a.dirs ? groups - a.sliced[d] : 0;
       }
       timing_begin(s);
-      cudaError_t e = rec_w4s_launch<20>(a, s);
+      cudaError_t e = a.w_bits == 8 ? rec_w4s_launch<20, true>(a, s) : rec_w4s_launch<20, false>(a, s);
       timing_end(s);
       ++g_launches;
       return e;
     }
+  }
+  // packed 4-bit weights with as few groups of 8 sequences per cluster as keeps all clusters resident
+  if (a.w_bits == 4 && a.hid_act.bits == 4 && a.hid_act.is_signed && a.H == 640 && !a.x_scale_b &&
+      !a.d[0].dbg_ih) {
+    const int maxc = rec_max_clusters(a.H);
     int nu = 1;
     while (nu <= 4 && a.dirs * ((groups + nu - 1) / nu) > maxc) ++nu;
     if (nu <= 4) {

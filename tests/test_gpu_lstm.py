@@ -145,6 +145,9 @@ def test_config0_layer_forward(Bd):
                                                    # 64 and 60 sequences x 2 directions of 640 cells: groups of 16
                                                    # sequences per cluster, full and ragged
                                                    (6, 64, 64, 640, 2, 4, 4, 4), (5, 60, 32, 640, 2, 8, 8, 4),
+                                                   # 8-bit layers of 640 cells, one group of 8 per cluster: int8
+                                                   # weights split between registers and shared memory
+                                                   (9, 20, 32, 640, 2, 8, 8, 4), (7, 30, 32, 640, 1, 8, 8, 8),
                                                    # 7620 rows x 1280 gate rows: 298 tiles of the input projection with a
                                                    # ragged last row tile, more than two per SM (the persistent GEMM)
                                                    (60, 127, 32, 320, 1, 4, 4, 4)])
@@ -157,6 +160,12 @@ def test_layer_clusters_taking_turns_at_a_surplus_group(Bd):
     # clusters of one direction take turns at its eighth group (9 of 64 steps each, one more on the
     # last; the group holds one live sequence), the other direction runs one group per cluster
     diff = layer_case(Bd, T=64, B=57, K=64, H=640, dirs=2, seed=23)
+    assert (diff > 0).sum() == 0
+
+
+def test_layer_clusters_taking_turns_eight_bit(Bd):
+    # the same with 8-bit weights and codes (the first encoder layer of the end-to-end workload)
+    diff = layer_case(Bd, T=64, B=57, K=64, H=640, dirs=2, xb=8, hb=8, ob=4, seed=37)
     assert (diff > 0).sum() == 0
 
 
@@ -181,8 +190,11 @@ def test_layer_time_slicing_equals_two_groups_per_cluster(Bd):
         assert torch.equal(a[k], b[k]), k
 
 
-def test_layer_per_sequence_input_scale(Bd):
-    T, B, K, H = 8, 5, 64, 32
+@pytest.mark.parametrize("T,B,K,H", [(8, 5, 64, 32),
+                                     # 640 cells: int8 weights mostly in registers; 20 sequences = one group per
+                                     # cluster, 57 over 64 steps = the clusters of one direction take turns
+                                     (8, 20, 64, 640), (64, 57, 64, 640)])
+def test_layer_per_sequence_input_scale(Bd, T, B, K, H):
     w = synth.single_layer(seed=5, T=T, B=B, K=K, H=H, bits=8, dirs=2)
     base = O.act_symmetric(1.0, 8)
     xq = np.empty((T, B, K), np.int16)
@@ -198,6 +210,7 @@ def test_layer_per_sequence_input_scale(Bd):
     got = Bd.qlstm_layer_forward(pack_codes(xq.reshape(T * B, K), base), to_act(base), T, B,
                                  [Bd.DeviceLstm(lw) for lw in w["layers"]],
                                  x_scale_b=torch.from_numpy(sc).cuda())
+    assert Bd.q4_poll_status(got["workspace"]) == 0
     yq = gpu_codes(got["yq"], 2 * H, hid).reshape(T, B, 2 * H)
     np.testing.assert_array_equal(yq, ref["yq"])
 
