@@ -47,6 +47,9 @@ WORKLOADS = {
     # reduced lengths of the same shapes, for profiler captures that must end by themselves
     "prof_encoder": dict(B=32, T=250, U_max=0, l1_bits=4, out_bits=4, enc=True, dec=False, seed=1),
     "prof_end_to_end": dict(B=64, T=24, U_max=12, l1_bits=8, out_bits=8, enc=True, dec=True, seed=4),
+    # the encoder of the end-to-end workload at a quarter of its length (64 utterances: one group of 8
+    # sequences more than resident clusters, so the clusters of one direction take turns)
+    "prof_encoder_64": dict(B=64, T=128, U_max=0, l1_bits=8, out_bits=4, enc=True, dec=False, seed=4),
     # the regime of the paper's run-time figure (Section 4.1): ONE utterance of 152 encoder frames,
     # everything at 4 bits, beam width from --beam (1..16): 16 hypothesis rows at most, so every
     # step streams all weights for a handful of rows
@@ -604,6 +607,10 @@ NCU_TRAFFIC = {
     "k_enc_recurrent": {"bytes": 167198464 + 7500288, "steps": 250, "sequences": 32,
                         "captured": "ncu capture of k_enc_recurrent_w4<1,20>, workload prof_encoder; scaled by steps x "
                                     "sequences (accumulators read once, codes written once)"},
+    # the same with one group of sequences more than clusters (clusters take turns), 128 steps x 64 sequences
+    "k_enc_recurrent_turns": {"bytes": 171157760 + 6593792, "steps": 128, "sequences": 64,
+                              "captured": "ncu capture of k_enc_recurrent_w4s<20,0>, workload prof_encoder_64; scaled by "
+                                          "steps x sequences (accumulators read once, codes written once)"},
 }
 
 
@@ -808,8 +815,9 @@ def roofline(job, tag, ms, n, pk, series=None):
                            "frac": ops / sec / 1e12 / int8_peak},
                    us_per_step=ms * 1e3 / Tn,
                    note="latency-bound: T dependent steps per launch, each waiting for the hidden codes of the other CTAs of its cluster")
-        t = NCU_TRAFFIC["k_enc_recurrent"]
-        if t is not None:
+        # more groups of 8 sequences than the 15 clusters that fit: the kernel whose clusters take turns
+        t = NCU_TRAFFIC["k_enc_recurrent_turns" if nd * ((Bn + 7) // 8) > 15 else "k_enc_recurrent"]
+        if t is not None and job.kind != "layer":
             # the traffic (input accumulators read once, codes written once) grows in proportion to
             # steps x sequences
             out["traffic"] = t["bytes"] * (Tn * Bn) / float(t["steps"] * t["sequences"])
