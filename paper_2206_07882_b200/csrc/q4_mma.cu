@@ -1188,15 +1188,30 @@ k_mma_lstm(const __grid_constant__ CUtensorMap tma_xa, const __grid_constant__ C
       const float cp[4] = {cprev.x, cprev.y, cprev.z, cprev.w};
       float cn[4], hn[4];
       int qh[4], qy[4];
+      // pre-activations of the four cells: acc_hh * s_hh + (acc_ih * s_ih + bias), gates (i, f) and (g, o)
+      // as pairs on the paired fp32 instructions (the same two roundings per value as the scalar form)
+      float pre[4][4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float4 s_ih = s_cst[0][ct + c], s_hh = s_cst[1][ct + c], bb = s_cst[2][ct + c];
+        const uint64_t sih0 = PREMUL ? pk2(s_ih.x, s_ih.y) : pk2(__fmul_rn(sx, s_ih.x), __fmul_rn(sx, s_ih.y));
+        const uint64_t sih1 = PREMUL ? pk2(s_ih.z, s_ih.w) : pk2(__fmul_rn(sx, s_ih.z), __fmul_rn(sx, s_ih.w));
+        const uint64_t shh0 = PREMUL ? pk2(s_hh.x, s_hh.y) : pk2(__fmul_rn(sh, s_hh.x), __fmul_rn(sh, s_hh.y));
+        const uint64_t shh1 = PREMUL ? pk2(s_hh.z, s_hh.w) : pk2(__fmul_rn(sh, s_hh.z), __fmul_rn(sh, s_hh.w));
+        const uint64_t v0 = fma2(pk2((float)hh[4 * c + 0], (float)hh[4 * c + 1]), shh0,
+                                 fma2(pk2((float)ih[4 * c + 0], (float)ih[4 * c + 1]), sih0, pk2(bb.x, bb.y)));
+        const uint64_t v1 = fma2(pk2((float)hh[4 * c + 2], (float)hh[4 * c + 3]), shh1,
+                                 fma2(pk2((float)ih[4 * c + 2], (float)ih[4 * c + 3]), sih1, pk2(bb.z, bb.w)));
+        upk2(v0, pre[c][0], pre[c][1]);
+        upk2(v1, pre[c][2], pre[c][3]);
+      }
+#pragma unroll
+      for (int c = 0; c < 4; c += 2)   // two cells per call
+        cell_fixed2(pre[c][0], pre[c][1], pre[c][2], pre[c][3], cp[c], pre[c + 1][0], pre[c + 1][1], pre[c + 1][2],
+                    pre[c + 1][3], cp[c + 1], cn[c], hn[c], cn[c + 1], hn[c + 1]);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const int cell = cell0 + c;
-        const float4 s_ih = s_cst[0][ct + c], s_hh = s_cst[1][ct + c], bb = s_cst[2][ct + c];
-        const float pi = __fmaf_rn((float)hh[4 * c + 0], (PREMUL ? s_hh.x : __fmul_rn(sh, s_hh.x)), __fmaf_rn((float)ih[4 * c + 0], (PREMUL ? s_ih.x : __fmul_rn(sx, s_ih.x)), bb.x));
-        const float pf = __fmaf_rn((float)hh[4 * c + 1], (PREMUL ? s_hh.y : __fmul_rn(sh, s_hh.y)), __fmaf_rn((float)ih[4 * c + 1], (PREMUL ? s_ih.y : __fmul_rn(sx, s_ih.y)), bb.y));
-        const float pg = __fmaf_rn((float)hh[4 * c + 2], (PREMUL ? s_hh.z : __fmul_rn(sh, s_hh.z)), __fmaf_rn((float)ih[4 * c + 2], (PREMUL ? s_ih.z : __fmul_rn(sx, s_ih.z)), bb.z));
-        const float po = __fmaf_rn((float)hh[4 * c + 3], (PREMUL ? s_hh.w : __fmul_rn(sh, s_hh.w)), __fmaf_rn((float)ih[4 * c + 3], (PREMUL ? s_ih.w : __fmul_rn(sx, s_ih.w)), bb.w));
-        cell_fixed(pi, pf, pg, po, cp[c], cn[c], hn[c]);
         qh[c] = quantize1(hn[c], a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
         qy[c] = EXTRAS ? quantize1(hn[c], a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi) : 0;
         if (EXTRAS && a.dbg_ih) {
