@@ -398,6 +398,17 @@ int q4_beam_select_exact_set(int32_t enabled);
  * and measurements; the results are identical).  Returns the previous setting. */
 int q4_encoder_time_slicing_set(int32_t enabled);
 
+/* How qlstm_layer_forward lays a layer's recurrence on thread-block clusters (host logic only, no
+ * launch; for tests and diagnostics; with no device present the cluster capacity defaults to 15).
+ * out[17]: [0] kernel (0 general, 1 packed 4-bit weights in registers, 2 the kernel whose clusters
+ * may take turns), [1] groups of 8 sequences per cluster, [2..3] clusters per direction, [4..5]
+ * whether the direction's clusters take turns at its last group, [6] groups per direction, [7]
+ * clusters that can be resident, [8..16] step bounds of the turns: cluster j of such a direction
+ * advances the shared group over steps [out[8+j], out[9+j]).  Assumes a signed hidden quantizer,
+ * no accumulator dump and a caller workspace (as qlstm_layer_forward provides). */
+int q4_encoder_recurrence_plan(int32_t T, int32_t B, int32_t dirs, int32_t H, int32_t w_bits, int32_t hid_bits,
+                               int32_t per_sequence_scale, int32_t* out);
+
 /* Test hook for the bounded device-side waits (not an operation of the paper): while skip_producer
  * is non-zero the tiled tensor-core GEMM (the tensor-core paths of q4_linear_forward and of the
  * projections) launches with a producer that issues no copy at all, so that the consumer's wait

@@ -81,7 +81,7 @@ EXPORTS = ["q4_act_symmetric", "q4_act_asymmetric", "quantize_pack_int4", "qlstm
            "qlstm_step", "q4_linear_forward", "qjoint_logprobs", "q4_beam_init",
            "dr_fusion_beam_step", "q4_traceback", "q4_feature_prologue", "q4_workspace_bytes",
            "q4_poll_status", "q4_version", "q4_launch_count", "q4_dependent_launch_set", "q4_beam_select_exact_set", "q4_timing_set", "q4_timing_count", "q4_prepared_bytes", "q4_prepare_model", "qjoint_logprobs_static", "q4_quantizer_calls", "q4_prepared_lstm_bytes", "q4_prepare_lstm",
-           "q4_prepared_linear_bytes", "q4_prepare_linear", "q4_test_wait_expiry_set", "q4_encoder_time_slicing_set"]
+           "q4_prepared_linear_bytes", "q4_prepare_linear", "q4_test_wait_expiry_set", "q4_encoder_time_slicing_set", "q4_encoder_recurrence_plan"]
 
 _lib = None
 
@@ -148,6 +148,18 @@ def dependent_launch_set(enabled: bool) -> bool:
 def encoder_time_slicing_set(enabled: bool) -> bool:
     """Let the clusters of the encoder recurrence take turns at a surplus group of sequences (default) or not; returns the previous setting."""
     return bool(lib().q4_encoder_time_slicing_set(1 if enabled else 0))
+
+
+def encoder_recurrence_plan(T: int, B: int, dirs: int, H: int, w_bits: int = 4, hid_bits: int = 4,
+                            per_sequence_scale: bool = False) -> dict:
+    """Host-side plan of a layer's recurrence (no launch): kernel, clusters per direction, turns."""
+    out = (C.c_int32 * 17)()
+    _chk(lib().q4_encoder_recurrence_plan(C.c_int32(T), C.c_int32(B), C.c_int32(dirs), C.c_int32(H), C.c_int32(w_bits),
+                                          C.c_int32(hid_bits), C.c_int32(1 if per_sequence_scale else 0), out),
+         "q4_encoder_recurrence_plan")
+    v = list(out)
+    return dict(kernel=v[0], groups_per_cluster=v[1], clusters=v[2:4], turns=v[4:6], groups=v[6], max_clusters=v[7],
+                windows=v[8:17])
 
 
 def beam_select_exact_set(enabled: bool) -> bool:

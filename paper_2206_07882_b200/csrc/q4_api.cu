@@ -103,6 +103,22 @@ int q4_test_wait_expiry_set(int32_t skip_producer, uint32_t wait_limit) {
   return Q4_OK;
 }
 int q4_encoder_time_slicing_set(int32_t enabled) { return enc_recurrent_sliced_set(enabled ? 1 : 0); }
+int q4_encoder_recurrence_plan(int32_t T, int32_t B, int32_t dirs, int32_t H, int32_t w_bits, int32_t hid_bits,
+                               int32_t per_sequence_scale, int32_t* out) {
+  if (!out) return Q4_ERR_NULL;
+  if (T <= 0 || B <= 0 || dirs < 1 || dirs > 2 || H <= 0) return Q4_ERR_DIM;
+  const EncRecPlan p = enc_recurrent_plan(T, B, dirs, H, w_bits, hid_bits, true, per_sequence_scale != 0, false, true);
+  out[0] = p.kernel;
+  out[1] = p.groups_per_cluster;
+  out[2] = p.ncl[0];
+  out[3] = p.ncl[1];
+  out[4] = p.sliced[0];
+  out[5] = p.sliced[1];
+  out[6] = p.groups;
+  out[7] = p.max_clusters;
+  for (int j = 0; j < 9; ++j) out[8 + j] = p.win[j];
+  return Q4_OK;
+}
 int q4_dependent_launch_set(int32_t enabled) {
   const int prev = g_dependent_launch;
   g_dependent_launch = enabled ? 1 : 0;

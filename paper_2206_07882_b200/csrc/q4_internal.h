@@ -191,12 +191,23 @@ struct EncRecArgs {
   int32_t ncl[2];           // clusters of each direction
   int32_t sliced[2];        // 1: the direction's clusters take turns at its last group
   int32_t groups;           // groups of 8 sequences per direction
+  int32_t win[9];           // cluster j of a sliced direction advances the shared group over steps [win[j], win[j+1])
   int32_t* flags;           // [2][8] hand-over counters, zero before the launch
   uint8_t* hand_h[2];       // [8][8][H / 8] hidden codes of the shared group at a hand-over, per direction
   float* hand_c[2];         // [8][H] its cell states
 };
 bool enc_recurrent_supported(int H, int B, int dirs);
 int enc_recurrent_sliced_set(int enabled);   // returns the previous setting
+// Which recurrence kernel a layer takes and how its groups of sequences are laid on clusters (host only).
+struct EncRecPlan {
+  int32_t kernel;           // 0: general kernel (int8 weights in shared memory), 1: packed weights in registers,
+                            // groups_per_cluster groups per cluster, 2: kernel whose clusters may take turns
+  int32_t groups_per_cluster;
+  int32_t ncl[2], sliced[2], groups, max_clusters;
+  int32_t win[9];
+};
+EncRecPlan enc_recurrent_plan(int T, int B, int dirs, int H, int w_bits, int hid_bits, bool hid_signed,
+                              bool per_sequence_scale, bool dump, bool scratch);
 cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s);
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }

@@ -638,7 +638,7 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
   const EncRecDir& D = a.d[d];
   const int T = a.T, B = a.B;
   // the shared group's steps [w0, w1) run here
-  const int w0 = host ? (int)((long long)j * T / C) : 0, w1 = host ? (int)((long long)(j + 1) * T / C) : 0;
+  const int w0 = host ? a.win[j] : 0, w1 = host ? a.win[j + 1] : 0;
   const int n_it = T + (w1 - w0);
   int8_t* hb = reinterpret_cast<int8_t*>(rec_smem);                       // [NS][2][source CTA][BG][cpc] h_{t-1}
   int4* pre_s = reinterpret_cast<int4*>(hb + (size_t)NS * 2 * UB);        // [2][threads] input accumulators
@@ -1065,49 +1065,77 @@ static cudaError_t rec_w4_launch(const EncRecArgs& a, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s) {
+EncRecPlan enc_recurrent_plan(int T, int B, int dirs, int H, int w_bits, int hid_bits, bool hid_signed,
+                              bool per_sequence_scale, bool dump, bool scratch) {
+  EncRecPlan p;
+  memset(&p, 0, sizeof(p));
+  const int groups = (B + REC_BG - 1) / REC_BG;
+  p.groups = groups;
+  p.max_clusters = rec_max_clusters(H);
   // 640 cells, no accumulator dump: the kernels that keep (most of) a CTA's recurrent weights in
   // registers; the general kernel otherwise
-  const int groups = (a.B + REC_BG - 1) / REC_BG;
-  const bool regs_ok = a.hid_act.is_signed && a.H == 640 && !a.d[0].dbg_ih && (a.w_bits == 4 || a.w_bits == 8) &&
-                       (a.hid_act.bits == 4 || a.hid_act.bits == 8);
+  const bool regs_ok = hid_signed && H == 640 && !dump && (w_bits == 4 || w_bits == 8) && (hid_bits == 4 || hid_bits == 8);
   if (regs_ok) {
     // The kernel whose clusters may take turns: with one group more than clusters per sliced
     // direction, and (all directions plain) for what the packed kernel below does not take: int8
     // weights, 8-bit hidden codes, an input scale per sequence.
-    const int maxc = rec_max_clusters(a.H);
-    const int lack = a.dirs * groups - maxc;
-    const bool plain_only = a.w_bits == 8 || a.hid_act.bits == 8 || a.x_scale_b;
-    const bool turns = g_rec_sliced && lack >= 1 && lack <= a.dirs && groups >= 2 && groups <= 8 && a.T >= 8 * groups &&
-                       a.flags && a.hand_h[0] && a.hand_c[0];
-    if (turns || (lack <= 0 && plain_only && groups <= 8 && a.flags)) {
-      a.groups = groups;
+    const int lack = dirs * groups - p.max_clusters;
+    const bool plain_only = w_bits == 8 || hid_bits == 8 || per_sequence_scale;
+    const bool turns = g_rec_sliced && lack >= 1 && lack <= dirs && groups >= 2 && groups <= 8 && T >= 8 * groups && scratch;
+    if (turns || (lack <= 0 && plain_only && groups <= 8 && scratch)) {
+      p.kernel = 2;
+      p.groups_per_cluster = 1;
       for (int d = 0; d < 2; ++d) {
-        a.sliced[d] = turns && d < a.dirs && d < lack ? 1 : 0;
-        a.ncl[d] = d < a.dirs ? groups - a.sliced[d] : 0;
+        p.sliced[d] = turns && d < dirs && d < lack ? 1 : 0;
+        p.ncl[d] = d < dirs ? groups - p.sliced[d] : 0;
       }
-      timing_begin(s);
-      cudaError_t e = a.w_bits == 8 ? rec_w4s_launch<20, true>(a, s) : rec_w4s_launch<20, false>(a, s);
-      timing_end(s);
-      ++g_launches;
-      return e;
+      if (turns)   // equal shares of the T steps, in cluster order
+        for (int j = 0; j <= groups - 1; ++j) p.win[j] = (int)((long long)j * T / (groups - 1));
+      return p;
     }
   }
   // packed 4-bit weights with as few groups of 8 sequences per cluster as keeps all clusters resident
-  if (a.w_bits == 4 && a.hid_act.bits == 4 && a.hid_act.is_signed && a.H == 640 && !a.x_scale_b &&
-      !a.d[0].dbg_ih) {
-    const int maxc = rec_max_clusters(a.H);
+  if (regs_ok && w_bits == 4 && hid_bits == 4 && !per_sequence_scale) {
     int nu = 1;
-    while (nu <= 4 && a.dirs * ((groups + nu - 1) / nu) > maxc) ++nu;
+    while (nu <= 4 && dirs * ((groups + nu - 1) / nu) > p.max_clusters) ++nu;
     if (nu <= 4) {
-      a.n_groups = (groups + nu - 1) / nu;   // clusters per direction
-      timing_begin(s);
-      cudaError_t e = nu == 1 ? rec_w4_launch<1, 20>(a, s) : nu == 2 ? rec_w4_launch<2, 20>(a, s)
-                      : nu == 3 ? rec_w4_launch<3, 20>(a, s) : rec_w4_launch<4, 20>(a, s);
-      timing_end(s);
-      ++g_launches;
-      return e;
+      p.kernel = 1;
+      p.groups_per_cluster = nu;
+      p.ncl[0] = (groups + nu - 1) / nu;
+      p.ncl[1] = dirs == 2 ? p.ncl[0] : 0;
+      return p;
     }
+  }
+  p.kernel = 0;
+  return p;
+}
+
+cudaError_t launch_enc_recurrent(EncRecArgs a, cudaStream_t s) {
+  const EncRecPlan p = enc_recurrent_plan(a.T, a.B, a.dirs, a.H, a.w_bits, a.hid_act.bits, a.hid_act.is_signed != 0,
+                                          a.x_scale_b != nullptr, a.d[0].dbg_ih != nullptr,
+                                          a.flags && a.hand_h[0] && a.hand_c[0]);
+  if (p.kernel == 2) {
+    a.groups = p.groups;
+    for (int d = 0; d < 2; ++d) {
+      a.sliced[d] = p.sliced[d];
+      a.ncl[d] = p.ncl[d];
+    }
+    for (int j = 0; j < 9; ++j) a.win[j] = p.win[j];
+    timing_begin(s);
+    cudaError_t e = a.w_bits == 8 ? rec_w4s_launch<20, true>(a, s) : rec_w4s_launch<20, false>(a, s);
+    timing_end(s);
+    ++g_launches;
+    return e;
+  }
+  if (p.kernel == 1) {
+    const int nu = p.groups_per_cluster;
+    a.n_groups = p.ncl[0];   // clusters per direction
+    timing_begin(s);
+    cudaError_t e = nu == 1 ? rec_w4_launch<1, 20>(a, s) : nu == 2 ? rec_w4_launch<2, 20>(a, s)
+                    : nu == 3 ? rec_w4_launch<3, 20>(a, s) : rec_w4_launch<4, 20>(a, s);
+    timing_end(s);
+    ++g_launches;
+    return e;
   }
   const int BG = enc_recurrent_group(a.B, a.dirs, a.H);
   a.n_groups = (a.B + BG - 1) / BG;

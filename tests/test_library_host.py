@@ -111,3 +111,38 @@ def test_no_cpu_fallback(Bd):
     x = torch.zeros((2, 32))
     with pytest.raises((RuntimeError, AssertionError)):
         Bd.quantize_pack_int4(x, Bd.q4_act_symmetric(1.0, 4))
+
+
+def test_encoder_recurrence_plan_lays_groups_on_clusters():
+    # host logic of qlstm_layer_forward's recurrence: which kernel, how many clusters, whose turn when
+    from paper_2206_07882_b200 import binding as Bd
+    plan = Bd.encoder_recurrence_plan
+    p = plan(500, 32, 2, 640)                      # 4 groups x 2 directions: one group per cluster
+    cap = p["max_clusters"]
+    assert cap >= 8 and p["kernel"] == 1 and p["groups_per_cluster"] == 1 and p["clusters"] == [4, 4]
+    for T, B in ((500, 64), (64, 57), (152, 60)):   # 8 groups x 2 directions
+        p = plan(T, B, 2, 640)
+        lack = 16 - cap
+        if 1 <= lack <= 2:                          # one group more than clusters in `lack` directions: turns
+            assert p["kernel"] == 2 and p["groups"] == 8
+            assert p["turns"] == [1, 1 if lack == 2 else 0]
+            assert sum(p["clusters"]) == cap and p["clusters"][0] == 7
+            w = p["windows"][:8]
+            assert w[0] == 0 and w[-1] == T and all(b > a for a, b in zip(w, w[1:]))      # a partition of the steps
+            assert max(b - a for a, b in zip(w, w[1:])) - min(b - a for a, b in zip(w, w[1:])) <= 1
+    p = plan(20, 64, 2, 640)                        # too few steps for turns: several groups per cluster
+    assert p["kernel"] == 1 and p["groups_per_cluster"] * sum(p["clusters"]) >= 16 and sum(p["clusters"]) <= cap
+    p = plan(500, 128, 2, 640)                      # 16 groups per direction
+    assert p["kernel"] == 1 and sum(p["clusters"]) <= cap and p["groups_per_cluster"] * p["clusters"][0] >= 16
+    # 8-bit weights or codes, or an input scale per sequence: the kernel with int8 fragments / per-sequence
+    # scales while one group per cluster fits, the general kernel beyond
+    assert plan(500, 32, 2, 640, w_bits=8, hid_bits=8)["kernel"] == 2
+    assert plan(500, 32, 2, 640, per_sequence_scale=True)["kernel"] == 2
+    assert plan(500, 64, 2, 640, w_bits=8, hid_bits=8)["kernel"] == (2 if 1 <= 16 - cap <= 2 else 0)
+    assert plan(500, 128, 2, 640, w_bits=8, hid_bits=8)["kernel"] == 0
+    assert plan(500, 32, 2, 320)["kernel"] == 0     # other widths: general kernel
+    import ctypes as C
+    assert Bd.lib().q4_encoder_recurrence_plan(C.c_int32(0), C.c_int32(4), C.c_int32(2), C.c_int32(640), C.c_int32(4),
+                                               C.c_int32(4), C.c_int32(0), (C.c_int32 * 17)()) == -2
+    assert Bd.lib().q4_encoder_recurrence_plan(C.c_int32(5), C.c_int32(4), C.c_int32(2), C.c_int32(640), C.c_int32(4),
+                                               C.c_int32(4), C.c_int32(0), None) == -1
