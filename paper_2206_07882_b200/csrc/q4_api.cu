@@ -271,7 +271,7 @@ int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_m
                                 Mp, s));
       Q4_TRY(launch_mma_gemm(x8, w->k_pad, M, static_cast<const int8_t*>(prepared), w->k_pad, w->rows, w->k_pad,
                              EPI_F32, out, w->rows, nullptr, w->scale, bias, x_act->scale, nullptr, status, nullptr,
-                             s));
+                             s, true));   // programmatic dependent of the gather before it
       return Q4_OK;
     }
   }
@@ -377,7 +377,8 @@ int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, co
       a.dbg_hh = dbg_acc_hh;
       a.dbg_ld = 4LL * H;
       a.status = status;
-      Q4_TRY(launch_mma_lstm(a, x8, (long long)Kx, xw8, (long long)Kx, h8, H, hw8, H, s));
+      // programmatic dependent of the second gather (which started after the first had completed)
+      Q4_TRY(launch_mma_lstm(a, x8, (long long)Kx, xw8, (long long)Kx, h8, H, hw8, H, s, true));
       return Q4_OK;
     }
   }
@@ -601,8 +602,8 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
     Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
     Q4_TRY(launch_unpack_rows(pq, row_bytes(Hp, p_act->bits), nullptr, *p_act, Hp, N, p8, Hp, 0, Np, s));
     Q4_TRY(launch_mma_gemm(p8, Hp, N, static_cast<const int8_t*>(prepared_pred), Hp, D, Hp, EPI_JOINTZ, z8, D,
-                           nullptr, w_pred->scale, b_pred, p_act->scale, z_act, status, nullptr, s, false, e,
-                           frame_idx));
+                           nullptr, w_pred->scale, b_pred, p_act->scale, z_act, status, nullptr, s, true, e,
+                           frame_idx));   // each kernel of the call is a programmatic dependent of the one before
     if (D == 256 && V <= 2048) {
       LmHeadArgs ja;
       memset(&ja, 0, sizeof(ja));
@@ -614,7 +615,7 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
       ja.b_out = b_out;
       ja.lp = logp;
       ja.status = status;
-      Q4_TRY(launch_mma_lmhead(ja, z8, D, nullptr, static_cast<const int8_t*>(prepared_out), s, false));
+      Q4_TRY(launch_mma_lmhead(ja, z8, D, nullptr, static_cast<const int8_t*>(prepared_out), s, true));
     } else {
       Q4_TRY(launch_mma_gemm(z8, D, N, static_cast<const int8_t*>(prepared_out), D, V, D, EPI_F32, logp, V, nullptr,
                              w_out->scale, b_out, z_act->scale, nullptr, status, nullptr, s));

@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(256) k_unpack_rows(const uint8_t* src, long lo
                                                      const int32_t* idx, int bits, int is_signed,
                                                      int zp, int k_pad, int n_rows, int8_t* dst,
                                                      long long dst_stride, int col0, int n_rows_pad) {
+  pdl_trigger();   // a dependent successor may set itself up; it reads nothing before this grid has completed
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = k_pad >> 5;  // 32 elements per thread
   if (i >= (long long)n_rows_pad * per_row) return;
