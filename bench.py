@@ -586,7 +586,8 @@ def main():
             from oracle import oracle as O
             O.build()
             cores = min(os.cpu_count() or 1, 8)
-            dt, audio, what = oracle_sample(args.workload, cores, frames=args.ref_frames)
+            # once per run: twice the frames of a step of the reference arm (10 - 20 s of CPU work at the default)
+            dt, audio, what = oracle_sample(args.workload, cores, frames=2 * args.ref_frames)
             line["cpu_baseline"] = {"value": dt / audio, "unit": "s/s", "cores": cores, "kind": "oracle",
                                     "sample": what, "seconds": dt}
         print(json.dumps(line), flush=True)

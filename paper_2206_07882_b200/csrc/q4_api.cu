@@ -266,9 +266,9 @@ int q4_linear_forward(const void* xq, const q4_act* x_act, int32_t M, const q4_m
       int8_t* x8 = reinterpret_cast<int8_t*>(ws + 256);
       const int Mp = (M + 127) / 128 * 128;
       TagScope tag(TAG_LINEAR);
-      Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
+      // the gather clears the status block and may start under the tail of whatever kernel precedes the call
       Q4_TRY(launch_unpack_rows(xq, row_bytes(w->k_pad, x_act->bits), nullptr, *x_act, w->k_pad, M, x8, w->k_pad, 0,
-                                Mp, s));
+                                Mp, s, status, true));
       Q4_TRY(launch_mma_gemm(x8, w->k_pad, M, static_cast<const int8_t*>(prepared), w->k_pad, w->rows, w->k_pad,
                              EPI_F32, out, w->rows, nullptr, w->scale, bias, x_act->scale, nullptr, status, nullptr,
                              s, true));   // programmatic dependent of the gather before it
@@ -353,10 +353,11 @@ int qlstm_step(const void* xq, const q4_act* x_act, const int32_t* x_row_idx, co
       int8_t* x8 = reinterpret_cast<int8_t*>(ws + 256);
       int8_t* h8 = x8 + align_up((size_t)Np * Kx);
       TagScope tag(TAG_PRED_LSTM);
-      Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
+      // every kernel of the call is a programmatic dependent of the one before (each waits for its
+      // predecessor's completion before it reads anything); the first gather clears the status block
       Q4_TRY(launch_unpack_rows(xq, row_bytes(w_ih->k_pad, x_act->bits), x_row_idx, *x_act, (int)Kx, N, x8, (long long)Kx,
-                                0, Np, s));
-      Q4_TRY(launch_unpack_rows(hq_in, row_bytes(H, hid_act->bits), nullptr, *hid_act, H, N, h8, H, 0, Np, s));
+                                0, Np, s, status, true));
+      Q4_TRY(launch_unpack_rows(hq_in, row_bytes(H, hid_act->bits), nullptr, *hid_act, H, N, h8, H, 0, Np, s, nullptr, true));
       MmaLstmArgs a;
       memset(&a, 0, sizeof(a));
       a.N = N;
@@ -599,8 +600,7 @@ int qjoint_logprobs(const float* e, const int32_t* frame_idx, const void* pq, co
     int32_t* status = reinterpret_cast<int32_t*>(ws);
     int8_t* p8 = reinterpret_cast<int8_t*>(ws + 256);
     int8_t* z8 = p8 + align_up((size_t)Np * Hp);
-    Q4_TRY(cudaMemsetAsync(status, 0, 256, s));
-    Q4_TRY(launch_unpack_rows(pq, row_bytes(Hp, p_act->bits), nullptr, *p_act, Hp, N, p8, Hp, 0, Np, s));
+    Q4_TRY(launch_unpack_rows(pq, row_bytes(Hp, p_act->bits), nullptr, *p_act, Hp, N, p8, Hp, 0, Np, s, status, true));
     Q4_TRY(launch_mma_gemm(p8, Hp, N, static_cast<const int8_t*>(prepared_pred), Hp, D, Hp, EPI_JOINTZ, z8, D,
                            nullptr, w_pred->scale, b_pred, p_act->scale, z_act, status, nullptr, s, true, e,
                            frame_idx));   // each kernel of the call is a programmatic dependent of the one before

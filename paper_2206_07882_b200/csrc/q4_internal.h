@@ -105,7 +105,10 @@ enum { EPI_QUANT8 = 3,      // re-quantize and store (code - zero_point) as int8
        EPI_JOINTZ = 4 };    // tanh(other factor * value), quantized, stored like EPI_QUANT8
 cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
                                const q4_act& act, int k_pad, int n_rows, int8_t* dst,
-                               long long dst_stride, int col0, int n_rows_pad, cudaStream_t s);
+                               long long dst_stride, int col0, int n_rows_pad, cudaStream_t s,
+                               int32_t* clear_status = nullptr, bool dependent = false);
+// clear_status: 64 status words zeroed by the kernel's first block (replaces a memset node in front of a
+// call); dependent: launched as a programmatic dependent (the kernel waits for its predecessor itself)
 struct UnpackJob {
   const uint8_t* src;       // packed code rows
   long long src_stride;

@@ -27,8 +27,10 @@ constexpr int LSTM_EPI_WARPS = 8;
 __global__ void __launch_bounds__(256) k_unpack_rows(const uint8_t* src, long long src_stride,
                                                      const int32_t* idx, int bits, int is_signed,
                                                      int zp, int k_pad, int n_rows, int8_t* dst,
-                                                     long long dst_stride, int col0, int n_rows_pad) {
+                                                     long long dst_stride, int col0, int n_rows_pad, int32_t* clear64) {
   pdl_trigger();   // a dependent successor may set itself up; it reads nothing before this grid has completed
+  pdl_wait();      // launched as a programmatic dependent itself: the source rows may be the predecessor's output
+  if (clear64 && blockIdx.x == 0 && threadIdx.x < 64) clear64[threadIdx.x] = 0;   // the call's status block
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = k_pad >> 5;  // 32 elements per thread
   if (i >= (long long)n_rows_pad * per_row) return;
@@ -76,16 +78,17 @@ __global__ void __launch_bounds__(256) k_unpack_rows(const uint8_t* src, long lo
 
 cudaError_t launch_unpack_rows(const void* src, long long src_stride, const int32_t* idx,
                                const q4_act& act, int k_pad, int n_rows, int8_t* dst,
-                               long long dst_stride, int col0, int n_rows_pad, cudaStream_t s) {
+                               long long dst_stride, int col0, int n_rows_pad, cudaStream_t s,
+                               int32_t* clear_status, bool dependent) {
   const long long total = (long long)n_rows_pad * (k_pad >> 5);
-  if (total <= 0) return cudaSuccess;
+  if (total <= 0) return clear_status ? cudaMemsetAsync(clear_status, 0, 256, s) : cudaSuccess;
   timing_begin(s);
-  k_unpack_rows<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
-      static_cast<const uint8_t*>(src), src_stride, idx, act.bits, act.is_signed, act.zero_point, k_pad,
-      n_rows, dst, dst_stride, col0, n_rows_pad);
+  cudaError_t le = launch_ex(k_unpack_rows, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, dependent, 1,
+                             static_cast<const uint8_t*>(src), src_stride, idx, (int)act.bits, (int)act.is_signed,
+                             (int)act.zero_point, k_pad, n_rows, dst, dst_stride, col0, n_rows_pad, clear_status);
   timing_end(s);
   ++g_launches;
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 // Several gather+unpack jobs in one launch (blockIdx.y selects the job).  The grid is sized for
