@@ -291,6 +291,28 @@ __device__ __forceinline__ void cell_fixed2(float pia, float pfa, float pga, flo
   hb = copysignf(h1, cb);
 }
 
+// One cell on the paired instructions: the (input, forget) and (output, candidate) exponentials of the
+// cell as pairs, the rest scalar; the same operations on the same operands as cell_fixed.
+__device__ __forceinline__ void cell_fixed_p(float pi, float pf, float pg, float po, float c_prev, float& c, float& h) {
+  const uint64_t one = pk2(1.0f, 1.0f);
+  const uint64_t e_if = exp2_fixed2(pk2(__fmul_rn(fminf(fmaxf(pi, -40.0f), 40.0f), NEG_LOG2E),
+                                        __fmul_rn(fminf(fmaxf(pf, -40.0f), 40.0f), NEG_LOG2E)));
+  const uint64_t e_og = exp2_fixed2(pk2(__fmul_rn(fminf(fmaxf(po, -40.0f), 40.0f), NEG_LOG2E),
+                                        __fmul_rn(fminf(fabsf(pg), 40.0f), NEG_2LOG2E)));
+  float I, F, O, G, t, m;
+  upk2(add2(one, e_if), I, F);
+  upk2(add2(one, e_og), O, G);
+  upk2(sub2(one, e_og), t, m);
+  (void)t;
+  const float ag = __fmul_rn(I, G);
+  const float R = rcp_fixed(__fmul_rn(ag, F));
+  const float ig = copysignf(__fmul_rn(__fmul_rn(m, F), R), pg);
+  c = __fmaf_rn(__fmul_rn(ag, R), c_prev, ig);
+  const float ec = exp2_fixed(__fmul_rn(fminf(fabsf(c), 40.0f), NEG_2LOG2E));
+  const float R2 = rcp_fixed(__fmul_rn(O, __fadd_rn(1.0f, ec)));
+  h = copysignf(__fmul_rn(__fsub_rn(1.0f, ec), R2), c);
+}
+
 // ---- argument blocks of the tile kernels -------------------------------------------
 enum { EPI_I32 = 0, EPI_F32 = 1, EPI_QUANT = 2 };
 

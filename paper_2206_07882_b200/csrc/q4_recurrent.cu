@@ -521,7 +521,7 @@ k_enc_recurrent_w4(const EncRecArgs a) {
           const float pg = __fmaf_rn((float)hh[2], s_hh.z, __fmaf_rn((float)pre.z, s_ih.z, bb.z));
           const float po = __fmaf_rn((float)hh[3], s_hh.w, __fmaf_rn((float)pre.w, s_ih.w, bb.w));
           float hval;
-          cell_fixed(pi, pf, pg, po, c_state[u], c_state[u], hval);
+          cell_fixed_p(pi, pf, pg, po, c_state[u], c_state[u], hval);
           q = quantize1(hval, a.hid_act.inv_scale, a.hid_act.zero_point, hlo, hhi);
           q2 = quantize1(hval, a.out_act.inv_scale, a.out_act.zero_point, ylo, yhi);
         }
@@ -873,7 +873,7 @@ k_enc_recurrent_w4s(const EncRecArgs a) {
       const float pg = __fmaf_rn((float)hh[2], s_hh.z, __fmaf_rn((float)pre.z, __fmul_rn(sx, s_ih.z), bb.z));
       const float po = __fmaf_rn((float)hh[3], s_hh.w, __fmaf_rn((float)pre.w, __fmul_rn(sx, s_ih.w), bb.w));
       float cs = u ? c_shared : c_own, hval;
-      cell_fixed(pi, pf, pg, po, cs, cs, hval);
+      cell_fixed_p(pi, pf, pg, po, cs, cs, hval);
       if (u)
         c_shared = cs;
       else
