@@ -248,6 +248,35 @@ def test_config1_full_size_sampled_utterances(Bd):
     encoder_case(Bd, enc, enc["features"], utts=[3, 28])
 
 
+def test_config4_encoder_full_size_sampled_utterances(Bd):
+    # The encoder of the end-to-end workload at its full size and in its launch configuration: 64
+    # utterances x 1000 log-mel frames (500 encoder steps), per-utterance MAX boundary, 8-bit first layer,
+    # 4-bit layers 2-6, replayed as a CUDA graph.  16 groups of 8 sequences on 15 clusters: the clusters of
+    # direction 0 take turns at the group of utterances 56-63 (71 or 72 steps each).  The oracle recomputes
+    # utterance 5 (a cluster's own group) and utterance 58 (the shared group).
+    B, T100 = 64, 1000
+    T = T100 // 2
+    enc_w = synth.encoder(4, T=T, B=B, first_layer_bits=8, in_max=True, features=False)
+    mel = synth.logmel(4, B, T100, 40)
+    mel_dev = torch.from_numpy(mel).cuda()
+    enc = Bd.Encoder(enc_w["enc"])
+    plan = Bd.encoder_recurrence_plan(T, B, 2, 640, 8, 8, True)
+    if plan["max_clusters"] == 15:
+        assert plan["kernel"] == 2 and plan["turns"] == [1, 0] and plan["clusters"] == [7, 8]
+    run = Bd.GraphedStep(lambda: enc.forward(Bd.q4_feature_prologue(mel_dev), want_layers=True))
+    got = run()
+    got = run()
+    torch.cuda.synchronize()
+    assert Bd.q4_poll_status(enc.ws) == 0
+    utts = [5, 58]
+    feats_ref = np.stack([O.features(mel[b]) for b in utts], axis=1).astype(np.float16)
+    ref = O.encoder_forward(enc_w["enc"], feats_ref, want_layers=True)
+    for l, yq in enumerate(got["layers"]):
+        g = gpu_codes(yq, 1280, enc.out_acts[l]).reshape(T, B, 1280)[:, utts]
+        np.testing.assert_array_equal(g, ref["layers"][l]["yq"], err_msg=f"encoder layer {l}")
+    np.testing.assert_array_equal(got["e"].cpu().numpy()[:, utts], ref["e"])
+
+
 # ------------------------------------------------------------------ against the PLAIN oracle path
 def plain_step_case(Bd, lw, x_act, hid, xq, hq, c):
     """qlstm_step against the textbook step (libm gates in double): real values within the
