@@ -281,14 +281,8 @@ def test_selection_paths_and_launch_modes_agree(Bd):
         np.testing.assert_array_equal(base[3], other[3])
 
 
-def test_config3_full_length_invariants(Bd):
-    # T=300, U_max=150 (450 iterations): properties that hold at any size.
-    dw = synth.decoder(seed=3, U_max=150)
-    T, B, W, U = 300, 16, 16, 150
-    e = config3_inputs(Bd, T, B)
-    dd = Bd.Decoder(dw)
-    tokens, lens, scores = dd.decode(e)
-    torch.cuda.synchronize()
+def check_search_invariants(dd, tokens, lens, scores, T, B, W, U, V=1024):
+    """Properties of an alignment-length synchronous search that hold at any size."""
     assert dd.tensors["status"].item() == 0
     IT = T + U
     par = dd.tensors["bp_parent"].cpu().numpy()[:IT]
@@ -303,7 +297,7 @@ def test_config3_full_length_invariants(Bd):
             assert (par[it, b, :n] >= 0).all() and (par[it, b, n:] < 0).all()     # slots are packed
             assert (np.diff(sc[it, b, :n]) <= 0).all()                            # rank order
             p, k = par[it, b, :n], tok[it, b, :n]
-            assert (p < len(strings)).all() and (k >= 0).all() and (k < 1024).all()
+            assert (p < len(strings)).all() and (k >= 0).all() and (k < V).all()
             t, u = t[p] + (k == 0), u[p] + (k > 0)
             assert ((t + u) == it + 1).all() and (t < T).all() and (u <= U).all()
             strings = [strings[pp] + ((int(kk),) if kk > 0 else ()) for pp, kk in zip(p, k)]
@@ -316,6 +310,37 @@ def test_config3_full_length_invariants(Bd):
         assert (np.diff(fs[b, :fin_n[b]]) <= 0).all()
         assert sc_h[b] == fs[b, 0] and 0 <= lens_h[b] <= U
         assert (tok_h[b, :lens_h[b]] > 0).all() and (tok_h[b, lens_h[b]:] == 0).all()
+
+
+def test_config3_full_length_invariants(Bd):
+    # T=300, U_max=150 (450 iterations): properties that hold at any size.
+    dw = synth.decoder(seed=3, U_max=150)
+    T, B, W, U = 300, 16, 16, 150
+    e = config3_inputs(Bd, T, B)
+    dd = Bd.Decoder(dw)
+    tokens, lens, scores = dd.decode(e)
+    torch.cuda.synchronize()
+    check_search_invariants(dd, tokens, lens, scores, T, B, W, U)
+
+
+def test_config4_search_full_size_invariants_in_graph_replay(Bd):
+    # The search of the end-to-end workload at its full size and in its launch configuration: 64 utterances,
+    # 500 frames, label budget 250 (750 iterations, 1024 hypothesis rows), 8-bit joint output layer, the
+    # whole search replayed as one CUDA graph.  Two replays give the same bits, and the properties that hold
+    # at any size hold (a search of this length is out of the oracle's reach; its first iterations are
+    # covered on sampled utterances by the composed test above).
+    dw = synth.decoder(seed=3, out_bits=8, U_max=250)
+    T, B, W, U = 500, 64, 16, 250
+    e = config3_inputs(Bd, T, B)
+    dd = Bd.Decoder(dw)
+    run = Bd.GraphedStep(lambda: dd.decode(e))
+    t1, l1, s1 = [x.clone() for x in run()]
+    par1 = dd.tensors["bp_parent"].clone()
+    t2, l2, s2 = run()
+    torch.cuda.synchronize()
+    assert torch.equal(t1, t2) and torch.equal(l1, l2) and torch.equal(s1, s2)
+    assert torch.equal(par1, dd.tensors["bp_parent"])
+    check_search_invariants(dd, t2, l2, s2, T, B, W, U)
 
 
 def run_tsd(Bd, dw, e, S_max, utts=None, tensor_cores=True):
