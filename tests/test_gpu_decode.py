@@ -496,6 +496,18 @@ def test_single_utterance_full_widths(Bd, W):
     assert tr == 1.0
 
 
+def test_single_utterance_full_length_beam_4(Bd):
+    # the run-time figure's utterance at its full length (152 frames, label budget 76: 228 iterations) and
+    # full widths, beam 4 (what the oracle decodes in a fraction of a minute): every beam of every iteration
+    # identical, through both regimes of the search (label iterations, then label-free ones)
+    dw = synth.decoder(seed=3, U_max=76, W=4)
+    T = 152
+    e = config3_inputs(Bd, T, 1).contiguous().cpu().numpy()
+    dd, tokens, lens, scores, ref = run_search(Bd, dw, e)
+    frac, tr = compare_search(dd, tokens, lens, scores, ref, [0], T, 76, 4, min_same=1.0)
+    assert tr == 1.0
+
+
 def test_config4_composed_full_widths_sampled_utterances(Bd):
     # The end-to-end workload as composed, at full widths and with its batch of 64: log-mel ->
     # prologue -> per-utterance MAX boundary, 8-bit first encoder layer -> 4-bit layers 2-6 ->
