@@ -47,6 +47,11 @@ extern "C" {
 #define Q4_ERR_TIMEOUT (-8)     /* a bounded device-side wait expired */
 
 typedef void* q4_stream; /* a cudaStream_t, passed as an opaque handle (NULL = default stream) */
+/* All work of a call is enqueued on its stream, in stream order with whatever the caller enqueued before.
+ * Kernels of the tensor-core paths are launched with programmatic stream serialization: one may be
+ * scheduled while its predecessor in the stream is draining, but every kernel waits for the completion of
+ * its predecessor (and the visibility of its writes) before it reads anything, so results never depend on
+ * it. */
 
 /* Integer weight matrix [rows, k_pad] with per-row scales (device pointers). */
 typedef struct {
