@@ -1095,11 +1095,39 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
     };
 
     const bool fused_head = D == 256 && V <= 2048;   // the fused head kernel: 256-wide bottleneck, one cluster per row tile
-    // Order of enqueueing = order in which a replayed graph submits kernels that do not depend on one
-    // another: the target LM (two wide layers, the longest chain of an iteration) first, so that its
-    // first kernel gets the SMs before the two shorter chains fill the rest.
-    // 1a. source LM (stream ss) and target LM (stream stt)
-    auto lm_chain = [&](int which) -> int {
+    // 1a. prediction network, then the joint network for every live slot (stream sp)
+    if (nets) {
+      Q4_CHECK(lstm_mma(sp, !forked || joint_on_call_stream, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
+                        st.pred_c, pred_h8));
+      Q4_CHECK(linear_mma(sp, true, TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
+                          st.pred_p, D, cst.adv_dst, nullptr, n_active));
+    }
+    {
+      TagScope tag(TAG_JOINT);
+      Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, sp, true));
+    }
+    joint_normalized = fused_head ? 1 : 0;
+    if (fused_head) {
+      // output layer of the joint network with the log-softmax over the vocabulary in its epilogue
+      TagScope tag(TAG_JOINT);
+      LmHeadArgs ja;
+      memset(&ja, 0, sizeof(ja));
+      ja.N = N;
+      ja.H = 0;
+      ja.V = V;
+      ja.q_scale = m.z_act.scale;
+      ja.sc_out = m.joint_out.w.scale;
+      ja.b_out = m.joint_out.bias;
+      ja.lp = logits;
+      ja.dst_row = live;
+      ja.status = st.status;
+      Q4_TRY(launch_mma_lmhead(ja, z8, D, nullptr, reinterpret_cast<const int8_t*>(pb + pp.lin[5]), sp, true));
+    } else {
+      Q4_CHECK(linear_mma(sp, true, TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr,
+                          nullptr));
+    }
+    // 1b. source LM (stream ss) and target LM (stream stt)
+    for (int which = 0; which < 2 && nets; ++which) {
       const q4_lm& lm = *lms[which];
       cudaStream_t sl = which == 0 ? ss : stt;
       const q4_lstm& L0 = lm.lstm[0];
@@ -1148,41 +1176,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
         Q4_CHECK(linear_mma(sl, true, head_tag, which == 0 ? 2 : 4, lm.out, bq8[which], lm.bott_act.scale, EPI_F32, lp,
                             V, cst.adv_dst, nullptr, n_active));
       }
-      return Q4_OK;
-    };
-    if (nets) Q4_CHECK(lm_chain(1));
-    // 1b. prediction network, then the joint network for every live slot (stream sp)
-    if (nets) {
-      Q4_CHECK(lstm_mma(sp, !forked || joint_on_call_stream, TAG_PRED_LSTM, 0, m.pred_lstm, m.pred_emb_act, xa8[0], ha8[0], st.pred_hq,
-                        st.pred_c, pred_h8));
-      Q4_CHECK(linear_mma(sp, true, TAG_PRED_PROJ, 0, m.pred_proj, pred_h8, m.pred_lstm.hid_act.scale, EPI_F32,
-                          st.pred_p, D, cst.adv_dst, nullptr, n_active));
     }
-    {
-      TagScope tag(TAG_JOINT);
-      Q4_TRY(launch_joint_z(e, nullptr, st.t, B, W, st.pred_p, st.row, N, D, m.z_act, nullptr, z8, live, sp, true));
-    }
-    joint_normalized = fused_head ? 1 : 0;
-    if (fused_head) {
-      // output layer of the joint network with the log-softmax over the vocabulary in its epilogue
-      TagScope tag(TAG_JOINT);
-      LmHeadArgs ja;
-      memset(&ja, 0, sizeof(ja));
-      ja.N = N;
-      ja.H = 0;
-      ja.V = V;
-      ja.q_scale = m.z_act.scale;
-      ja.sc_out = m.joint_out.w.scale;
-      ja.b_out = m.joint_out.bias;
-      ja.lp = logits;
-      ja.dst_row = live;
-      ja.status = st.status;
-      Q4_TRY(launch_mma_lmhead(ja, z8, D, nullptr, reinterpret_cast<const int8_t*>(pb + pp.lin[5]), sp, true));
-    } else {
-      Q4_CHECK(linear_mma(sp, true, TAG_JOINT, 5, m.joint_out, z8, m.z_act.scale, EPI_F32, logits, V, live, nullptr,
-                          nullptr));
-    }
-    if (nets) Q4_CHECK(lm_chain(0));
     if (forked) {   // join: the call's stream waits for both side chains
       cudaEvent_t j0 = reinterpret_cast<cudaEvent_t>(st.aux_event[1]);
       cudaEvent_t j1 = reinterpret_cast<cudaEvent_t>(st.aux_event[2]);
