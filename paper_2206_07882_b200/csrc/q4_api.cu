@@ -1263,7 +1263,7 @@ int dr_fusion_beam_step(const q4_model* model, q4_beam_state* state, const float
   sel.mode = mode;
   TagScope tag_sel(TAG_SELECT);
   if (mode != 0)
-    Q4_TRY(launch_tsd_select(sel, s));
+    Q4_TRY(launch_tsd_select(sel, s, use_mma));
   else
     Q4_TRY(launch_beam_select(sel, s, use_mma));
   return Q4_OK;

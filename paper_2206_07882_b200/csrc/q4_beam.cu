@@ -990,7 +990,7 @@ __global__ void __launch_bounds__(SEL_NT) k_tsd_select(const __grid_constant__ B
   }
 }
 
-cudaError_t launch_tsd_select(const BeamSelArgs& a, cudaStream_t s) {
+cudaError_t launch_tsd_select(const BeamSelArgs& a, cudaStream_t s, bool dependent) {
   const size_t smem = (size_t)a.W * a.V * sizeof(float) + (size_t)16 * ((a.V + 31) / 32) * sizeof(uint64_t);
   static size_t configured = 0;
   if (smem > configured) {
@@ -999,7 +999,7 @@ cudaError_t launch_tsd_select(const BeamSelArgs& a, cudaStream_t s) {
     configured = smem;
   }
   timing_begin(s);
-  cudaError_t le = launch_ex(k_tsd_select, dim3(a.B), dim3(SEL_NT), smem, s, false, 1, a);
+  cudaError_t le = launch_ex(k_tsd_select, dim3(a.B), dim3(SEL_NT), smem, s, dependent, 1, a);
   timing_end(s);
   ++g_launches;
   return le != cudaSuccess ? le : cudaGetLastError();

@@ -30,7 +30,7 @@ struct BeamSelArgs {
   int32_t exact_only;       // 1 = skip the register-resident fast filter (the exact threshold path alone)
 };
 cudaError_t launch_beam_select(const BeamSelArgs& a, cudaStream_t s, bool dependent = false);
-cudaError_t launch_tsd_select(const BeamSelArgs& a, cudaStream_t s);
+cudaError_t launch_tsd_select(const BeamSelArgs& a, cudaStream_t s, bool dependent = false);
 cudaError_t launch_beam_init(const q4_beam_state& st, int B, int W, int n_iters, cudaStream_t s);
 cudaError_t launch_traceback(const q4_beam_state& st, int B, int W, int n_iters, int u_max,
                              int32_t* tokens, int32_t* lens, float* scores, cudaStream_t s);
