@@ -460,6 +460,7 @@ def main():
     ms_total = t_start.elapsed_time(t_stop)
     enc_ms = sum(tmarks[i].elapsed_time(tmarks[i + 1]) for i in range(0, len(tmarks), 3)) / K
     dec_ms = sum(tmarks[i + 1].elapsed_time(tmarks[i + 2]) for i in range(0, len(tmarks), 3)) / K
+    per_step = sorted(tmarks[i].elapsed_time(tmarks[i + 2]) for i in range(0, len(tmarks), 3))   # each step by itself
 
     # ---- timed region 2: end to end through the public API with host buffers
     barrier()
@@ -552,6 +553,8 @@ def main():
         pk = peaks()
         line = {"metric": "end_to_end_rtf", "value": rtf, "unit": "s/s", "n_gpus": world, "steps": K,
                 "warmup": W, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+                "ms_per_step_best": per_step[0] if per_step else None,
+                "ms_per_step_median": statistics.median(per_step) if per_step else None,
                 "vs_baseline": None, "dtype": "int4/int8 codes, int32 accumulate, fp32 gates",
                 "data": "synthetic",
                 "config": {"workload": args.workload, "utterances_per_gpu": B, "frames": T,
