@@ -996,6 +996,36 @@ static int rec_max_clusters(int H) {
   return cached;
 }
 
+// The same question for the kernel whose clusters may take turns (its int8 variant, the one with the
+// larger shared-memory footprint); asked once.  The plan takes the smaller of the two answers, so that
+// every cluster of a launch is resident at once (a cluster that was not would only start later: a
+// waiting cluster only waits for lower-numbered ones; but its direction would finish that much later).
+static int rec_turns_max_clusters() {
+  static int cached = 0;
+  if (cached > 0) return cached;
+  constexpr int H = 640, cpc = H / REC_CLUSTER;
+  const size_t smem = (size_t)2 * 2 * REC_BG * H + (size_t)2 * REC_THREADS * sizeof(int4) + (size_t)3 * cpc * sizeof(float4) +
+                      (size_t)4 * 2 * REC_BG * cpc + (size_t)2 * 2 * sizeof(uint64_t) + 32 +
+                      (size_t)rec_turns_ksmem(true) * REC_THREADS * sizeof(uint4);
+  int n = 0;
+  if (cudaFuncSetAttribute(k_enc_recurrent_w4s<20, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(REC_CLUSTER * 16);
+    cfg.blockDim = dim3(REC4_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = REC_CLUSTER;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (cudaOccupancyMaxActiveClusters(&n, k_enc_recurrent_w4s<20, true>, &cfg) != cudaSuccess) n = 0;
+  }
+  cached = n > 0 ? n : 15;
+  return cached;
+}
+
 // Sequences per cluster: 8 or 16 (one or two MMA tiles), whichever gives the smaller estimated
 // layer time = waves * (fixed cost + cost per sequence); a step's work grows with the group
 // size, a second wave doubles everything.
@@ -1072,6 +1102,7 @@ EncRecPlan enc_recurrent_plan(int T, int B, int dirs, int H, int w_bits, int hid
   const int groups = (B + REC_BG - 1) / REC_BG;
   p.groups = groups;
   p.max_clusters = rec_max_clusters(H);
+  if (H == 640) p.max_clusters = p.max_clusters < rec_turns_max_clusters() ? p.max_clusters : rec_turns_max_clusters();
   // 640 cells, no accumulator dump: the kernels that keep (most of) a CTA's recurrent weights in
   // registers; the general kernel otherwise
   const bool regs_ok = hid_signed && H == 640 && !dump && (w_bits == 4 || w_bits == 8) && (hid_bits == 4 || hid_bits == 8);
